@@ -1,0 +1,183 @@
+/*
+ * fasa.h - C ABI of the B200 (sm_100a) decode-time hot path of FASA,
+ * Frequency-Aware Sparse Attention (arxiv 2602.03152).
+ *
+ * One decode step per (batch b, KV head h), in the paper's order:
+ *   fasa_kv_append          cache update, incl. the dominant part of the key cache
+ *                           (C_key^dom of Algorithm 2, kept here as a packed
+ *                           "proxy-K" side buffer)
+ *   fasa_fc_score           TIP: S_t = sum_{i in I_dom} alpha^(i)       (Sec. 4.1)
+ *   fasa_topk               T_t = TopK-I(S_t, N_fac)                    (Sec. 4.1)
+ *   fasa_sparse_decode_attn FAC: Softmax(q K_T^T / sqrt(d)) V_T         (Sec. 4.2, Eq. 6-7)
+ *   fasa_full_decode_attn   full-KV attention, the FKV baseline         (Sec. 5.1)
+ *
+ * Conventions
+ *   - Every tensor argument is a DEVICE pointer owned by the caller unless its
+ *     name ends in _host.  The library owns only the context and a few hundred
+ *     bytes of device tables inside it.  Nothing is allocated per call.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream) and return without synchronising, except where
+ *     stated.  A non-zero return means nothing was enqueued by that call.
+ *   - bf16 = IEEE binary32 upper half, 2 bytes.  head_dim is 128.
+ *   - Layouts are row-major.  K and V: [batch][n_kv_heads][max_len][128] bf16
+ *     (or the strides in fasa_config_t), keys stored post-RoPE at their
+ *     absolute positions.  q: [batch][n_q_heads][128] bf16, post-RoPE; query
+ *     head g belongs to KV head g / (n_q_heads / n_kv_heads).
+ *   - Frequency chunk (FC) i, 0 <= i < 64, is the channel pair (i, i+64) with
+ *     rope_pairing 0 (rotate-half layout) or (2i, 2i+1) with rope_pairing 1
+ *     (the paper's Eq. 1 layout).  An FC is never split (Appendix, design choices).
+ *   - Proxy-K buffer: [batch][n_kv_heads][max_len][proxy_row_elems] bf16 where
+ *     proxy_row_elems = 8 * ceil(n_dom / 4) (fasa_proxy_row_elems).  Row j holds,
+ *     for the head's dominant FCs sorted ascending, the pairs (K[j][c0], K[j][c1]);
+ *     padding elements are zero.  Base pointer 16-byte aligned.
+ *   - Data-dependent problems (a sequence longer than max_len, an index out of
+ *     range) never fault: the kernel clamps and ORs a bit into a device status
+ *     word read by fasa_get_device_status.
+ */
+#ifndef FASA_H_
+#define FASA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FASA_OK                 0
+#define FASA_ERR_INVALID_ARG   -1   /* null pointer, non-positive size, bad alignment      */
+#define FASA_ERR_UNSUPPORTED   -2   /* head_dim != 128, n_dom outside 1..64, group > 8 ... */
+#define FASA_ERR_WORKSPACE     -3   /* n_sel_max / budget larger than the workspace covers */
+#define FASA_ERR_CUDA          -4   /* a CUDA runtime call failed (see fasa_last_cuda_error) */
+#define FASA_ERR_TIMEOUT       -5   /* reserved: no kernel of this library waits           */
+
+/* Bits of the device status word. */
+#define FASA_DEV_LEN_CLAMPED    1   /* a seq_lens entry was < 0 or > max_len               */
+#define FASA_DEV_APPEND_FULL    2   /* kv_append ran out of rows; the excess was dropped   */
+#define FASA_DEV_IDX_CLAMPED    4   /* sparse attention met an index outside [0, max_len)  */
+#define FASA_DEV_NSEL_CLAMPED   8   /* n_sel exceeded n_sel_max                            */
+
+typedef struct fasa_ctx fasa_ctx_t;
+
+typedef struct {
+  int32_t batch, n_q_heads, n_kv_heads, head_dim; /* head_dim must be 128                  */
+  int32_t max_len;        /* rows allocated per (b, kv head) in K, V, proxy and scores     */
+  int32_t n_dom;          /* F = N_tip: dominant FCs per KV head, 1..64                    */
+  int32_t rope_pairing;   /* 0: FC i = (i, i+64); 1: FC i = (2i, 2i+1)                     */
+  int32_t group_reduce;   /* score of a KV head over its query heads: 0 sum, 1 max         */
+  int32_t n_sink;         /* first n_sink positions are always selected                    */
+  int32_t n_recent;       /* last n_recent positions are always selected                   */
+  float   softmax_scale;  /* 0 => 1/sqrt(head_dim)                                         */
+  int64_t k_stride_b, k_stride_h, k_stride_t; /* in elements; all 0 => dense layout above  */
+  int64_t v_stride_b, v_stride_h, v_stride_t; /* stride_t must be a multiple of 8          */
+} fasa_config_t;
+
+/* ---- context (off the hot path) ----------------------------------------- */
+
+/* Validates cfg, sorts each head's dominant-FC list and uploads the channel
+ * table to the current device.  dom_fc_host: [n_kv_heads][n_dom] distinct FC
+ * indices in 0..63 (the calibrated I_dom of Sec. 4.1; Algorithm 1 produces it).
+ * Synchronises the device once.  Errors: INVALID_ARG (null, duplicate or
+ * out-of-range FC), UNSUPPORTED, CUDA. */
+int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_host, fasa_ctx_t** out);
+int32_t fasa_destroy(fasa_ctx_t* ctx);
+
+/* Elements per proxy-K row for n_dom dominant FCs: 8 * ceil(n_dom / 4). */
+int32_t fasa_proxy_row_elems(int32_t n_dom);
+
+/* Bytes of caller-provided scratch that fasa_topk, the two attention calls and
+ * fasa_decode_step need for selections of at most n_sel_max tokens.  The
+ * workspace must be 256-byte aligned; its contents need not be preserved
+ * between calls, and two calls that overlap on the GPU need separate ones. */
+int32_t fasa_workspace_bytes(const fasa_ctx_t* ctx, int32_t n_sel_max, size_t* out_bytes);
+
+const char* fasa_status_string(int32_t status);
+/* Text of the last CUDA error a call of this library met in this thread's context. */
+const char* fasa_last_cuda_error(const fasa_ctx_t* ctx);
+/* Synchronises `stream`, copies the device status word to *host_out and clears it. */
+int32_t fasa_get_device_status(fasa_ctx_t* ctx, void* stream, int32_t* host_out);
+/* Number of kernels this context has launched so far (host-side counter). */
+int64_t fasa_launch_count(const fasa_ctx_t* ctx);
+
+/* ---- cache update (Algorithm 2: Split + UpdateCache) -------------------- */
+
+/* Appends n_new rows per (b, kv head): K and V rows go to rows seq_lens[b] ..
+ * seq_lens[b]+n_new-1 of the caches, the dominant-FC slices of the new keys go
+ * to the same rows of proxy_k, then seq_lens[b] += n_new (on the device, in
+ * stream order).  k_new, v_new: bf16 [batch][n_kv_heads][n_new][128], post-RoPE.
+ * Rows that would pass max_len are dropped and FASA_DEV_APPEND_FULL is set. */
+int32_t fasa_kv_append(fasa_ctx_t* ctx, void* k_cache, void* v_cache, void* proxy_k,
+                       int32_t* seq_lens, const void* k_new, const void* v_new,
+                       int32_t n_new, void* stream);
+
+/* Fills proxy_k rows 0 .. seq_lens[b]-1 from a key cache that was written by
+ * other means (a prefill): the Split of Algorithm 2 applied to the whole cache. */
+int32_t fasa_proxy_build(fasa_ctx_t* ctx, const void* k_cache, void* proxy_k,
+                         const int32_t* seq_lens, void* stream);
+
+/* ---- TIP: importance scores (Sec. 4.1) ---------------------------------- */
+
+/* scores[b][h][j] = reduce_{g in group(h)} sum_{i in I_dom(h)}
+ *                   (q[b][g][c0(i)] K[j][c0(i)] + q[b][g][c1(i)] K[j][c1(i)])
+ * for j < seq_lens[b], read from proxy_k; fp32 accumulation of exact bf16
+ * products; no scaling.  scores: fp32 [batch][n_kv_heads][max_len]; entries at
+ * j >= seq_lens[b] are left untouched.  -0 is stored as +0. */
+int32_t fasa_fc_score(fasa_ctx_t* ctx, const void* q, const void* proxy_k,
+                      const int32_t* seq_lens, float* scores, void* stream);
+
+/* ---- TopK-I (Sec. 4.1) --------------------------------------------------- */
+
+/* Per (b, h) with L = seq_lens[b]: forced = positions < n_sink or >= L - n_recent;
+ * T = forced U the `budget` best-scoring other positions, higher score first and
+ * lower index first among equal scores; n_sel = min(L, |forced| + budget).
+ * budget > 0 is N_fac itself; budget < 0 means ceil(-budget/1000 * L) (device-side,
+ * so a length that grows each step needs no host round trip).
+ * idx: int32 [batch][n_kv_heads][n_sel_max], ascending; entries past n_sel are
+ * left untouched.  n_sel: int32 [batch][n_kv_heads].  If n_sel would exceed
+ * n_sel_max the selection is cut to the n_sel_max best and FASA_DEV_NSEL_CLAMPED
+ * is set.  NaN scores rank above +inf (their sign bit clear) or below -inf. */
+int32_t fasa_topk(fasa_ctx_t* ctx, const float* scores, const int32_t* seq_lens,
+                  int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
+                  void* workspace, void* stream);
+
+/* ---- FAC (Sec. 4.2, Eq. 6-7) and FKV (Sec. 5.1) -------------------------- */
+
+/* out[b][g][:] = sum_j p_j V[idx_j],  p = softmax_j(q[b][g] . K[idx_j] * scale) over
+ * the n_sel[b][h] rows listed in idx (any order, rows used as stored).  fp32
+ * accumulation; out fp32 [batch][n_q_heads][128]; lse (nullable) fp32
+ * [batch][n_q_heads] = log sum_j exp(logit_j).  n_sel == 0 gives out = 0,
+ * lse = -inf.  Split over the selection, merged by a second kernel. */
+int32_t fasa_sparse_decode_attn(fasa_ctx_t* ctx, const void* q, const void* k_cache,
+                                const void* v_cache, const int32_t* idx, const int32_t* n_sel,
+                                int32_t n_sel_max, float* out, float* lse, void* workspace,
+                                void* stream);
+
+/* The same over all rows j < seq_lens[b], no index list. */
+int32_t fasa_full_decode_attn(fasa_ctx_t* ctx, const void* q, const void* k_cache,
+                              const void* v_cache, const int32_t* seq_lens, float* out,
+                              float* lse, void* workspace, void* stream);
+
+/* ---- whole step ---------------------------------------------------------- */
+
+/* fasa_fc_score -> fasa_topk -> fasa_sparse_decode_attn on one stream with no
+ * host round trip in between.  scores, idx and n_sel are outputs too. */
+int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_cache,
+                         const void* v_cache, const void* proxy_k, const int32_t* seq_lens,
+                         int32_t budget, int32_t n_sel_max, float* scores, int32_t* idx,
+                         int32_t* n_sel, float* out, float* lse, void* workspace, void* stream);
+
+/* End-to-end step from HOST buffers (pinned memory recommended): copies q_host,
+ * k_new_host, v_new_host (layouts as fasa_kv_append with n_new = 1) to the device
+ * staging area dev_stage (>= fasa_stage_bytes), appends, runs fasa_decode_step,
+ * copies out to out_host (fp32 [batch][n_q_heads][128]) and synchronises the stream. */
+int32_t fasa_stage_bytes(const fasa_ctx_t* ctx, size_t* out_bytes);
+int32_t fasa_decode_step_host(fasa_ctx_t* ctx, const void* q_host, const void* k_new_host,
+                              const void* v_new_host, void* dev_stage, void* k_cache,
+                              void* v_cache, void* proxy_k, int32_t* seq_lens, int32_t budget,
+                              int32_t n_sel_max, float* scores, int32_t* idx, int32_t* n_sel,
+                              float* out, float* out_host, void* workspace, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FASA_H_ */

@@ -1,0 +1,200 @@
+"""ctypes front end of the fp64 CPU oracle (`fasa_oracle.c`).
+
+TEST INFRASTRUCTURE ONLY.  Tests, the smoke check and the benchmark's CPU-baseline
+leg import this module; nothing on the product path does, and this module never
+imports the CUDA package.  It compiles the C file with gcc on first use.
+
+Each wrapper passes numpy arrays to one C function and cites the passage that
+function follows (arxiv 2602.03152).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fasa_oracle.c")
+_LIB = os.path.join(_HERE, "libfasa_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+_f64p = ctypes.POINTER(ctypes.c_double)
+_i32p = ctypes.POINTER(ctypes.c_int32)
+_u16p = ctypes.POINTER(ctypes.c_uint16)
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle into a shared object next to its source."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + ".tmp.%d" % os.getpid()
+            subprocess.check_call(
+                ["gcc", "-O2", "-std=c99", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"]
+            )
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.fasa_oracle_bf16_to_f64.restype = ctypes.c_double
+        _lib.fasa_oracle_bf16_to_f64.argtypes = [ctypes.c_uint16]
+        _lib.fasa_oracle_f32_to_bf16.restype = ctypes.c_uint16
+        _lib.fasa_oracle_f32_to_bf16.argtypes = [ctypes.c_float]
+        _lib.fasa_oracle_theta.restype = ctypes.c_double
+        _lib.fasa_oracle_theta.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_double]
+        _lib.fasa_oracle_select.restype = ctypes.c_int
+        _lib.fasa_oracle_decode_bf16.restype = ctypes.c_int
+    return _lib
+
+
+def _f64(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _ptr(a, t):
+    return a.ctypes.data_as(t) if a is not None else None
+
+
+def bf16_bits_to_f64(bits) -> np.ndarray:
+    """Exact widening of bf16 bit patterns (uint16) to float64."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    out = np.empty(bits.shape, dtype=np.float64)
+    _load().fasa_oracle_widen_bf16(_ptr(bits, _u16p), ctypes.c_int64(bits.size), _ptr(out, _f64p))
+    return out
+
+
+def f32_to_bf16_bits(x: float) -> int:
+    """Round-to-nearest-even binary32 -> bf16 bits."""
+    return int(_load().fasa_oracle_f32_to_bf16(ctypes.c_float(x)))
+
+
+def theta(i: int, d: int, base: float) -> float:
+    """theta_i = B^(-2i/d), 0-based FC index (Sec. 3.1)."""
+    return float(_load().fasa_oracle_theta(i, d, ctypes.c_double(base)))
+
+
+def rope(x, pos: float, base: float, pairing: int = 0) -> np.ndarray:
+    """Rotate every FC of one d-vector to position `pos` (Sec. 3.1, Eq. 1)."""
+    x = _f64(x)
+    assert x.ndim == 1 and x.size % 2 == 0
+    out = np.empty_like(x)
+    _load().fasa_oracle_rope(_ptr(x, _f64p), ctypes.c_int(x.size), ctypes.c_double(pos),
+                             ctypes.c_double(base), ctypes.c_int(pairing), _ptr(out, _f64p))
+    return out
+
+
+def fc_partial_logits(q, K, pairing: int = 0) -> np.ndarray:
+    """Single-FC raw scores alpha^(i)[j] for all i, shape [d/2, L] (Sec. 3.3, Eq. 3)."""
+    q, K = _f64(q), _f64(K)
+    L, d = K.shape
+    a = np.empty((d // 2, L), dtype=np.float64)
+    _load().fasa_oracle_fc_partial_logits(_ptr(q, _f64p), _ptr(K, _f64p), ctypes.c_int(L),
+                                          ctypes.c_int(d), ctypes.c_int(pairing), _ptr(a, _f64p))
+    return a
+
+
+def fc_score(q, K, dom, pairing: int = 0, group_reduce: int = 0) -> np.ndarray:
+    """Importance scores S_t[j] of one KV head from its G query heads (Sec. 4.1, TIP)."""
+    q, K = _f64(q), _f64(K)
+    if q.ndim == 1:
+        q = q[None, :]
+    G, d = q.shape
+    L = K.shape[0]
+    dom = np.ascontiguousarray(dom, dtype=np.int32)
+    S = np.empty(L, dtype=np.float64)
+    _load().fasa_oracle_fc_score(_ptr(q, _f64p), ctypes.c_int(G), _ptr(K, _f64p), ctypes.c_int(L),
+                                 ctypes.c_int(d), ctypes.c_int(pairing), _ptr(dom, _i32p),
+                                 ctypes.c_int(dom.size), ctypes.c_int(group_reduce), _ptr(S, _f64p))
+    return S
+
+
+def select(S, k: int, n_sink: int = 0, n_recent: int = 0, tie_rel: float = 1e-3):
+    """T_t = forced U TopK-I(S_t, k), ascending; also the boundary record (Sec. 4.1)."""
+    S = _f64(S)
+    L = S.size
+    idx = np.empty(max(L, 1), dtype=np.int32)
+    band = np.zeros(4, dtype=np.float64)
+    n = _load().fasa_oracle_select(_ptr(S, _f64p), ctypes.c_int(L), ctypes.c_int(k),
+                                   ctypes.c_int(n_sink), ctypes.c_int(n_recent),
+                                   ctypes.c_double(tie_rel), _ptr(idx, _i32p), _ptr(band, _f64p))
+    info = {"has_boundary": bool(band[0]), "s_k": band[1], "s_k1": band[2], "tie": bool(band[3])}
+    return idx[:n].copy(), info
+
+
+def attn_subset(q, K, V, idx, scale: float):
+    """FAC on the selected rows: (O [G,d], lse [G]) (Sec. 4.2, Eq. 6-7)."""
+    q, K, V = _f64(q), _f64(K), _f64(V)
+    if q.ndim == 1:
+        q = q[None, :]
+    G, d = q.shape
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    O = np.empty((G, d), dtype=np.float64)
+    lse = np.empty(G, dtype=np.float64)
+    _load().fasa_oracle_attn_subset(_ptr(q, _f64p), ctypes.c_int(G), _ptr(K, _f64p), _ptr(V, _f64p),
+                                    ctypes.c_int(d), _ptr(idx, _i32p), ctypes.c_int(idx.size),
+                                    ctypes.c_double(scale), _ptr(O, _f64p), _ptr(lse, _f64p))
+    return O, lse
+
+
+def attn_dense(q, K, V, L: int, scale: float):
+    """Full-KV attention over rows 0..L-1 (FKV, Sec. 5.1)."""
+    q, K, V = _f64(q), _f64(K), _f64(V)
+    if q.ndim == 1:
+        q = q[None, :]
+    G, d = q.shape
+    O = np.empty((G, d), dtype=np.float64)
+    lse = np.empty(G, dtype=np.float64)
+    _load().fasa_oracle_attn_dense(_ptr(q, _f64p), ctypes.c_int(G), _ptr(K, _f64p), _ptr(V, _f64p),
+                                   ctypes.c_int(d), ctypes.c_int(L), ctypes.c_double(scale),
+                                   _ptr(O, _f64p), _ptr(lse, _f64p))
+    return O, lse
+
+
+def decode_bf16(q_bits, K_bits, V_bits, seq_lens, dom, *, pairing=0, group_reduce=0, n_sink=0,
+                n_recent=0, budget=256, n_sel_max=None, scale=None, tie_rel=1e-3, n_threads=0,
+                want_scores=True, want_sparse=True, want_dense=True):
+    """One whole decode step on bf16 bit patterns, unit by unit in the paper's order.
+
+    q_bits [B,Hq,d], K_bits/V_bits [B,Hkv,Lmax,d] (uint16), seq_lens [B], dom [Hkv,F].
+    Returns a dict with scores, idx, n_sel, band, out, lse, dense_out, dense_lse, threads.
+    """
+    q_bits = np.ascontiguousarray(q_bits, dtype=np.uint16)
+    K_bits = np.ascontiguousarray(K_bits, dtype=np.uint16)
+    V_bits = np.ascontiguousarray(V_bits, dtype=np.uint16)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    dom = np.ascontiguousarray(dom, dtype=np.int32)
+    B, Hq, d = q_bits.shape
+    _, Hkv, Lmax, _ = K_bits.shape
+    F = dom.shape[1]
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    if n_sel_max is None:
+        n_sel_max = Lmax
+    U = B * Hkv
+    scores = np.full((B, Hkv, Lmax), np.nan, dtype=np.float64) if want_scores else None
+    idx = np.full((B, Hkv, n_sel_max), -1, dtype=np.int32)
+    n_sel = np.zeros((B, Hkv), dtype=np.int32)
+    band = np.zeros((B, Hkv, 4), dtype=np.float64)
+    out = np.zeros((B, Hq, d), dtype=np.float64) if want_sparse else None
+    lse = np.zeros((B, Hq), dtype=np.float64) if want_sparse else None
+    dout = np.zeros((B, Hq, d), dtype=np.float64) if want_dense else None
+    dlse = np.zeros((B, Hq), dtype=np.float64) if want_dense else None
+    used = _load().fasa_oracle_decode_bf16(
+        _ptr(q_bits, _u16p), _ptr(K_bits, _u16p), _ptr(V_bits, _u16p), _ptr(seq_lens, _i32p),
+        _ptr(dom, _i32p), ctypes.c_int(B), ctypes.c_int(Hq), ctypes.c_int(Hkv), ctypes.c_int(d),
+        ctypes.c_int(Lmax), ctypes.c_int(F), ctypes.c_int(pairing), ctypes.c_int(group_reduce),
+        ctypes.c_int(n_sink), ctypes.c_int(n_recent), ctypes.c_int(budget),
+        ctypes.c_int(n_sel_max), ctypes.c_double(scale), ctypes.c_double(tie_rel),
+        ctypes.c_int(n_threads), _ptr(scores, _f64p), _ptr(idx, _i32p), _ptr(n_sel, _i32p),
+        _ptr(band, _f64p), _ptr(out, _f64p), _ptr(lse, _f64p), _ptr(dout, _f64p), _ptr(dlse, _f64p))
+    assert U >= 0
+    return {"scores": scores, "idx": idx, "n_sel": n_sel, "band": band, "out": out, "lse": lse,
+            "dense_out": dout, "dense_lse": dlse, "threads": int(used)}
