@@ -1,0 +1,225 @@
+// Context, validation, workspace sizing and the composite calls of the C ABI.
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "fasa_common.cuh"
+
+namespace {
+
+bool valid_cfg(const fasa_config_t& c, int32_t* why) {
+  *why = FASA_ERR_INVALID_ARG;
+  if (c.batch <= 0 || c.n_q_heads <= 0 || c.n_kv_heads <= 0 || c.max_len <= 0) return false;
+  if (c.n_sink < 0 || c.n_recent < 0) return false;
+  if (c.softmax_scale < 0.f || c.softmax_scale != c.softmax_scale) return false;
+  *why = FASA_ERR_UNSUPPORTED;
+  if (c.head_dim != FASA_HEAD_DIM) return false;
+  if (c.n_dom < 1 || c.n_dom > FASA_MAX_DOM) return false;
+  if (c.n_q_heads % c.n_kv_heads != 0) return false;
+  if (c.n_q_heads / c.n_kv_heads > FASA_MAX_GROUP) return false;
+  if (c.rope_pairing != 0 && c.rope_pairing != 1) return false;
+  if (c.group_reduce != 0 && c.group_reduce != 1) return false;
+  if ((long long)c.batch * c.n_kv_heads > 65535) return false;  // grid.y
+  return true;
+}
+
+bool fill_strides(int64_t& sb, int64_t& sh, int64_t& st, const fasa_config_t& c) {
+  if (sb == 0 && sh == 0 && st == 0) {
+    st = FASA_HEAD_DIM;
+    sh = (int64_t)c.max_len * FASA_HEAD_DIM;
+    sb = sh * c.n_kv_heads;
+    return true;
+  }
+  // rows are read with 16-byte loads
+  return st >= FASA_HEAD_DIM && st % 8 == 0 && sh % 8 == 0 && sb % 8 == 0 && sh > 0 && sb > 0;
+}
+
+}  // namespace
+
+extern "C" int32_t fasa_proxy_row_elems(int32_t n_dom) {
+  if (n_dom < 1 || n_dom > FASA_MAX_DOM) return 0;
+  return 8 * ((n_dom + 3) / 4);
+}
+
+extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_host,
+                               fasa_ctx_t** out) {
+  if (!cfg || !dom_fc_host || !out) return FASA_ERR_INVALID_ARG;
+  *out = nullptr;
+  int32_t why;
+  if (!valid_cfg(*cfg, &why)) return why;
+
+  fasa_ctx* ctx = new (std::nothrow) fasa_ctx();
+  if (!ctx) return FASA_ERR_INVALID_ARG;
+  memset(ctx, 0, sizeof(*ctx));
+  ctx->cfg = *cfg;
+  fasa_config_t& c = ctx->cfg;
+  if (!fill_strides(c.k_stride_b, c.k_stride_h, c.k_stride_t, c) ||
+      !fill_strides(c.v_stride_b, c.v_stride_h, c.v_stride_t, c)) {
+    delete ctx;
+    return FASA_ERR_INVALID_ARG;
+  }
+  if (c.softmax_scale == 0.f) c.softmax_scale = 0.08838834764831845f;  // 1/sqrt(128)
+  ctx->group = c.n_q_heads / c.n_kv_heads;
+  ctx->chunks = (c.n_dom + 3) / 4;
+  ctx->row_elems = 8 * ctx->chunks;
+
+  // Channel table: dominant FCs sorted ascending, FC r of head h at elements 2r, 2r+1.
+  std::vector<int16_t> chan((size_t)c.n_kv_heads * ctx->row_elems, (int16_t)-1);
+  for (int h = 0; h < c.n_kv_heads; ++h) {
+    std::vector<int32_t> fcs(dom_fc_host + (size_t)h * c.n_dom, dom_fc_host + (size_t)(h + 1) * c.n_dom);
+    std::sort(fcs.begin(), fcs.end());
+    for (int r = 0; r < c.n_dom; ++r) {
+      bool bad = fcs[r] < 0 || fcs[r] >= FASA_HEAD_DIM / 2 || (r > 0 && fcs[r] == fcs[r - 1]);
+      if (bad) {
+        delete ctx;
+        return FASA_ERR_INVALID_ARG;
+      }
+      int c0 = c.rope_pairing == 0 ? fcs[r] : 2 * fcs[r];
+      int c1 = c.rope_pairing == 0 ? fcs[r] + FASA_HEAD_DIM / 2 : 2 * fcs[r] + 1;
+      chan[(size_t)h * ctx->row_elems + 2 * r] = (int16_t)c0;
+      chan[(size_t)h * ctx->row_elems + 2 * r + 1] = (int16_t)c1;
+    }
+  }
+
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  cudaDeviceProp prop;
+  if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, ctx->device);
+  if (e == cudaSuccess && prop.major != 10) {
+    delete ctx;
+    return FASA_ERR_UNSUPPORTED;  // built for sm_100a only
+  }
+  if (e == cudaSuccess) ctx->n_sm = prop.multiProcessorCount;
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_chan, chan.size() * sizeof(int16_t));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, 256);
+  if (e == cudaSuccess)
+    e = cudaMemcpy(ctx->d_chan, chan.data(), chan.size() * sizeof(int16_t), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    cudaFree(ctx->d_chan);
+    cudaFree(ctx->d_status);
+    delete ctx;
+    return FASA_ERR_CUDA;
+  }
+  *out = ctx;
+  return FASA_OK;
+}
+
+extern "C" int32_t fasa_destroy(fasa_ctx_t* ctx) {
+  if (!ctx) return FASA_ERR_INVALID_ARG;
+  cudaFree(ctx->d_chan);
+  cudaFree(ctx->d_status);
+  delete ctx;
+  return FASA_OK;
+}
+
+extern "C" const char* fasa_status_string(int32_t s) {
+  switch (s) {
+    case FASA_OK: return "ok";
+    case FASA_ERR_INVALID_ARG: return "invalid argument";
+    case FASA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case FASA_ERR_WORKSPACE: return "workspace too small for this selection size";
+    case FASA_ERR_CUDA: return "CUDA runtime error";
+    case FASA_ERR_TIMEOUT: return "timeout";
+    default: return "unknown status";
+  }
+}
+
+extern "C" const char* fasa_last_cuda_error(const fasa_ctx_t* ctx) {
+  return ctx ? ctx->cuda_err : "";
+}
+
+extern "C" int64_t fasa_launch_count(const fasa_ctx_t* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" int32_t fasa_get_device_status(fasa_ctx_t* ctx, void* stream, int32_t* host_out) {
+  if (!ctx || !host_out) return FASA_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  FASA_CUDA_TRY(ctx, cudaMemcpyAsync(host_out, ctx->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  FASA_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(int32_t), s));
+  FASA_CUDA_TRY(ctx, cudaStreamSynchronize(s));
+  return FASA_OK;
+}
+
+// Splits: enough CTAs to fill the GPU a few times over, between 64 and 2048 rows each.
+static int split_count_bound(const fasa_ctx* ctx, int n_upper) {
+  const int units = ctx->cfg.batch * ctx->cfg.n_kv_heads;
+  const int target = 4 * (ctx->n_sm > 0 ? ctx->n_sm : 148);
+  const int want = std::max((target + units - 1) / units, (n_upper + 2047) / 2048);
+  const int most = (n_upper + 63) / 64;
+  return std::max(1, std::min(want, most));   // non-decreasing in n_upper
+}
+
+fasa_split_plan fasa_plan_splits(const fasa_ctx* ctx, int n_upper) {
+  const int n = split_count_bound(ctx, n_upper);
+  int chunk = (n_upper + n - 1) / n;
+  chunk = (chunk + 31) / 32 * 32;
+  fasa_split_plan p;
+  p.chunk = chunk;
+  p.n_splits = std::max(1, (n_upper + chunk - 1) / chunk);  // <= n
+  return p;
+}
+
+// The partial-result area is sized for the largest split count any call can use
+// (the bound at max_len), so it does not depend on the selection size.
+extern "C" int32_t fasa_workspace_bytes(const fasa_ctx_t* ctx, int32_t n_sel_max, size_t* out_bytes) {
+  if (!ctx || !out_bytes || n_sel_max < 0) return FASA_ERR_INVALID_ARG;
+  const int n = split_count_bound(ctx, ctx->cfg.max_len);
+  size_t per_split = (size_t)ctx->cfg.batch * ctx->cfg.n_q_heads * (FASA_HEAD_DIM + 2) * sizeof(float);
+  *out_bytes = fasa_align_up(per_split * (size_t)n, 256) + 256;
+  return FASA_OK;
+}
+
+extern "C" int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_cache,
+                                    const void* v_cache, const void* proxy_k,
+                                    const int32_t* seq_lens, int32_t budget, int32_t n_sel_max,
+                                    float* scores, int32_t* idx, int32_t* n_sel, float* out,
+                                    float* lse, void* workspace, void* stream) {
+  if (!ctx || !q || !k_cache || !v_cache || !proxy_k || !seq_lens || !scores || !idx || !n_sel ||
+      !out || !workspace || budget == 0 || n_sel_max <= 0)
+    return FASA_ERR_INVALID_ARG;
+  int32_t st = fasa_fc_score(ctx, q, proxy_k, seq_lens, scores, stream);
+  if (st != FASA_OK) return st;
+  st = fasa_topk(ctx, scores, seq_lens, budget, n_sel_max, idx, n_sel, workspace, stream);
+  if (st != FASA_OK) return st;
+  return fasa_sparse_decode_attn(ctx, q, k_cache, v_cache, idx, n_sel, n_sel_max, out, lse,
+                                 workspace, stream);
+}
+
+extern "C" int32_t fasa_stage_bytes(const fasa_ctx_t* ctx, size_t* out_bytes) {
+  if (!ctx || !out_bytes) return FASA_ERR_INVALID_ARG;
+  const fasa_config_t& c = ctx->cfg;
+  size_t qb = fasa_align_up((size_t)c.batch * c.n_q_heads * FASA_HEAD_DIM * 2, 256);
+  size_t kb = fasa_align_up((size_t)c.batch * c.n_kv_heads * FASA_HEAD_DIM * 2, 256);
+  *out_bytes = qb + 2 * kb;
+  return FASA_OK;
+}
+
+extern "C" int32_t fasa_decode_step_host(fasa_ctx_t* ctx, const void* q_host,
+                                         const void* k_new_host, const void* v_new_host,
+                                         void* dev_stage, void* k_cache, void* v_cache,
+                                         void* proxy_k, int32_t* seq_lens, int32_t budget,
+                                         int32_t n_sel_max, float* scores, int32_t* idx,
+                                         int32_t* n_sel, float* out, float* out_host,
+                                         void* workspace, void* stream) {
+  if (!ctx || !q_host || !k_new_host || !v_new_host || !dev_stage || !out_host || !out)
+    return FASA_ERR_INVALID_ARG;
+  const fasa_config_t& c = ctx->cfg;
+  cudaStream_t s = (cudaStream_t)stream;
+  size_t q_bytes = (size_t)c.batch * c.n_q_heads * FASA_HEAD_DIM * 2;
+  size_t kv_bytes = (size_t)c.batch * c.n_kv_heads * FASA_HEAD_DIM * 2;
+  char* dq = (char*)dev_stage;
+  char* dk = dq + fasa_align_up(q_bytes, 256);
+  char* dv = dk + fasa_align_up(kv_bytes, 256);
+  FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
+  FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
+  FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
+  int32_t st = fasa_kv_append(ctx, k_cache, v_cache, proxy_k, seq_lens, dk, dv, 1, stream);
+  if (st != FASA_OK) return st;
+  st = fasa_decode_step(ctx, dq, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
+                        idx, n_sel, out, nullptr, workspace, stream);
+  if (st != FASA_OK) return st;
+  size_t o_bytes = (size_t)c.batch * c.n_q_heads * FASA_HEAD_DIM * sizeof(float);
+  FASA_CUDA_TRY(ctx, cudaMemcpyAsync(out_host, out, o_bytes, cudaMemcpyDeviceToHost, s));
+  FASA_CUDA_TRY(ctx, cudaStreamSynchronize(s));
+  return FASA_OK;
+}

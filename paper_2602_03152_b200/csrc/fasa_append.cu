@@ -1,0 +1,132 @@
+// Cache update: K/V rows plus the packed dominant-FC proxy rows (Algorithm 2: Split,
+// UpdateCache), and the one-off proxy build from an existing key cache.
+#include "fasa_common.cuh"
+
+namespace {
+
+// 64 threads per appended row: 16 copy the K row, 16 the V row (16 bytes each),
+// up to 16 assemble the proxy row (8 gathered channels = 16 bytes each).
+__global__ void __launch_bounds__(256)
+kv_append_kernel(uint16_t* __restrict__ k_cache, uint16_t* __restrict__ v_cache,
+                 uint16_t* __restrict__ proxy, const int32_t* __restrict__ seq_lens,
+                 const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
+                 const int16_t* __restrict__ chan, int32_t* __restrict__ status, int n_rows,
+                 int n_new, int n_kv_heads, int max_len, int chunks, int64_t ksb, int64_t ksh,
+                 int64_t kst, int64_t vsb, int64_t vsh, int64_t vst) {
+  const int row = blockIdx.x * 4 + (threadIdx.x >> 6);
+  if (row >= n_rows) return;
+  const int t = threadIdx.x & 63;
+  const int n = row % n_new;
+  const int u = row / n_new;  // unit = b * n_kv_heads + h
+  const int h = u % n_kv_heads;
+  const int b = u / n_kv_heads;
+  const int len = clamp_len(seq_lens[b], max_len, status);
+  const int pos = len + n;
+  if (pos >= max_len) {
+    if (t == 0) atomicOr(status, FASA_DEV_APPEND_FULL);
+    return;
+  }
+  const uint16_t* ksrc = k_new + (int64_t)row * FASA_HEAD_DIM;
+  if (t < 16) {
+    uint4 x = *reinterpret_cast<const uint4*>(ksrc + t * 8);
+    *reinterpret_cast<uint4*>(k_cache + b * ksb + h * ksh + pos * kst + t * 8) = x;
+  } else if (t < 32) {
+    const int c = t - 16;
+    uint4 x = *reinterpret_cast<const uint4*>(v_new + (int64_t)row * FASA_HEAD_DIM + c * 8);
+    *reinterpret_cast<uint4*>(v_cache + b * vsb + h * vsh + pos * vst + c * 8) = x;
+  } else if (t - 32 < chunks) {
+    const int c = t - 32;
+    const int row_elems = chunks * 8;
+    const int16_t* ch = chan + h * row_elems + c * 8;
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      int c0 = ch[2 * e], c1 = ch[2 * e + 1];
+      uint32_t lo = c0 >= 0 ? ksrc[c0] : 0u;
+      uint32_t hi = c1 >= 0 ? ksrc[c1] : 0u;
+      w[e] = lo | (hi << 16);
+    }
+    uint16_t* dst = proxy + ((int64_t)u * max_len + pos) * row_elems + c * 8;
+    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+__global__ void seq_len_bump_kernel(int32_t* __restrict__ seq_lens, int batch, int n_new,
+                                    int max_len, int32_t* __restrict__ status) {
+  int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= batch) return;
+  int len = clamp_len(seq_lens[b], max_len, status);
+  len += n_new;
+  seq_lens[b] = len > max_len ? max_len : len;
+}
+
+// One thread per 16-byte proxy chunk of rows 0 .. seq_lens[b]-1.
+__global__ void __launch_bounds__(256)
+proxy_build_kernel(const uint16_t* __restrict__ k_cache, uint16_t* __restrict__ proxy,
+                   const int32_t* __restrict__ seq_lens, const int16_t* __restrict__ chan,
+                   int32_t* __restrict__ status, int n_kv_heads, int max_len, int chunks,
+                   int64_t ksb, int64_t ksh, int64_t kst) {
+  const int u = blockIdx.y;
+  const int h = u % n_kv_heads;
+  const int b = u / n_kv_heads;
+  const int len = clamp_len(seq_lens[b], max_len, status);
+  const int64_t item = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int j = (int)(item / chunks);
+  const int c = (int)(item % chunks);
+  if (j >= len) return;
+  const int row_elems = chunks * 8;
+  const int16_t* ch = chan + h * row_elems + c * 8;
+  const uint16_t* ksrc = k_cache + b * ksb + h * ksh + (int64_t)j * kst;
+  uint32_t w[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    int c0 = ch[2 * e], c1 = ch[2 * e + 1];
+    uint32_t lo = c0 >= 0 ? ksrc[c0] : 0u;
+    uint32_t hi = c1 >= 0 ? ksrc[c1] : 0u;
+    w[e] = lo | (hi << 16);
+  }
+  uint16_t* dst = proxy + ((int64_t)u * max_len + j) * row_elems + c * 8;
+  *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+}  // namespace
+
+extern "C" int32_t fasa_kv_append(fasa_ctx_t* ctx, void* k_cache, void* v_cache, void* proxy_k,
+                                  int32_t* seq_lens, const void* k_new, const void* v_new,
+                                  int32_t n_new, void* stream) {
+  if (!ctx || !k_cache || !v_cache || !proxy_k || !seq_lens || !k_new || !v_new || n_new <= 0)
+    return FASA_ERR_INVALID_ARG;
+  if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(proxy_k) || !aligned16(k_new) ||
+      !aligned16(v_new))
+    return FASA_ERR_INVALID_ARG;
+  const fasa_config_t& c = ctx->cfg;
+  long long n_rows = (long long)c.batch * c.n_kv_heads * n_new;
+  if (n_rows > (1ll << 30)) return FASA_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  kv_append_kernel<<<(unsigned)((n_rows + 3) / 4), 256, 0, s>>>(
+      (uint16_t*)k_cache, (uint16_t*)v_cache, (uint16_t*)proxy_k, seq_lens, (const uint16_t*)k_new,
+      (const uint16_t*)v_new, ctx->d_chan, ctx->d_status, (int)n_rows, n_new, c.n_kv_heads,
+      c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h, c.k_stride_t, c.v_stride_b,
+      c.v_stride_h, c.v_stride_t);
+  FASA_LAUNCH_CHECK(ctx);
+  seq_len_bump_kernel<<<(c.batch + 127) / 128, 128, 0, s>>>(seq_lens, c.batch, n_new, c.max_len,
+                                                            ctx->d_status);
+  FASA_LAUNCH_CHECK(ctx);
+  return FASA_OK;
+}
+
+extern "C" int32_t fasa_proxy_build(fasa_ctx_t* ctx, const void* k_cache, void* proxy_k,
+                                    const int32_t* seq_lens, void* stream) {
+  if (!ctx || !k_cache || !proxy_k || !seq_lens) return FASA_ERR_INVALID_ARG;
+  if (!aligned16(k_cache) || !aligned16(proxy_k)) return FASA_ERR_INVALID_ARG;
+  const fasa_config_t& c = ctx->cfg;
+  long long items = (long long)c.max_len * ctx->chunks;
+  dim3 grid((unsigned)((items + 255) / 256), (unsigned)(c.batch * c.n_kv_heads));
+  proxy_build_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(
+      (const uint16_t*)k_cache, (uint16_t*)proxy_k, seq_lens, ctx->d_chan, ctx->d_status,
+      c.n_kv_heads, c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h, c.k_stride_t);
+  FASA_LAUNCH_CHECK(ctx);
+  return FASA_OK;
+}

@@ -1,0 +1,342 @@
+// FAC (Sec. 4.2, Eq. 6-7) and the dense FKV path (Sec. 5.1): split-K flash decoding with an
+// online softmax, rows gathered by index for the sparse form, followed by a merge pass.
+//
+// Mapping.  A KV row (128 bf16 = 256 bytes) is read by a half-warp, 16 bytes per lane, so a
+// lane owns 8 channels of every row it sees and keeps, for up to 4 query heads of the GQA
+// group, its slice of q and of the output accumulator in registers.  One K/V row therefore
+// serves the whole group from a single load.  Groups of 5-8 heads use both half-warps of a
+// warp on the same row (the second load is merged by the coalescer).  Logits of a batch of
+// 8 rows are completed with a transposing xor-shuffle reduction (8 shuffles per head per
+// batch); probabilities travel back to all lanes through shared memory.  All multiply-adds
+// are packed two-wide fp32 FMAs.  No tensor cores: one query token per sequence.
+#include "fasa_common.cuh"
+
+namespace {
+
+constexpr int kAttnThreads = 128;
+constexpr int kAttnHalfWarps = kAttnThreads / 16;  // 8
+constexpr int kRB = 8;                              // rows per half-warp batch
+constexpr int kPartialStride = FASA_HEAD_DIM + 2;   // m, l, acc[128] (base-2 domain)
+
+struct AttnParams {
+  const uint16_t* q;
+  const uint16_t* k;
+  const uint16_t* v;
+  const int32_t* idx;      // sparse: [units][n_sel_max]
+  const int32_t* n_rows;   // sparse: n_sel [units]; dense: seq_lens [batch]
+  float* partial;          // [batch][n_q_heads][n_splits][kPartialStride]
+  int32_t* status;
+  int n_q_heads, n_kv_heads, group, max_len, n_sel_max, n_cap, chunk, n_splits;
+  int64_t ksb, ksh, kst, vsb, vsh, vst;
+  float scale_log2;        // softmax_scale * log2(e)
+};
+
+// GP: heads per half-warp (1..4).  HWS: half-warps sharing a row (1: group <= 4, 2: group <= 8).
+template <int GP, int HWS, bool SPARSE>
+__global__ void __launch_bounds__(kAttnThreads)
+decode_attn_kernel(const AttnParams p) {
+  const int u = blockIdx.y;
+  const int h = u % p.n_kv_heads;
+  const int b = u / p.n_kv_heads;
+  int n;
+  if (SPARSE) {
+    n = p.n_rows[u];
+    if (n < 0 || n > p.n_cap) {
+      atomicOr(p.status, FASA_DEV_NSEL_CLAMPED);
+      n = n < 0 ? 0 : p.n_cap;
+    }
+  } else {
+    n = clamp_len(p.n_rows[b], p.max_len, p.status);
+  }
+  const int split = blockIdx.x;
+  const int r0 = split * p.chunk;
+  if (r0 >= n) return;
+  const int r1 = min(n, r0 + p.chunk);
+
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int l16 = lane & 15;
+  const int hw = lane >> 4;
+  const int hwid = warp * 2 + hw;                          // half-warp within the CTA
+  constexpr int kSlots = kAttnHalfWarps / HWS;             // row-batch streams per CTA
+  constexpr int kWarpRows = kRB * (2 / HWS);               // rows one warp covers per iteration
+  const int g0 = HWS == 1 ? 0 : hw * GP;                   // first head (within the group) of this half-warp
+
+  __shared__ __align__(16) float s_p[kAttnHalfWarps][kRB][4];
+  __shared__ __align__(16) float s_acc[kAttnHalfWarps][GP][FASA_HEAD_DIM];
+  __shared__ float s_m[kAttnHalfWarps][GP];
+  __shared__ float s_l[kAttnHalfWarps][GP];
+
+  // q slice of this lane, pre-multiplied by scale * log2(e): logits live in the base-2 domain.
+  float2 qf[GP][4];
+#pragma unroll
+  for (int g = 0; g < GP; ++g) {
+    const bool head_ok = g0 + g < p.group;
+    const uint16_t* qp =
+        p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group + (head_ok ? g0 + g : 0)) * FASA_HEAD_DIM + l16 * 8;
+    uint4 w = *reinterpret_cast<const uint4*>(qp);
+    const float sc = head_ok ? p.scale_log2 : 0.f;
+    float2 t;
+    t = bf16x2_to_f32x2(w.x); qf[g][0] = make_float2(t.x * sc, t.y * sc);
+    t = bf16x2_to_f32x2(w.y); qf[g][1] = make_float2(t.x * sc, t.y * sc);
+    t = bf16x2_to_f32x2(w.z); qf[g][2] = make_float2(t.x * sc, t.y * sc);
+    t = bf16x2_to_f32x2(w.w); qf[g][3] = make_float2(t.x * sc, t.y * sc);
+  }
+
+  float2 acc[GP][4];
+  float m[GP], lsum[GP];
+#pragma unroll
+  for (int g = 0; g < GP; ++g) {
+    m[g] = -INFINITY;
+    lsum[g] = 0.f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc[g][e] = make_float2(0.f, 0.f);
+  }
+
+  const uint16_t* kbase = p.k + b * p.ksb + h * p.ksh + l16 * 8;
+  const uint16_t* vbase = p.v + b * p.vsb + h * p.vsh + l16 * 8;
+  const int32_t* irow = SPARSE ? p.idx + (int64_t)u * p.n_sel_max : nullptr;
+  // The row of the batch whose finished logit lands in this lane after the reduction.
+  const int my_row = ((l16 >> 3) & 1) * 4 + ((l16 >> 2) & 1) * 2 + ((l16 >> 1) & 1);
+
+  // The trip count is the same for both half-warps of a warp (the shuffles below name all
+  // 32 lanes); a half-warp whose batch starts past r1 runs it fully masked.
+  for (int wbase = r0 + warp * kWarpRows; wbase < r1; wbase += (kAttnThreads / 32) * kWarpRows) {
+    const int base = wbase + (HWS == 1 ? hw * kRB : 0);
+    uint4 kk[kRB], vv[kRB];
+#pragma unroll
+    for (int i = 0; i < kRB; ++i) {
+      const int r = base + i;
+      int tok = 0;
+      if (r < r1) {
+        if (SPARSE) {
+          tok = __ldg(irow + r);
+          if (tok < 0 || tok >= p.max_len) {
+            atomicOr(p.status, FASA_DEV_IDX_CLAMPED);
+            tok = 0;
+          }
+        } else {
+          tok = r;
+        }
+        kk[i] = ld_stream_u4(kbase + (int64_t)tok * p.kst);
+        vv[i] = ld_stream_u4(vbase + (int64_t)tok * p.vst);
+      } else {
+        kk[i] = make_uint4(0u, 0u, 0u, 0u);
+        vv[i] = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+
+    float alpha[GP];
+#pragma unroll
+    for (int g = 0; g < GP; ++g) {
+      // partial logits of the 8 rows over this lane's 8 channels
+      float part[kRB];
+#pragma unroll
+      for (int i = 0; i < kRB; ++i) part[i] = dot8(qf[g], kk[i]);
+      // transposing reduction over the 16 lanes: 8 -> 4 -> 2 -> 1 rows per lane
+      float p4[4], p2[2], p1;
+      {
+        const bool up = (l16 & 8) != 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float send = up ? part[i] : part[i + 4];
+          const float keep = up ? part[i + 4] : part[i];
+          p4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+        }
+      }
+      {
+        const bool up = (l16 & 4) != 0;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const float send = up ? p4[i] : p4[i + 2];
+          const float keep = up ? p4[i + 2] : p4[i];
+          p2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+        }
+      }
+      {
+        const bool up = (l16 & 2) != 0;
+        const float send = up ? p2[0] : p2[1];
+        const float keep = up ? p2[1] : p2[0];
+        p1 = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+      }
+      p1 += __shfl_xor_sync(0xffffffffu, p1, 1);
+      const float logit = (base + my_row < r1) ? p1 : -INFINITY;
+      float bmax = logit;
+      bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 8));
+      bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 4));
+      bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
+      const float m_new = fmaxf(m[g], bmax);
+      // m_new is finite here: the batch holds at least one real row with finite inputs.
+      const float m_safe = m_new == -INFINITY ? 0.f : m_new;
+      alpha[g] = exp2f(m[g] - m_safe);
+      const float pr = exp2f(logit - m_safe);
+      lsum[g] = lsum[g] * alpha[g] + ((l16 & 1) ? 0.f : pr);
+      m[g] = m_new;
+      if ((l16 & 1) == 0) s_p[hwid][my_row][g] = pr;
+    }
+    __syncwarp();
+
+#pragma unroll
+    for (int g = 0; g < GP; ++g) {
+      const float2 a2 = make_float2(alpha[g], alpha[g]);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[g][e] = __ffma2_rn(acc[g][e], a2, make_float2(0.f, 0.f));
+    }
+#pragma unroll
+    for (int i = 0; i < kRB; ++i) {
+      const float4 pi = *reinterpret_cast<const float4*>(&s_p[hwid][i][0]);
+      const float pg[4] = {pi.x, pi.y, pi.z, pi.w};
+      float2 vf[4];
+      vf[0] = bf16x2_to_f32x2(vv[i].x);
+      vf[1] = bf16x2_to_f32x2(vv[i].y);
+      vf[2] = bf16x2_to_f32x2(vv[i].z);
+      vf[3] = bf16x2_to_f32x2(vv[i].w);
+#pragma unroll
+      for (int g = 0; g < GP; ++g) {
+        const float2 p2 = make_float2(pg[g], pg[g]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[g][e] = __ffma2_rn(p2, vf[e], acc[g][e]);
+      }
+    }
+    __syncwarp();  // s_p is rewritten by the next batch
+  }
+
+  // ---- combine the half-warps of this CTA, then write one partial per head -----------
+#pragma unroll
+  for (int g = 0; g < GP; ++g) {
+    float l = lsum[g];
+    l += __shfl_xor_sync(0xffffffffu, l, 8);
+    l += __shfl_xor_sync(0xffffffffu, l, 4);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    if (l16 == 0) {
+      s_m[hwid][g] = m[g];
+      s_l[hwid][g] = l;
+    }
+    float4* dst = reinterpret_cast<float4*>(&s_acc[hwid][g][l16 * 8]);
+    dst[0] = make_float4(acc[g][0].x, acc[g][0].y, acc[g][1].x, acc[g][1].y);
+    dst[1] = make_float4(acc[g][2].x, acc[g][2].y, acc[g][3].x, acc[g][3].y);
+  }
+  __syncthreads();
+
+  const int c = threadIdx.x;  // one channel per thread
+  for (int gl = 0; gl < p.group; ++gl) {
+    const int gi = HWS == 1 ? gl : gl % GP;      // index inside the half-warp
+    const int hsel = HWS == 1 ? 0 : gl / GP;     // which half of each warp holds it
+    float mx = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < kSlots; ++s) {
+      const int hwi = HWS == 1 ? s : s * 2 + hsel;
+      mx = fmaxf(mx, s_m[hwi][gi]);
+    }
+    float a = 0.f, l = 0.f;
+#pragma unroll
+    for (int s = 0; s < kSlots; ++s) {
+      const int hwi = HWS == 1 ? s : s * 2 + hsel;
+      const float ms = s_m[hwi][gi];
+      const float w = ms == -INFINITY ? 0.f : exp2f(ms - mx);
+      a += w * s_acc[hwi][gi][c];
+      l += w * s_l[hwi][gi];
+    }
+    float* dst = p.partial +
+                 (((int64_t)b * p.n_q_heads + (int64_t)h * p.group + gl) * p.n_splits + split) * kPartialStride;
+    dst[2 + c] = a;
+    if (c == 0) {
+      dst[0] = mx;
+      dst[1] = l;
+    }
+  }
+}
+
+// Merge pass: one CTA per (batch, query head), one channel per thread.
+template <bool SPARSE>
+__global__ void __launch_bounds__(FASA_HEAD_DIM)
+decode_attn_merge_kernel(const float* __restrict__ partial, const int32_t* __restrict__ n_rows,
+                         float* __restrict__ out, float* __restrict__ lse,
+                         int32_t* __restrict__ status, int n_q_heads, int n_kv_heads, int group,
+                         int max_len, int n_cap, int chunk, int n_splits) {
+  const int bh = blockIdx.x;
+  const int b = bh / n_q_heads;
+  const int hq = bh % n_q_heads;
+  int n;
+  if (SPARSE) {
+    n = n_rows[b * n_kv_heads + hq / group];
+    n = n < 0 ? 0 : (n > n_cap ? n_cap : n);
+  } else {
+    n = n_rows[b];
+    n = n < 0 ? 0 : (n > max_len ? max_len : n);
+  }
+  const int ns = min(n_splits, (n + chunk - 1) / chunk);
+  const int c = threadIdx.x;
+  const float* src = partial + (int64_t)bh * n_splits * kPartialStride;
+  float mx = -INFINITY;
+  for (int s = 0; s < ns; ++s) mx = fmaxf(mx, src[s * kPartialStride]);
+  float a = 0.f, l = 0.f;
+  for (int s = 0; s < ns; ++s) {
+    const float ms = src[s * kPartialStride];
+    const float w = ms == -INFINITY ? 0.f : exp2f(ms - mx);
+    a += w * src[s * kPartialStride + 2 + c];
+    l += w * src[s * kPartialStride + 1];
+  }
+  out[(int64_t)bh * FASA_HEAD_DIM + c] = (ns > 0 && l > 0.f) ? a / l : 0.f;
+  if (lse && c == 0)
+    lse[bh] = (ns > 0 && l > 0.f) ? (mx + log2f(l)) * 0.6931471805599453f : -INFINITY;
+}
+
+template <bool SPARSE>
+int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
+                    const int32_t* idx, const int32_t* n_rows, int n_upper, int n_sel_max,
+                    float* out, float* lse, void* workspace, cudaStream_t s) {
+  const fasa_config_t& c = ctx->cfg;
+  const fasa_split_plan plan = fasa_plan_splits(ctx, n_upper);
+  AttnParams p;
+  p.q = (const uint16_t*)q; p.k = (const uint16_t*)k; p.v = (const uint16_t*)v;
+  p.idx = idx; p.n_rows = n_rows; p.partial = (float*)workspace; p.status = ctx->d_status;
+  p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group;
+  p.max_len = c.max_len; p.n_sel_max = n_sel_max; p.n_cap = n_upper; p.chunk = plan.chunk; p.n_splits = plan.n_splits;
+  p.ksb = c.k_stride_b; p.ksh = c.k_stride_h; p.kst = c.k_stride_t;
+  p.vsb = c.v_stride_b; p.vsh = c.v_stride_h; p.vst = c.v_stride_t;
+  p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
+  dim3 grid((unsigned)plan.n_splits, (unsigned)(c.batch * c.n_kv_heads));
+  const int G = ctx->group;
+  if (G == 1) decode_attn_kernel<1, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
+  else if (G == 2) decode_attn_kernel<2, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
+  else if (G == 3) decode_attn_kernel<3, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
+  else if (G == 4) decode_attn_kernel<4, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
+  else if (G <= 6) decode_attn_kernel<3, 2, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
+  else decode_attn_kernel<4, 2, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
+  FASA_LAUNCH_CHECK(ctx);
+  decode_attn_merge_kernel<SPARSE><<<c.batch * c.n_q_heads, FASA_HEAD_DIM, 0, s>>>(
+      (const float*)workspace, n_rows, out, lse, ctx->d_status, c.n_q_heads, c.n_kv_heads,
+      ctx->group, c.max_len, n_upper, plan.chunk, plan.n_splits);
+  FASA_LAUNCH_CHECK(ctx);
+  return FASA_OK;
+}
+
+bool aligned(const void* p, uintptr_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
+
+}  // namespace
+
+extern "C" int32_t fasa_sparse_decode_attn(fasa_ctx_t* ctx, const void* q, const void* k_cache,
+                                           const void* v_cache, const int32_t* idx,
+                                           const int32_t* n_sel, int32_t n_sel_max, float* out,
+                                           float* lse, void* workspace, void* stream) {
+  if (!ctx || !q || !k_cache || !v_cache || !idx || !n_sel || !out || !workspace || n_sel_max <= 0)
+    return FASA_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(workspace, 256))
+    return FASA_ERR_INVALID_ARG;
+  const int n_upper = n_sel_max < ctx->cfg.max_len ? n_sel_max : ctx->cfg.max_len;
+  return launch_attn<true>(ctx, q, k_cache, v_cache, idx, n_sel, n_upper, n_sel_max, out, lse,
+                           workspace, (cudaStream_t)stream);
+}
+
+extern "C" int32_t fasa_full_decode_attn(fasa_ctx_t* ctx, const void* q, const void* k_cache,
+                                         const void* v_cache, const int32_t* seq_lens, float* out,
+                                         float* lse, void* workspace, void* stream) {
+  if (!ctx || !q || !k_cache || !v_cache || !seq_lens || !out || !workspace)
+    return FASA_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(workspace, 256))
+    return FASA_ERR_INVALID_ARG;
+  return launch_attn<false>(ctx, q, k_cache, v_cache, nullptr, seq_lens, ctx->cfg.max_len, 0, out,
+                            lse, workspace, (cudaStream_t)stream);
+}

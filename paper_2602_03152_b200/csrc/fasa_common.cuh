@@ -1,0 +1,93 @@
+// Shared declarations of the FASA CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "fasa.h"
+
+#define FASA_HEAD_DIM 128
+#define FASA_MAX_GROUP 8
+#define FASA_MAX_DOM 64
+
+// Context: the normalised configuration plus a small device table.
+struct fasa_ctx {
+  fasa_config_t cfg;      // strides and softmax_scale filled in
+  int group;              // query heads per KV head
+  int chunks;             // 16-byte chunks per proxy row = ceil(n_dom / 4)
+  int row_elems;          // bf16 elements per proxy row = 8 * chunks
+  int device;
+  int n_sm;
+  int16_t* d_chan;        // device [n_kv_heads][row_elems]: K channel of each proxy element, -1 = padding
+  int32_t* d_status;      // device status word (FASA_DEV_* bits)
+  long long launches;     // kernels launched through this context
+  char cuda_err[256];
+};
+
+// Records a CUDA failure in the context and returns FASA_ERR_CUDA from the caller.
+#define FASA_CUDA_TRY(ctx, expr)                                                       \
+  do {                                                                                 \
+    cudaError_t e_ = (expr);                                                           \
+    if (e_ != cudaSuccess) {                                                           \
+      snprintf((ctx)->cuda_err, sizeof((ctx)->cuda_err), "%s: %s", #expr,              \
+               cudaGetErrorString(e_));                                                \
+      return FASA_ERR_CUDA;                                                            \
+    }                                                                                  \
+  } while (0)
+
+#define FASA_LAUNCH_CHECK(ctx)                                                         \
+  do {                                                                                 \
+    (ctx)->launches += 1;                                                              \
+    FASA_CUDA_TRY(ctx, cudaGetLastError());                                            \
+  } while (0)
+
+// How the attention kernels cut a list of at most n_upper rows into splits.
+struct fasa_split_plan {
+  int n_splits;   // grid.x
+  int chunk;      // rows per split (multiple of 32)
+};
+fasa_split_plan fasa_plan_splits(const fasa_ctx* ctx, int n_upper);
+
+static inline size_t fasa_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+#ifdef __CUDACC__
+
+// Two bf16 packed in a 32-bit word -> two fp32 (exact).
+__device__ __forceinline__ float2 bf16x2_to_f32x2(uint32_t w) {
+  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint16_t b) {
+  return __uint_as_float(((uint32_t)b) << 16);
+}
+
+// 128-bit read-only load that does not allocate in L1 (streamed once).
+__device__ __forceinline__ uint4 ld_stream_u4(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+
+// Dot product of 8 fp32 (as 4 float2) with 8 bf16 (one uint4), packed FMAs.
+__device__ __forceinline__ float dot8(const float2 (&q)[4], const uint4& k) {
+  float2 a = make_float2(0.f, 0.f);
+  a = __ffma2_rn(q[0], bf16x2_to_f32x2(k.x), a);
+  a = __ffma2_rn(q[1], bf16x2_to_f32x2(k.y), a);
+  a = __ffma2_rn(q[2], bf16x2_to_f32x2(k.z), a);
+  a = __ffma2_rn(q[3], bf16x2_to_f32x2(k.w), a);
+  return a.x + a.y;
+}
+
+__device__ __forceinline__ int clamp_len(int len, int max_len, int32_t* status) {
+  if (len < 0 || len > max_len) {
+    atomicOr(status, FASA_DEV_LEN_CLAMPED);
+    len = len < 0 ? 0 : max_len;
+  }
+  return len;
+}
+
+#endif  // __CUDACC__

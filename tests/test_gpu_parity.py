@@ -1,0 +1,384 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 CPU oracle, element by
+element on the same seeded bf16 inputs.  Index sets are bit-exact outside a 1e-3-relative
+tie band; attention is within max-abs 2e-3; scores within 1e-5 of sum |q_c k_c|."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import fasa_oracle as O
+from oracle import parity
+from paper_2602_03152_b200 import binding, synth
+
+from gpu_harness import SENTINEL, Run
+
+pytestmark = pytest.mark.gpu
+
+C = synth.CONFIGS
+
+
+def _full_check(r: Run, budget=None, dense=True):
+    r.build_proxy()
+    r.step(budget)
+    if dense:
+        r.dense_step()
+    h = r.host()
+    rep = parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
+                            n_sel=h["n_sel"], out=h["out"], dense_out=h["dense"] if dense else None,
+                            what=r.w.name, **r.oracle_kwargs(budget))
+    # rows at and past the sequence length are never written
+    for b in range(r.w.batch):
+        L = int(h["seq_lens"][b])
+        assert np.all(h["scores"][b, :, L:] == SENTINEL)
+        for hh in range(r.w.n_kv_heads):
+            assert np.all(h["idx"][b, hh, int(h["n_sel"][b, hh]):] == -7)
+    assert r.fasa.device_status() == 0
+    return rep, h
+
+
+def test_config0_full_size():
+    rep, h = _full_check(Run(C["c0"]))
+    assert rep["units"] == 1 and int(h["n_sel"][0, 0]) == 256
+
+
+def test_config1_shape_scaled_ragged_tail():
+    w = C["c1"].replace(max_len=3001, len_lo=2999, len_hi=2999)
+    rep, h = _full_check(Run(w))
+    assert rep["units"] == 8 and np.all(h["n_sel"] == 256 + 68)
+
+
+def test_config2_shape_scaled_ragged_batch():
+    w = C["c2"].replace(batch=3, max_len=2100, len_lo=500, len_hi=2100, budget=100)
+    rep, _ = _full_check(Run(w))
+    assert rep["units"] == 24
+
+
+def test_config3_shape_group_of_7_permille_budget():
+    w = C["c3"].replace(batch=2, max_len=1500, len_lo=900, len_hi=1400)
+    r = Run(w)
+    rep, h = _full_check(r)
+    for b in range(2):
+        assert np.all(h["n_sel"][b] == math.ceil(189 * int(h["seq_lens"][b]) / 1000))
+
+
+@pytest.mark.parametrize("F", [1, 3, 4, 5, 8, 13, 32, 64])
+def test_dominant_fc_counts(F):
+    w = C["c4"].replace(batch=1, max_len=777, len_lo=700, len_hi=700, n_dom=F, budget=64)
+    _full_check(Run(w), dense=False)
+
+
+def test_all_fcs_equal_dense_topk_on_gpu():
+    # F = 64: the GPU selection must be the top-k of the full logits (the "Oracle" baseline).
+    w = C["c4"].replace(batch=1, max_len=2048, len_lo=2048, len_hi=2048, n_dom=64, budget=128)
+    r = Run(w)
+    _, h = _full_check(r, dense=False)
+    G = w.group
+    for hh in range(w.n_kv_heads):
+        full = (h["k"][0, hh] @ h["q"][0, hh * G:(hh + 1) * G].T).sum(1)
+        ref = np.sort(np.argsort(-full, kind="stable")[:128])
+        got = h["idx"][0, hh, :128]
+        if not np.array_equal(got, ref):
+            parity.check_selection(got, full, 2048, 128, 0, 0, "F=64")
+
+
+@pytest.mark.parametrize("G,Hkv", [(1, 2), (2, 2), (3, 1), (4, 2), (5, 1), (6, 1), (7, 2), (8, 1)])
+def test_group_sizes(G, Hkv):
+    w = C["c1"].replace(n_q_heads=G * Hkv, n_kv_heads=Hkv, max_len=900, len_lo=850, len_hi=850, budget=77)
+    _full_check(Run(w))
+
+
+def test_interleaved_pairing_and_max_reduce():
+    w = C["c1"].replace(max_len=1000, len_lo=1000, len_hi=1000, pairing=1, budget=50)
+    _full_check(Run(w), dense=False)
+    w = C["c1"].replace(max_len=1000, len_lo=1000, len_hi=1000, group_reduce=1, budget=50)
+    _full_check(Run(w), dense=False)
+    w = C["c3"].replace(batch=1, max_len=600, len_lo=600, len_hi=600, group_reduce=1, budget=50)
+    _full_check(Run(w), dense=False)
+
+
+@pytest.mark.parametrize("L,budget,sink,recent", [
+    (1, 256, 0, 0), (1, 256, 4, 64), (2, 1, 0, 0), (100, 256, 0, 0), (256, 256, 0, 0), (257, 256, 0, 0),
+    (50, 8, 30, 30), (300, 10, 4, 64), (68, 256, 4, 64), (69, 1, 4, 64), (1000, 1, 0, 0), (1000, 999, 0, 0),
+])
+def test_length_and_budget_edges(L, budget, sink, recent):
+    w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, max_len=1024, len_lo=L, len_hi=L, budget=budget,
+                        n_sink=sink, n_recent=recent)
+    _, h = _full_check(Run(w, n_sel_max=1024))
+    assert np.all(h["n_sel"] == min(L, budget + min(L, sink) + min(recent, L - min(L, sink))))
+
+
+def test_budget_covering_context_equals_dense():
+    w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, max_len=1500, len_lo=1234, len_hi=1234, budget=1500)
+    r = Run(w, n_sel_max=1500)
+    _, h = _full_check(r)
+    assert np.all(h["n_sel"] == 1234)
+    assert np.array_equal(h["idx"][0, 0, :1234], np.arange(1234))
+    assert np.abs(h["out"] - h["dense"]).max() <= 2e-5
+    assert np.abs(h["lse"] - h["dense_lse"]).max() <= 1e-4
+
+
+def test_empty_sequence_gives_zero_output():
+    w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, batch=2, max_len=256, len_lo=256, len_hi=256, budget=16)
+    t = synth.make_inputs(w, "cpu")
+    t["seq_lens"] = torch.tensor([0, 200], dtype=torch.int32)
+    r = Run(w, t)
+    _, h = _full_check(r)
+    assert np.all(h["n_sel"][0] == 0) and np.all(h["out"][0] == 0) and np.all(h["dense"][0] == 0)
+    assert np.all(np.isneginf(h["lse"][0])) and np.all(np.isneginf(h["dense_lse"][0]))
+
+
+def test_zero_query_ties_resolve_to_lowest_indices():
+    w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, max_len=500, len_lo=500, len_hi=500, budget=20, n_sink=0,
+                        n_recent=0)
+    t = synth.make_inputs(w, "cpu")
+    t["q"] = torch.zeros_like(t["q"])
+    r = Run(w, t)
+    _, h = _full_check(r)
+    assert np.array_equal(h["idx"][0, 0, :20], np.arange(20))
+    # q = 0: attention is the plain mean of the selected value rows
+    assert np.abs(h["out"][0, 0] - h["v"][0, 0, :20].mean(0)).max() <= 2e-3
+
+
+def test_lse_matches_oracle():
+    w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, max_len=700, len_lo=700, len_hi=700, budget=90)
+    r = Run(w)
+    _, h = _full_check(r)
+    G = w.group
+    for hh in range(2):
+        n = int(h["n_sel"][0, hh])
+        _, lse = O.attn_subset(h["q"][0, hh * G:(hh + 1) * G], h["k"][0, hh], h["v"][0, hh], h["idx"][0, hh, :n],
+                               1 / math.sqrt(128))
+        assert np.abs(h["lse"][0, hh * G:(hh + 1) * G] - lse).max() <= 1e-3
+        _, dlse = O.attn_dense(h["q"][0, hh * G:(hh + 1) * G], h["k"][0, hh], h["v"][0, hh], 700, 1 / math.sqrt(128))
+        assert np.abs(h["dense_lse"][0, hh * G:(hh + 1) * G] - dlse).max() <= 1e-3
+
+
+def test_results_are_deterministic():
+    w = C["c2"].replace(batch=2, max_len=5000, len_lo=3000, len_hi=5000, budget=300)
+    r = Run(w)
+    r.build_proxy()
+    r.step(); r.dense_step()
+    a = [x.clone() for x in (r.scores, r.idx, r.n_sel, r.out, r.dense)]
+    r.step(); r.dense_step()
+    for x, y in zip(a, (r.scores, r.idx, r.n_sel, r.out, r.dense)):
+        assert torch.equal(x, y)
+
+
+def test_decode_step_equals_separate_calls_and_host_variant():
+    w = C["c1"].replace(max_len=2000, len_lo=1500, len_hi=1500, budget=128)
+    r = Run(w)
+    r.build_proxy()
+    r.step()
+    ref = [x.clone() for x in (r.scores, r.idx, r.n_sel, r.out)]
+    for x in (r.scores, r.out):
+        x.fill_(SENTINEL)
+    r.fasa.decode_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel, r.out, r.ws)
+    torch.cuda.synchronize()
+    for x, y in zip(ref, (r.scores, r.idx, r.n_sel, r.out)):
+        assert torch.equal(x, y)
+    # host variant: append one token, then the same step; compare with the oracle on the grown cache
+    s = synth.make_step_inputs(w, 0, "cpu")
+    stage = torch.empty(r.fasa.stage_bytes(), dtype=torch.uint8, device="cuda")
+    out_host = torch.empty((w.batch, w.n_q_heads, 128), dtype=torch.float32).pin_memory()
+    r.fasa.decode_step_host(s["q"].pin_memory(), s["k_new"].pin_memory(), s["v_new"].pin_memory(), stage, r.k, r.v,
+                            r.proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel, r.out, out_host, r.ws)
+    assert r.seq_lens.cpu().tolist() == [1501]
+    kc, vc = r.k.cpu(), r.v.cpu()
+    assert torch.equal(kc[:, :, 1500], s["k_new"][:, :, 0]) and torch.equal(vc[:, :, 1500], s["v_new"][:, :, 0])
+    rep = parity.check_step(s["q"].double().numpy(), kc.double().numpy(), vc.double().numpy(), [1501],
+                            np.sort(r.dom.numpy(), axis=1), scores=r.scores.cpu().numpy(), idx=r.idx.cpu().numpy(),
+                            n_sel=r.n_sel.cpu().numpy(), out=out_host.numpy(), what="host step", **r.oracle_kwargs())
+    assert rep["units"] == 8
+    assert torch.equal(out_host, r.out.cpu())
+
+
+def test_strided_token_major_cache():
+    # K/V stored [B][L][Hkv][128] (token-major), addressed through the stride fields.
+    w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, batch=2, max_len=640, len_lo=400, len_hi=640, budget=40)
+    t = synth.make_inputs(w, "cpu")
+    r = Run(w, t)
+    kt = r.k.permute(0, 2, 1, 3).contiguous()   # [B][L][H][d]
+    vt = r.v.permute(0, 2, 1, 3).contiguous()
+    st = (640 * 2 * 128, 128, 2 * 128)          # stride_b, stride_h, stride_t in elements
+    f = binding.Fasa(w.batch, w.n_q_heads, w.n_kv_heads, w.max_len, r.dom, n_sink=w.n_sink, n_recent=w.n_recent,
+                     k_strides=st, v_strides=st)
+    proxy = f.alloc_proxy()
+    f.proxy_build(kt, proxy, r.seq_lens)
+    r.build_proxy()
+    assert torch.equal(proxy, r.proxy)
+    f.decode_step(r.q, kt, vt, proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel, r.out, r.ws)
+    f.full_decode_attn(r.q, kt, vt, r.seq_lens, r.dense, r.ws)
+    torch.cuda.synchronize()
+    h = r.host()
+    parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
+                      n_sel=h["n_sel"], out=h["out"], dense_out=h["dense"], what="strided", **r.oracle_kwargs())
+
+
+# ------------------------------------------------------------------ cache update ----
+
+def _expected_proxy(k_bits_cpu, dom_sorted, pairing, row_elems, lens):
+    """Proxy layout by plain indexing: pairs (K[c0], K[c1]) of the sorted dominant FCs, zero padded."""
+    B, H, Lm, _ = k_bits_cpu.shape
+    out = torch.zeros((B, H, Lm, row_elems), dtype=torch.int16)
+    for h in range(H):
+        for r, i in enumerate(dom_sorted[h].tolist()):
+            c0, c1 = (i, i + 64) if pairing == 0 else (2 * i, 2 * i + 1)
+            out[:, h, :, 2 * r] = k_bits_cpu[:, h, :, c0]
+            out[:, h, :, 2 * r + 1] = k_bits_cpu[:, h, :, c1]
+    for b in range(B):
+        out[b, :, int(lens[b]):] = 0
+    return out
+
+
+@pytest.mark.parametrize("F,pairing", [(16, 0), (5, 0), (16, 1), (64, 0), (1, 1)])
+def test_proxy_build_layout_is_bit_exact(F, pairing):
+    w = C["c2"].replace(batch=2, max_len=300, len_lo=100, len_hi=300, n_dom=F, pairing=pairing)
+    r = Run(w)
+    r.build_proxy()
+    torch.cuda.synchronize()
+    exp = _expected_proxy(r.t["k"].view(torch.int16), torch.sort(r.dom, dim=1).values, pairing, r.fasa.row_elems,
+                          r.t["seq_lens"])
+    assert torch.equal(r.proxy.cpu().view(torch.int16), exp)
+
+
+def test_kv_append_bulk_then_stepwise():
+    w = C["c3"].replace(batch=3, max_len=200, len_lo=0, len_hi=0)
+    t = synth.make_inputs(w, "cpu")
+    r = Run(w, t)
+    src_k, src_v = r.k.clone(), r.v.clone()
+    r.k.zero_(); r.v.zero_()
+    lens = torch.zeros(3, dtype=torch.int32, device="cuda")
+    # bulk prefill of 150 rows, then 20 single-token appends
+    r.fasa.kv_append(r.k, r.v, r.proxy, lens, src_k[:, :, :150].contiguous(), src_v[:, :, :150].contiguous())
+    for s in range(150, 170):
+        r.fasa.kv_append(r.k, r.v, r.proxy, lens, src_k[:, :, s:s + 1].contiguous(), src_v[:, :, s:s + 1].contiguous())
+    torch.cuda.synchronize()
+    assert lens.cpu().tolist() == [170, 170, 170]
+    assert torch.equal(r.k[:, :, :170], src_k[:, :, :170]) and torch.equal(r.v[:, :, :170], src_v[:, :, :170])
+    assert torch.count_nonzero(r.k[:, :, 170:].view(torch.int16)) == 0
+    exp = _expected_proxy(src_k.cpu().view(torch.int16), torch.sort(r.dom, dim=1).values, 0, r.fasa.row_elems,
+                          [170, 170, 170])
+    assert torch.equal(r.proxy.cpu().view(torch.int16), exp)
+    assert r.fasa.device_status() == 0
+    # attention over the appended cache agrees with the oracle
+    r.seq_lens = lens
+    r.t["seq_lens"] = lens.cpu()
+    r.t["k"], r.t["v"] = r.k.cpu(), r.v.cpu()
+    r.step(); r.dense_step()
+    h = r.host()
+    parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
+                      n_sel=h["n_sel"], out=h["out"], dense_out=h["dense"], what="appended", **r.oracle_kwargs())
+
+
+def test_device_status_bits_instead_of_faults():
+    w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, max_len=128, len_lo=128, len_hi=128, budget=16)
+    r = Run(w)
+    r.build_proxy()
+    # cache full: the appended row is dropped, the length stays at max_len
+    s = synth.make_step_inputs(w, 0, "cuda")
+    r.fasa.kv_append(r.k, r.v, r.proxy, r.seq_lens, s["k_new"], s["v_new"])
+    assert r.fasa.device_status() & binding.DEV_APPEND_FULL
+    assert r.seq_lens.cpu().tolist() == [128]
+    # a length beyond max_len is clamped
+    r.seq_lens.fill_(100000)
+    r.step()
+    assert r.fasa.device_status() & binding.DEV_LEN_CLAMPED
+    assert int(r.n_sel[0, 0]) == 16 + 68
+    # an out-of-range index is clamped to row 0, n_sel beyond the list to its capacity
+    r.seq_lens.fill_(128)
+    r.idx.fill_(10 ** 6)
+    r.n_sel.fill_(10 ** 6)
+    r.fasa.sparse_decode_attn(r.q, r.k, r.v, r.idx, r.n_sel, r.out, r.ws)
+    st = r.fasa.device_status()
+    assert st & binding.DEV_IDX_CLAMPED and st & binding.DEV_NSEL_CLAMPED
+    assert torch.isfinite(r.out).all()
+    # selection larger than the index list: cut to the best n_sel_max
+    small = torch.empty((1, 2, 10), dtype=torch.int32, device="cuda")
+    r.fasa.topk(r.scores, r.seq_lens, 50, small, r.n_sel, r.ws)
+    assert r.fasa.device_status() & binding.DEV_NSEL_CLAMPED
+    assert r.n_sel.cpu().tolist() == [[10, 10]]
+    assert r.fasa.device_status() == 0
+
+
+# ------------------------------------------------------------------ top-k alone ----
+
+def _topk_only(scores_cpu, lens, budget, n_sink, n_recent, n_sel_max):
+    B, H, Lm = scores_cpu.shape
+    dom = torch.arange(4, dtype=torch.int32).repeat(H, 1)
+    f = binding.Fasa(B, H, H, Lm, dom, n_sink=n_sink, n_recent=n_recent)
+    sc = scores_cpu.cuda()
+    ln = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    idx = torch.full((B, H, n_sel_max), -7, dtype=torch.int32, device="cuda")
+    ns = torch.full((B, H), -7, dtype=torch.int32, device="cuda")
+    f.topk(sc, ln, budget, idx, ns)
+    torch.cuda.synchronize()
+    assert f.device_status() == 0
+    return idx.cpu().numpy(), ns.cpu().numpy()
+
+
+def _assert_topk_exact(scores_cpu, lens, budget, n_sink=0, n_recent=0, n_sel_max=None):
+    """Given the same fp32 scores, the GPU set equals the oracle's bit for bit, ties included."""
+    B, H, Lm = scores_cpu.shape
+    n_sel_max = n_sel_max or Lm
+    idx, ns = _topk_only(scores_cpu, lens, budget, n_sink, n_recent, n_sel_max)
+    for b in range(B):
+        L = lens[b]
+        k = budget if budget > 0 else (-budget * L + 999) // 1000
+        for h in range(H):
+            ref, _ = O.select(scores_cpu[b, h, :L].double().numpy(), k, n_sink, n_recent)
+            assert int(ns[b, h]) == ref.size
+            assert np.array_equal(idx[b, h, :ref.size], ref), (b, h)
+
+
+def test_topk_exact_on_heavy_ties():
+    g = torch.Generator().manual_seed(5)
+    # few distinct values: the k-th rank always falls inside a run of equal scores
+    sc = torch.randint(-3, 4, (2, 3, 5000), generator=g).float()
+    for budget in (1, 100, 2500, 4999):
+        _assert_topk_exact(sc, [5000, 4321], budget)
+    _assert_topk_exact(sc, [5000, 4321], 64, n_sink=4, n_recent=64)
+    _assert_topk_exact(torch.zeros(1, 2, 3000), [3000], 17)
+    _assert_topk_exact(torch.full((1, 2, 3000), -1.5), [2999], -189)
+
+
+def test_topk_exact_on_special_values():
+    g = torch.Generator().manual_seed(6)
+    sc = torch.randn(1, 4, 4096, generator=g)
+    sc[0, 0, ::7] = float("inf")
+    sc[0, 1, ::5] = float("-inf")
+    sc[0, 2, 100:300] = 0.0             # (+0 only: fc_score never emits -0, which would rank below +0)
+    sc[0, 3] = sc[0, 3].abs() * 1e-40   # subnormals
+    for budget in (10, 600, 3000):
+        _assert_topk_exact(sc, [4096], budget)
+
+
+@pytest.mark.parametrize("L,B,H", [(32768, 1, 8), (131072, 2, 2), (140001, 1, 2), (20000, 3, 5)])
+def test_topk_exact_at_scale(L, B, H):
+    # 131072 fills the register-resident capacity of an 8-CTA cluster; 140001 takes the
+    # streaming fallback; 20000 x 15 units uses small clusters.
+    g = torch.Generator().manual_seed(L)
+    sc = torch.randn(B, H, L, generator=g) * 40.0
+    lens = [L - 13 * b for b in range(B)]
+    for budget in (256, 4096):
+        _assert_topk_exact(sc, lens, budget, n_sink=4, n_recent=64, n_sel_max=4096 + 68)
+    _assert_topk_exact(sc, lens, -189, n_sel_max=(189 * L + 999) // 1000)
+
+
+# ------------------------------------------------------------------ full sizes ----
+
+def test_config1_full_size():
+    rep, h = _full_check(Run(C["c1"]))
+    assert rep["units"] == 8 and np.all(h["n_sel"] == 324)
+
+
+def test_config4_point_full_length_sampled_units():
+    # One sweep point at the full 65536 context, batch reduced to keep host memory modest.
+    w = C["c4"].replace(batch=2, n_q_heads=16, n_kv_heads=4, budget=2048, n_dom=32)
+    r = Run(w)
+    r.build_proxy()
+    r.step(); r.dense_step()
+    h = r.host()
+    parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
+                      n_sel=h["n_sel"], out=h["out"], dense_out=h["dense"], units=[(0, 0), (1, 3), (1, 1)],
+                      what="c4", **r.oracle_kwargs())
