@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of the FASA decode hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c1] [--impl reference]
+
+One step = one pass of the whole hot path over one batch: append one token per sequence
+(K, V and proxy-K rows), score every cached key on the dominant FCs, select the top-budget
+tokens, run exact attention over the selected rows and merge the splits.  Inputs are
+synthetic (paper_2602_03152_b200.synth) and resident in HBM before the timed region; L2 is
+flushed between steps.  Rank 0 prints one JSON line.
+
+Headline metric: effective HBM GB/s = algorithmic bytes of the step (proxy bytes of every
+cached token + K/V rows of the selected tokens + q + out) / device time, summed over ranks;
+`us_per_step`, the dense-path time and the speedup ride along.  `roofline` describes the
+dominant kernel (the FC scoring stream), `cpu_baseline` the fp64 oracle timed on the host.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fasa_decode_attn_effective_hbm_gbs"
+UNIT = "GB/s"
+L2_FLUSH_BYTES = 256 << 20
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, burst copy)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+# ---------------------------------------------------------------- byte model ----
+
+def step_bytes(w, lens, n_sel):
+    """Algorithmic bytes of one FASA step and of one dense step (Sec. 4.4 byte model).
+    lens: per-sequence context at scoring time; n_sel: tokens attended per unit."""
+    units_len = sum(int(l) for l in lens) * w.n_kv_heads
+    qo = w.batch * w.n_q_heads * 128 * (2 + 4)
+    proxy = units_len * 4 * w.n_dom
+    gathered = int(n_sel) * 512
+    return {"proxy": proxy, "gathered": gathered, "qo": qo, "fasa": proxy + gathered + qo,
+            "dense": units_len * 512 + qo}
+
+
+# ---------------------------------------------------------------- clocks ----
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.rows, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", gpu_id, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        # the busiest half of the samples stands for "under load"
+        sm_sorted = sorted(sm)
+        load = sm_sorted[len(sm_sorted) // 2:] if sm_sorted else []
+        return {"sm_mhz": statistics.median(load) if load else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------- reference arm ----
+
+def run_reference(args, w):
+    """Times the fp64 CPU oracle, as it stands, on the host cores: each step is one oracle
+    pass (score -> select -> attention) over a bounded sample of the workload's units."""
+    import numpy as np
+    from oracle import fasa_oracle as O
+    from paper_2602_03152_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = os.cpu_count() or 1
+    # sample: at most 8 units, sequences cut to 32768 rows (about a second of CPU work per step)
+    sw = w.replace(batch=1, max_len=min(w.max_len, 32768), len_lo=min(w.len_lo, 32768), len_hi=min(w.len_hi, 32768))
+    t = synth.make_inputs(sw, "cpu")
+    qb, kb, vb = synth.bf16_bits(t["q"]), synth.bf16_bits(t["k"]), synth.bf16_bits(t["v"])
+    lens, dom = t["seq_lens"].numpy(), t["dom"].numpy()
+    kw = dict(pairing=sw.pairing, group_reduce=sw.group_reduce, n_sink=sw.n_sink, n_recent=sw.n_recent,
+              budget=sw.budget, n_sel_max=sw.n_sel_max(), n_threads=cores, want_scores=False, want_dense=False)
+    steps, warm = max(1, min(args.steps, 20)), max(1, min(args.warmup, 3))
+    for _ in range(warm):
+        r = O.decode_bf16(qb, kb, vb, lens, dom, **kw)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        r = O.decode_bf16(qb, kb, vb, lens, dom, **kw)
+    dt = (time.perf_counter() - t0) / steps
+    by = step_bytes(sw, lens, int(r["n_sel"].sum()))
+    val = by["fasa"] / dt / 1e9
+    sample = f"{sw.n_kv_heads} units (batch 1 of {w.batch}), context {int(lens[0])}, one oracle pass per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": int(r["threads"]), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+# ---------------------------------------------------------------- our arm ----
+
+def run_fasa(args, w):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2602_03152_b200 import binding, build, synth
+
+    build.build()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the FASA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    # Weak scaling: every rank holds its own batch of independent (batch, KV head) units.
+    # The cache has one spare row so each step appends at row L-1 and scores L rows.
+    wl = w.replace(index=w.index + 100 * rank)
+    t = synth.make_inputs(wl, dev)
+    lens_full = t["seq_lens"].clone()
+    lens_start = (lens_full - 1).clamp_(min=0)
+    f = binding.Fasa.from_workload(wl, t["dom"])
+    q, k, v = t["q"], t["k"], t["v"]
+    n_sel_max = wl.n_sel_max()
+    B, Hq, Hkv, Lm = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.max_len
+    proxy = f.alloc_proxy(dev)
+    ws = f.alloc_workspace(n_sel_max, dev)
+    scores = torch.zeros((B, Hkv, Lm), dtype=torch.float32, device=dev)
+    idx = torch.zeros((B, Hkv, n_sel_max), dtype=torch.int32, device=dev)
+    n_sel = torch.zeros((B, Hkv), dtype=torch.int32, device=dev)
+    out = torch.zeros((B, Hq, 128), dtype=torch.float32, device=dev)
+    dense_out = torch.zeros_like(out)
+    lens = lens_full.clone()
+    f.proxy_build(k, proxy, lens)
+    # the token appended each step: the cache's own last row, so the cache content never changes
+    bi = torch.arange(B, device=dev)
+    last = lens_start.long()
+    k_new = k[bi, :, last].unsqueeze(2).contiguous()
+    v_new = v[bi, :, last].unsqueeze(2).contiguous()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, n, warm):
+        """n event-timed calls of fn on the current stream, L2 flushed and the sequence
+        lengths reset before each; returns the list of durations in microseconds."""
+        durs = []
+        for i in range(warm + n):
+            lens.copy_(lens_start)
+            flush.fill_(i & 0xff)
+            a, b = ev(), ev()
+            a.record()
+            fn()
+            b.record()
+            b.synchronize()
+            if i >= warm:
+                durs.append(a.elapsed_time(b) * 1e3)
+        return durs
+
+    def fasa_step():
+        f.kv_append(k, v, proxy, lens, k_new, v_new)
+        f.decode_step(q, k, v, proxy, lens, wl.budget, scores, idx, n_sel, out, ws)
+
+    def dense_step():
+        f.kv_append(k, v, proxy, lens, k_new, v_new)
+        f.full_decode_attn(q, k, v, lens, dense_out, ws)
+
+    K, W = args.steps, max(3, args.warmup)
+    gpu_id = str(local)
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(gpu_id) if rank == 0 else None
+
+    # ---- timed region: K whole steps ------------------------------------------------
+    timed(fasa_step, 0, W)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    l0 = f.launch_count()
+    step_us = timed(fasa_step, K, 0)
+    torch.cuda.synchronize()
+    launches = f.launch_count() - l0
+    if world > 1:
+        dist.barrier()
+    total_us = sum(step_us)
+    if world > 1:
+        tt = torch.tensor([total_us], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_us = float(tt.item())
+    us_per_step = total_us / K
+
+    n_sel_total = int(n_sel.sum().item())
+    by = step_bytes(wl, lens_full.cpu().tolist(), n_sel_total)
+    status = f.device_status()
+
+    # ---- per-kernel breakdown (same launches, one C-ABI call at a time) ----------------
+    parts = {"kv_append": [], "fc_score": [], "topk": [], "sparse_attn": []}
+    Kk = min(K, 200)
+    for i in range(W + Kk):
+        lens.copy_(lens_start)
+        flush.fill_(i & 0xff)
+        e = [ev() for _ in range(5)]
+        e[0].record(); f.kv_append(k, v, proxy, lens, k_new, v_new)
+        e[1].record(); f.fc_score(q, proxy, lens, scores)
+        e[2].record(); f.topk(scores, lens, wl.budget, idx, n_sel, ws)
+        e[3].record(); f.sparse_decode_attn(q, k, v, idx, n_sel, out, ws)
+        e[4].record(); e[4].synchronize()
+        if i >= W:
+            for j, name in enumerate(parts):
+                parts[name].append(e[j].elapsed_time(e[j + 1]) * 1e3)
+    kern_us = {n: statistics.mean(v_) for n, v_ in parts.items()}
+    dense_us = statistics.mean(timed(dense_step, Kk, W))
+
+    # ---- end to end from host buffers ---------------------------------------------------
+    stage = torch.empty(f.stage_bytes(), dtype=torch.uint8, device=dev)
+    qh, knh, vnh = q.cpu().pin_memory(), k_new.cpu().pin_memory(), v_new.cpu().pin_memory()
+    oh = torch.empty((B, Hq, 128), dtype=torch.float32).pin_memory()
+
+    def e2e_step():
+        f.decode_step_host(qh, knh, vnh, stage, k, v, proxy, lens, wl.budget, scores, idx, n_sel, out, oh, ws)
+
+    e2e_us = statistics.mean(timed(e2e_step, Kk, W))
+    if world > 1:
+        tt = torch.tensor([e2e_us], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_us = float(tt.item())
+    h2d = qh.numel() * 2 + knh.numel() * 2 + vnh.numel() * 2
+    d2h = oh.numel() * 4
+    clocks = sampler.stop() if sampler else None
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = _peaks()
+    fc_bytes = by["proxy"]                      # the scoring kernel's algorithmic bytes per launch
+    roof_us = by["fasa"] / (peak * 1e9) * 1e6
+    line = {
+        "metric": METRIC, "value": world * by["fasa"] / (us_per_step * 1e-6) / 1e9, "unit": UNIT,
+        "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": us_per_step / 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, f32 accumulate",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "batch": B, "n_q_heads": Hq, "n_kv_heads": Hkv, "context": int(lens_full.max()),
+                   "context_mean": float(lens_full.float().mean()), "n_dom": wl.n_dom, "budget": wl.budget,
+                   "n_sink": wl.n_sink, "n_recent": wl.n_recent, "n_sel_per_unit": n_sel_total / (B * Hkv),
+                   "l2": f"flushed before every step ({L2_FLUSH_BYTES >> 20} MiB write)",
+                   "per_rank": "each rank runs its own batch of independent units, no collective"},
+        "us_per_step": us_per_step,
+        "us_per_step_median": statistics.median(step_us),
+        "step_bytes": by["fasa"], "step_roofline_us": roof_us, "step_frac_of_roofline": roof_us / us_per_step,
+        "dense_us_per_step": dense_us, "dense_bytes": by["dense"],
+        "dense_gbs": by["dense"] / (dense_us * 1e-6) / 1e9, "dense_frac_of_roofline": by["dense"] / (dense_us * 1e-6) / 1e9 / peak,
+        "speedup_vs_dense": dense_us / us_per_step, "byte_ratio_dense_over_fasa": by["dense"] / by["fasa"],
+        "kernels_us": kern_us,
+        "kernels_gbs": {"fc_score": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9,
+                        "sparse_attn": by["gathered"] / (kern_us["sparse_attn"] * 1e-6) / 1e9,
+                        "topk": (by["proxy"] // wl.n_dom) / (kern_us["topk"] * 1e-6) / 1e9},
+        "roofline": {"kernel": "fc_score_kernel", "bound": "hbm",
+                     "achieved": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
+                     "frac": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9 / peak, "traffic": None,
+                     "bytes_per_launch": fc_bytes, "us_per_launch": kern_us["fc_score"], "peak_source": peak_src},
+        "e2e": {"value": world * by["fasa"] / (e2e_us * 1e-6) / 1e9, "unit": UNIT, "us_per_step": e2e_us,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches), "device_status": status, "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl, t, by)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(w, t, by):
+    """The fp64 oracle, as it stands, timed on the host cores on a bounded sample: the units
+    of the first sequence, one whole pass (score -> select -> attention)."""
+    from oracle import fasa_oracle as O
+    from paper_2602_03152_b200 import synth
+
+    cores = os.cpu_count() or 1
+    L = int(t["seq_lens"][0])
+    qb = synth.bf16_bits(t["q"][:1])
+    kb = synth.bf16_bits(t["k"][:1, :, :L])
+    vb = synth.bf16_bits(t["v"][:1, :, :L])
+    lens = t["seq_lens"][:1].cpu().numpy()
+    kw = dict(pairing=w.pairing, group_reduce=w.group_reduce, n_sink=w.n_sink, n_recent=w.n_recent,
+              budget=w.budget, n_sel_max=w.n_sel_max(), n_threads=cores, want_scores=False, want_dense=False)
+    r = O.decode_bf16(qb, kb, vb, lens, t["dom"].numpy(), **kw)      # warm-up, page in
+    reps, t0 = 0, time.perf_counter()
+    while reps < 3 or (time.perf_counter() - t0 < 10.0 and reps < 50):
+        r = O.decode_bf16(qb, kb, vb, lens, t["dom"].numpy(), **kw)
+        reps += 1
+    dt = (time.perf_counter() - t0) / reps
+    sb = step_bytes(w.replace(batch=1), [L], int(r["n_sel"].sum()))
+    return {"value": sb["fasa"] / dt / 1e9, "unit": UNIT, "cores": int(r["threads"]), "kind": "oracle",
+            "us_per_step_sample": dt * 1e6,
+            "sample": f"{w.n_kv_heads} units of sequence 0 (context {L}) out of batch {w.batch}, {reps} passes"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="fasa", choices=["fasa", "reference"])
+    ap.add_argument("--config", default="c1", help="workload: c0, c1 (default), c2, c4")
+    ap.add_argument("--budget", type=int, default=None)
+    ap.add_argument("--n-dom", type=int, default=None)
+    ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (profiling)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2602_03152_b200 import synth
+    w = synth.CONFIGS[args.config]
+    if args.budget is not None:
+        w = w.replace(budget=args.budget)
+    if args.n_dom is not None:
+        w = w.replace(n_dom=args.n_dom)
+    if args.batch is not None:
+        w = w.replace(batch=args.batch)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_fasa(args, w)
+
+
+if __name__ == "__main__":
+    main()
