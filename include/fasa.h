@@ -157,6 +157,37 @@ int32_t fasa_full_decode_attn(fasa_ctx_t* ctx, const void* q, const void* k_cach
                               const void* v_cache, const int32_t* seq_lens, float* out,
                               float* lse, void* workspace, void* stream);
 
+/* ---- for callers that cannot allocate ------------------------------------ */
+
+/* Size of the built-in scratch area of fasa_sparse_decode_attn_static (bytes). */
+#define FASA_STATIC_SCRATCH_BYTES (4u << 20)
+
+/* (No counterpart in the paper: a packaging variant of fasa_sparse_decode_attn.)
+ * Some callers have no way to hand the library a workspace: code that runs where
+ * cudaMalloc is off limits (inside a memory pool it does not own, under a plugin
+ * interface that passes only inputs and outputs, in a real-time loop that may not
+ * touch the allocator).  For them this call computes exactly what
+ * fasa_sparse_decode_attn computes, with the split-K partial results kept in a
+ * fixed FASA_STATIC_SCRATCH_BYTES array that is part of the library image; each
+ * GPU that loads the library holds that array until the process exits.  The call
+ * allocates and frees nothing, on the host or the device.
+ *   - Arguments, layouts and results: as fasa_sparse_decode_attn, minus `workspace`.
+ *   - Limit: batch * n_q_heads * n_splits * 130 * 4 bytes must fit the array, where
+ *     n_splits is the split count the library picks for n_sel_max (at most
+ *     ceil(n_sel_max / 64)); otherwise FASA_ERR_WORKSPACE is returned and nothing is
+ *     enqueued.  Configuration 1 of the benchmarks needs 0.1 MB, configuration 2 1.4 MB.
+ *   - The context's device must be current (FASA_ERR_INVALID_ARG otherwise).  The first
+ *     call on a device looks up the array's device address (a CUDA runtime query, no
+ *     allocation); make that first call before any stream capture begins.
+ *   - All calls in the process share the one array per device.  Nothing in it has to
+ *     start at zero (every partial that is read was written by the same call), but
+ *     two calls whose kernels overlap on the GPU (different streams, or different
+ *     contexts on the same device) race on it: keep them on one stream, or ordered. */
+int32_t fasa_sparse_decode_attn_static(fasa_ctx_t* ctx, const void* q, const void* k_cache,
+                                       const void* v_cache, const int32_t* idx,
+                                       const int32_t* n_sel, int32_t n_sel_max, float* out,
+                                       float* lse, void* stream);
+
 /* ---- whole step ---------------------------------------------------------- */
 
 /* fasa_fc_score -> fasa_topk -> fasa_sparse_decode_attn on one stream with no

@@ -25,6 +25,7 @@ SYMBOLS = [
     "fasa_status_string", "fasa_last_cuda_error", "fasa_get_device_status", "fasa_launch_count",
     "fasa_kv_append", "fasa_proxy_build", "fasa_fc_score", "fasa_topk", "fasa_sparse_decode_attn",
     "fasa_full_decode_attn", "fasa_decode_step", "fasa_stage_bytes", "fasa_decode_step_host",
+    "fasa_sparse_decode_attn_static",
 ]
 
 
@@ -74,6 +75,7 @@ def load_library() -> ctypes.CDLL:
         "fasa_topk": (i32, [vp, vp, vp, i32, i32, vp, vp, vp, vp]),
         "fasa_sparse_decode_attn": (i32, [vp] * 6 + [i32] + [vp] * 4),
         "fasa_full_decode_attn": (i32, [vp] * 9),
+        "fasa_sparse_decode_attn_static": (i32, [vp] * 6 + [i32] + [vp] * 3),
         "fasa_decode_step": (i32, [vp] * 6 + [i32, i32] + [vp] * 7),
         "fasa_stage_bytes": (i32, [vp, ctypes.POINTER(ctypes.c_size_t)]),
         "fasa_decode_step_host": (i32, [vp] * 9 + [i32, i32] + [vp] * 7),
@@ -206,6 +208,16 @@ class Fasa:
                                                       v_cache.data_ptr(), _dp(idx, torch.int32),
                                                       _dp(n_sel, torch.int32), n_sel_max, _dp(out, torch.float32),
                                                       _dp(lse), _dp(workspace), _stream()), "fasa_sparse_decode_attn")
+
+    def sparse_decode_attn_static(self, q, k_cache, v_cache, idx, n_sel, out, lse=None):
+        """fasa_sparse_decode_attn for callers that cannot provide a workspace: the split-K
+        partials go to a fixed array inside the library (no allocation anywhere).  Calls share
+        that array, so keep them ordered on one stream."""
+        n_sel_max = idx.shape[-1]
+        self._check(self._lib.fasa_sparse_decode_attn_static(
+            self._h, _dp(q, torch.bfloat16), k_cache.data_ptr(), v_cache.data_ptr(), _dp(idx, torch.int32),
+            _dp(n_sel, torch.int32), n_sel_max, _dp(out, torch.float32), _dp(lse), _stream()),
+            "fasa_sparse_decode_attn_static")
 
     def full_decode_attn(self, q, k_cache, v_cache, seq_lens, out, workspace, lse=None):
         self._check(self._lib.fasa_full_decode_attn(self._h, _dp(q, torch.bfloat16), k_cache.data_ptr(),

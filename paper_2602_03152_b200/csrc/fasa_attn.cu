@@ -9,9 +9,16 @@
 // 8 rows are completed with a transposing xor-shuffle reduction (8 shuffles per head per
 // batch); probabilities travel back to all lanes through shared memory.  All multiply-adds
 // are packed two-wide fp32 FMAs.  No tensor cores: one query token per sequence.
+#include <mutex>
+
 #include "fasa_common.cuh"
 
 namespace {
+
+// Split-K partials of fasa_sparse_decode_attn_static: lives in the library image, so every
+// GPU that loads the library holds these bytes until the process exits.
+constexpr size_t kStaticScratchBytes = FASA_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 constexpr int kAttnThreads = 128;
 constexpr int kAttnHalfWarps = kAttnThreads / 16;  // 8
@@ -339,4 +346,45 @@ extern "C" int32_t fasa_full_decode_attn(fasa_ctx_t* ctx, const void* q, const v
     return FASA_ERR_INVALID_ARG;
   return launch_attn<false>(ctx, q, k_cache, v_cache, nullptr, seq_lens, ctx->cfg.max_len, 0, out,
                             lse, workspace, (cudaStream_t)stream);
+}
+
+// ---- variant for callers that cannot allocate device memory --------------------------------
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_ptr[kMaxDevices];   // device address of g_static_scratch, per device ordinal
+}  // namespace
+
+extern "C" int32_t fasa_sparse_decode_attn_static(fasa_ctx_t* ctx, const void* q,
+                                                  const void* k_cache, const void* v_cache,
+                                                  const int32_t* idx, const int32_t* n_sel,
+                                                  int32_t n_sel_max, float* out, float* lse,
+                                                  void* stream) {
+  if (!ctx || !q || !k_cache || !v_cache || !idx || !n_sel || !out || n_sel_max <= 0)
+    return FASA_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16)) return FASA_ERR_INVALID_ARG;
+  const fasa_config_t& c = ctx->cfg;
+  const int n_upper = n_sel_max < c.max_len ? n_sel_max : c.max_len;
+  const fasa_split_plan plan = fasa_plan_splits(ctx, n_upper);
+  const size_t need = (size_t)c.batch * c.n_q_heads * (size_t)plan.n_splits * kPartialStride * sizeof(float);
+  if (need > kStaticScratchBytes) return FASA_ERR_WORKSPACE;
+
+  // The symbol names a different copy of the array on each device: its address is looked up
+  // once per device, with that device current (the name itself is not a device pointer).
+  int dev = -1;
+  FASA_CUDA_TRY(ctx, cudaGetDevice(&dev));
+  if (dev != ctx->device || dev < 0 || dev >= kMaxDevices) return FASA_ERR_INVALID_ARG;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ptr[dev]) {
+      void* p = nullptr;
+      FASA_CUDA_TRY(ctx, cudaGetSymbolAddress(&p, g_static_scratch));
+      g_scratch_ptr[dev] = p;
+    }
+    scratch = g_scratch_ptr[dev];
+  }
+  return launch_attn<true>(ctx, q, k_cache, v_cache, idx, n_sel, n_upper, n_sel_max, out, lse,
+                           scratch, (cudaStream_t)stream);
 }
