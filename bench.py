@@ -5,14 +5,18 @@
 
 One step = one pass of the whole hot path over one batch: append one token per sequence
 (K, V and proxy-K rows), score every cached key on the dominant FCs, select the top-budget
-tokens, run exact attention over the selected rows and merge the splits.  Inputs are
+tokens, run exact attention over the selected rows and merge the splits.  The step calls
+fasa_kv_append and fasa_decode_step (one cluster kernel: score -> select -> attention); the
+three stand-alone calls (fasa_fc_score, fasa_topk, fasa_sparse_decode_attn) and the dense
+path are timed beside it.  Inputs are
 synthetic (paper_2602_03152_b200.synth) and resident in HBM before the timed region; L2 is
 flushed between steps.  Rank 0 prints one JSON line.
 
 Headline metric: effective HBM GB/s = algorithmic bytes of the step (proxy bytes of every
 cached token + K/V rows of the selected tokens + q + out) / device time, summed over ranks;
 `us_per_step`, the dense-path time and the speedup ride along.  `roofline` describes the
-dominant kernel (the FC scoring stream), `cpu_baseline` the fp64 oracle timed on the host.
+dominant kernel (the one-launch decode step, or the FC scoring stream where the step runs as
+three kernels), `cpu_baseline` the fp64 oracle timed on the host.
 """
 from __future__ import annotations
 
@@ -207,9 +211,13 @@ def run_fasa(args, w):
                 durs.append(a.elapsed_time(b) * 1e3)
         return durs
 
+    if args.step_mode is not None:
+        f.set_step_mode(args.step_mode)
+    fused = f.step_cluster_size() > 0
+
     def fasa_step():
         f.kv_append(k, v, proxy, lens, k_new, v_new)
-        f.decode_step(q, k, v, proxy, lens, wl.budget, scores, idx, n_sel, out, ws)
+        f.decode_step(q, k, v, proxy, lens, wl.budget, None if fused else scores, idx, n_sel, out, ws)
 
     def dense_step():
         f.kv_append(k, v, proxy, lens, k_new, v_new)
@@ -262,6 +270,24 @@ def run_fasa(args, w):
                 parts[name].append(e[j].elapsed_time(e[j + 1]) * 1e3)
     kern_us = {n: statistics.mean(v_) for n, v_ in parts.items()}
     dense_us = statistics.mean(timed(dense_step, Kk, W))
+    # the decode step alone (no append): one launch when the cluster kernel is in use
+    lens.copy_(lens_full)
+
+    def step_only():
+        lens.copy_(lens_full)
+        f.decode_step(q, k, v, proxy, lens, wl.budget, None if fused else scores, idx, n_sel, out, ws)
+
+    step_only_us = []
+    for i in range(W + Kk):
+        flush.fill_(i & 0xff)
+        lens.copy_(lens_full)
+        a, b = ev(), ev()
+        a.record()
+        f.decode_step(q, k, v, proxy, lens, wl.budget, None if fused else scores, idx, n_sel, out, ws)
+        b.record(); b.synchronize()
+        if i >= W:
+            step_only_us.append(a.elapsed_time(b) * 1e3)
+    step_only_us = statistics.mean(step_only_us)
 
     # ---- end to end from host buffers ---------------------------------------------------
     stage = torch.empty(f.stage_bytes(), dtype=torch.uint8, device=dev)
@@ -288,6 +314,17 @@ def run_fasa(args, w):
     peak, peak_src = _peaks()
     fc_bytes = by["proxy"]                      # the scoring kernel's algorithmic bytes per launch
     roof_us = by["fasa"] / (peak * 1e9) * 1e6
+    if fused:
+        roofline = {"kernel": "fused_decode_kernel", "bound": "hbm",
+                    "achieved": by["fasa"] / (step_only_us * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
+                    "frac": by["fasa"] / (step_only_us * 1e-6) / 1e9 / peak, "traffic": None,
+                    "bytes_per_launch": by["fasa"], "us_per_launch": step_only_us, "peak_source": peak_src,
+                    "cluster_size": f.step_cluster_size()}
+    else:
+        roofline = {"kernel": "fc_score_kernel", "bound": "hbm",
+                    "achieved": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
+                    "frac": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9 / peak, "traffic": None,
+                    "bytes_per_launch": fc_bytes, "us_per_launch": kern_us["fc_score"], "peak_source": peak_src}
     line = {
         "metric": METRIC, "value": world * by["fasa"] / (us_per_step * 1e-6) / 1e9, "unit": UNIT,
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": us_per_step / 1e3,
@@ -308,10 +345,11 @@ def run_fasa(args, w):
         "kernels_gbs": {"fc_score": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9,
                         "sparse_attn": by["gathered"] / (kern_us["sparse_attn"] * 1e-6) / 1e9,
                         "topk": (by["proxy"] // wl.n_dom) / (kern_us["topk"] * 1e-6) / 1e9},
-        "roofline": {"kernel": "fc_score_kernel", "bound": "hbm",
-                     "achieved": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
-                     "frac": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9 / peak, "traffic": None,
-                     "bytes_per_launch": fc_bytes, "us_per_launch": kern_us["fc_score"], "peak_source": peak_src},
+        "kernels_frac_of_peak": {"fc_score": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9 / peak,
+                                 "sparse_attn": by["gathered"] / (kern_us["sparse_attn"] * 1e-6) / 1e9 / peak,
+                                 "topk": (by["proxy"] // wl.n_dom) / (kern_us["topk"] * 1e-6) / 1e9 / peak},
+        "decode_step_only_us": step_only_us, "step_mode": "one cluster kernel" if fused else "three kernels",
+        "roofline": roofline,
         "e2e": {"value": world * by["fasa"] / (e2e_us * 1e-6) / 1e9, "unit": UNIT, "us_per_step": e2e_us,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches), "device_status": status, "clocks": clocks,
@@ -360,6 +398,8 @@ def main():
     ap.add_argument("--n-dom", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--step-mode", type=int, default=None, choices=[0, 1],
+                    help="0: fasa_decode_step as three kernels; 1 (default): one cluster kernel where available")
     args = ap.parse_args()
 
     from paper_2602_03152_b200 import synth

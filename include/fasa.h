@@ -190,8 +190,19 @@ int32_t fasa_sparse_decode_attn_static(fasa_ctx_t* ctx, const void* q, const voi
 
 /* ---- whole step ---------------------------------------------------------- */
 
-/* fasa_fc_score -> fasa_topk -> fasa_sparse_decode_attn on one stream with no
- * host round trip in between.  scores, idx and n_sel are outputs too. */
+/* Scoring, selection and attention of one step, on one stream with no host round trip.
+ * idx and n_sel are outputs too; so is scores unless it is NULL.
+ *
+ * Mode 1 (default where available): ONE kernel, one thread-block cluster per (batch, KV
+ * head); scores, histograms and split partials stay in (distributed) shared memory, so
+ * `workspace` may be NULL and `scores` may be NULL (they are then not written).  Available
+ * when group_reduce == 0 and ceil(max_len / 16) <= 45056; fasa_step_cluster_size tells.
+ * Mode 0, and every configuration mode 1 cannot take: fasa_fc_score -> fasa_topk ->
+ * fasa_sparse_decode_attn; scores and workspace are then required (INVALID_ARG if NULL).
+ * Both modes select identical index sets; outputs agree to fp32 rounding. */
+int32_t fasa_set_step_mode(fasa_ctx_t* ctx, int32_t mode);
+/* Cluster size mode 1 runs with for this context; 0 = fasa_decode_step uses mode 0. */
+int32_t fasa_step_cluster_size(const fasa_ctx_t* ctx);
 int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_cache,
                          const void* v_cache, const void* proxy_k, const int32_t* seq_lens,
                          int32_t budget, int32_t n_sel_max, float* scores, int32_t* idx,

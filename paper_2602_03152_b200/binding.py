@@ -25,7 +25,7 @@ SYMBOLS = [
     "fasa_status_string", "fasa_last_cuda_error", "fasa_get_device_status", "fasa_launch_count",
     "fasa_kv_append", "fasa_proxy_build", "fasa_fc_score", "fasa_topk", "fasa_sparse_decode_attn",
     "fasa_full_decode_attn", "fasa_decode_step", "fasa_stage_bytes", "fasa_decode_step_host",
-    "fasa_sparse_decode_attn_static",
+    "fasa_sparse_decode_attn_static", "fasa_set_step_mode", "fasa_step_cluster_size",
 ]
 
 
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
         "fasa_full_decode_attn": (i32, [vp] * 9),
         "fasa_sparse_decode_attn_static": (i32, [vp] * 6 + [i32] + [vp] * 3),
         "fasa_decode_step": (i32, [vp] * 6 + [i32, i32] + [vp] * 7),
+        "fasa_set_step_mode": (i32, [vp, i32]),
+        "fasa_step_cluster_size": (i32, [vp]),
         "fasa_stage_bytes": (i32, [vp, ctypes.POINTER(ctypes.c_size_t)]),
         "fasa_decode_step_host": (i32, [vp] * 9 + [i32, i32] + [vp] * 7),
     }
@@ -164,6 +166,13 @@ class Fasa:
         self._check(self._lib.fasa_stage_bytes(self._h, ctypes.byref(out)), "fasa_stage_bytes")
         return int(out.value)
 
+    def set_step_mode(self, mode: int):
+        """1: decode_step runs as one cluster kernel where available; 0: three separate calls."""
+        self._check(self._lib.fasa_set_step_mode(self._h, mode), "fasa_set_step_mode")
+
+    def step_cluster_size(self) -> int:
+        return int(self._lib.fasa_step_cluster_size(self._h))
+
     def launch_count(self) -> int:
         return int(self._lib.fasa_launch_count(self._h))
 
@@ -225,7 +234,7 @@ class Fasa:
                                                     _dp(out, torch.float32), _dp(lse), _dp(workspace), _stream()),
                     "fasa_full_decode_attn")
 
-    def decode_step(self, q, k_cache, v_cache, proxy_k, seq_lens, budget, scores, idx, n_sel, out, workspace,
+    def decode_step(self, q, k_cache, v_cache, proxy_k, seq_lens, budget, scores, idx, n_sel, out, workspace=None,
                     lse=None):
         n_sel_max = idx.shape[-1]
         self._check(self._lib.fasa_decode_step(self._h, _dp(q, torch.bfloat16), k_cache.data_ptr(),

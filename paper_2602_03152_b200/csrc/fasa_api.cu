@@ -101,6 +101,8 @@ extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_h
     delete ctx;
     return FASA_ERR_CUDA;
   }
+  fasa_fused_plan(ctx);
+  ctx->use_fused = 1;
   *out = ctx;
   return FASA_OK;
 }
@@ -127,6 +129,16 @@ extern "C" const char* fasa_status_string(int32_t s) {
 
 extern "C" const char* fasa_last_cuda_error(const fasa_ctx_t* ctx) {
   return ctx ? ctx->cuda_err : "";
+}
+
+extern "C" int32_t fasa_set_step_mode(fasa_ctx_t* ctx, int32_t mode) {
+  if (!ctx || (mode != 0 && mode != 1)) return FASA_ERR_INVALID_ARG;
+  ctx->use_fused = mode;
+  return FASA_OK;
+}
+
+extern "C" int32_t fasa_step_cluster_size(const fasa_ctx_t* ctx) {
+  return ctx && ctx->use_fused ? ctx->fused_cs : 0;
 }
 
 extern "C" int64_t fasa_launch_count(const fasa_ctx_t* ctx) { return ctx ? ctx->launches : 0; }
@@ -174,9 +186,17 @@ extern "C" int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* 
                                     const int32_t* seq_lens, int32_t budget, int32_t n_sel_max,
                                     float* scores, int32_t* idx, int32_t* n_sel, float* out,
                                     float* lse, void* workspace, void* stream) {
-  if (!ctx || !q || !k_cache || !v_cache || !proxy_k || !seq_lens || !scores || !idx || !n_sel ||
-      !out || !workspace || budget == 0 || n_sel_max <= 0)
+  if (!ctx || !q || !k_cache || !v_cache || !proxy_k || !seq_lens || !idx || !n_sel || !out ||
+      budget == 0 || budget < -1000 || n_sel_max <= 0)
     return FASA_ERR_INVALID_ARG;
+  if (ctx->use_fused && ctx->fused_cs > 0) {
+    if (((uintptr_t)proxy_k & 15) || ((uintptr_t)q & 1) || ((uintptr_t)k_cache & 15) ||
+        ((uintptr_t)v_cache & 15) || (scores && ((uintptr_t)scores & 3)))
+      return FASA_ERR_INVALID_ARG;
+    return fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
+                             idx, n_sel, out, lse, (cudaStream_t)stream);
+  }
+  if (!scores || !workspace) return FASA_ERR_INVALID_ARG;
   int32_t st = fasa_fc_score(ctx, q, proxy_k, seq_lens, scores, stream);
   if (st != FASA_OK) return st;
   st = fasa_topk(ctx, scores, seq_lens, budget, n_sel_max, idx, n_sel, workspace, stream);

@@ -22,6 +22,9 @@ struct fasa_ctx {
   int n_sm;
   int16_t* d_chan;        // device [n_kv_heads][row_elems]: K channel of each proxy element, -1 = padding
   int32_t* d_status;      // device status word (FASA_DEV_* bits)
+  int fused_cs;           // cluster size of the one-launch decode step, 0 = not available
+  size_t fused_smem;      // its dynamic shared memory
+  int use_fused;          // fasa_decode_step takes the one-launch kernel when it is available
   long long launches;     // kernels launched through this context
   char cuda_err[256];
 };
@@ -49,6 +52,13 @@ struct fasa_split_plan {
   int chunk;      // rows per split (multiple of 32)
 };
 fasa_split_plan fasa_plan_splits(const fasa_ctx* ctx, int n_upper);
+
+// One-launch decode step (fasa_fused.cu): plan at context creation, launch per step.
+int fasa_fused_plan(fasa_ctx* ctx);
+int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                          const void* proxy_k, const int32_t* seq_lens, int32_t budget,
+                          int32_t n_sel_max, float* scores, int32_t* idx, int32_t* n_sel,
+                          float* out, float* lse, cudaStream_t stream);
 
 static inline size_t fasa_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -1,0 +1,656 @@
+// One decode step in one launch: TIP scoring -> TopK-I -> FAC (Sec. 4.1-4.2, Eq. 6-7).
+//
+// One thread-block cluster per (batch, KV head) unit.  The CTAs of the cluster cut the unit's
+// cached tokens into contiguous slices and
+//   1. stream their slice of the proxy-K buffer once (16-byte loads, 8 in flight per thread),
+//      keep every token's selection key in shared memory and histogram its top 11 bits;
+//   2. find the budget-th largest key by an MSB-first radix select (11 + 11 + 10 bits): each
+//      pass needs one cluster barrier, after which every CTA reads the other CTAs' coarse and
+//      fine bin counts through distributed shared memory and locates the bin redundantly;
+//   3. write the selected positions in ascending order (ballot / prefix-sum compaction, equal
+//      keys lowest index first, so the result equals a stable sort);
+//   4. share the selected rows evenly, gather K/V rows by index with an online softmax, and
+//   5. merge the per-CTA partial results through distributed shared memory.
+// Scores, histograms and split-K partials never travel through HBM: the launch moves the
+// proxy rows of every token, the K/V rows of the selected tokens, q and the outputs.
+//
+// Every cluster barrier sits at the top level of the kernel and is reached by all threads of
+// all CTAs the same number of times, whatever the data; no thread waits on anything else.
+#include <cooperative_groups.h>
+
+#include "fasa_common.cuh"
+#include "fasa_score_core.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace {
+
+constexpr int kFT = 256;               // threads per CTA (two CTAs share an SM)
+constexpr int kFW = kFT / 32;          // warps per CTA
+constexpr int kFBins = 2048;           // bins of the widest radix pass
+constexpr int kFUnroll = 8;            // proxy loads in flight per thread
+constexpr int kPartStride = FASA_HEAD_DIM + 2;   // m, l, acc[128]
+constexpr int kCapMax = 22528;         // keys a CTA can hold (88 KB of shared memory)
+constexpr int kCapPair = 16384;        // ... and still leave room for a second CTA on the SM
+
+struct FusedParams {
+  const uint16_t* q;
+  const uint16_t* k;
+  const uint16_t* v;
+  const uint4* proxy;
+  const int32_t* seq_lens;
+  const int16_t* chan;
+  float* scores;           // nullable
+  int32_t* idx;
+  int32_t* n_sel;
+  float* out;
+  float* lse;              // nullable
+  int32_t* status;
+  int n_q_heads, n_kv_heads, group, max_len, chunks, n_sink, n_recent, budget, n_sel_max;
+  int64_t ksb, ksh, kst, vsb, vsh, vst;
+  float scale_log2;        // softmax_scale * log2(e)
+};
+
+__device__ __forceinline__ uint2 ld_stream_u2(const void* p) {
+  uint2 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
+  return r;
+}
+
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xffffffffu, v, o);
+    if (lane >= o) v += t;
+  }
+  return v;
+}
+
+// Among per-lane counts v (lane 0 first), finds the lane where the running sum reaches kth.
+// Returns true when found; *hit_lane and *residual (= kth minus the sum before that lane) are
+// then uniform over the warp.  *total is the sum over the warp.
+__device__ __forceinline__ bool warp_find_kth(uint32_t v, uint32_t kth, int lane, int* hit_lane,
+                                              uint32_t* residual, uint32_t* total) {
+  const uint32_t incl = warp_incl_scan(v, lane);
+  *total = __shfl_sync(0xffffffffu, incl, 31);
+  const uint32_t hits = __ballot_sync(0xffffffffu, incl >= kth);
+  if (hits == 0u) return false;
+  const int first = __ffs(hits) - 1;
+  const uint32_t before = __shfl_sync(0xffffffffu, incl - v, first);
+  *hit_lane = first;
+  *residual = kth - before;
+  return true;
+}
+
+// LPR = lanes per proxy row; GP = query heads padded to 4 or 8.
+template <int LPR, int GP>
+__global__ void __launch_bounds__(kFT, 2)
+fused_decode_kernel(const FusedParams p) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const int cs = (int)cluster.num_blocks();
+  const int crank = (int)cluster.block_rank();
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const int warp = tid >> 5;
+  const int u = blockIdx.y;
+  const int h = u % p.n_kv_heads;
+  const int b = u / p.n_kv_heads;
+
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ uint32_t s_coarse[2][kFBins / 32];
+  __shared__ uint32_t s_gather[16][kFBins / 32];   // remote counts, one row per cluster rank
+  __shared__ unsigned long long s_wcnt[kFW];
+  __shared__ unsigned long long s_tot;
+  __shared__ uint32_t s_bin, s_kth;
+  __shared__ __align__(16) float s_q[GP][FASA_HEAD_DIM];
+  __shared__ __align__(16) float s_part[GP][kPartStride + 2];
+  __shared__ __align__(16) float s_p[kFW][32];
+  __shared__ __align__(16) float s_al[kFW][GP];
+  __shared__ float s_m[kFW][GP];
+  __shared__ float s_l[kFW][GP];
+
+  // ---- slices -------------------------------------------------------------------------
+  const int len = clamp_len(p.seq_lens[b], p.max_len, p.status);
+  const int per = (((len + cs - 1) / cs) + 31) & ~31;          // <= the capacity the host sized
+  const int c0 = min(len, crank * per);
+  const int c1 = min(len, c0 + per);
+  const int nloc = c1 - c0;
+  const int cap = (((p.max_len + cs - 1) / cs) + 31) & ~31;
+  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw);
+  uint32_t* hist0 = keys + cap;
+  uint32_t* hist1 = hist0 + kFBins;
+
+  const long long k_budget =
+      p.budget > 0 ? (long long)p.budget : ((long long)(-p.budget) * len + 999) / 1000;
+  const int sink = min(len, p.n_sink);
+  const int n_forced = sink + min(p.n_recent, len - sink);
+  long long ktot_ll = min((long long)len, (long long)n_forced + k_budget);
+  if (ktot_ll > p.n_sel_max) {
+    ktot_ll = p.n_sel_max;
+    if (crank == 0 && tid == 0) atomicOr(p.status, FASA_DEV_NSEL_CLAMPED);
+  }
+  const uint32_t ktot = (uint32_t)ktot_ll;
+
+  for (int i = tid; i < 2 * kFBins; i += kFT) hist0[i] = 0u;
+  // query, scaled into the base-2 logit domain, for the attention phase
+  for (int i = tid; i < GP * (FASA_HEAD_DIM / 8); i += kFT) {
+    const int g = i / (FASA_HEAD_DIM / 8), c = (i % (FASA_HEAD_DIM / 8)) * 8;
+    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+    if (g < p.group)
+      w = *reinterpret_cast<const uint4*>(p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group + g) * FASA_HEAD_DIM + c);
+    const float2 f0 = bf16x2_to_f32x2(w.x), f1 = bf16x2_to_f32x2(w.y), f2 = bf16x2_to_f32x2(w.z), f3 = bf16x2_to_f32x2(w.w);
+    const float sc = p.scale_log2;
+    *reinterpret_cast<float4*>(&s_q[g][c]) = make_float4(f0.x * sc, f0.y * sc, f1.x * sc, f1.y * sc);
+    *reinterpret_cast<float4*>(&s_q[g][c + 4]) = make_float4(f2.x * sc, f2.y * sc, f3.x * sc, f3.y * sc);
+  }
+  __syncthreads();
+
+  // ---- 1. scoring stream -> keys + first histogram ------------------------------------------
+  {
+    constexpr int RPL = 32 / LPR;
+    constexpr int RPI = RPL * kFUnroll;
+    const int sub = lane & (LPR - 1);
+    const int grp = lane / LPR;
+    const bool live = sub < p.chunks;
+    const uint4* prow = p.proxy + (int64_t)u * p.max_len * p.chunks;
+    float* srow = p.scores ? p.scores + (int64_t)u * p.max_len : nullptr;
+
+    auto issue = [&](uint4 (&x)[kFUnroll], int base) {
+#pragma unroll
+      for (int i = 0; i < kFUnroll; ++i) {
+        const int row = base + i * RPL + grp;
+        x[i] = (live && row < c1) ? ld_stream_u4(prow + (int64_t)row * p.chunks + sub)
+                                  : make_uint4(0u, 0u, 0u, 0u);
+      }
+    };
+    const int stride = kFW * RPI;
+    int base = c0 + warp * RPI;
+    uint4 x[kFUnroll];
+    issue(x, base);
+    ScoreQ<false> sq;
+    load_score_q<false>(sq, p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM,
+                        p.chan + h * p.chunks * 8 + (live ? sub : 0) * 8, p.group, live);
+    while (base < c1) {
+      float sc[kFUnroll];
+#pragma unroll
+      for (int i = 0; i < kFUnroll; ++i) sc[i] = score_row<LPR, false>(sq, x[i], p.group);
+      if (base + stride < c1) issue(x, base + stride);   // next loads fly while keys are made
+#pragma unroll
+      for (int i = 0; i < kFUnroll; ++i) {
+        const int row = base + i * RPL + grp;
+        if (sub == 0 && row < c1) {
+          const uint32_t key = fasa_item_key(sc[i], row, len, p.n_sink, p.n_recent);
+          atomicAdd(&hist0[key >> 21], 1u);
+          keys[row - c0] = key;
+          if (srow) srow[row] = sc[i];
+        }
+      }
+      base += stride;
+    }
+  }
+  __syncthreads();
+
+  // ---- 2. radix select of the ktot-th largest key ------------------------------------------
+  uint32_t prefix = 0, kth = ktot;
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    const int bits = pass == 2 ? 10 : 11;
+    const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+    const int nb = 1 << bits;
+    const int ng = nb / 32;
+    uint32_t* buf = (pass & 1) ? hist1 : hist0;
+    uint32_t* coarse = s_coarse[pass & 1];
+    if (pass > 0) {
+      if (pass == 2) {
+        for (int i = tid; i < nb; i += kFT) buf[i] = 0u;
+        __syncthreads();
+      }
+      for (int i = tid * 4; i < nloc; i += kFT * 4) {
+        const uint4 kq = *reinterpret_cast<const uint4*>(&keys[i]);
+        const uint32_t kv[4] = {kq.x, kq.y, kq.z, kq.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (i + e < nloc && (kv[e] >> (shift + bits)) == prefix)
+            atomicAdd(&buf[(kv[e] >> shift) & (uint32_t)(nb - 1)], 1u);
+      }
+      __syncthreads();
+    }
+    {
+      // group sums: each warp reduces its kFBins/32/kFW groups side by side
+      constexpr int GPW = kFBins / 32 / kFW;
+      uint32_t v[GPW];
+#pragma unroll
+      for (int j = 0; j < GPW; ++j) {
+        const int g = warp + j * kFW;
+        v[j] = g < ng ? buf[g * 32 + lane] : 0u;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int j = 0; j < GPW; ++j) v[j] += __shfl_xor_sync(0xffffffffu, v[j], o);
+      if (lane == 0) {
+#pragma unroll
+        for (int j = 0; j < GPW; ++j)
+          if (warp + j * kFW < ng) coarse[warp + j * kFW] = v[j];
+      }
+    }
+    cluster.sync();   // barrier 1..3
+
+    // Every thread fetches a few of the other CTAs' coarse counts (all loads in flight at
+    // once); warp 0 adds them up and finds the group of 32 bins that holds the kth key.
+    for (int i = tid; i < ng * cs; i += kFT) {
+      const int r = i / ng, g = i % ng;
+      s_gather[r][g] = cluster.map_shared_rank(coarse, r)[g];
+    }
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t res = kth, tot = 0;
+      int hit = 0, group_id = -1;
+      for (int g0 = ng - 1; g0 >= 0 && group_id < 0; g0 -= 32) {   // groups, highest first
+        const int g = g0 - lane;
+        uint32_t v = 0;
+        for (int r = 0; r < cs; ++r) v += s_gather[r][g];
+        if (warp_find_kth(v, res, lane, &hit, &res, &tot)) group_id = g0 - hit;
+        else res -= tot;
+      }
+      if (group_id < 0) { group_id = 0; res = 1; }   // cannot happen: kth <= number of keys
+      if (lane == 0) { s_bin = (uint32_t)group_id; s_kth = res; }
+    }
+    __syncthreads();
+    const int group_id = (int)s_bin;
+    const uint32_t kth_in_group = s_kth;
+    __syncthreads();
+    // the 32 bins of that group, from every CTA
+    for (int i = tid; i < 32 * cs; i += kFT) {
+      const int r = i / 32, bl = i % 32;
+      s_gather[r][bl] = cluster.map_shared_rank(buf, r)[group_id * 32 + bl];
+    }
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t v = 0, res2 = kth_in_group, tot = 0;
+      int hit = 0;
+      for (int r = 0; r < cs; ++r) v += s_gather[r][31 - lane];   // lane 0 = highest bin
+      if (!warp_find_kth(v, kth_in_group, lane, &hit, &res2, &tot)) { hit = 31; res2 = 1; }
+      if (lane == 0) {
+        s_bin = (uint32_t)(group_id * 32 + 31 - hit);
+        s_kth = res2;
+      }
+    }
+    __syncthreads();
+    prefix = (prefix << bits) | s_bin;
+    kth = s_kth;
+    __syncthreads();
+  }
+  const uint32_t thr = prefix;
+  const uint32_t tie_quota = kth;
+
+  // ---- 3. ascending compaction ---------------------------------------------------------------
+  // A warp owns a contiguous run of keys and walks it 128 at a time, four consecutive keys
+  // per lane, so positions come out in index order.
+  const int wper = (((nloc + kFW - 1) / kFW) + 127) & ~127;
+  const int w0 = min(nloc, warp * wper);
+  const int w1 = min(nloc, w0 + wper);
+  {
+    uint32_t n_gt = 0, n_eq = 0;
+    for (int i = w0 + lane * 4; i < w1; i += 128) {
+      const uint4 kq = *reinterpret_cast<const uint4*>(&keys[i]);
+      const uint32_t kv[4] = {kq.x, kq.y, kq.z, kq.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool ok = i + e < w1;
+        n_gt += ok && kv[e] > thr;
+        n_eq += ok && kv[e] == thr;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      n_gt += __shfl_xor_sync(0xffffffffu, n_gt, o);
+      n_eq += __shfl_xor_sync(0xffffffffu, n_eq, o);
+    }
+    if (lane == 0) s_wcnt[warp] = ((unsigned long long)n_gt << 32) | n_eq;
+  }
+  __syncthreads();
+  unsigned long long before = 0;
+  {
+    unsigned long long all = 0;
+    for (int w = 0; w < kFW; ++w) {
+      const unsigned long long c = s_wcnt[w];
+      if (w < warp) before += c;
+      all += c;
+    }
+    if (tid == 0) s_tot = all;
+  }
+  cluster.sync();   // barrier 4
+  for (int r = 0; r < crank; ++r) before += *cluster.map_shared_rank(&s_tot, r);
+  {
+    uint32_t g_run = (uint32_t)(before >> 32), e_run = (uint32_t)before;
+    int32_t* out_idx = p.idx + (int64_t)u * p.n_sel_max;
+    for (int i0 = w0; i0 < w1; i0 += 128) {   // uniform trip count over the warp
+      const int i = i0 + lane * 4;
+      uint32_t kv[4] = {0u, 0u, 0u, 0u};
+      if (i < w1) {
+        const uint4 kq = *reinterpret_cast<const uint4*>(&keys[i]);
+        kv[0] = kq.x; kv[1] = kq.y; kv[2] = kq.z; kv[3] = kq.w;
+      }
+      uint32_t c_gt = 0, c_eq = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool ok = i + e < w1;
+        c_gt += ok && kv[e] > thr;
+        c_eq += ok && kv[e] == thr;
+      }
+      const uint32_t packed = c_gt | (c_eq << 16);          // at most 128 of each per step
+      if (!__any_sync(0xffffffffu, packed != 0u)) continue;   // nothing selected in these 128 keys
+      const uint32_t incl = warp_incl_scan(packed, lane);
+      const uint32_t excl = incl - packed;
+      uint32_t g_before = g_run + (excl & 0xffffu);
+      uint32_t e_before = e_run + (excl >> 16);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool ok = i + e < w1;
+        // (positions are < ktot by construction; the comparison keeps a write inside the
+        // list whatever the scores hold)
+        uint32_t pos = 0xffffffffu;
+        if (ok && kv[e] > thr) { pos = g_before + min(e_before, tie_quota); ++g_before; }
+        else if (ok && kv[e] == thr) { if (e_before < tie_quota) pos = g_before + e_before; ++e_before; }
+        if (pos < ktot) out_idx[pos] = c0 + i + e;
+      }
+      const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+      g_run += tot & 0xffffu;
+      e_run += tot >> 16;
+    }
+    if (crank == 0 && tid == 0) p.n_sel[u] = (int32_t)ktot;
+  }
+  cluster.sync();   // barrier 5: the index list is complete and visible to the whole cluster
+
+  // ---- 4. attention over this CTA's share of the selected rows -----------------------------
+  constexpr int R = 32 / GP;                                   // rows per warp batch
+  const int m_per = ((((int)ktot + cs - 1) / cs) + R - 1) / R * R;
+  const int a0 = min((int)ktot, crank * m_per);
+  const int a1 = min((int)ktot, a0 + m_per);
+  float2 acc[GP][2];
+#pragma unroll
+  for (int g = 0; g < GP; ++g) acc[g][0] = acc[g][1] = make_float2(0.f, 0.f);
+  float m_run = -INFINITY, l_run = 0.f;   // of head (lane % GP); replicated over the row lanes
+  {
+    const int32_t* irow = p.idx + (int64_t)u * p.n_sel_max;
+    const uint16_t* kbase = p.k + b * p.ksb + h * p.ksh + lane * 4;
+    const uint16_t* vbase = p.v + b * p.vsb + h * p.vsh + lane * 4;
+    const int my_g = lane % GP;
+    const int my_i = lane / GP;
+    for (int base = a0 + warp * R; base < a1; base += kFW * R) {
+      uint2 kk[R], vv[R];
+#pragma unroll
+      for (int i = 0; i < R; ++i) {
+        const int r = base + i;
+        if (r < a1) {
+          int tok = __ldcg(irow + r);
+          tok = min(max(tok, 0), p.max_len - 1);
+          kk[i] = ld_stream_u2(kbase + (int64_t)tok * p.kst);
+          vv[i] = ld_stream_u2(vbase + (int64_t)tok * p.vst);
+        } else {
+          kk[i] = make_uint2(0u, 0u);
+          vv[i] = make_uint2(0u, 0u);
+        }
+      }
+      // partial logits of R rows x GP heads over this lane's 4 channels
+      float part[32];
+#pragma unroll
+      for (int g = 0; g < GP; ++g) {
+        const float4 qg = *reinterpret_cast<const float4*>(&s_q[g][lane * 4]);
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+          const float2 k0 = bf16x2_to_f32x2(kk[i].x), k1 = bf16x2_to_f32x2(kk[i].y);
+          part[i * GP + g] = qg.x * k0.x + qg.y * k0.y + qg.z * k1.x + qg.w * k1.y;
+        }
+      }
+      // transposing reduction over the 32 lanes: lane L ends with the full sum of value L
+      float logit;
+      {
+        float p16[16], p8[8], p4[4], p2[2];
+        const bool u16 = (lane & 16) != 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float send = u16 ? part[i] : part[i + 16];
+          const float keep = u16 ? part[i + 16] : part[i];
+          p16[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+        }
+        const bool u8 = (lane & 8) != 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float send = u8 ? p16[i] : p16[i + 8];
+          const float keep = u8 ? p16[i + 8] : p16[i];
+          p8[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+        }
+        const bool u4 = (lane & 4) != 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float send = u4 ? p8[i] : p8[i + 4];
+          const float keep = u4 ? p8[i + 4] : p8[i];
+          p4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+        }
+        const bool u2 = (lane & 2) != 0;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const float send = u2 ? p4[i] : p4[i + 2];
+          const float keep = u2 ? p4[i + 2] : p4[i];
+          p2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+        }
+        const bool u1 = (lane & 1) != 0;
+        const float send = u1 ? p2[0] : p2[1];
+        const float keep = u1 ? p2[1] : p2[0];
+        logit = keep + __shfl_xor_sync(0xffffffffu, send, 1);
+      }
+      if (!(base + my_i < a1 && my_g < p.group)) logit = -INFINITY;
+      float bmax = logit;
+#pragma unroll
+      for (int o = GP; o < 32; o <<= 1) bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, o));
+      const float m_new = fmaxf(m_run, bmax);
+      const float m_safe = m_new == -INFINITY ? 0.f : m_new;
+      const float alpha = exp2f(m_run - m_safe);
+      const float pr = exp2f(logit - m_safe);
+      l_run = l_run * alpha + pr;
+      m_run = m_new;
+      s_p[warp][lane] = pr;
+      if (lane < GP) s_al[warp][lane] = alpha;
+      __syncwarp();
+#pragma unroll
+      for (int g = 0; g < GP; ++g) {
+        const float a = s_al[warp][g];
+        const float2 a2 = make_float2(a, a);
+        acc[g][0] = __ffma2_rn(acc[g][0], a2, make_float2(0.f, 0.f));
+        acc[g][1] = __ffma2_rn(acc[g][1], a2, make_float2(0.f, 0.f));
+      }
+#pragma unroll
+      for (int i = 0; i < R; ++i) {
+        const float2 v0 = bf16x2_to_f32x2(vv[i].x), v1 = bf16x2_to_f32x2(vv[i].y);
+#pragma unroll
+        for (int g = 0; g < GP; ++g) {
+          const float pg = s_p[warp][i * GP + g];
+          const float2 p2 = make_float2(pg, pg);
+          acc[g][0] = __ffma2_rn(p2, v0, acc[g][0]);
+          acc[g][1] = __ffma2_rn(p2, v1, acc[g][1]);
+        }
+      }
+      __syncwarp();
+    }
+    // row lanes of a head add their partial sums of probabilities
+#pragma unroll
+    for (int o = GP; o < 32; o <<= 1) l_run += __shfl_xor_sync(0xffffffffu, l_run, o);
+  }
+
+  // ---- 5. combine the warps of this CTA, then the CTAs of the cluster ------------------------
+  // The warp accumulators reuse the key / histogram area: every read of it, local or remote,
+  // happened before barrier 4.
+  float* s_acc = reinterpret_cast<float*>(smem_raw);           // [kFW][GP][128]
+  if (lane < GP) {
+    s_m[warp][lane] = m_run;
+    s_l[warp][lane] = l_run;
+  }
+#pragma unroll
+  for (int g = 0; g < GP; ++g)
+    *reinterpret_cast<float4*>(&s_acc[((warp * GP) + g) * FASA_HEAD_DIM + lane * 4]) =
+        make_float4(acc[g][0].x, acc[g][0].y, acc[g][1].x, acc[g][1].y);
+  __syncthreads();
+  for (int o = tid; o < GP * FASA_HEAD_DIM; o += kFT) {
+    const int g = o / FASA_HEAD_DIM, c = o % FASA_HEAD_DIM;
+    float mx = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kFW; ++w) mx = fmaxf(mx, s_m[w][g]);
+    float a = 0.f, l = 0.f;
+#pragma unroll
+    for (int w = 0; w < kFW; ++w) {
+      const float ms = s_m[w][g];
+      const float wt = ms == -INFINITY ? 0.f : exp2f(ms - mx);
+      a += wt * s_acc[((w * GP) + g) * FASA_HEAD_DIM + c];
+      l += wt * s_l[w][g];
+    }
+    s_part[g][2 + c] = a;
+    if (c == 0) {
+      s_part[g][0] = mx;
+      s_part[g][1] = l;
+    }
+  }
+  cluster.sync();   // barrier 6: every CTA's partial result is in its shared memory
+
+  {
+    const int n_out = p.group * FASA_HEAD_DIM;
+    const int per_o = (n_out + cs - 1) / cs;
+    for (int t = tid; t < per_o; t += kFT) {
+      const int o = crank * per_o + t;
+      if (o >= n_out) break;
+      const int g = o / FASA_HEAD_DIM, c = o % FASA_HEAD_DIM;
+      float mx = -INFINITY;
+      for (int r = 0; r < cs; ++r) mx = fmaxf(mx, cluster.map_shared_rank(&s_part[g][0], r)[0]);
+      float a = 0.f, l = 0.f;
+      for (int r = 0; r < cs; ++r) {
+        const float* pr = cluster.map_shared_rank(&s_part[g][0], r);
+        const float ms = pr[0];
+        const float wt = ms == -INFINITY ? 0.f : exp2f(ms - mx);
+        a += wt * pr[2 + c];
+        l += wt * pr[1];
+      }
+      const int64_t hq = (int64_t)b * p.n_q_heads + (int64_t)h * p.group + g;
+      p.out[hq * FASA_HEAD_DIM + c] = l > 0.f ? a / l : 0.f;
+      if (p.lse && c == 0) p.lse[hq] = l > 0.f ? (mx + log2f(l)) * 0.6931471805599453f : -INFINITY;
+    }
+  }
+  cluster.sync();   // barrier 7: no CTA leaves while a peer can still read its shared memory
+}
+
+struct FusedPlan {
+  int cs;        // cluster size, 0 = the fused kernel cannot take this configuration
+  int cap;       // keys per CTA
+  size_t smem;   // dynamic shared memory
+};
+
+template <int GP>
+size_t fused_smem_bytes(int cap) {
+  const size_t sel = (size_t)cap * 4 + 2 * kFBins * 4;
+  const size_t att = (size_t)kFW * GP * FASA_HEAD_DIM * 4;
+  return sel > att ? sel : att;
+}
+
+using FusedFn = void (*)(const FusedParams);
+
+template <int GP>
+FusedFn fused_fn_lpr(int chunks) {
+  if (chunks <= 1) return fused_decode_kernel<1, GP>;
+  if (chunks <= 2) return fused_decode_kernel<2, GP>;
+  if (chunks <= 4) return fused_decode_kernel<4, GP>;
+  if (chunks <= 8) return fused_decode_kernel<8, GP>;
+  return fused_decode_kernel<16, GP>;
+}
+
+}  // namespace
+
+// Decides once per context whether and how the fused kernel runs: the smallest cluster whose
+// CTAs can hold their slice of max_len keys, grown while that leaves SMs idle, then shrunk
+// again if the device cannot co-schedule a cluster of that size.
+int fasa_fused_plan(fasa_ctx* ctx) {
+  const fasa_config_t& c = ctx->cfg;
+  ctx->fused_cs = 0;
+  ctx->fused_smem = 0;
+  if (c.group_reduce != 0) return 0;          // the max reduction takes the three-kernel path
+  const int units = c.batch * c.n_kv_heads;
+  const bool gp8 = ctx->group > 4;
+  FusedFn fn = gp8 ? fused_fn_lpr<8>(ctx->chunks) : fused_fn_lpr<4>(ctx->chunks);
+  auto cap_of = [&](int cs) { return (((c.max_len + cs - 1) / cs) + 31) & ~31; };
+  // Two CTAs per SM can be resident; a cluster is doubled while the whole grid still fits
+  // in one wave of them and every CTA keeps at least 512 tokens.
+  const int slots = 2 * ctx->n_sm;
+  int want = 1;
+  while (want < 16 && cap_of(want) > kCapPair) want *= 2;
+  while (want < 16 && units * want * 2 <= slots && c.max_len / (2 * want) >= 512) want *= 2;
+  if (cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+    cudaGetLastError();
+    if (want > 8) want = 8;
+  }
+  for (int cs = want; cs >= 1; cs /= 2) {
+    const int cap = cap_of(cs);
+    if (cap > kCapMax) break;
+    const size_t smem = gp8 ? fused_smem_bytes<8>(cap) : fused_smem_bytes<4>(cap);
+    if (cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+      cudaGetLastError();
+      continue;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)cs, (unsigned)units, 1);
+    cfg.blockDim = dim3(kFT, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&n_clusters, (const void*)fn, &cfg) != cudaSuccess || n_clusters < 1) {
+      cudaGetLastError();
+      continue;
+    }
+    ctx->fused_cs = cs;
+    ctx->fused_smem = smem;
+    return cs;
+  }
+  return 0;
+}
+
+int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                          const void* proxy_k, const int32_t* seq_lens, int32_t budget,
+                          int32_t n_sel_max, float* scores, int32_t* idx, int32_t* n_sel,
+                          float* out, float* lse, cudaStream_t stream) {
+  const fasa_config_t& c = ctx->cfg;
+  FusedParams p;
+  p.q = (const uint16_t*)q; p.k = (const uint16_t*)k_cache; p.v = (const uint16_t*)v_cache;
+  p.proxy = (const uint4*)proxy_k; p.seq_lens = seq_lens; p.chan = ctx->d_chan;
+  p.scores = scores; p.idx = idx; p.n_sel = n_sel; p.out = out; p.lse = lse; p.status = ctx->d_status;
+  p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group; p.max_len = c.max_len;
+  p.chunks = ctx->chunks; p.n_sink = c.n_sink; p.n_recent = c.n_recent; p.budget = budget;
+  p.n_sel_max = n_sel_max;
+  p.ksb = c.k_stride_b; p.ksh = c.k_stride_h; p.kst = c.k_stride_t;
+  p.vsb = c.v_stride_b; p.vsh = c.v_stride_h; p.vst = c.v_stride_t;
+  p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
+  const bool gp8 = ctx->group > 4;
+  FusedFn fn = gp8 ? fused_fn_lpr<8>(ctx->chunks) : fused_fn_lpr<4>(ctx->chunks);
+
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)ctx->fused_cs, (unsigned)(c.batch * c.n_kv_heads), 1);
+  cfg.blockDim = dim3(kFT, 1, 1);
+  cfg.dynamicSmemBytes = ctx->fused_smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)ctx->fused_cs;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, fn, p);
+  ctx->launches += 1;
+  FASA_CUDA_TRY(ctx, e);
+  return FASA_OK;
+}

@@ -3,6 +3,7 @@
 // are contiguous across the warp, each thread keeps UNROLL loads in flight, and the lanes
 // that share a row combine their partial sums with xor-shuffles.
 #include "fasa_common.cuh"
+#include "fasa_score_core.cuh"
 
 namespace {
 
@@ -19,82 +20,60 @@ fc_score_kernel(const uint16_t* __restrict__ q, const uint4* __restrict__ proxy,
                 int n_kv_heads, int group, int max_len, int chunks, int rows_per_cta) {
   constexpr int RPL = 32 / LPR;                 // rows covered by one warp-wide load
   constexpr int RPI = RPL * kScoreUnroll;       // rows per warp iteration
-  constexpr int NG = MAXRED ? FASA_MAX_GROUP : 1;
 
   const int u = blockIdx.y;
   const int h = u % n_kv_heads;
   const int b = u / n_kv_heads;
-  const int len = clamp_len(seq_lens[b], max_len, status);
   const int cta_row0 = blockIdx.x * rows_per_cta;
-  if (cta_row0 >= len) return;
-  const int cta_row1 = min(len, cta_row0 + rows_per_cta);
-
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int sub = lane & (LPR - 1);             // which 16-byte chunk of the row
   const int grp = lane / LPR;                   // which row of the warp-wide load
   const bool live = sub < chunks;
+  const uint4* prow = proxy + (int64_t)u * max_len * chunks;
 
-  // This lane's 8 query values (summed over the group, or kept per head for MAXRED).
-  float2 qv[NG][4];
+  // The first batch of proxy loads is issued before anything else is known: rows up to
+  // max_len are allocated, so reading past the sequence length is harmless, and the loads of
+  // the length, the channel table and the query overlap with the stream instead of
+  // preceding it.
+  const int alloc_row1 = min(max_len, cta_row0 + rows_per_cta);
+  int base = cta_row0 + warp * RPI;
+  uint4 x[kScoreUnroll];
 #pragma unroll
-  for (int g = 0; g < NG; ++g)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) qv[g][e] = make_float2(0.f, 0.f);
-  if (live) {
-    const int16_t* ch = chan + h * chunks * 8 + sub * 8;
-    const uint16_t* qb = q + ((int64_t)b * n_q_heads + (int64_t)h * group) * FASA_HEAD_DIM;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int c0 = ch[2 * e], c1 = ch[2 * e + 1];
-      for (int g = 0; g < group; ++g) {
-        const float x = c0 >= 0 ? bf16_bits_to_f32(qb[g * FASA_HEAD_DIM + c0]) : 0.f;
-        const float y = c1 >= 0 ? bf16_bits_to_f32(qb[g * FASA_HEAD_DIM + c1]) : 0.f;
-        if (MAXRED) {
-#pragma unroll
-          for (int gg = 0; gg < NG; ++gg)
-            if (gg == g) qv[gg][e] = make_float2(x, y);
-        } else {
-          qv[0][e].x += x;
-          qv[0][e].y += y;
-        }
-      }
-    }
+  for (int i = 0; i < kScoreUnroll; ++i) {
+    const int row = base + i * RPL + grp;
+    x[i] = (live && row < alloc_row1) ? ld_stream_u4(prow + (int64_t)row * chunks + sub)
+                                      : make_uint4(0u, 0u, 0u, 0u);
   }
 
-  const uint4* prow = proxy + (int64_t)u * max_len * chunks;
+  const int len = clamp_len(seq_lens[b], max_len, status);
+  if (cta_row0 >= len) return;
+  const int cta_row1 = min(len, cta_row0 + rows_per_cta);
+
+  ScoreQ<MAXRED> sq;
+  load_score_q<MAXRED>(sq, q + ((int64_t)b * n_q_heads + (int64_t)h * group) * FASA_HEAD_DIM,
+                       chan + h * chunks * 8 + (live ? sub : 0) * 8, group, live);
   float* srow = scores + (int64_t)u * max_len;
 
-  for (int base = cta_row0 + warp * RPI; base < cta_row1; base += (kScoreThreads / 32) * RPI) {
-    uint4 x[kScoreUnroll];
+  while (base < cta_row1) {
+    float s[kScoreUnroll];
 #pragma unroll
-    for (int i = 0; i < kScoreUnroll; ++i) {
-      const int row = base + i * RPL + grp;
-      x[i] = (live && row < cta_row1) ? ld_stream_u4(prow + (int64_t)row * chunks + sub)
-                                      : make_uint4(0u, 0u, 0u, 0u);
-    }
+    for (int i = 0; i < kScoreUnroll; ++i) s[i] = score_row<LPR, MAXRED>(sq, x[i], group);
+    const int next = base + (kScoreThreads / 32) * RPI;
+    if (next < cta_row1) {
 #pragma unroll
-    for (int i = 0; i < kScoreUnroll; ++i) {
-      float s;
-      if (!MAXRED) {
-        s = dot8(qv[0], x[i]);
-#pragma unroll
-        for (int o = LPR / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      } else {
-        s = -INFINITY;
-#pragma unroll
-        for (int g = 0; g < NG; ++g) {
-          if (g < group) {
-            float sg = dot8(qv[g], x[i]);
-#pragma unroll
-            for (int o = LPR / 2; o > 0; o >>= 1) sg += __shfl_xor_sync(0xffffffffu, sg, o);
-            s = fmaxf(s, sg);
-          }
-        }
+      for (int i = 0; i < kScoreUnroll; ++i) {
+        const int row = next + i * RPL + grp;
+        x[i] = (live && row < cta_row1) ? ld_stream_u4(prow + (int64_t)row * chunks + sub)
+                                        : make_uint4(0u, 0u, 0u, 0u);
       }
-      const int row = base + i * RPL + grp;
-      if (sub == 0 && row < cta_row1) srow[row] = s + 0.0f;  // -0 becomes +0
     }
+#pragma unroll
+    for (int i = 0; i < kScoreUnroll; ++i) {
+      const int row = base + i * RPL + grp;
+      if (sub == 0 && row < cta_row1) srow[row] = s[i];
+    }
+    base = next;
   }
 }
 

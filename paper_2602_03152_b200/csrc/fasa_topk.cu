@@ -12,6 +12,7 @@
 #include <cooperative_groups.h>
 
 #include "fasa_common.cuh"
+#include "fasa_score_core.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -21,18 +22,6 @@ constexpr int kTopkThreads = 1024;
 constexpr int kTopkItems = 16;                         // keys a thread can hold
 constexpr int kTopkCtaCap = kTopkThreads * kTopkItems;  // 16384 scores per CTA in registers
 constexpr int kMaxBins = 2048;
-
-__device__ __forceinline__ uint32_t order_key(float f) {
-  uint32_t u = __float_as_uint(f);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
-// Forced positions outrank every score; scores are capped just below them.
-__device__ __forceinline__ uint32_t item_key(float s, int j, int len, int n_sink, int n_recent) {
-  if (j < n_sink || j >= len - n_recent) return 0xffffffffu;
-  uint32_t k = order_key(s);
-  return k == 0xffffffffu ? 0xfffffffeu : k;
-}
 
 // Block-wide inclusive scan of a 64-bit value (1024 threads).
 __device__ __forceinline__ unsigned long long block_scan_incl(unsigned long long v,
@@ -122,7 +111,7 @@ topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ seq_le
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const bool ok = (i < ipt) && (j + e < c1);
-        keys[i + e] = ok ? item_key(s[e], j + e, len, n_sink, n_recent) : 0u;
+        keys[i + e] = ok ? fasa_item_key(s[e], j + e, len, n_sink, n_recent) : 0u;
         vmask |= ok ? (1u << (i + e)) : 0u;
       }
     }
@@ -137,7 +126,7 @@ topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ seq_le
     } else {
       for (int i = 0; i < ipt; ++i) {
         const int j = j0 + i;
-        if (j < c1) f(item_key(srow[j], j, len, n_sink, n_recent), j);
+        if (j < c1) f(fasa_item_key(srow[j], j, len, n_sink, n_recent), j);
       }
     }
   };

@@ -43,12 +43,27 @@ class Run:
     def build_proxy(self):
         self.fasa.proxy_build(self.k, self.proxy, self.seq_lens)
 
-    def step(self, budget=None):
+    def reset_outputs(self):
+        self.scores.fill_(SENTINEL)
+        self.idx.fill_(-7)
+        self.n_sel.fill_(-7)
+        self.out.fill_(SENTINEL)
+        self.lse.fill_(SENTINEL)
+
+    def step(self, budget=None, fused=False):
+        """The three calls one after another, or fasa_decode_step as one cluster kernel."""
         budget = self.w.budget if budget is None else budget
         f = self.fasa
-        f.fc_score(self.q, self.proxy, self.seq_lens, self.scores)
-        f.topk(self.scores, self.seq_lens, budget, self.idx, self.n_sel, self.ws)
-        f.sparse_decode_attn(self.q, self.k, self.v, self.idx, self.n_sel, self.out, self.ws, self.lse)
+        if fused:
+            assert f.step_cluster_size() > 0, "the one-launch step is not available for this configuration"
+            n0 = f.launch_count()
+            f.decode_step(self.q, self.k, self.v, self.proxy, self.seq_lens, budget, self.scores, self.idx,
+                          self.n_sel, self.out, None, self.lse)
+            assert f.launch_count() == n0 + 1
+        else:
+            f.fc_score(self.q, self.proxy, self.seq_lens, self.scores)
+            f.topk(self.scores, self.seq_lens, budget, self.idx, self.n_sel, self.ws)
+            f.sparse_decode_attn(self.q, self.k, self.v, self.idx, self.n_sel, self.out, self.ws, self.lse)
         torch.cuda.synchronize()
 
     def dense_step(self):

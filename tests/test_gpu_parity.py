@@ -19,22 +19,39 @@ C = synth.CONFIGS
 
 
 def _full_check(r: Run, budget=None, dense=True):
+    """Checks the three separate calls against the oracle, then the one-launch step (where the
+    configuration has one) against the oracle and against the separate calls."""
     r.build_proxy()
-    r.step(budget)
     if dense:
         r.dense_step()
-    h = r.host()
-    rep = parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
-                            n_sel=h["n_sel"], out=h["out"], dense_out=h["dense"] if dense else None,
-                            what=r.w.name, **r.oracle_kwargs(budget))
-    # rows at and past the sequence length are never written
-    for b in range(r.w.batch):
-        L = int(h["seq_lens"][b])
-        assert np.all(h["scores"][b, :, L:] == SENTINEL)
-        for hh in range(r.w.n_kv_heads):
-            assert np.all(h["idx"][b, hh, int(h["n_sel"][b, hh]):] == -7)
-    assert r.fasa.device_status() == 0
-    return rep, h
+    first = None
+    for fused in (False, True):
+        if fused and r.fasa.step_cluster_size() == 0:
+            assert r.w.group_reduce == 1
+            break
+        r.reset_outputs()
+        r.step(budget, fused=fused)
+        h = r.host()
+        rep = parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
+                                n_sel=h["n_sel"], out=h["out"], dense_out=h["dense"] if dense and not fused else None,
+                                what=r.w.name + (" fused" if fused else ""), **r.oracle_kwargs(budget))
+        # rows at and past the sequence length are never written
+        for b in range(r.w.batch):
+            L = int(h["seq_lens"][b])
+            assert np.all(h["scores"][b, :, L:] == SENTINEL)
+            for hh in range(r.w.n_kv_heads):
+                assert np.all(h["idx"][b, hh, int(h["n_sel"][b, hh]):] == -7)
+        assert r.fasa.device_status() == 0
+        if not fused:
+            first = (rep, h)
+        else:
+            h0 = first[1]
+            assert np.array_equal(h["scores"], h0["scores"]) and np.array_equal(h["idx"], h0["idx"])
+            assert np.array_equal(h["n_sel"], h0["n_sel"])
+            assert np.abs(h["out"] - h0["out"]).max() <= 1e-4
+            fin = np.isfinite(h0["lse"])
+            assert np.array_equal(np.isfinite(h["lse"]), fin) and np.abs(h["lse"][fin] - h0["lse"][fin]).max() <= 1e-4
+    return first
 
 
 def test_config0_full_size():
@@ -158,11 +175,13 @@ def test_results_are_deterministic():
     w = C["c2"].replace(batch=2, max_len=5000, len_lo=3000, len_hi=5000, budget=300)
     r = Run(w)
     r.build_proxy()
-    r.step(); r.dense_step()
-    a = [x.clone() for x in (r.scores, r.idx, r.n_sel, r.out, r.dense)]
-    r.step(); r.dense_step()
-    for x, y in zip(a, (r.scores, r.idx, r.n_sel, r.out, r.dense)):
-        assert torch.equal(x, y)
+    for fused in (False, True):
+        r.step(fused=fused); r.dense_step()
+        a = [x.clone() for x in (r.scores, r.idx, r.n_sel, r.out, r.dense)]
+        r.reset_outputs()
+        r.step(fused=fused); r.dense_step()
+        for x, y in zip(a, (r.scores, r.idx, r.n_sel, r.out, r.dense)):
+            assert torch.equal(x, y)
 
 
 def test_decode_step_equals_separate_calls_and_host_variant():
@@ -175,8 +194,15 @@ def test_decode_step_equals_separate_calls_and_host_variant():
         x.fill_(SENTINEL)
     r.fasa.decode_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel, r.out, r.ws)
     torch.cuda.synchronize()
-    for x, y in zip(ref, (r.scores, r.idx, r.n_sel, r.out)):
+    for x, y in zip(ref[:3], (r.scores, r.idx, r.n_sel)):
         assert torch.equal(x, y)
+    assert float((ref[3] - r.out).abs().max()) <= 1e-4      # another split of the rows: fp32 rounding only
+    r.fasa.set_step_mode(0)
+    r.out.fill_(SENTINEL)
+    r.fasa.decode_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel, r.out, r.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(ref[3], r.out)                        # mode 0 is the three calls themselves
+    r.fasa.set_step_mode(1)
     # host variant: append one token, then the same step; compare with the oracle on the grown cache
     s = synth.make_step_inputs(w, 0, "cpu")
     stage = torch.empty(r.fasa.stage_bytes(), dtype=torch.uint8, device="cuda")
@@ -282,9 +308,11 @@ def test_device_status_bits_instead_of_faults():
     assert r.seq_lens.cpu().tolist() == [128]
     # a length beyond max_len is clamped
     r.seq_lens.fill_(100000)
-    r.step()
-    assert r.fasa.device_status() & binding.DEV_LEN_CLAMPED
-    assert int(r.n_sel[0, 0]) == 16 + 68
+    for fused in (False, True):
+        r.reset_outputs()
+        r.step(fused=fused)
+        assert r.fasa.device_status() & binding.DEV_LEN_CLAMPED
+        assert int(r.n_sel[0, 0]) == 16 + 68
     # an out-of-range index is clamped to row 0, n_sel beyond the list to its capacity
     r.seq_lens.fill_(128)
     r.idx.fill_(10 ** 6)
@@ -299,6 +327,9 @@ def test_device_status_bits_instead_of_faults():
     assert r.fasa.device_status() & binding.DEV_NSEL_CLAMPED
     assert r.n_sel.cpu().tolist() == [[10, 10]]
     assert r.fasa.device_status() == 0
+    r.fasa.decode_step(r.q, r.k, r.v, r.proxy, r.seq_lens, 50, None, small, r.n_sel, r.out)
+    assert r.fasa.device_status() & binding.DEV_NSEL_CLAMPED
+    assert r.n_sel.cpu().tolist() == [[10, 10]]
 
 
 # ------------------------------------------------------------------ top-k alone ----
@@ -377,8 +408,11 @@ def test_config4_point_full_length_sampled_units():
     w = C["c4"].replace(batch=2, n_q_heads=16, n_kv_heads=4, budget=2048, n_dom=32)
     r = Run(w)
     r.build_proxy()
-    r.step(); r.dense_step()
-    h = r.host()
-    parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
-                      n_sel=h["n_sel"], out=h["out"], dense_out=h["dense"], units=[(0, 0), (1, 3), (1, 1)],
-                      what="c4", **r.oracle_kwargs())
+    r.dense_step()
+    for fused in (False, True):
+        r.reset_outputs()
+        r.step(fused=fused)
+        h = r.host()
+        parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
+                          n_sel=h["n_sel"], out=h["out"], dense_out=h["dense"], units=[(0, 0), (1, 3), (1, 1)],
+                          what="c4", **r.oracle_kwargs())
