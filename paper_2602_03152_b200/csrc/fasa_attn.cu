@@ -110,23 +110,25 @@ decode_attn_kernel(const AttnParams p) {
   // 32 lanes); a half-warp whose batch starts past r1 runs it fully masked.
   for (int wbase = r0 + warp * kWarpRows; wbase < r1; wbase += (kAttnThreads / 32) * kWarpRows) {
     const int base = wbase + (HWS == 1 ? hw * kRB : 0);
+    // all row indices first, then all row loads, so that no load waits on a previous row
+    int tok[kRB];
+#pragma unroll
+    for (int i = 0; i < kRB; ++i) {
+      const int r = base + i;
+      tok[i] = SPARSE ? (r < r1 ? __ldg(irow + r) : 0) : r;
+    }
     uint4 kk[kRB], vv[kRB];
 #pragma unroll
     for (int i = 0; i < kRB; ++i) {
       const int r = base + i;
-      int tok = 0;
       if (r < r1) {
-        if (SPARSE) {
-          tok = __ldg(irow + r);
-          if (tok < 0 || tok >= p.max_len) {
-            atomicOr(p.status, FASA_DEV_IDX_CLAMPED);
-            tok = 0;
-          }
-        } else {
-          tok = r;
+        int t = tok[i];
+        if (SPARSE && (t < 0 || t >= p.max_len)) {
+          atomicOr(p.status, FASA_DEV_IDX_CLAMPED);
+          t = 0;
         }
-        kk[i] = ld_stream_u4(kbase + (int64_t)tok * p.kst);
-        vv[i] = ld_stream_u4(vbase + (int64_t)tok * p.vst);
+        kk[i] = ld_stream_u4(kbase + (int64_t)t * p.kst);
+        vv[i] = ld_stream_u4(vbase + (int64_t)t * p.vst);
       } else {
         kk[i] = make_uint4(0u, 0u, 0u, 0u);
         vv[i] = make_uint4(0u, 0u, 0u, 0u);

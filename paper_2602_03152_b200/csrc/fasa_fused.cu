@@ -101,7 +101,7 @@ fused_decode_kernel(const FusedParams p) {
   __shared__ uint32_t s_gather[16][kFBins / 32];   // remote counts, one row per cluster rank
   __shared__ unsigned long long s_wcnt[kFW];
   __shared__ unsigned long long s_tot;
-  __shared__ uint32_t s_bin, s_kth;
+  __shared__ uint32_t s_bin, s_kth, s_cnt;
   __shared__ __align__(16) float s_q[GP][FASA_HEAD_DIM];
   __shared__ __align__(16) float s_part[GP][kPartStride + 2];
   __shared__ __align__(16) float s_p[kFW][32];
@@ -191,7 +191,11 @@ fused_decode_kernel(const FusedParams p) {
   __syncthreads();
 
   // ---- 2. radix select of the ktot-th largest key ------------------------------------------
-  uint32_t prefix = 0, kth = ktot;
+  // `done` (the bin that holds the kth key is needed whole, so its remaining bits do not
+  // matter) is computed from cluster-wide sums and is the same in every CTA; the barrier is
+  // taken in every pass regardless.
+  uint32_t prefix = 0, kth = ktot, thr = 0, tie_quota = 0;
+  bool done = false;
 #pragma unroll 1
   for (int pass = 0; pass < 3; ++pass) {
     const int bits = pass == 2 ? 10 : 11;
@@ -200,7 +204,7 @@ fused_decode_kernel(const FusedParams p) {
     const int ng = nb / 32;
     uint32_t* buf = (pass & 1) ? hist1 : hist0;
     uint32_t* coarse = s_coarse[pass & 1];
-    if (pass > 0) {
+    if (pass > 0 && !done) {
       if (pass == 2) {
         for (int i = tid; i < nb; i += kFT) buf[i] = 0u;
         __syncthreads();
@@ -215,7 +219,7 @@ fused_decode_kernel(const FusedParams p) {
       }
       __syncthreads();
     }
-    {
+    if (!done) {
       // group sums: each warp reduces its kFBins/32/kFW groups side by side
       constexpr int GPW = kFBins / 32 / kFW;
       uint32_t v[GPW];
@@ -235,6 +239,7 @@ fused_decode_kernel(const FusedParams p) {
       }
     }
     cluster.sync();   // barrier 1..3
+    if (done) continue;
 
     // Every thread fetches a few of the other CTAs' coarse counts (all loads in flight at
     // once); warp 0 adds them up and finds the group of 32 bins that holds the kth key.
@@ -271,22 +276,31 @@ fused_decode_kernel(const FusedParams p) {
       int hit = 0;
       for (int r = 0; r < cs; ++r) v += s_gather[r][31 - lane];   // lane 0 = highest bin
       if (!warp_find_kth(v, kth_in_group, lane, &hit, &res2, &tot)) { hit = 31; res2 = 1; }
+      const uint32_t in_bin = __shfl_sync(0xffffffffu, v, hit);
       if (lane == 0) {
         s_bin = (uint32_t)(group_id * 32 + 31 - hit);
         s_kth = res2;
+        s_cnt = in_bin;
       }
     }
     __syncthreads();
     prefix = (prefix << bits) | s_bin;
     kth = s_kth;
+    if (s_cnt == kth && pass < 2) {   // every key of this bin is selected
+      thr = prefix << shift;
+      tie_quota = 0xffffffffu;
+      done = true;
+    }
     __syncthreads();
   }
-  const uint32_t thr = prefix;
-  const uint32_t tie_quota = kth;
+  if (!done) {
+    thr = prefix;
+    tie_quota = kth;
+  }
 
   // ---- 3. ascending compaction ---------------------------------------------------------------
-  // A warp owns a contiguous run of keys and walks it 128 at a time, four consecutive keys
-  // per lane, so positions come out in index order.
+  // A warp owns a contiguous run of keys and walks it 128 at a time (four rows of 32
+  // consecutive keys, one key per lane and row), so positions come out in index order.
   const int wper = (((nloc + kFW - 1) / kFW) + 127) & ~127;
   const int w0 = min(nloc, warp * wper);
   const int w1 = min(nloc, w0 + wper);
@@ -321,43 +335,45 @@ fused_decode_kernel(const FusedParams p) {
     if (tid == 0) s_tot = all;
   }
   cluster.sync();   // barrier 4
-  for (int r = 0; r < crank; ++r) before += *cluster.map_shared_rank(&s_tot, r);
+  {
+    // totals of the lower-ranked CTAs, one per lane, fetched side by side
+    unsigned long long t = lane < crank ? *cluster.map_shared_rank(&s_tot, lane) : 0ull;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    before += t;
+  }
   {
     uint32_t g_run = (uint32_t)(before >> 32), e_run = (uint32_t)before;
     int32_t* out_idx = p.idx + (int64_t)u * p.n_sel_max;
+    const uint32_t lt = (1u << lane) - 1u;
     for (int i0 = w0; i0 < w1; i0 += 128) {   // uniform trip count over the warp
-      const int i = i0 + lane * 4;
-      uint32_t kv[4] = {0u, 0u, 0u, 0u};
-      if (i < w1) {
-        const uint4 kq = *reinterpret_cast<const uint4*>(&keys[i]);
-        kv[0] = kq.x; kv[1] = kq.y; kv[2] = kq.z; kv[3] = kq.w;
-      }
-      uint32_t c_gt = 0, c_eq = 0;
+      uint32_t kv[4];
+      bool ok[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const bool ok = i + e < w1;
-        c_gt += ok && kv[e] > thr;
-        c_eq += ok && kv[e] == thr;
+        const int i = i0 + e * 32 + lane;
+        ok[e] = i < w1;
+        kv[e] = ok[e] ? keys[i] : 0u;
       }
-      const uint32_t packed = c_gt | (c_eq << 16);          // at most 128 of each per step
-      if (!__any_sync(0xffffffffu, packed != 0u)) continue;   // nothing selected in these 128 keys
-      const uint32_t incl = warp_incl_scan(packed, lane);
-      const uint32_t excl = incl - packed;
-      uint32_t g_before = g_run + (excl & 0xffffu);
-      uint32_t e_before = e_run + (excl >> 16);
+      uint32_t mg[4], me[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const bool ok = i + e < w1;
+        mg[e] = __ballot_sync(0xffffffffu, ok[e] && kv[e] > thr);
+        me[e] = __ballot_sync(0xffffffffu, ok[e] && kv[e] == thr);
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t g_before = g_run + __popc(mg[e] & lt);
+        const uint32_t e_before = e_run + __popc(me[e] & lt);
         // (positions are < ktot by construction; the comparison keeps a write inside the
         // list whatever the scores hold)
         uint32_t pos = 0xffffffffu;
-        if (ok && kv[e] > thr) { pos = g_before + min(e_before, tie_quota); ++g_before; }
-        else if (ok && kv[e] == thr) { if (e_before < tie_quota) pos = g_before + e_before; ++e_before; }
-        if (pos < ktot) out_idx[pos] = c0 + i + e;
+        if (ok[e] && kv[e] > thr) pos = g_before + min(e_before, tie_quota);
+        else if (ok[e] && kv[e] == thr && e_before < tie_quota) pos = g_before + e_before;
+        if (pos < ktot) out_idx[pos] = c0 + i0 + e * 32 + lane;
+        g_run += __popc(mg[e]);
+        e_run += __popc(me[e]);
       }
-      const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
-      g_run += tot & 0xffffu;
-      e_run += tot >> 16;
     }
     if (crank == 0 && tid == 0) p.n_sel[u] = (int32_t)ktot;
   }
@@ -379,19 +395,17 @@ fused_decode_kernel(const FusedParams p) {
     const int my_g = lane % GP;
     const int my_i = lane / GP;
     for (int base = a0 + warp * R; base < a1; base += kFW * R) {
+      // all row indices first, then all row loads: nothing waits on a previous row (rows
+      // past the end repeat the last one and are masked below)
+      int tok[R];
+#pragma unroll
+      for (int i = 0; i < R; ++i) tok[i] = __ldcg(irow + min(base + i, a1 - 1));
       uint2 kk[R], vv[R];
 #pragma unroll
       for (int i = 0; i < R; ++i) {
-        const int r = base + i;
-        if (r < a1) {
-          int tok = __ldcg(irow + r);
-          tok = min(max(tok, 0), p.max_len - 1);
-          kk[i] = ld_stream_u2(kbase + (int64_t)tok * p.kst);
-          vv[i] = ld_stream_u2(vbase + (int64_t)tok * p.vst);
-        } else {
-          kk[i] = make_uint2(0u, 0u);
-          vv[i] = make_uint2(0u, 0u);
-        }
+        const int t = min(max(tok[i], 0), p.max_len - 1);
+        kk[i] = ld_stream_u2(kbase + (int64_t)t * p.kst);
+        vv[i] = ld_stream_u2(vbase + (int64_t)t * p.vst);
       }
       // partial logits of R rows x GP heads over this lane's 4 channels
       float part[32];
@@ -514,25 +528,33 @@ fused_decode_kernel(const FusedParams p) {
   cluster.sync();   // barrier 6: every CTA's partial result is in its shared memory
 
   {
+    // This CTA finishes a contiguous share of the unit's outputs.  cs neighbouring lanes take
+    // one output together, each fetching one CTA's (m, l, acc) from its shared memory, and
+    // combine with xor-shuffles: one round of remote loads whatever the cluster size.
     const int n_out = p.group * FASA_HEAD_DIM;
     const int per_o = (n_out + cs - 1) / cs;
-    for (int t = tid; t < per_o; t += kFT) {
+    const int opp = kFT / cs;                // outputs per pass (cs is a power of two <= 16)
+    const int r = tid % cs, tl = tid / cs;
+    for (int t0 = 0; t0 < per_o; t0 += opp) {   // uniform trip count
+      const int t = t0 + tl;
       const int o = crank * per_o + t;
-      if (o >= n_out) break;
-      const int g = o / FASA_HEAD_DIM, c = o % FASA_HEAD_DIM;
-      float mx = -INFINITY;
-      for (int r = 0; r < cs; ++r) mx = fmaxf(mx, cluster.map_shared_rank(&s_part[g][0], r)[0]);
-      float a = 0.f, l = 0.f;
-      for (int r = 0; r < cs; ++r) {
-        const float* pr = cluster.map_shared_rank(&s_part[g][0], r);
-        const float ms = pr[0];
-        const float wt = ms == -INFINITY ? 0.f : exp2f(ms - mx);
-        a += wt * pr[2 + c];
-        l += wt * pr[1];
+      const bool ok = t < per_o && o < n_out;
+      const int g = ok ? o / FASA_HEAD_DIM : 0, c = ok ? o % FASA_HEAD_DIM : 0;
+      const float* pr = cluster.map_shared_rank(&s_part[g][0], r);
+      const float ms = pr[0], ls = pr[1], as = pr[2 + c];
+      float mx = ms;
+      for (int off = cs >> 1; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+      const float wt = ms == -INFINITY ? 0.f : exp2f(ms - mx);
+      float a = wt * as, l = wt * ls;
+      for (int off = cs >> 1; off > 0; off >>= 1) {
+        a += __shfl_xor_sync(0xffffffffu, a, off);
+        l += __shfl_xor_sync(0xffffffffu, l, off);
       }
-      const int64_t hq = (int64_t)b * p.n_q_heads + (int64_t)h * p.group + g;
-      p.out[hq * FASA_HEAD_DIM + c] = l > 0.f ? a / l : 0.f;
-      if (p.lse && c == 0) p.lse[hq] = l > 0.f ? (mx + log2f(l)) * 0.6931471805599453f : -INFINITY;
+      if (ok && r == 0) {
+        const int64_t hq = (int64_t)b * p.n_q_heads + (int64_t)h * p.group + g;
+        p.out[hq * FASA_HEAD_DIM + c] = l > 0.f ? a / l : 0.f;
+        if (p.lse && c == 0) p.lse[hq] = l > 0.f ? (mx + log2f(l)) * 0.6931471805599453f : -INFINITY;
+      }
     }
   }
   cluster.sync();   // barrier 7: no CTA leaves while a peer can still read its shared memory
