@@ -208,6 +208,19 @@ int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_cache,
                          int32_t budget, int32_t n_sel_max, float* scores, int32_t* idx,
                          int32_t* n_sel, float* out, float* lse, void* workspace, void* stream);
 
+/* Algorithm 2's order for one new token per sequence: UpdateCache (K, V and the dominant
+ * part of the key cache), then the step above on the grown cache; seq_lens[b] += 1 on the
+ * device.  k_new, v_new: bf16 [batch][n_kv_heads][1][128], post-RoPE, 16-byte aligned.
+ * In mode 1 the append happens inside the same kernel (the CTA whose slice ends the
+ * sequence writes the three rows before it scores them), so the whole step is one launch;
+ * otherwise it is fasa_kv_append followed by fasa_decode_step.  A full cache drops the
+ * token and sets FASA_DEV_APPEND_FULL, as fasa_kv_append does. */
+int32_t fasa_append_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_new,
+                                const void* v_new, void* k_cache, void* v_cache, void* proxy_k,
+                                int32_t* seq_lens, int32_t budget, int32_t n_sel_max,
+                                float* scores, int32_t* idx, int32_t* n_sel, float* out,
+                                float* lse, void* workspace, void* stream);
+
 /* End-to-end step from HOST buffers (pinned memory recommended): copies q_host,
  * k_new_host, v_new_host (layouts as fasa_kv_append with n_new = 1) to the device
  * staging area dev_stage (>= fasa_stage_bytes), appends, runs fasa_decode_step,

@@ -91,6 +91,8 @@ extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_h
   if (e == cudaSuccess) ctx->n_sm = prop.multiProcessorCount;
   if (e == cudaSuccess) e = cudaMalloc(&ctx->d_chan, chan.size() * sizeof(int16_t));
   if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, 256);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_arrive, (size_t)c.batch * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_arrive, 0, (size_t)c.batch * sizeof(int32_t));
   if (e == cudaSuccess)
     e = cudaMemcpy(ctx->d_chan, chan.data(), chan.size() * sizeof(int16_t), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
@@ -98,6 +100,7 @@ extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_h
   if (e != cudaSuccess) {
     cudaFree(ctx->d_chan);
     cudaFree(ctx->d_status);
+    cudaFree(ctx->d_arrive);
     delete ctx;
     return FASA_ERR_CUDA;
   }
@@ -111,6 +114,7 @@ extern "C" int32_t fasa_destroy(fasa_ctx_t* ctx) {
   if (!ctx) return FASA_ERR_INVALID_ARG;
   cudaFree(ctx->d_chan);
   cudaFree(ctx->d_status);
+  cudaFree(ctx->d_arrive);
   delete ctx;
   return FASA_OK;
 }
@@ -190,11 +194,11 @@ extern "C" int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* 
       budget == 0 || budget < -1000 || n_sel_max <= 0)
     return FASA_ERR_INVALID_ARG;
   if (ctx->use_fused && ctx->fused_cs > 0) {
-    if (((uintptr_t)proxy_k & 15) || ((uintptr_t)q & 1) || ((uintptr_t)k_cache & 15) ||
+    if (((uintptr_t)proxy_k & 15) || ((uintptr_t)q & 15) || ((uintptr_t)k_cache & 15) ||
         ((uintptr_t)v_cache & 15) || (scores && ((uintptr_t)scores & 3)))
       return FASA_ERR_INVALID_ARG;
     return fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
-                             idx, n_sel, out, lse, (cudaStream_t)stream);
+                             idx, n_sel, out, lse, nullptr, nullptr, (cudaStream_t)stream);
   }
   if (!scores || !workspace) return FASA_ERR_INVALID_ARG;
   int32_t st = fasa_fc_score(ctx, q, proxy_k, seq_lens, scores, stream);
@@ -203,6 +207,29 @@ extern "C" int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* 
   if (st != FASA_OK) return st;
   return fasa_sparse_decode_attn(ctx, q, k_cache, v_cache, idx, n_sel, n_sel_max, out, lse,
                                  workspace, stream);
+}
+
+extern "C" int32_t fasa_append_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_new,
+                                           const void* v_new, void* k_cache, void* v_cache,
+                                           void* proxy_k, int32_t* seq_lens, int32_t budget,
+                                           int32_t n_sel_max, float* scores, int32_t* idx,
+                                           int32_t* n_sel, float* out, float* lse, void* workspace,
+                                           void* stream) {
+  if (!ctx || !q || !k_new || !v_new || !k_cache || !v_cache || !proxy_k || !seq_lens || !idx ||
+      !n_sel || !out || budget == 0 || budget < -1000 || n_sel_max <= 0)
+    return FASA_ERR_INVALID_ARG;
+  if (ctx->use_fused && ctx->fused_cs > 0) {
+    if (((uintptr_t)proxy_k & 15) || ((uintptr_t)q & 15) || ((uintptr_t)k_cache & 15) ||
+        ((uintptr_t)v_cache & 15) || ((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15) ||
+        (scores && ((uintptr_t)scores & 3)))
+      return FASA_ERR_INVALID_ARG;
+    return fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
+                             idx, n_sel, out, lse, k_new, v_new, (cudaStream_t)stream);
+  }
+  int32_t st = fasa_kv_append(ctx, k_cache, v_cache, proxy_k, seq_lens, k_new, v_new, 1, stream);
+  if (st != FASA_OK) return st;
+  return fasa_decode_step(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores, idx,
+                          n_sel, out, lse, workspace, stream);
 }
 
 extern "C" int32_t fasa_stage_bytes(const fasa_ctx_t* ctx, size_t* out_bytes) {
@@ -233,10 +260,8 @@ extern "C" int32_t fasa_decode_step_host(fasa_ctx_t* ctx, const void* q_host,
   FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
   FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
   FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
-  int32_t st = fasa_kv_append(ctx, k_cache, v_cache, proxy_k, seq_lens, dk, dv, 1, stream);
-  if (st != FASA_OK) return st;
-  st = fasa_decode_step(ctx, dq, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
-                        idx, n_sel, out, nullptr, workspace, stream);
+  int32_t st = fasa_append_decode_step(ctx, dq, dk, dv, k_cache, v_cache, proxy_k, seq_lens, budget,
+                                       n_sel_max, scores, idx, n_sel, out, nullptr, workspace, stream);
   if (st != FASA_OK) return st;
   size_t o_bytes = (size_t)c.batch * c.n_q_heads * FASA_HEAD_DIM * sizeof(float);
   FASA_CUDA_TRY(ctx, cudaMemcpyAsync(out_host, out, o_bytes, cudaMemcpyDeviceToHost, s));

@@ -40,6 +40,15 @@ struct FusedParams {
   const uint4* proxy;
   const int32_t* seq_lens;
   const int16_t* chan;
+  // append-then-step form (all null / unused otherwise): the new token's rows, the buffers
+  // they are written to, the length to update and a per-sequence arrival counter
+  const uint16_t* k_new;
+  const uint16_t* v_new;
+  uint16_t* k_w;
+  uint16_t* v_w;
+  uint16_t* proxy_w;
+  int32_t* seq_lens_w;
+  int32_t* arrive;
   float* scores;           // nullable
   int32_t* idx;
   int32_t* n_sel;
@@ -53,7 +62,18 @@ struct FusedParams {
 
 __device__ __forceinline__ uint2 ld_stream_u2(const void* p) {
   uint2 r;
-  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
+  asm volatile("ld.global.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p) : "memory");
+  return r;
+}
+
+// 128-bit load through the coherent path (not .nc): in the append-then-step form the last
+// proxy / K / V row was written earlier in this same launch.
+__device__ __forceinline__ uint4 ld_coherent_u4(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p)
+               : "memory");
   return r;
 }
 
@@ -102,6 +122,9 @@ fused_decode_kernel(const FusedParams p) {
   __shared__ unsigned long long s_wcnt[kFW];
   __shared__ unsigned long long s_tot;
   __shared__ uint32_t s_bin, s_kth, s_cnt;
+  __shared__ int s_len_old;
+  __shared__ uint32_t s_mg[kCapMax / 32], s_me[kCapMax / 32];   // per 32 keys: above / equal masks
+  __shared__ unsigned long long s_roff[kCapMax / 32];           // per 32 keys: (gt, eq) selected before
   __shared__ __align__(16) float s_q[GP][FASA_HEAD_DIM];
   __shared__ __align__(16) float s_part[GP][kPartStride + 2];
   __shared__ __align__(16) float s_p[kFW][32];
@@ -110,7 +133,29 @@ fused_decode_kernel(const FusedParams p) {
   __shared__ float s_l[kFW][GP];
 
   // ---- slices -------------------------------------------------------------------------
-  const int len = clamp_len(p.seq_lens[b], p.max_len, p.status);
+  // Append-then-step: one thread reads the length for the whole CTA, so that the CTA's arrival
+  // (below) certifies that it no longer needs the old value; the last CTA of the sequence to
+  // arrive stores the new length.  Nothing waits on the counter.
+  const bool append = p.k_new != nullptr;
+  int len_old;
+  if (append) {
+    if (tid == 0) s_len_old = clamp_len(p.seq_lens[b], p.max_len, p.status);
+    __syncthreads();
+    len_old = s_len_old;
+  } else {
+    len_old = clamp_len(p.seq_lens[b], p.max_len, p.status);
+  }
+  const bool grows = append && len_old < p.max_len;
+  const int len = len_old + (grows ? 1 : 0);
+  if (append && tid == 0) {
+    if (!grows && crank == 0) atomicOr(p.status, FASA_DEV_APPEND_FULL);
+    __threadfence();
+    const int total = p.n_kv_heads * cs;
+    if (atomicAdd(&p.arrive[b], 1) == total - 1) {
+      p.seq_lens_w[b] = len;
+      p.arrive[b] = 0;
+    }
+  }
   const int per = (((len + cs - 1) / cs) + 31) & ~31;          // <= the capacity the host sized
   const int c0 = min(len, crank * per);
   const int c1 = min(len, c0 + per);
@@ -131,6 +176,32 @@ fused_decode_kernel(const FusedParams p) {
   }
   const uint32_t ktot = (uint32_t)ktot_ll;
 
+  if (grows && c0 <= len_old && len_old < c1) {
+    // this CTA's slice holds the new row: K and V copies (16 lanes each) and the packed
+    // dominant-FC pairs of the key (one lane per 16-byte chunk), as in fasa_kv_append
+    const uint16_t* ksrc = p.k_new + (int64_t)u * FASA_HEAD_DIM;
+    if (tid < 16) {
+      *reinterpret_cast<uint4*>(p.k_w + b * p.ksb + h * p.ksh + (int64_t)len_old * p.kst + tid * 8) =
+          *reinterpret_cast<const uint4*>(ksrc + tid * 8);
+    } else if (tid < 32) {
+      const int c = tid - 16;
+      *reinterpret_cast<uint4*>(p.v_w + b * p.vsb + h * p.vsh + (int64_t)len_old * p.vst + c * 8) =
+          *reinterpret_cast<const uint4*>(p.v_new + (int64_t)u * FASA_HEAD_DIM + c * 8);
+    } else if (tid - 32 < p.chunks) {
+      const int c = tid - 32;
+      const int16_t* ch = p.chan + h * p.chunks * 8 + c * 8;
+      uint32_t w[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int ch0 = ch[2 * e], ch1 = ch[2 * e + 1];
+        const uint32_t lo = ch0 >= 0 ? ksrc[ch0] : 0u;
+        const uint32_t hi = ch1 >= 0 ? ksrc[ch1] : 0u;
+        w[e] = lo | (hi << 16);
+      }
+      *reinterpret_cast<uint4*>(p.proxy_w + ((int64_t)u * p.max_len + len_old) * (p.chunks * 8) + c * 8) =
+          make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
   for (int i = tid; i < 2 * kFBins; i += kFT) hist0[i] = 0u;
   // query, scaled into the base-2 logit domain, for the attention phase
   for (int i = tid; i < GP * (FASA_HEAD_DIM / 8); i += kFT) {
@@ -159,7 +230,7 @@ fused_decode_kernel(const FusedParams p) {
 #pragma unroll
       for (int i = 0; i < kFUnroll; ++i) {
         const int row = base + i * RPL + grp;
-        x[i] = (live && row < c1) ? ld_stream_u4(prow + (int64_t)row * p.chunks + sub)
+        x[i] = (live && row < c1) ? ld_coherent_u4(prow + (int64_t)row * p.chunks + sub)
                                   : make_uint4(0u, 0u, 0u, 0u);
       }
     };
@@ -209,6 +280,7 @@ fused_decode_kernel(const FusedParams p) {
         for (int i = tid; i < nb; i += kFT) buf[i] = 0u;
         __syncthreads();
       }
+#pragma unroll 4
       for (int i = tid * 4; i < nloc; i += kFT * 4) {
         const uint4 kq = *reinterpret_cast<const uint4*>(&keys[i]);
         const uint32_t kv[4] = {kq.x, kq.y, kq.z, kq.w};
@@ -299,32 +371,46 @@ fused_decode_kernel(const FusedParams p) {
   }
 
   // ---- 3. ascending compaction ---------------------------------------------------------------
-  // A warp owns a contiguous run of keys and walks it 128 at a time (four rows of 32
-  // consecutive keys, one key per lane and row), so positions come out in index order.
-  const int wper = (((nloc + kFW - 1) / kFW) + 127) & ~127;
-  const int w0 = min(nloc, warp * wper);
-  const int w1 = min(nloc, w0 + wper);
-  {
-    uint32_t n_gt = 0, n_eq = 0;
-    for (int i = w0 + lane * 4; i < w1; i += 128) {
-      const uint4 kq = *reinterpret_cast<const uint4*>(&keys[i]);
-      const uint32_t kv[4] = {kq.x, kq.y, kq.z, kq.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const bool ok = i + e < w1;
-        n_gt += ok && kv[e] > thr;
-        n_eq += ok && kv[e] == thr;
-      }
+  // Rows of 32 consecutive keys.  (a) every warp turns its rows into two bit masks (key above
+  // the threshold / equal to it) with independent ballots; (b) a block scan over the rows'
+  // bit counts gives each row its offsets; (c) after the cluster-wide prefix, set bits become
+  // positions.  No step carries a running counter through a loop, so the loops pipeline.
+  const int n_rows = (nloc + 31) >> 5;
+  for (int r0 = warp * 32; r0 < n_rows; r0 += kFW * 32) {   // 32 rows per warp step
+    uint32_t my_g = 0, my_e = 0;
+#pragma unroll 8
+    for (int j = 0; j < 32; ++j) {
+      const int i = (r0 + j) * 32 + lane;
+      const bool ok = i < nloc;
+      const uint32_t key = ok ? keys[i] : 0u;
+      const uint32_t mg = __ballot_sync(0xffffffffu, ok && key > thr);
+      const uint32_t me = __ballot_sync(0xffffffffu, ok && key == thr);
+      if (lane == j) { my_g = mg; my_e = me; }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      n_gt += __shfl_xor_sync(0xffffffffu, n_gt, o);
-      n_eq += __shfl_xor_sync(0xffffffffu, n_eq, o);
+    if (r0 + lane < n_rows) {
+      s_mg[r0 + lane] = my_g;
+      s_me[r0 + lane] = my_e;
     }
-    if (lane == 0) s_wcnt[warp] = ((unsigned long long)n_gt << 32) | n_eq;
   }
   __syncthreads();
-  unsigned long long before = 0;
+  // block scan of the per-row counts (gt in the high half, eq in the low half)
+  constexpr int RPT = (kCapMax / 32 + kFT - 1) / kFT;       // rows per thread
+  unsigned long long row_cnt[RPT], mine = 0;
+#pragma unroll
+  for (int j = 0; j < RPT; ++j) {
+    const int r = tid * RPT + j;
+    row_cnt[j] = r < n_rows ? (((unsigned long long)__popc(s_mg[r]) << 32) | (unsigned)__popc(s_me[r])) : 0ull;
+    mine += row_cnt[j];
+  }
+  unsigned long long incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) s_wcnt[warp] = incl;
+  __syncthreads();
+  unsigned long long before = incl - mine;
   {
     unsigned long long all = 0;
     for (int w = 0; w < kFW; ++w) {
@@ -342,38 +428,28 @@ fused_decode_kernel(const FusedParams p) {
     for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
     before += t;
   }
+#pragma unroll
+  for (int j = 0; j < RPT; ++j) {            // offsets of this thread's rows
+    const int r = tid * RPT + j;
+    if (r < n_rows) s_roff[r] = before;
+    before += row_cnt[j];
+  }
+  __syncthreads();
   {
-    uint32_t g_run = (uint32_t)(before >> 32), e_run = (uint32_t)before;
     int32_t* out_idx = p.idx + (int64_t)u * p.n_sel_max;
     const uint32_t lt = (1u << lane) - 1u;
-    for (int i0 = w0; i0 < w1; i0 += 128) {   // uniform trip count over the warp
-      uint32_t kv[4];
-      bool ok[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int i = i0 + e * 32 + lane;
-        ok[e] = i < w1;
-        kv[e] = ok[e] ? keys[i] : 0u;
-      }
-      uint32_t mg[4], me[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        mg[e] = __ballot_sync(0xffffffffu, ok[e] && kv[e] > thr);
-        me[e] = __ballot_sync(0xffffffffu, ok[e] && kv[e] == thr);
-      }
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const uint32_t g_before = g_run + __popc(mg[e] & lt);
-        const uint32_t e_before = e_run + __popc(me[e] & lt);
-        // (positions are < ktot by construction; the comparison keeps a write inside the
-        // list whatever the scores hold)
-        uint32_t pos = 0xffffffffu;
-        if (ok[e] && kv[e] > thr) pos = g_before + min(e_before, tie_quota);
-        else if (ok[e] && kv[e] == thr && e_before < tie_quota) pos = g_before + e_before;
-        if (pos < ktot) out_idx[pos] = c0 + i0 + e * 32 + lane;
-        g_run += __popc(mg[e]);
-        e_run += __popc(me[e]);
-      }
+    for (int r = warp; r < n_rows; r += kFW) {
+      const uint32_t mg = s_mg[r], me = s_me[r];
+      if ((mg | me) == 0u) continue;                         // uniform over the warp
+      const unsigned long long off = s_roff[r];
+      const uint32_t g_before = (uint32_t)(off >> 32) + __popc(mg & lt);
+      const uint32_t e_before = (uint32_t)off + __popc(me & lt);
+      // (positions are < ktot by construction; the comparison keeps a write inside the list
+      // whatever the scores hold)
+      uint32_t pos = 0xffffffffu;
+      if ((mg >> lane) & 1u) pos = g_before + min(e_before, tie_quota);
+      else if (((me >> lane) & 1u) && e_before < tie_quota) pos = g_before + e_before;
+      if (pos < ktot) out_idx[pos] = c0 + r * 32 + lane;
     }
     if (crank == 0 && tid == 0) p.n_sel[u] = (int32_t)ktot;
   }
@@ -643,11 +719,15 @@ int fasa_fused_plan(fasa_ctx* ctx) {
 int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                           const void* proxy_k, const int32_t* seq_lens, int32_t budget,
                           int32_t n_sel_max, float* scores, int32_t* idx, int32_t* n_sel,
-                          float* out, float* lse, cudaStream_t stream) {
+                          float* out, float* lse, const void* k_new, const void* v_new,
+                          cudaStream_t stream) {
   const fasa_config_t& c = ctx->cfg;
   FusedParams p;
   p.q = (const uint16_t*)q; p.k = (const uint16_t*)k_cache; p.v = (const uint16_t*)v_cache;
   p.proxy = (const uint4*)proxy_k; p.seq_lens = seq_lens; p.chan = ctx->d_chan;
+  p.k_new = (const uint16_t*)k_new; p.v_new = (const uint16_t*)v_new;
+  p.k_w = (uint16_t*)k_cache; p.v_w = (uint16_t*)v_cache; p.proxy_w = (uint16_t*)proxy_k;
+  p.seq_lens_w = (int32_t*)seq_lens; p.arrive = ctx->d_arrive;
   p.scores = scores; p.idx = idx; p.n_sel = n_sel; p.out = out; p.lse = lse; p.status = ctx->d_status;
   p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group; p.max_len = c.max_len;
   p.chunks = ctx->chunks; p.n_sink = c.n_sink; p.n_recent = c.n_recent; p.budget = budget;

@@ -219,6 +219,40 @@ def test_decode_step_equals_separate_calls_and_host_variant():
     assert torch.equal(out_host, r.out.cpu())
 
 
+@pytest.mark.parametrize("mode", [1, 0])
+def test_append_decode_step_equals_append_then_step(mode):
+    # ragged batch, group of 7, permille budget; several steps in a row so the per-sequence
+    # arrival counter of the one-launch form is reused
+    w = C["c3"].replace(batch=3, max_len=1300, len_lo=700, len_hi=1297)
+    t = synth.make_inputs(w, "cpu")
+    t["seq_lens"] = torch.tensor([700, 1297, 1001], dtype=torch.int32)
+    a, b = Run(w, t), Run(w, {k_: (v_.clone() if torch.is_tensor(v_) else v_) for k_, v_ in t.items()})
+    for r in (a, b):
+        r.fasa.set_step_mode(mode)
+        r.build_proxy()
+    for step in range(5):
+        s = synth.make_step_inputs(w, step, "cuda")
+        a.fasa.kv_append(a.k, a.v, a.proxy, a.seq_lens, s["k_new"], s["v_new"])
+        a.fasa.decode_step(s["q"], a.k, a.v, a.proxy, a.seq_lens, w.budget, a.scores, a.idx, a.n_sel, a.out, a.ws)
+        n0 = b.fasa.launch_count()
+        b.fasa.append_decode_step(s["q"], s["k_new"], s["v_new"], b.k, b.v, b.proxy, b.seq_lens, w.budget, b.scores,
+                                  b.idx, b.n_sel, b.out, b.ws)
+        torch.cuda.synchronize()
+        assert b.fasa.launch_count() - n0 == (1 if mode == 1 else 6)
+        for x, y in ((a.k, b.k), (a.v, b.v), (a.proxy, b.proxy), (a.seq_lens, b.seq_lens), (a.scores, b.scores),
+                     (a.idx, b.idx), (a.n_sel, b.n_sel)):
+            assert torch.equal(x, y)
+        assert float((a.out - b.out).abs().max()) <= 1e-5
+    # sequence 1 filled up after 3 steps: later tokens are dropped and flagged, on both routes
+    assert a.seq_lens.cpu().tolist() == [705, 1300, 1006]
+    assert a.fasa.device_status() & binding.DEV_APPEND_FULL and b.fasa.device_status() & binding.DEV_APPEND_FULL
+    # and the result of the last step agrees with the oracle on the grown cache
+    kc, vc = b.k.cpu(), b.v.cpu()
+    parity.check_step(s["q"].cpu().double().numpy(), kc.double().numpy(), vc.double().numpy(), [705, 1300, 1006],
+                      np.sort(b.dom.numpy(), axis=1), scores=b.scores.cpu().numpy(), idx=b.idx.cpu().numpy(),
+                      n_sel=b.n_sel.cpu().numpy(), out=b.out.cpu().numpy(), what="append+step", **b.oracle_kwargs())
+
+
 def test_strided_token_major_cache():
     # K/V stored [B][L][Hkv][128] (token-major), addressed through the stride fields.
     w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, batch=2, max_len=640, len_lo=400, len_hi=640, budget=40)
