@@ -5,10 +5,11 @@
 
 One step = one pass of the whole hot path over one batch: append one token per sequence
 (K, V and proxy-K rows), score every cached key on the dominant FCs, select the top-budget
-tokens, run exact attention over the selected rows and merge the splits.  The step calls
-fasa_kv_append and fasa_decode_step (one cluster kernel: score -> select -> attention); the
-three stand-alone calls (fasa_fc_score, fasa_topk, fasa_sparse_decode_attn) and the dense
-path are timed beside it.  Inputs are
+tokens, run exact attention over the selected rows and merge the splits.  The step is one
+call, fasa_append_decode_step (one cluster kernel: append -> score -> select -> attention);
+the stand-alone calls (fasa_kv_append, fasa_fc_score, fasa_topk, fasa_sparse_decode_attn)
+and the dense path are timed beside it, and the large batched workloads are reported under
+`other_workloads`.  Inputs are
 synthetic (paper_2602_03152_b200.synth) and resident in HBM before the timed region; L2 is
 flushed between steps.  Rank 0 prints one JSON line.
 
@@ -148,34 +149,25 @@ def run_reference(args, w):
 
 # ---------------------------------------------------------------- our arm ----
 
-def run_fasa(args, w):
-    import numpy as np
+def measure(w, K, W, dev, world, step_mode=None, sampler_factory=None, want_e2e=True):
+    """Times one workload on this rank's GPU; returns a dict of measurements (durations are
+    max over ranks where that matters)."""
     import torch
     import torch.distributed as dist
 
-    from paper_2602_03152_b200 import binding, build, synth
+    from paper_2602_03152_b200 import binding, synth
 
-    build.build()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: the FASA path has no CPU fallback")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    # Weak scaling: every rank holds its own batch of independent (batch, KV head) units.
-    # The cache has one spare row so each step appends at row L-1 and scores L rows.
-    wl = w.replace(index=w.index + 100 * rank)
-    t = synth.make_inputs(wl, dev)
+    t = synth.make_inputs(w, dev)
     lens_full = t["seq_lens"].clone()
+    # The cache has one spare row so each step appends at row L-1 and scores L rows.
     lens_start = (lens_full - 1).clamp_(min=0)
-    f = binding.Fasa.from_workload(wl, t["dom"])
+    f = binding.Fasa.from_workload(w, t["dom"])
+    if step_mode is not None:
+        f.set_step_mode(step_mode)
+    fused = f.step_cluster_size() > 0
     q, k, v = t["q"], t["k"], t["v"]
-    n_sel_max = wl.n_sel_max()
-    B, Hq, Hkv, Lm = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.max_len
+    n_sel_max = w.n_sel_max()
+    B, Hq, Hkv, Lm = w.batch, w.n_q_heads, w.n_kv_heads, w.max_len
     proxy = f.alloc_proxy(dev)
     ws = f.alloc_workspace(n_sel_max, dev)
     scores = torch.zeros((B, Hkv, Lm), dtype=torch.float32, device=dev)
@@ -211,25 +203,22 @@ def run_fasa(args, w):
                 durs.append(a.elapsed_time(b) * 1e3)
         return durs
 
-    if args.step_mode is not None:
-        f.set_step_mode(args.step_mode)
-    fused = f.step_cluster_size() > 0
+    def rank_max(x):
+        if world > 1:
+            tt = torch.tensor([x], dtype=torch.float64, device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            return float(tt.item())
+        return x
 
     def fasa_step():
-        f.kv_append(k, v, proxy, lens, k_new, v_new)
-        f.decode_step(q, k, v, proxy, lens, wl.budget, None if fused else scores, idx, n_sel, out, ws)
+        f.append_decode_step(q, k_new, v_new, k, v, proxy, lens, w.budget, None if fused else scores, idx, n_sel,
+                             out, ws)
 
     def dense_step():
         f.kv_append(k, v, proxy, lens, k_new, v_new)
         f.full_decode_attn(q, k, v, lens, dense_out, ws)
 
-    K, W = args.steps, max(3, args.warmup)
-    gpu_id = str(local)
-    try:
-        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
-    except Exception:
-        pass
-    sampler = ClockSampler(gpu_id) if rank == 0 else None
+    sampler = sampler_factory() if sampler_factory else None
 
     # ---- timed region: K whole steps ------------------------------------------------
     timed(fasa_step, 0, W)
@@ -242,18 +231,12 @@ def run_fasa(args, w):
     launches = f.launch_count() - l0
     if world > 1:
         dist.barrier()
-    total_us = sum(step_us)
-    if world > 1:
-        tt = torch.tensor([total_us], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_us = float(tt.item())
-    us_per_step = total_us / K
+    us_per_step = rank_max(sum(step_us)) / K
 
     n_sel_total = int(n_sel.sum().item())
-    by = step_bytes(wl, lens_full.cpu().tolist(), n_sel_total)
-    status = f.device_status()
+    by = step_bytes(w, lens_full.cpu().tolist(), n_sel_total)
 
-    # ---- per-kernel breakdown (same launches, one C-ABI call at a time) ----------------
+    # ---- the stand-alone calls, one C-ABI call at a time ---------------------------------
     parts = {"kv_append": [], "fc_score": [], "topk": [], "sparse_attn": []}
     Kk = min(K, 200)
     for i in range(W + Kk):
@@ -262,7 +245,7 @@ def run_fasa(args, w):
         e = [ev() for _ in range(5)]
         e[0].record(); f.kv_append(k, v, proxy, lens, k_new, v_new)
         e[1].record(); f.fc_score(q, proxy, lens, scores)
-        e[2].record(); f.topk(scores, lens, wl.budget, idx, n_sel, ws)
+        e[2].record(); f.topk(scores, lens, w.budget, idx, n_sel, ws)
         e[3].record(); f.sparse_decode_attn(q, k, v, idx, n_sel, out, ws)
         e[4].record(); e[4].synchronize()
         if i >= W:
@@ -270,41 +253,89 @@ def run_fasa(args, w):
                 parts[name].append(e[j].elapsed_time(e[j + 1]) * 1e3)
     kern_us = {n: statistics.mean(v_) for n, v_ in parts.items()}
     dense_us = statistics.mean(timed(dense_step, Kk, W))
-    # the decode step alone (no append): one launch when the cluster kernel is in use
-    lens.copy_(lens_full)
-
-    def step_only():
-        lens.copy_(lens_full)
-        f.decode_step(q, k, v, proxy, lens, wl.budget, None if fused else scores, idx, n_sel, out, ws)
-
-    step_only_us = []
-    for i in range(W + Kk):
-        flush.fill_(i & 0xff)
-        lens.copy_(lens_full)
-        a, b = ev(), ev()
-        a.record()
-        f.decode_step(q, k, v, proxy, lens, wl.budget, None if fused else scores, idx, n_sel, out, ws)
-        b.record(); b.synchronize()
-        if i >= W:
-            step_only_us.append(a.elapsed_time(b) * 1e3)
-    step_only_us = statistics.mean(step_only_us)
 
     # ---- end to end from host buffers ---------------------------------------------------
-    stage = torch.empty(f.stage_bytes(), dtype=torch.uint8, device=dev)
-    qh, knh, vnh = q.cpu().pin_memory(), k_new.cpu().pin_memory(), v_new.cpu().pin_memory()
-    oh = torch.empty((B, Hq, 128), dtype=torch.float32).pin_memory()
+    e2e_us = h2d = d2h = None
+    if want_e2e:
+        stage = torch.empty(f.stage_bytes(), dtype=torch.uint8, device=dev)
+        qh, knh, vnh = q.cpu().pin_memory(), k_new.cpu().pin_memory(), v_new.cpu().pin_memory()
+        oh = torch.empty((B, Hq, 128), dtype=torch.float32).pin_memory()
 
-    def e2e_step():
-        f.decode_step_host(qh, knh, vnh, stage, k, v, proxy, lens, wl.budget, scores, idx, n_sel, out, oh, ws)
+        def e2e_step():
+            f.decode_step_host(qh, knh, vnh, stage, k, v, proxy, lens, w.budget, None if fused else scores, idx,
+                               n_sel, out, oh, ws)
 
-    e2e_us = statistics.mean(timed(e2e_step, Kk, W))
-    if world > 1:
-        tt = torch.tensor([e2e_us], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_us = float(tt.item())
-    h2d = qh.numel() * 2 + knh.numel() * 2 + vnh.numel() * 2
-    d2h = oh.numel() * 4
+        e2e_us = rank_max(statistics.mean(timed(e2e_step, Kk, W)))
+        h2d = qh.numel() * 2 + knh.numel() * 2 + vnh.numel() * 2
+        d2h = oh.numel() * 4
+    status = f.device_status()
     clocks = sampler.stop() if sampler else None
+    return dict(w=w, t=t, by=by, us_per_step=us_per_step, step_us_median=statistics.median(step_us), launches=launches,
+                kern_us=kern_us, dense_us=dense_us, e2e_us=e2e_us, h2d=h2d, d2h=d2h, status=status, clocks=clocks,
+                fused=fused, cluster_size=f.step_cluster_size(), n_sel_total=n_sel_total, lens_full=lens_full)
+
+
+def summarize(m, peak):
+    """The figures every workload reports (the headline workload adds the contract's keys)."""
+    w, by, ku = m["w"], m["by"], m["kern_us"]
+    gbs = lambda nbytes, us: nbytes / (us * 1e-6) / 1e9
+    score_bytes = by["proxy"]
+    topk_bytes = by["proxy"] // w.n_dom           # one fp32 score per cached token
+    return {
+        "workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
+        "context": int(m["lens_full"].max()), "context_mean": float(m["lens_full"].float().mean()),
+        "n_dom": w.n_dom, "budget": w.budget, "n_sink": w.n_sink, "n_recent": w.n_recent,
+        "n_sel_per_unit": m["n_sel_total"] / (w.batch * w.n_kv_heads),
+        "step_mode": f"one cluster kernel (cluster of {m['cluster_size']})" if m["fused"] else "three kernels",
+        "us_per_step": m["us_per_step"], "step_bytes": by["fasa"],
+        "step_gbs": gbs(by["fasa"], m["us_per_step"]), "step_frac_of_peak": gbs(by["fasa"], m["us_per_step"]) / peak,
+        "dense_us_per_step": m["dense_us"], "dense_bytes": by["dense"],
+        "dense_frac_of_peak": gbs(by["dense"], m["dense_us"]) / peak,
+        "speedup_vs_dense": m["dense_us"] / m["us_per_step"], "byte_ratio_dense_over_fasa": by["dense"] / by["fasa"],
+        "standalone_us": ku,
+        "standalone_frac_of_peak": {"fc_score": gbs(score_bytes, ku["fc_score"]) / peak,
+                                    "topk": gbs(topk_bytes, ku["topk"]) / peak,
+                                    "sparse_attn": gbs(by["gathered"], ku["sparse_attn"]) / peak},
+        "device_status": m["status"],
+    }
+
+
+def run_fasa(args, w):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2602_03152_b200 import build, synth
+
+    build.build()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the FASA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    gpu_id = str(local)
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        pass
+    K, W = args.steps, max(3, args.warmup)
+    # Weak scaling: every rank holds its own batch of independent (batch, KV head) units.
+    wl = w.replace(index=w.index + 100 * rank)
+    m = measure(wl, K, W, dev, world, args.step_mode, (lambda: ClockSampler(gpu_id)) if rank == 0 else None)
+
+    # Other configurations of the same path, a few steps each (single GPU only): the large
+    # batched shapes, where the stream is long enough to approach the HBM roofline.
+    others = []
+    if world == 1 and not args.no_extras:
+        for name in args.extras.split(","):
+            if name and name in synth.CONFIGS and name != args.config:
+                mo = measure(synth.CONFIGS[name], 30, 3, dev, 1, args.step_mode, None, want_e2e=False)
+                mo.pop("t")
+                others.append(mo)
 
     if rank != 0:
         if world > 1:
@@ -312,50 +343,42 @@ def run_fasa(args, w):
         return
 
     peak, peak_src = _peaks()
-    fc_bytes = by["proxy"]                      # the scoring kernel's algorithmic bytes per launch
+    by, us_per_step = m["by"], m["us_per_step"]
+    head = summarize(m, peak)
     roof_us = by["fasa"] / (peak * 1e9) * 1e6
-    if fused:
-        roofline = {"kernel": "fused_decode_kernel", "bound": "hbm",
-                    "achieved": by["fasa"] / (step_only_us * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
-                    "frac": by["fasa"] / (step_only_us * 1e-6) / 1e9 / peak, "traffic": None,
-                    "bytes_per_launch": by["fasa"], "us_per_launch": step_only_us, "peak_source": peak_src,
-                    "cluster_size": f.step_cluster_size()}
+    if m["fused"]:
+        # dominant kernel = the whole step in one launch: its algorithmic bytes are the step's
+        roofline = {"kernel": "fused_decode_kernel", "bound": "hbm", "achieved": head["step_gbs"], "peak": peak,
+                    "unit": "GB/s", "frac": head["step_frac_of_peak"], "traffic": None,
+                    "bytes_per_launch": by["fasa"], "us_per_launch": us_per_step, "peak_source": peak_src,
+                    "cluster_size": m["cluster_size"]}
     else:
-        roofline = {"kernel": "fc_score_kernel", "bound": "hbm",
-                    "achieved": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
-                    "frac": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9 / peak, "traffic": None,
-                    "bytes_per_launch": fc_bytes, "us_per_launch": kern_us["fc_score"], "peak_source": peak_src}
+        fc_us = m["kern_us"]["fc_score"]
+        roofline = {"kernel": "fc_score_kernel", "bound": "hbm", "achieved": by["proxy"] / (fc_us * 1e-6) / 1e9,
+                    "peak": peak, "unit": "GB/s", "frac": by["proxy"] / (fc_us * 1e-6) / 1e9 / peak, "traffic": None,
+                    "bytes_per_launch": by["proxy"], "us_per_launch": fc_us, "peak_source": peak_src}
+    cfg = {k_: head[k_] for k_ in ("workload", "batch", "n_q_heads", "n_kv_heads", "context", "context_mean", "n_dom",
+                                   "budget", "n_sink", "n_recent", "n_sel_per_unit", "step_mode")}
+    cfg["l2"] = f"flushed before every step ({L2_FLUSH_BYTES >> 20} MiB write)"
+    cfg["per_rank"] = "each rank runs its own batch of independent units, no collective"
     line = {
         "metric": METRIC, "value": world * by["fasa"] / (us_per_step * 1e-6) / 1e9, "unit": UNIT,
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": us_per_step / 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, f32 accumulate",
-        "data": "synthetic",
-        "config": {"workload": wl.name, "batch": B, "n_q_heads": Hq, "n_kv_heads": Hkv, "context": int(lens_full.max()),
-                   "context_mean": float(lens_full.float().mean()), "n_dom": wl.n_dom, "budget": wl.budget,
-                   "n_sink": wl.n_sink, "n_recent": wl.n_recent, "n_sel_per_unit": n_sel_total / (B * Hkv),
-                   "l2": f"flushed before every step ({L2_FLUSH_BYTES >> 20} MiB write)",
-                   "per_rank": "each rank runs its own batch of independent units, no collective"},
-        "us_per_step": us_per_step,
-        "us_per_step_median": statistics.median(step_us),
+        "data": "synthetic", "config": cfg,
+        "us_per_step": us_per_step, "us_per_step_median": m["step_us_median"],
         "step_bytes": by["fasa"], "step_roofline_us": roof_us, "step_frac_of_roofline": roof_us / us_per_step,
-        "dense_us_per_step": dense_us, "dense_bytes": by["dense"],
-        "dense_gbs": by["dense"] / (dense_us * 1e-6) / 1e9, "dense_frac_of_roofline": by["dense"] / (dense_us * 1e-6) / 1e9 / peak,
-        "speedup_vs_dense": dense_us / us_per_step, "byte_ratio_dense_over_fasa": by["dense"] / by["fasa"],
-        "kernels_us": kern_us,
-        "kernels_gbs": {"fc_score": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9,
-                        "sparse_attn": by["gathered"] / (kern_us["sparse_attn"] * 1e-6) / 1e9,
-                        "topk": (by["proxy"] // wl.n_dom) / (kern_us["topk"] * 1e-6) / 1e9},
-        "kernels_frac_of_peak": {"fc_score": fc_bytes / (kern_us["fc_score"] * 1e-6) / 1e9 / peak,
-                                 "sparse_attn": by["gathered"] / (kern_us["sparse_attn"] * 1e-6) / 1e9 / peak,
-                                 "topk": (by["proxy"] // wl.n_dom) / (kern_us["topk"] * 1e-6) / 1e9 / peak},
-        "decode_step_only_us": step_only_us, "step_mode": "one cluster kernel" if fused else "three kernels",
+        "dense_us_per_step": m["dense_us"], "dense_bytes": by["dense"], "dense_frac_of_roofline": head["dense_frac_of_peak"],
+        "speedup_vs_dense": head["speedup_vs_dense"], "byte_ratio_dense_over_fasa": head["byte_ratio_dense_over_fasa"],
+        "standalone_kernels_us": m["kern_us"], "standalone_kernels_frac_of_peak": head["standalone_frac_of_peak"],
         "roofline": roofline,
-        "e2e": {"value": world * by["fasa"] / (e2e_us * 1e-6) / 1e9, "unit": UNIT, "us_per_step": e2e_us,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": int(launches), "device_status": status, "clocks": clocks,
+        "e2e": {"value": world * by["fasa"] / (m["e2e_us"] * 1e-6) / 1e9, "unit": UNIT, "us_per_step": m["e2e_us"],
+                "h2d_bytes_per_step": m["h2d"], "d2h_bytes_per_step": m["d2h"]},
+        "gpu_launches": int(m["launches"]), "device_status": m["status"], "clocks": m["clocks"],
+        "other_workloads": [summarize(mo, peak) for mo in others],
     }
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(wl, t, by)
+        line["cpu_baseline"] = cpu_baseline(wl, m["t"], by)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -398,6 +421,8 @@ def main():
     ap.add_argument("--n-dom", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--extras", default="c4,c2", help="other workloads reported under other_workloads (30 steps each)")
+    ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--step-mode", type=int, default=None, choices=[0, 1],
                     help="0: fasa_decode_step as three kernels; 1 (default): one cluster kernel where available")
     args = ap.parse_args()
