@@ -26,10 +26,16 @@
  *   - Frequency chunk (FC) i, 0 <= i < 64, is the channel pair (i, i+64) with
  *     rope_pairing 0 (rotate-half layout) or (2i, 2i+1) with rope_pairing 1
  *     (the paper's Eq. 1 layout).  An FC is never split (Appendix, design choices).
- *   - Proxy-K buffer: [batch][n_kv_heads][max_len][proxy_row_elems] bf16 where
- *     proxy_row_elems = 8 * ceil(n_dom / 4) (fasa_proxy_row_elems).  Row j holds,
- *     for the head's dominant FCs sorted ascending, the pairs (K[j][c0], K[j][c1]);
- *     padding elements are zero.  Base pointer 16-byte aligned.
+ *   - Proxy-K buffer: fasa_proxy_bytes() bytes, 16-byte aligned, zero-filled once by
+ *     the caller.  Per (batch, kv head) it holds ceil(max_len / 16) tiles of 16 tokens;
+ *     a token owns proxy_row_elems = 8 * ceil(n_dom / 4) bf16 values: for the head's
+ *     dominant FCs sorted ascending, the pairs (K[j][c0], K[j][c1]), zero padded.
+ *     Inside a tile the values are stored in the operand order of the tensor-core
+ *     instruction that scores them (blocks of 16 channels, 512 bytes each, lane
+ *     4g+t of a warp owning {P[g][2t..2t+1], P[g+8][2t..2t+1], P[g][2t+8..2t+9],
+ *     P[g+8][2t+8..2t+9]}; a trailing block of 8 channels, 256 bytes, when
+ *     ceil(n_dom / 4) is odd).  Only fasa_kv_append, fasa_proxy_build and
+ *     fasa_append_decode_step write it; treat it as opaque.
  *   - Data-dependent problems (a sequence longer than max_len, an index out of
  *     range) never fault: the kernel clamps and ORs a bit into a device status
  *     word read by fasa_get_device_status.
@@ -82,8 +88,11 @@ typedef struct {
 int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_host, fasa_ctx_t** out);
 int32_t fasa_destroy(fasa_ctx_t* ctx);
 
-/* Elements per proxy-K row for n_dom dominant FCs: 8 * ceil(n_dom / 4). */
+/* bf16 values per token in the proxy-K buffer for n_dom dominant FCs: 8 * ceil(n_dom / 4). */
 int32_t fasa_proxy_row_elems(int32_t n_dom);
+/* Size of the proxy-K buffer of this context:
+ * batch * n_kv_heads * 16 * ceil(max_len / 16) * proxy_row_elems * 2 bytes. */
+int32_t fasa_proxy_bytes(const fasa_ctx_t* ctx, size_t* out_bytes);
 
 /* Bytes of caller-provided scratch that fasa_topk, the two attention calls and
  * fasa_decode_step need for selections of at most n_sel_max tokens.  The

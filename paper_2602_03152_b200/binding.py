@@ -26,7 +26,7 @@ SYMBOLS = [
     "fasa_kv_append", "fasa_proxy_build", "fasa_fc_score", "fasa_topk", "fasa_sparse_decode_attn",
     "fasa_full_decode_attn", "fasa_decode_step", "fasa_stage_bytes", "fasa_decode_step_host",
     "fasa_sparse_decode_attn_static", "fasa_set_step_mode", "fasa_step_cluster_size",
-    "fasa_append_decode_step",
+    "fasa_append_decode_step", "fasa_proxy_bytes",
 ]
 
 
@@ -65,6 +65,7 @@ def load_library() -> ctypes.CDLL:
         "fasa_create": (i32, [ctypes.POINTER(FasaConfig), vp, ctypes.POINTER(vp)]),
         "fasa_destroy": (i32, [vp]),
         "fasa_proxy_row_elems": (i32, [i32]),
+        "fasa_proxy_bytes": (i32, [vp, ctypes.POINTER(ctypes.c_size_t)]),
         "fasa_workspace_bytes": (i32, [vp, i32, ctypes.POINTER(ctypes.c_size_t)]),
         "fasa_status_string": (ctypes.c_char_p, [i32]),
         "fasa_last_cuda_error": (ctypes.c_char_p, [vp]),
@@ -184,9 +185,18 @@ class Fasa:
         return int(out.value)
 
     # -- device buffers (torch is the allocator) -------------------------------
+    def proxy_bytes(self) -> int:
+        out = ctypes.c_size_t()
+        self._check(self._lib.fasa_proxy_bytes(self._h, ctypes.byref(out)), "fasa_proxy_bytes")
+        return int(out.value)
+
     def alloc_proxy(self, device="cuda") -> torch.Tensor:
-        return torch.zeros((self.batch, self.n_kv_heads, self.max_len, self.row_elems),
-                           dtype=torch.bfloat16, device=device)
+        """Zero-filled proxy-K buffer: [batch, kv heads, tiles of 16 tokens, 16 * row_elems] bf16
+        (opaque tile-internal order, see include/fasa.h)."""
+        tiles = (self.max_len + 15) // 16
+        t = torch.zeros((self.batch, self.n_kv_heads, tiles, 16 * self.row_elems), dtype=torch.bfloat16, device=device)
+        assert t.numel() * 2 == self.proxy_bytes()
+        return t
 
     def alloc_workspace(self, n_sel_max: int, device="cuda") -> torch.Tensor:
         return torch.empty(self.workspace_bytes(n_sel_max), dtype=torch.uint8, device=device)

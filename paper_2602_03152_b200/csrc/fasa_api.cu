@@ -41,6 +41,14 @@ extern "C" int32_t fasa_proxy_row_elems(int32_t n_dom) {
   return 8 * ((n_dom + 3) / 4);
 }
 
+extern "C" int32_t fasa_proxy_bytes(const fasa_ctx_t* ctx, size_t* out_bytes) {
+  if (!ctx || !out_bytes) return FASA_ERR_INVALID_ARG;
+  const fasa_config_t& c = ctx->cfg;
+  const size_t rows = (size_t)((c.max_len + 15) / 16) * 16;
+  *out_bytes = (size_t)c.batch * c.n_kv_heads * rows * ctx->row_elems * 2;
+  return FASA_OK;
+}
+
 extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_host,
                                fasa_ctx_t** out) {
   if (!cfg || !dom_fc_host || !out) return FASA_ERR_INVALID_ARG;

@@ -1,21 +1,23 @@
 // Cache update: K/V rows plus the packed dominant-FC proxy rows (Algorithm 2: Split,
 // UpdateCache), and the one-off proxy build from an existing key cache.
 #include "fasa_common.cuh"
+#include "fasa_score_core.cuh"
 
 namespace {
 
-// 64 threads per appended row: 16 copy the K row, 16 the V row (16 bytes each),
-// up to 16 assemble the proxy row (8 gathered channels = 16 bytes each).
+// 128 threads per appended row: 16 copy the K row, 16 the V row (16 bytes each), up to 64
+// write the proxy words (one dominant FC = one 4-byte channel pair each) to their places in
+// the tiled proxy layout.
 __global__ void __launch_bounds__(256)
 kv_append_kernel(uint16_t* __restrict__ k_cache, uint16_t* __restrict__ v_cache,
-                 uint16_t* __restrict__ proxy, const int32_t* __restrict__ seq_lens,
+                 unsigned char* __restrict__ proxy, const int32_t* __restrict__ seq_lens,
                  const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
                  const int16_t* __restrict__ chan, int32_t* __restrict__ status, int n_rows,
                  int n_new, int n_kv_heads, int max_len, int chunks, int64_t ksb, int64_t ksh,
                  int64_t kst, int64_t vsb, int64_t vsh, int64_t vst) {
-  const int row = blockIdx.x * 4 + (threadIdx.x >> 6);
+  const int row = blockIdx.x * 2 + (threadIdx.x >> 7);
   if (row >= n_rows) return;
-  const int t = threadIdx.x & 63;
+  const int t = threadIdx.x & 127;
   const int n = row % n_new;
   const int u = row / n_new;  // unit = b * n_kv_heads + h
   const int h = u % n_kv_heads;
@@ -34,20 +36,15 @@ kv_append_kernel(uint16_t* __restrict__ k_cache, uint16_t* __restrict__ v_cache,
     const int c = t - 16;
     uint4 x = *reinterpret_cast<const uint4*>(v_new + (int64_t)row * FASA_HEAD_DIM + c * 8);
     *reinterpret_cast<uint4*>(v_cache + b * vsb + h * vsh + pos * vst + c * 8) = x;
-  } else if (t - 32 < chunks) {
-    const int c = t - 32;
-    const int row_elems = chunks * 8;
-    const int16_t* ch = chan + h * row_elems + c * 8;
-    uint32_t w[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      int c0 = ch[2 * e], c1 = ch[2 * e + 1];
-      uint32_t lo = c0 >= 0 ? ksrc[c0] : 0u;
-      uint32_t hi = c1 >= 0 ? ksrc[c1] : 0u;
-      w[e] = lo | (hi << 16);
-    }
-    uint16_t* dst = proxy + ((int64_t)u * max_len + pos) * row_elems + c * 8;
-    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+  } else if (t - 32 < 4 * chunks) {
+    const int w = t - 32;
+    const ProxyGeom pg = proxy_geom(chunks);
+    const int16_t* ch = chan + h * chunks * 8 + 2 * w;
+    const int c0 = ch[0], c1 = ch[1];
+    const uint32_t lo = c0 >= 0 ? ksrc[c0] : 0u;
+    const uint32_t hi = c1 >= 0 ? ksrc[c1] : 0u;
+    unsigned char* unit = proxy + (int64_t)u * ((max_len + 15) >> 4) * pg.tile_bytes;
+    *reinterpret_cast<uint32_t*>(unit + proxy_word_offset(pg, pos, w)) = lo | (hi << 16);
   }
 }
 
@@ -60,9 +57,9 @@ __global__ void seq_len_bump_kernel(int32_t* __restrict__ seq_lens, int batch, i
   seq_lens[b] = len > max_len ? max_len : len;
 }
 
-// One thread per 16-byte proxy chunk of rows 0 .. seq_lens[b]-1.
+// One thread per proxy word of rows 0 .. seq_lens[b]-1.
 __global__ void __launch_bounds__(256)
-proxy_build_kernel(const uint16_t* __restrict__ k_cache, uint16_t* __restrict__ proxy,
+proxy_build_kernel(const uint16_t* __restrict__ k_cache, unsigned char* __restrict__ proxy,
                    const int32_t* __restrict__ seq_lens, const int16_t* __restrict__ chan,
                    int32_t* __restrict__ status, int n_kv_heads, int max_len, int chunks,
                    int64_t ksb, int64_t ksh, int64_t kst) {
@@ -70,23 +67,19 @@ proxy_build_kernel(const uint16_t* __restrict__ k_cache, uint16_t* __restrict__ 
   const int h = u % n_kv_heads;
   const int b = u / n_kv_heads;
   const int len = clamp_len(seq_lens[b], max_len, status);
+  const int words = 4 * chunks;
   const int64_t item = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int j = (int)(item / chunks);
-  const int c = (int)(item % chunks);
+  const int j = (int)(item / words);
+  const int w = (int)(item % words);
   if (j >= len) return;
-  const int row_elems = chunks * 8;
-  const int16_t* ch = chan + h * row_elems + c * 8;
+  const ProxyGeom pg = proxy_geom(chunks);
+  const int16_t* ch = chan + h * chunks * 8 + 2 * w;
   const uint16_t* ksrc = k_cache + b * ksb + h * ksh + (int64_t)j * kst;
-  uint32_t w[4];
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    int c0 = ch[2 * e], c1 = ch[2 * e + 1];
-    uint32_t lo = c0 >= 0 ? ksrc[c0] : 0u;
-    uint32_t hi = c1 >= 0 ? ksrc[c1] : 0u;
-    w[e] = lo | (hi << 16);
-  }
-  uint16_t* dst = proxy + ((int64_t)u * max_len + j) * row_elems + c * 8;
-  *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+  const int c0 = ch[0], c1 = ch[1];
+  const uint32_t lo = c0 >= 0 ? ksrc[c0] : 0u;
+  const uint32_t hi = c1 >= 0 ? ksrc[c1] : 0u;
+  unsigned char* unit = proxy + (int64_t)u * ((max_len + 15) >> 4) * pg.tile_bytes;
+  *reinterpret_cast<uint32_t*>(unit + proxy_word_offset(pg, j, w)) = lo | (hi << 16);
 }
 
 bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
@@ -105,8 +98,8 @@ extern "C" int32_t fasa_kv_append(fasa_ctx_t* ctx, void* k_cache, void* v_cache,
   long long n_rows = (long long)c.batch * c.n_kv_heads * n_new;
   if (n_rows > (1ll << 30)) return FASA_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  kv_append_kernel<<<(unsigned)((n_rows + 3) / 4), 256, 0, s>>>(
-      (uint16_t*)k_cache, (uint16_t*)v_cache, (uint16_t*)proxy_k, seq_lens, (const uint16_t*)k_new,
+  kv_append_kernel<<<(unsigned)((n_rows + 1) / 2), 256, 0, s>>>(
+      (uint16_t*)k_cache, (uint16_t*)v_cache, (unsigned char*)proxy_k, seq_lens, (const uint16_t*)k_new,
       (const uint16_t*)v_new, ctx->d_chan, ctx->d_status, (int)n_rows, n_new, c.n_kv_heads,
       c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h, c.k_stride_t, c.v_stride_b,
       c.v_stride_h, c.v_stride_t);
@@ -122,10 +115,10 @@ extern "C" int32_t fasa_proxy_build(fasa_ctx_t* ctx, const void* k_cache, void* 
   if (!ctx || !k_cache || !proxy_k || !seq_lens) return FASA_ERR_INVALID_ARG;
   if (!aligned16(k_cache) || !aligned16(proxy_k)) return FASA_ERR_INVALID_ARG;
   const fasa_config_t& c = ctx->cfg;
-  long long items = (long long)c.max_len * ctx->chunks;
+  long long items = (long long)c.max_len * ctx->chunks * 4;
   dim3 grid((unsigned)((items + 255) / 256), (unsigned)(c.batch * c.n_kv_heads));
   proxy_build_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(
-      (const uint16_t*)k_cache, (uint16_t*)proxy_k, seq_lens, ctx->d_chan, ctx->d_status,
+      (const uint16_t*)k_cache, (unsigned char*)proxy_k, seq_lens, ctx->d_chan, ctx->d_status,
       c.n_kv_heads, c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h, c.k_stride_t);
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;

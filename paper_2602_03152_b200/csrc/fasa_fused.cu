@@ -2,8 +2,9 @@
 //
 // One thread-block cluster per (batch, KV head) unit.  The CTAs of the cluster cut the unit's
 // cached tokens into contiguous slices and
-//   1. stream their slice of the proxy-K buffer once (16-byte loads, 8 in flight per thread),
-//      keep every token's selection key in shared memory and histogram its top 11 bits;
+//   1. stream their slice of the tiled proxy-K buffer once (16-byte loads in tensor-core
+//      fragment order, scored with mma.sync), keep every token's selection key in shared
+//      memory and histogram its top 11 bits;
 //   2. find the budget-th largest key by an MSB-first radix select (11 + 11 + 10 bits): each
 //      pass needs one cluster barrier, after which every CTA reads the other CTAs' coarse and
 //      fine bin counts through distributed shared memory and locates the bin redundantly;
@@ -28,7 +29,6 @@ namespace {
 constexpr int kFT = 256;               // threads per CTA (two CTAs share an SM)
 constexpr int kFW = kFT / 32;          // warps per CTA
 constexpr int kFBins = 2048;           // bins of the widest radix pass
-constexpr int kFUnroll = 8;            // proxy loads in flight per thread
 constexpr int kPartStride = FASA_HEAD_DIM + 2;   // m, l, acc[128]
 constexpr int kCapMax = 22528;         // keys a CTA can hold (88 KB of shared memory)
 constexpr int kCapPair = 16384;        // ... and still leave room for a second CTA on the SM
@@ -37,7 +37,7 @@ struct FusedParams {
   const uint16_t* q;
   const uint16_t* k;
   const uint16_t* v;
-  const uint4* proxy;
+  const unsigned char* proxy;
   const int32_t* seq_lens;
   const int16_t* chan;
   // append-then-step form (all null / unused otherwise): the new token's rows, the buffers
@@ -46,7 +46,7 @@ struct FusedParams {
   const uint16_t* v_new;
   uint16_t* k_w;
   uint16_t* v_w;
-  uint16_t* proxy_w;
+  unsigned char* proxy_w;
   int32_t* seq_lens_w;
   int32_t* arrive;
   float* scores;           // nullable
@@ -63,17 +63,6 @@ struct FusedParams {
 __device__ __forceinline__ uint2 ld_stream_u2(const void* p) {
   uint2 r;
   asm volatile("ld.global.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p) : "memory");
-  return r;
-}
-
-// 128-bit load through the coherent path (not .nc): in the append-then-step form the last
-// proxy / K / V row was written earlier in this same launch.
-__device__ __forceinline__ uint4 ld_coherent_u4(const void* p) {
-  uint4 r;
-  asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-               : "l"(p)
-               : "memory");
   return r;
 }
 
@@ -102,8 +91,9 @@ __device__ __forceinline__ bool warp_find_kth(uint32_t v, uint32_t kth, int lane
   return true;
 }
 
-// LPR = lanes per proxy row; GP = query heads padded to 4 or 8.
-template <int LPR, int GP>
+// KB = 16-channel blocks per proxy tile rounded up to a power of two; GP = query heads padded
+// to 4 or 8.
+template <int KB, int GP>
 __global__ void __launch_bounds__(kFT, 2)
 fused_decode_kernel(const FusedParams p) {
   cg::cluster_group cluster = cg::this_cluster();
@@ -187,19 +177,15 @@ fused_decode_kernel(const FusedParams p) {
       const int c = tid - 16;
       *reinterpret_cast<uint4*>(p.v_w + b * p.vsb + h * p.vsh + (int64_t)len_old * p.vst + c * 8) =
           *reinterpret_cast<const uint4*>(p.v_new + (int64_t)u * FASA_HEAD_DIM + c * 8);
-    } else if (tid - 32 < p.chunks) {
-      const int c = tid - 32;
-      const int16_t* ch = p.chan + h * p.chunks * 8 + c * 8;
-      uint32_t w[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int ch0 = ch[2 * e], ch1 = ch[2 * e + 1];
-        const uint32_t lo = ch0 >= 0 ? ksrc[ch0] : 0u;
-        const uint32_t hi = ch1 >= 0 ? ksrc[ch1] : 0u;
-        w[e] = lo | (hi << 16);
-      }
-      *reinterpret_cast<uint4*>(p.proxy_w + ((int64_t)u * p.max_len + len_old) * (p.chunks * 8) + c * 8) =
-          make_uint4(w[0], w[1], w[2], w[3]);
+    } else if (tid - 32 < 4 * p.chunks) {
+      const int w = tid - 32;                       // one dominant FC = one 4-byte channel pair
+      const ProxyGeom pg = proxy_geom(p.chunks);
+      const int16_t* ch = p.chan + h * p.chunks * 8 + 2 * w;
+      const int ch0 = ch[0], ch1 = ch[1];
+      const uint32_t lo = ch0 >= 0 ? ksrc[ch0] : 0u;
+      const uint32_t hi = ch1 >= 0 ? ksrc[ch1] : 0u;
+      unsigned char* unit = p.proxy_w + (int64_t)u * ((p.max_len + 15) >> 4) * pg.tile_bytes;
+      *reinterpret_cast<uint32_t*>(unit + proxy_word_offset(pg, len_old, w)) = lo | (hi << 16);
     }
   }
   for (int i = tid; i < 2 * kFBins; i += kFT) hist0[i] = 0u;
@@ -218,45 +204,43 @@ fused_decode_kernel(const FusedParams p) {
 
   // ---- 1. scoring stream -> keys + first histogram ------------------------------------------
   {
-    constexpr int RPL = 32 / LPR;
-    constexpr int RPI = RPL * kFUnroll;
-    const int sub = lane & (LPR - 1);
-    const int grp = lane / LPR;
-    const bool live = sub < p.chunks;
-    const uint4* prow = p.proxy + (int64_t)u * p.max_len * p.chunks;
+    constexpr int TPI = KB == 1 ? 8 : (KB == 2 ? 4 : 2);      // tiles per warp iteration
+    const ProxyGeom pg = proxy_geom(p.chunks);
+    const int n_blocks = pg.n16 + pg.n8;
+    const unsigned char* unit = p.proxy + (int64_t)u * ((p.max_len + 15) >> 4) * pg.tile_bytes;
     float* srow = p.scores ? p.scores + (int64_t)u * p.max_len : nullptr;
 
-    auto issue = [&](uint4 (&x)[kFUnroll], int base) {
+    int T = ((crank * per) >> 4) + warp * TPI;                // slices start on a tile boundary
+    uint4 a[TPI][KB];
 #pragma unroll
-      for (int i = 0; i < kFUnroll; ++i) {
-        const int row = base + i * RPL + grp;
-        x[i] = (live && row < c1) ? ld_coherent_u4(prow + (int64_t)row * p.chunks + sub)
-                                  : make_uint4(0u, 0u, 0u, 0u);
+    for (int j = 0; j < TPI; ++j)
+      load_tile<KB>(a[j], unit + (int64_t)(T + j) * pg.tile_bytes, pg, lane, (T + j) * 16 < c1);
+    ScoreFrag<KB> f;
+    load_score_b<KB>(f, p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM,
+                     p.chan + h * p.chunks * 8, p.chunks, p.group, lane);
+    while (T * 16 < c1) {       // uniform over the warp
+      float s_lo[TPI], s_hi[TPI];
+#pragma unroll
+      for (int j = 0; j < TPI; ++j) score_tile<KB, false>(a[j], f, n_blocks, p.group, lane, s_lo[j], s_hi[j]);
+      const int next = T + kFW * TPI;
+      if (next * 16 < c1) {     // next loads fly while keys are made
+#pragma unroll
+        for (int j = 0; j < TPI; ++j)
+          load_tile<KB>(a[j], unit + (int64_t)(next + j) * pg.tile_bytes, pg, lane, (next + j) * 16 < c1);
       }
-    };
-    const int stride = kFW * RPI;
-    int base = c0 + warp * RPI;
-    uint4 x[kFUnroll];
-    issue(x, base);
-    ScoreQ<false> sq;
-    load_score_q<false>(sq, p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM,
-                        p.chan + h * p.chunks * 8 + (live ? sub : 0) * 8, p.group, live);
-    while (base < c1) {
-      float sc[kFUnroll];
 #pragma unroll
-      for (int i = 0; i < kFUnroll; ++i) sc[i] = score_row<LPR, false>(sq, x[i], p.group);
-      if (base + stride < c1) issue(x, base + stride);   // next loads fly while keys are made
-#pragma unroll
-      for (int i = 0; i < kFUnroll; ++i) {
-        const int row = base + i * RPL + grp;
-        if (sub == 0 && row < c1) {
-          const uint32_t key = fasa_item_key(sc[i], row, len, p.n_sink, p.n_recent);
+      for (int pr = 0; pr < TPI / 2; ++pr) {
+        float sc;
+        const int row = (T + 2 * pr) * 16 +
+                        pick_row_of_pair(lane, s_lo[2 * pr], s_hi[2 * pr], s_lo[2 * pr + 1], s_hi[2 * pr + 1], sc);
+        if (row < c1) {
+          const uint32_t key = fasa_item_key(sc, row, len, p.n_sink, p.n_recent);
           atomicAdd(&hist0[key >> 21], 1u);
           keys[row - c0] = key;
-          if (srow) srow[row] = sc[i];
+          if (srow) srow[row] = sc;
         }
       }
-      base += stride;
+      T = next;
     }
   }
   __syncthreads();
@@ -653,11 +637,11 @@ using FusedFn = void (*)(const FusedParams);
 
 template <int GP>
 FusedFn fused_fn_lpr(int chunks) {
-  if (chunks <= 1) return fused_decode_kernel<1, GP>;
-  if (chunks <= 2) return fused_decode_kernel<2, GP>;
-  if (chunks <= 4) return fused_decode_kernel<4, GP>;
-  if (chunks <= 8) return fused_decode_kernel<8, GP>;
-  return fused_decode_kernel<16, GP>;
+  const int nb = (chunks + 1) / 2;      // 16-channel blocks per tile, the 8-channel one included
+  if (nb <= 1) return fused_decode_kernel<1, GP>;
+  if (nb <= 2) return fused_decode_kernel<2, GP>;
+  if (nb <= 4) return fused_decode_kernel<4, GP>;
+  return fused_decode_kernel<8, GP>;
 }
 
 }  // namespace
@@ -724,9 +708,9 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
   const fasa_config_t& c = ctx->cfg;
   FusedParams p;
   p.q = (const uint16_t*)q; p.k = (const uint16_t*)k_cache; p.v = (const uint16_t*)v_cache;
-  p.proxy = (const uint4*)proxy_k; p.seq_lens = seq_lens; p.chan = ctx->d_chan;
+  p.proxy = (const unsigned char*)proxy_k; p.seq_lens = seq_lens; p.chan = ctx->d_chan;
   p.k_new = (const uint16_t*)k_new; p.v_new = (const uint16_t*)v_new;
-  p.k_w = (uint16_t*)k_cache; p.v_w = (uint16_t*)v_cache; p.proxy_w = (uint16_t*)proxy_k;
+  p.k_w = (uint16_t*)k_cache; p.v_w = (uint16_t*)v_cache; p.proxy_w = (unsigned char*)proxy_k;
   p.seq_lens_w = (int32_t*)seq_lens; p.arrive = ctx->d_arrive;
   p.scores = scores; p.idx = idx; p.n_sel = n_sel; p.out = out; p.lse = lse; p.status = ctx->d_status;
   p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group; p.max_len = c.max_len;

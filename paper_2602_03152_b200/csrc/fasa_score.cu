@@ -1,102 +1,100 @@
 // TIP scoring (Sec. 4.1): S[j] = reduce_g sum_{i in I_dom} alpha^(i)_g[j], streamed from the
-// packed proxy-K buffer.  HBM-bound: every proxy byte is read once with 128-bit loads that
-// are contiguous across the warp, each thread keeps UNROLL loads in flight, and the lanes
-// that share a row combine their partial sums with xor-shuffles.
+// tiled proxy-K buffer.  Every proxy byte is read once: a warp fetches whole 512-byte blocks
+// (16 bytes per lane, already in tensor-core fragment order) and turns 16 tokens x 16
+// channels x up to 8 query heads into partial scores with one mma.sync; several tiles are in
+// flight per warp, and the first batch of loads is issued before the sequence length, the
+// channel table and the query are known.
 #include "fasa_common.cuh"
 #include "fasa_score_core.cuh"
 
 namespace {
 
 constexpr int kScoreThreads = 256;
-constexpr int kScoreUnroll = 8;
+constexpr int kScoreWarps = kScoreThreads / 32;
 
-// LPR = lanes per proxy row (power of two >= chunks).  MAXRED = reduce the group by max
-// (one dot product per query head) instead of by sum (one dot product with sum_g q_g).
-template <int LPR, bool MAXRED>
+// Tiles a warp handles per iteration (even; about 8 loads in flight per lane).
+template <int KB>
+struct TilesPerIter {
+  static constexpr int value = KB == 1 ? 8 : (KB == 2 ? 4 : 2);
+};
+
+// KB = 16-channel blocks per tile rounded up to a power of two (1, 2, 4, 8).
+template <int KB, bool MAXRED>
 __global__ void __launch_bounds__(kScoreThreads)
-fc_score_kernel(const uint16_t* __restrict__ q, const uint4* __restrict__ proxy,
+fc_score_kernel(const uint16_t* __restrict__ q, const unsigned char* __restrict__ proxy,
                 const int32_t* __restrict__ seq_lens, const int16_t* __restrict__ chan,
                 float* __restrict__ scores, int32_t* __restrict__ status, int n_q_heads,
-                int n_kv_heads, int group, int max_len, int chunks, int rows_per_cta) {
-  constexpr int RPL = 32 / LPR;                 // rows covered by one warp-wide load
-  constexpr int RPI = RPL * kScoreUnroll;       // rows per warp iteration
-
+                int n_kv_heads, int group, int max_len, int chunks, int tiles_per_cta) {
+  constexpr int TPI = TilesPerIter<KB>::value;
   const int u = blockIdx.y;
   const int h = u % n_kv_heads;
   const int b = u / n_kv_heads;
-  const int cta_row0 = blockIdx.x * rows_per_cta;
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
-  const int sub = lane & (LPR - 1);             // which 16-byte chunk of the row
-  const int grp = lane / LPR;                   // which row of the warp-wide load
-  const bool live = sub < chunks;
-  const uint4* prow = proxy + (int64_t)u * max_len * chunks;
+  const ProxyGeom pg = proxy_geom(chunks);
+  const int n_blocks = pg.n16 + pg.n8;
+  const int tiles_alloc = (max_len + 15) >> 4;
+  const int cta_tile0 = blockIdx.x * tiles_per_cta;
+  const int cta_tile1 = min(tiles_alloc, cta_tile0 + tiles_per_cta);
+  const unsigned char* unit = proxy + (int64_t)u * tiles_alloc * pg.tile_bytes;
 
-  // The first batch of proxy loads is issued before anything else is known: rows up to
-  // max_len are allocated, so reading past the sequence length is harmless, and the loads of
-  // the length, the channel table and the query overlap with the stream instead of
-  // preceding it.
-  const int alloc_row1 = min(max_len, cta_row0 + rows_per_cta);
-  int base = cta_row0 + warp * RPI;
-  uint4 x[kScoreUnroll];
+  // First batch of loads: every tile up to max_len is allocated, so reading past the
+  // sequence length is harmless and overlaps with the loads of the length and the query.
+  int T = cta_tile0 + warp * TPI;
+  uint4 a[TPI][KB];
 #pragma unroll
-  for (int i = 0; i < kScoreUnroll; ++i) {
-    const int row = base + i * RPL + grp;
-    x[i] = (live && row < alloc_row1) ? ld_stream_u4(prow + (int64_t)row * chunks + sub)
-                                      : make_uint4(0u, 0u, 0u, 0u);
-  }
+  for (int j = 0; j < TPI; ++j)
+    load_tile<KB>(a[j], unit + (int64_t)(T + j) * pg.tile_bytes, pg, lane, T + j < cta_tile1);
 
   const int len = clamp_len(seq_lens[b], max_len, status);
-  if (cta_row0 >= len) return;
-  const int cta_row1 = min(len, cta_row0 + rows_per_cta);
+  if (cta_tile0 * 16 >= len) return;
+  const int row1 = min(len, cta_tile1 * 16);
 
-  ScoreQ<MAXRED> sq;
-  load_score_q<MAXRED>(sq, q + ((int64_t)b * n_q_heads + (int64_t)h * group) * FASA_HEAD_DIM,
-                       chan + h * chunks * 8 + (live ? sub : 0) * 8, group, live);
+  ScoreFrag<KB> f;
+  load_score_b<KB>(f, q + ((int64_t)b * n_q_heads + (int64_t)h * group) * FASA_HEAD_DIM,
+                   chan + h * chunks * 8, chunks, group, lane);
   float* srow = scores + (int64_t)u * max_len;
 
-  while (base < cta_row1) {
-    float s[kScoreUnroll];
+  while (T * 16 < row1) {       // uniform over the warp
+    float s_lo[TPI], s_hi[TPI];
 #pragma unroll
-    for (int i = 0; i < kScoreUnroll; ++i) s[i] = score_row<LPR, MAXRED>(sq, x[i], group);
-    const int next = base + (kScoreThreads / 32) * RPI;
-    if (next < cta_row1) {
+    for (int j = 0; j < TPI; ++j) score_tile<KB, MAXRED>(a[j], f, n_blocks, group, lane, s_lo[j], s_hi[j]);
+    const int next = T + kScoreWarps * TPI;
+    if (next * 16 < row1) {
 #pragma unroll
-      for (int i = 0; i < kScoreUnroll; ++i) {
-        const int row = next + i * RPL + grp;
-        x[i] = (live && row < cta_row1) ? ld_stream_u4(prow + (int64_t)row * chunks + sub)
-                                        : make_uint4(0u, 0u, 0u, 0u);
-      }
+      for (int j = 0; j < TPI; ++j)
+        load_tile<KB>(a[j], unit + (int64_t)(next + j) * pg.tile_bytes, pg, lane, (next + j) * 16 < row1);
     }
 #pragma unroll
-    for (int i = 0; i < kScoreUnroll; ++i) {
-      const int row = base + i * RPL + grp;
-      if (sub == 0 && row < cta_row1) srow[row] = s[i];
+    for (int p = 0; p < TPI / 2; ++p) {
+      float v;
+      const int row = (T + 2 * p) * 16 + pick_row_of_pair(lane, s_lo[2 * p], s_hi[2 * p], s_lo[2 * p + 1], s_hi[2 * p + 1], v);
+      if (row < row1) srow[row] = v;
     }
-    base = next;
+    T = next;
   }
 }
 
-template <int LPR>
+template <int KB>
 void launch_score(fasa_ctx* ctx, const void* q, const void* proxy, const int32_t* seq_lens,
                   float* scores, cudaStream_t s) {
   const fasa_config_t& c = ctx->cfg;
   const int units = c.batch * c.n_kv_heads;
   // Enough CTAs to cover the SMs several times, at least one warp iteration each.
-  constexpr int RPI_CTA = (32 / LPR) * kScoreUnroll * (kScoreThreads / 32);
-  int want_ctas = (8 * ctx->n_sm + units - 1) / units;
-  int rows = (c.max_len + want_ctas - 1) / want_ctas;
-  rows = (rows + RPI_CTA - 1) / RPI_CTA * RPI_CTA;
-  if (rows < RPI_CTA) rows = RPI_CTA;
-  dim3 grid((unsigned)((c.max_len + rows - 1) / rows), (unsigned)units);
+  constexpr int kStep = TilesPerIter<KB>::value * kScoreWarps;
+  const int tiles = (c.max_len + 15) / 16;
+  const int want_ctas = (8 * ctx->n_sm + units - 1) / units;
+  int per = (tiles + want_ctas - 1) / want_ctas;
+  per = (per + kStep - 1) / kStep * kStep;
+  dim3 grid((unsigned)((tiles + per - 1) / per), (unsigned)units);
   if (c.group_reduce == 0)
-    fc_score_kernel<LPR, false><<<grid, kScoreThreads, 0, s>>>(
-        (const uint16_t*)q, (const uint4*)proxy, seq_lens, ctx->d_chan, scores, ctx->d_status,
-        c.n_q_heads, c.n_kv_heads, ctx->group, c.max_len, ctx->chunks, rows);
+    fc_score_kernel<KB, false><<<grid, kScoreThreads, 0, s>>>(
+        (const uint16_t*)q, (const unsigned char*)proxy, seq_lens, ctx->d_chan, scores, ctx->d_status,
+        c.n_q_heads, c.n_kv_heads, ctx->group, c.max_len, ctx->chunks, per);
   else
-    fc_score_kernel<LPR, true><<<grid, kScoreThreads, 0, s>>>(
-        (const uint16_t*)q, (const uint4*)proxy, seq_lens, ctx->d_chan, scores, ctx->d_status,
-        c.n_q_heads, c.n_kv_heads, ctx->group, c.max_len, ctx->chunks, rows);
+    fc_score_kernel<KB, true><<<grid, kScoreThreads, 0, s>>>(
+        (const uint16_t*)q, (const unsigned char*)proxy, seq_lens, ctx->d_chan, scores, ctx->d_status,
+        c.n_q_heads, c.n_kv_heads, ctx->group, c.max_len, ctx->chunks, per);
 }
 
 }  // namespace
@@ -107,12 +105,11 @@ extern "C" int32_t fasa_fc_score(fasa_ctx_t* ctx, const void* q, const void* pro
   if (((uintptr_t)proxy_k & 15) != 0 || ((uintptr_t)q & 1) != 0 || ((uintptr_t)scores & 3) != 0)
     return FASA_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  const int ch = ctx->chunks;
-  if (ch <= 1) launch_score<1>(ctx, q, proxy_k, seq_lens, scores, s);
-  else if (ch <= 2) launch_score<2>(ctx, q, proxy_k, seq_lens, scores, s);
-  else if (ch <= 4) launch_score<4>(ctx, q, proxy_k, seq_lens, scores, s);
-  else if (ch <= 8) launch_score<8>(ctx, q, proxy_k, seq_lens, scores, s);
-  else launch_score<16>(ctx, q, proxy_k, seq_lens, scores, s);
+  const int nb = (ctx->chunks + 1) / 2;      // 16-channel blocks per tile, the 8-channel one included
+  if (nb <= 1) launch_score<1>(ctx, q, proxy_k, seq_lens, scores, s);
+  else if (nb <= 2) launch_score<2>(ctx, q, proxy_k, seq_lens, scores, s);
+  else if (nb <= 4) launch_score<4>(ctx, q, proxy_k, seq_lens, scores, s);
+  else launch_score<8>(ctx, q, proxy_k, seq_lens, scores, s);
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
 }

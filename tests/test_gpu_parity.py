@@ -278,20 +278,41 @@ def test_strided_token_major_cache():
 # ------------------------------------------------------------------ cache update ----
 
 def _expected_proxy(k_bits_cpu, dom_sorted, pairing, row_elems, lens):
-    """Proxy layout by plain indexing: pairs (K[c0], K[c1]) of the sorted dominant FCs, zero padded."""
+    """The documented proxy layout by plain indexing.  Logical row j of a head = the pairs
+    (K[j][c0], K[j][c1]) of its sorted dominant FCs, zero padded; tiles of 16 rows; inside a tile
+    blocks of 16 channels in tensor-core operand order (lane 4g+t: P[g][2t..2t+1], P[g+8][2t..2t+1],
+    P[g][2t+8..2t+9], P[g+8][2t+8..2t+9]), then one block of 8 channels if the chunk count is odd."""
     B, H, Lm, _ = k_bits_cpu.shape
-    out = torch.zeros((B, H, Lm, row_elems), dtype=torch.int16)
+    tiles = (Lm + 15) // 16
+    logical = torch.zeros((B, H, tiles * 16, row_elems), dtype=torch.int16)
     for h in range(H):
         for r, i in enumerate(dom_sorted[h].tolist()):
             c0, c1 = (i, i + 64) if pairing == 0 else (2 * i, 2 * i + 1)
-            out[:, h, :, 2 * r] = k_bits_cpu[:, h, :, c0]
-            out[:, h, :, 2 * r + 1] = k_bits_cpu[:, h, :, c1]
+            logical[:, h, :Lm, 2 * r] = k_bits_cpu[:, h, :, c0]
+            logical[:, h, :Lm, 2 * r + 1] = k_bits_cpu[:, h, :, c1]
     for b in range(B):
-        out[b, :, int(lens[b]):] = 0
+        logical[b, :, int(lens[b]):] = 0
+    chunks = row_elems // 8
+    n16, n8 = chunks // 2, chunks % 2
+    out = torch.zeros((B, H, tiles, 16 * row_elems), dtype=torch.int16)
+    lg = logical.view(B, H, tiles, 16, row_elems)
+    for kb in range(n16):
+        for g in range(8):
+            for t in range(4):
+                base = kb * 256 + (g * 4 + t) * 8                  # in 2-byte elements
+                for e, (rr, cc) in enumerate([(g, 2 * t), (g, 2 * t + 1), (g + 8, 2 * t), (g + 8, 2 * t + 1),
+                                              (g, 2 * t + 8), (g, 2 * t + 9), (g + 8, 2 * t + 8), (g + 8, 2 * t + 9)]):
+                    out[:, :, :, base + e] = lg[:, :, :, rr, kb * 16 + cc]
+    if n8:
+        for g in range(8):
+            for t in range(4):
+                base = n16 * 256 + (g * 4 + t) * 4
+                for e, (rr, cc) in enumerate([(g, 2 * t), (g, 2 * t + 1), (g + 8, 2 * t), (g + 8, 2 * t + 1)]):
+                    out[:, :, :, base + e] = lg[:, :, :, rr, n16 * 16 + cc]
     return out
 
 
-@pytest.mark.parametrize("F,pairing", [(16, 0), (5, 0), (16, 1), (64, 0), (1, 1)])
+@pytest.mark.parametrize("F,pairing", [(16, 0), (5, 0), (16, 1), (64, 0), (1, 1), (12, 0), (40, 1)])
 def test_proxy_build_layout_is_bit_exact(F, pairing):
     w = C["c2"].replace(batch=2, max_len=300, len_lo=100, len_hi=300, n_dom=F, pairing=pairing)
     r = Run(w)
