@@ -26,7 +26,8 @@ namespace cg = cooperative_groups;
 
 namespace {
 
-constexpr int kFT = 256;               // threads per CTA (two CTAs share an SM)
+constexpr int kFT = 512;               // threads per CTA; two CTAs share an SM (64 registers per thread):
+                                       // what one SM can pull from HBM grows with its resident warps
 constexpr int kFW = kFT / 32;          // warps per CTA
 constexpr int kFBins = 2048;           // bins of the widest radix pass
 constexpr int kPartStride = FASA_HEAD_DIM + 2;   // m, l, acc[128]
@@ -91,9 +92,9 @@ __device__ __forceinline__ bool warp_find_kth(uint32_t v, uint32_t kth, int lane
   return true;
 }
 
-// KB = 16-channel blocks per proxy tile rounded up to a power of two; GP = query heads padded
-// to 4 or 8.
-template <int KB, int GP>
+// A tile's 16-channel blocks are taken NG groups of KB at a time (KB = 1, 2, 4; NG = 2 only with
+// KB = 4, for more than 4 blocks), which bounds the registers the loads in flight need.
+template <int KB, int NG>
 __global__ void __launch_bounds__(kFT, 2)
 fused_decode_kernel(const FusedParams p) {
   cg::cluster_group cluster = cg::this_cluster();
@@ -115,12 +116,14 @@ fused_decode_kernel(const FusedParams p) {
   __shared__ int s_len_old;
   __shared__ uint32_t s_mg[kCapMax / 32], s_me[kCapMax / 32];   // per 32 keys: above / equal masks
   __shared__ unsigned long long s_roff[kCapMax / 32];           // per 32 keys: (gt, eq) selected before
+  constexpr int GP = FASA_MAX_GROUP;     // query heads a KV head can serve
+  constexpr int HP = 4;                  // heads per attention pass
   __shared__ __align__(16) float s_q[GP][FASA_HEAD_DIM];
   __shared__ __align__(16) float s_part[GP][kPartStride + 2];
-  __shared__ __align__(16) float s_p[kFW][32];
-  __shared__ __align__(16) float s_al[kFW][GP];
-  __shared__ float s_m[kFW][GP];
-  __shared__ float s_l[kFW][GP];
+  __shared__ __align__(16) float s_p[kFW][16];
+  __shared__ __align__(16) float s_al[kFW][HP];
+  __shared__ float s_m[kFW][HP];
+  __shared__ float s_l[kFW][HP];
 
   // ---- slices -------------------------------------------------------------------------
   // Append-then-step: one thread reads the length for the whole CTA, so that the CTA's arrival
@@ -204,35 +207,46 @@ fused_decode_kernel(const FusedParams p) {
 
   // ---- 1. scoring stream -> keys + first histogram ------------------------------------------
   {
-    constexpr int TPI = KB == 1 ? 8 : (KB == 2 ? 4 : 2);      // tiles per warp iteration
+    // A warp keeps about four 16-byte loads per lane in flight (more do not raise what a warp
+    // can pull); the SM's bandwidth comes from its 32 resident warps.
+    constexpr int TPI = KB == 1 ? 4 : 2;                      // tiles per warp iteration (even)
     const ProxyGeom pg = proxy_geom(p.chunks);
     const int n_blocks = pg.n16 + pg.n8;
     const unsigned char* unit = p.proxy + (int64_t)u * ((p.max_len + 15) >> 4) * pg.tile_bytes;
     float* srow = p.scores ? p.scores + (int64_t)u * p.max_len : nullptr;
 
+    auto fetch = [&](uint4 (&a)[TPI][KB], int T, int grp) {
+#pragma unroll
+      for (int j = 0; j < TPI; ++j)
+        load_tile<KB>(a[j], unit + (int64_t)(T + j) * pg.tile_bytes, pg, lane, (T + j) * 16 < c1, grp * KB);
+    };
+    const int step = kFW * TPI;
     int T = ((crank * per) >> 4) + warp * TPI;                // slices start on a tile boundary
     uint4 a[TPI][KB];
+    fetch(a, T, 0);
+    ScoreFrag<KB> f[NG];
 #pragma unroll
-    for (int j = 0; j < TPI; ++j)
-      load_tile<KB>(a[j], unit + (int64_t)(T + j) * pg.tile_bytes, pg, lane, (T + j) * 16 < c1);
-    ScoreFrag<KB> f;
-    load_score_b<KB>(f, p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM,
-                     p.chan + h * p.chunks * 8, p.chunks, p.group, lane);
+    for (int grp = 0; grp < NG; ++grp)
+      load_score_b<KB>(f[grp], p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM,
+                       p.chan + h * p.chunks * 8, p.chunks, p.group, lane, grp * KB);
     while (T * 16 < c1) {       // uniform over the warp
-      float s_lo[TPI], s_hi[TPI];
+      float c[TPI][4];
 #pragma unroll
-      for (int j = 0; j < TPI; ++j) score_tile<KB, false>(a[j], f, n_blocks, p.group, lane, s_lo[j], s_hi[j]);
-      const int next = T + kFW * TPI;
-      if (next * 16 < c1) {     // next loads fly while keys are made
+      for (int j = 0; j < TPI; ++j) c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.f;
 #pragma unroll
-        for (int j = 0; j < TPI; ++j)
-          load_tile<KB>(a[j], unit + (int64_t)(next + j) * pg.tile_bytes, pg, lane, (next + j) * 16 < c1);
+      for (int grp = 0; grp < NG; ++grp) {
+#pragma unroll
+        for (int j = 0; j < TPI; ++j) mma_tile<KB>(c[j], a[j], f[grp], n_blocks - grp * KB);
+        // the registers are free again: the next group, or the next batch of tiles, at once
+        if (grp + 1 < NG) fetch(a, T, grp + 1);
+        else if ((T + step) * 16 < c1) fetch(a, T + step, 0);
       }
 #pragma unroll
       for (int pr = 0; pr < TPI / 2; ++pr) {
-        float sc;
-        const int row = (T + 2 * pr) * 16 +
-                        pick_row_of_pair(lane, s_lo[2 * pr], s_hi[2 * pr], s_lo[2 * pr + 1], s_hi[2 * pr + 1], sc);
+        float a_lo, a_hi, b_lo, b_hi, sc;
+        reduce_heads<false>(c[2 * pr], p.group, lane, a_lo, a_hi);
+        reduce_heads<false>(c[2 * pr + 1], p.group, lane, b_lo, b_hi);
+        const int row = (T + 2 * pr) * 16 + pick_row_of_pair(lane, a_lo, a_hi, b_lo, b_hi, sc);
         if (row < c1) {
           const uint32_t key = fasa_item_key(sc, row, len, p.n_sink, p.n_recent);
           atomicAdd(&hist0[key >> 21], 1u);
@@ -240,7 +254,7 @@ fused_decode_kernel(const FusedParams p) {
           if (srow) srow[row] = sc;
         }
       }
-      T = next;
+      T += step;
     }
   }
   __syncthreads();
@@ -440,20 +454,28 @@ fused_decode_kernel(const FusedParams p) {
   cluster.sync();   // barrier 5: the index list is complete and visible to the whole cluster
 
   // ---- 4. attention over this CTA's share of the selected rows -----------------------------
-  constexpr int R = 32 / GP;                                   // rows per warp batch
+  // Register-lean form (64 registers per thread): four query heads per pass (two passes for
+  // groups of 5-8 heads; the second pass finds the rows in L2), four rows per warp step, a
+  // lane owning 4 channels of every row.  The 16 partial logits (4 rows x 4 heads) of a step
+  // are completed by a transposing xor-shuffle reduction, one shuffle per value.
+  constexpr int R = 4;
   const int m_per = ((((int)ktot + cs - 1) / cs) + R - 1) / R * R;
   const int a0 = min((int)ktot, crank * m_per);
   const int a1 = min((int)ktot, a0 + m_per);
-  float2 acc[GP][2];
+  float* s_acc = reinterpret_cast<float*>(smem_raw);           // [kFW][HP][128]; the key / histogram
+                                                               // area is free: all reads of it, local
+                                                               // or remote, happened before barrier 4
+  const int n_hp = (p.group + HP - 1) / HP;
+  for (int hp = 0; hp < n_hp; ++hp) {                          // uniform
+    float2 acc[HP][2];
 #pragma unroll
-  for (int g = 0; g < GP; ++g) acc[g][0] = acc[g][1] = make_float2(0.f, 0.f);
-  float m_run = -INFINITY, l_run = 0.f;   // of head (lane % GP); replicated over the row lanes
-  {
+    for (int g = 0; g < HP; ++g) acc[g][0] = acc[g][1] = make_float2(0.f, 0.f);
+    float m_run = -INFINITY, l_run = 0.f;   // of value (lane >> 1) = row * 4 + head
     const int32_t* irow = p.idx + (int64_t)u * p.n_sel_max;
     const uint16_t* kbase = p.k + b * p.ksb + h * p.ksh + lane * 4;
     const uint16_t* vbase = p.v + b * p.vsb + h * p.vsh + lane * 4;
-    const int my_g = lane % GP;
-    const int my_i = lane / GP;
+    const int my_g = (lane >> 1) & 3;
+    const int my_i = lane >> 3;
     for (int base = a0 + warp * R; base < a1; base += kFW * R) {
       // all row indices first, then all row loads: nothing waits on a previous row (rows
       // past the end repeat the last one and are masked below)
@@ -467,123 +489,117 @@ fused_decode_kernel(const FusedParams p) {
         kk[i] = ld_stream_u2(kbase + (int64_t)t * p.kst);
         vv[i] = ld_stream_u2(vbase + (int64_t)t * p.vst);
       }
-      // partial logits of R rows x GP heads over this lane's 4 channels
-      float part[32];
+      float part[16];
 #pragma unroll
-      for (int g = 0; g < GP; ++g) {
-        const float4 qg = *reinterpret_cast<const float4*>(&s_q[g][lane * 4]);
+      for (int g = 0; g < HP; ++g) {
+        const float4 qg = *reinterpret_cast<const float4*>(&s_q[hp * HP + g][lane * 4]);
 #pragma unroll
         for (int i = 0; i < R; ++i) {
           const float2 k0 = bf16x2_to_f32x2(kk[i].x), k1 = bf16x2_to_f32x2(kk[i].y);
-          part[i * GP + g] = qg.x * k0.x + qg.y * k0.y + qg.z * k1.x + qg.w * k1.y;
+          part[i * HP + g] = qg.x * k0.x + qg.y * k0.y + qg.z * k1.x + qg.w * k1.y;
         }
       }
-      // transposing reduction over the 32 lanes: lane L ends with the full sum of value L
+      // transposing reduction: lane L ends with the full sum of value L >> 1
       float logit;
       {
-        float p16[16], p8[8], p4[4], p2[2];
+        float p8[8], p4[4], p2[2];
         const bool u16 = (lane & 16) != 0;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float send = u16 ? part[i] : part[i + 16];
-          const float keep = u16 ? part[i + 16] : part[i];
-          p16[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+        for (int i = 0; i < 8; ++i) {
+          const float send = u16 ? part[i] : part[i + 8];
+          const float keep = u16 ? part[i + 8] : part[i];
+          p8[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
         }
         const bool u8 = (lane & 8) != 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float send = u8 ? p16[i] : p16[i + 8];
-          const float keep = u8 ? p16[i + 8] : p16[i];
-          p8[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+        for (int i = 0; i < 4; ++i) {
+          const float send = u8 ? p8[i] : p8[i + 4];
+          const float keep = u8 ? p8[i + 4] : p8[i];
+          p4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
         }
         const bool u4 = (lane & 4) != 0;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float send = u4 ? p8[i] : p8[i + 4];
-          const float keep = u4 ? p8[i + 4] : p8[i];
-          p4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+        for (int i = 0; i < 2; ++i) {
+          const float send = u4 ? p4[i] : p4[i + 2];
+          const float keep = u4 ? p4[i + 2] : p4[i];
+          p2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
         }
         const bool u2 = (lane & 2) != 0;
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const float send = u2 ? p4[i] : p4[i + 2];
-          const float keep = u2 ? p4[i + 2] : p4[i];
-          p2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-        }
-        const bool u1 = (lane & 1) != 0;
-        const float send = u1 ? p2[0] : p2[1];
-        const float keep = u1 ? p2[1] : p2[0];
-        logit = keep + __shfl_xor_sync(0xffffffffu, send, 1);
+        const float send = u2 ? p2[0] : p2[1];
+        const float keep = u2 ? p2[1] : p2[0];
+        logit = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+        logit += __shfl_xor_sync(0xffffffffu, logit, 1);
       }
-      if (!(base + my_i < a1 && my_g < p.group)) logit = -INFINITY;
-      float bmax = logit;
-#pragma unroll
-      for (int o = GP; o < 32; o <<= 1) bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, o));
+      if (!(base + my_i < a1 && hp * HP + my_g < p.group)) logit = -INFINITY;
+      float bmax = logit;                                      // over the 4 rows of this head
+      bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 8));
+      bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 16));
       const float m_new = fmaxf(m_run, bmax);
       const float m_safe = m_new == -INFINITY ? 0.f : m_new;
       const float alpha = exp2f(m_run - m_safe);
       const float pr = exp2f(logit - m_safe);
       l_run = l_run * alpha + pr;
       m_run = m_new;
-      s_p[warp][lane] = pr;
-      if (lane < GP) s_al[warp][lane] = alpha;
+      if ((lane & 1) == 0) {
+        s_p[warp][lane >> 1] = pr;
+        if (lane < 2 * HP) s_al[warp][lane >> 1] = alpha;      // row 0 lanes: one per head
+      }
       __syncwarp();
 #pragma unroll
-      for (int g = 0; g < GP; ++g) {
-        const float a = s_al[warp][g];
-        const float2 a2 = make_float2(a, a);
+      for (int g = 0; g < HP; ++g) {
+        const float al = s_al[warp][g];
+        const float2 a2 = make_float2(al, al);
         acc[g][0] = __ffma2_rn(acc[g][0], a2, make_float2(0.f, 0.f));
         acc[g][1] = __ffma2_rn(acc[g][1], a2, make_float2(0.f, 0.f));
       }
 #pragma unroll
       for (int i = 0; i < R; ++i) {
         const float2 v0 = bf16x2_to_f32x2(vv[i].x), v1 = bf16x2_to_f32x2(vv[i].y);
+        const float4 pi = *reinterpret_cast<const float4*>(&s_p[warp][i * HP]);
+        const float pg4[4] = {pi.x, pi.y, pi.z, pi.w};
 #pragma unroll
-        for (int g = 0; g < GP; ++g) {
-          const float pg = s_p[warp][i * GP + g];
-          const float2 p2 = make_float2(pg, pg);
+        for (int g = 0; g < HP; ++g) {
+          const float2 p2 = make_float2(pg4[g], pg4[g]);
           acc[g][0] = __ffma2_rn(p2, v0, acc[g][0]);
           acc[g][1] = __ffma2_rn(p2, v1, acc[g][1]);
         }
       }
       __syncwarp();
     }
-    // row lanes of a head add their partial sums of probabilities
-#pragma unroll
-    for (int o = GP; o < 32; o <<= 1) l_run += __shfl_xor_sync(0xffffffffu, l_run, o);
-  }
+    // the four row lanes of a head add their partial sums of probabilities
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 8);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 16);
 
-  // ---- 5. combine the warps of this CTA, then the CTAs of the cluster ------------------------
-  // The warp accumulators reuse the key / histogram area: every read of it, local or remote,
-  // happened before barrier 4.
-  float* s_acc = reinterpret_cast<float*>(smem_raw);           // [kFW][GP][128]
-  if (lane < GP) {
-    s_m[warp][lane] = m_run;
-    s_l[warp][lane] = l_run;
-  }
-#pragma unroll
-  for (int g = 0; g < GP; ++g)
-    *reinterpret_cast<float4*>(&s_acc[((warp * GP) + g) * FASA_HEAD_DIM + lane * 4]) =
-        make_float4(acc[g][0].x, acc[g][0].y, acc[g][1].x, acc[g][1].y);
-  __syncthreads();
-  for (int o = tid; o < GP * FASA_HEAD_DIM; o += kFT) {
-    const int g = o / FASA_HEAD_DIM, c = o % FASA_HEAD_DIM;
-    float mx = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < kFW; ++w) mx = fmaxf(mx, s_m[w][g]);
-    float a = 0.f, l = 0.f;
-#pragma unroll
-    for (int w = 0; w < kFW; ++w) {
-      const float ms = s_m[w][g];
-      const float wt = ms == -INFINITY ? 0.f : exp2f(ms - mx);
-      a += wt * s_acc[((w * GP) + g) * FASA_HEAD_DIM + c];
-      l += wt * s_l[w][g];
+    // ---- 5a. combine the warps of this CTA for these heads ---------------------------------
+    if (lane < 2 * HP && (lane & 1) == 0) {
+      s_m[warp][lane >> 1] = m_run;
+      s_l[warp][lane >> 1] = l_run;
     }
-    s_part[g][2 + c] = a;
-    if (c == 0) {
-      s_part[g][0] = mx;
-      s_part[g][1] = l;
+#pragma unroll
+    for (int g = 0; g < HP; ++g)
+      *reinterpret_cast<float4*>(&s_acc[((warp * HP) + g) * FASA_HEAD_DIM + lane * 4]) =
+          make_float4(acc[g][0].x, acc[g][0].y, acc[g][1].x, acc[g][1].y);
+    __syncthreads();
+    for (int o = tid; o < HP * FASA_HEAD_DIM; o += kFT) {
+      const int g = o / FASA_HEAD_DIM, c = o % FASA_HEAD_DIM;
+      float mx = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < kFW; ++w) mx = fmaxf(mx, s_m[w][g]);
+      float av = 0.f, l = 0.f;
+#pragma unroll
+      for (int w = 0; w < kFW; ++w) {
+        const float ms = s_m[w][g];
+        const float wt = ms == -INFINITY ? 0.f : exp2f(ms - mx);
+        av += wt * s_acc[((w * HP) + g) * FASA_HEAD_DIM + c];
+        l += wt * s_l[w][g];
+      }
+      s_part[hp * HP + g][2 + c] = av;
+      if (c == 0) {
+        s_part[hp * HP + g][0] = mx;
+        s_part[hp * HP + g][1] = l;
+      }
     }
+    __syncthreads();                                           // s_acc / s_m are reused by the next pass
   }
   cluster.sync();   // barrier 6: every CTA's partial result is in its shared memory
 
@@ -626,22 +642,20 @@ struct FusedPlan {
   size_t smem;   // dynamic shared memory
 };
 
-template <int GP>
 size_t fused_smem_bytes(int cap) {
   const size_t sel = (size_t)cap * 4 + 2 * kFBins * 4;
-  const size_t att = (size_t)kFW * GP * FASA_HEAD_DIM * 4;
+  const size_t att = (size_t)kFW * 4 * FASA_HEAD_DIM * 4;
   return sel > att ? sel : att;
 }
 
 using FusedFn = void (*)(const FusedParams);
 
-template <int GP>
-FusedFn fused_fn_lpr(int chunks) {
+FusedFn fused_fn(int chunks) {
   const int nb = (chunks + 1) / 2;      // 16-channel blocks per tile, the 8-channel one included
-  if (nb <= 1) return fused_decode_kernel<1, GP>;
-  if (nb <= 2) return fused_decode_kernel<2, GP>;
-  if (nb <= 4) return fused_decode_kernel<4, GP>;
-  return fused_decode_kernel<8, GP>;
+  if (nb <= 1) return fused_decode_kernel<1, 1>;
+  if (nb <= 2) return fused_decode_kernel<2, 1>;
+  if (nb <= 4) return fused_decode_kernel<4, 1>;
+  return fused_decode_kernel<4, 2>;
 }
 
 }  // namespace
@@ -655,8 +669,7 @@ int fasa_fused_plan(fasa_ctx* ctx) {
   ctx->fused_smem = 0;
   if (c.group_reduce != 0) return 0;          // the max reduction takes the three-kernel path
   const int units = c.batch * c.n_kv_heads;
-  const bool gp8 = ctx->group > 4;
-  FusedFn fn = gp8 ? fused_fn_lpr<8>(ctx->chunks) : fused_fn_lpr<4>(ctx->chunks);
+  FusedFn fn = fused_fn(ctx->chunks);
   auto cap_of = [&](int cs) { return (((c.max_len + cs - 1) / cs) + 31) & ~31; };
   // Two CTAs per SM can be resident; a cluster is doubled while the whole grid still fits
   // in one wave of them and every CTA keeps at least 512 tokens.
@@ -671,7 +684,7 @@ int fasa_fused_plan(fasa_ctx* ctx) {
   for (int cs = want; cs >= 1; cs /= 2) {
     const int cap = cap_of(cs);
     if (cap > kCapMax) break;
-    const size_t smem = gp8 ? fused_smem_bytes<8>(cap) : fused_smem_bytes<4>(cap);
+    const size_t smem = fused_smem_bytes(cap);
     if (cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
       cudaGetLastError();
       continue;
@@ -719,8 +732,7 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
   p.ksb = c.k_stride_b; p.ksh = c.k_stride_h; p.kst = c.k_stride_t;
   p.vsb = c.v_stride_b; p.vsh = c.v_stride_h; p.vst = c.v_stride_t;
   p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
-  const bool gp8 = ctx->group > 4;
-  FusedFn fn = gp8 ? fused_fn_lpr<8>(ctx->chunks) : fused_fn_lpr<4>(ctx->chunks);
+  FusedFn fn = fused_fn(ctx->chunks);
 
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));

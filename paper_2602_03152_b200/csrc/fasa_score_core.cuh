@@ -67,7 +67,7 @@ struct ScoreFrag {
 template <int KB>
 __device__ __forceinline__ void load_score_b(ScoreFrag<KB>& f, const uint16_t* __restrict__ q_unit,
                                              const int16_t* __restrict__ chan_h, int chunks,
-                                             int group, int lane) {
+                                             int group, int lane, int kb0 = 0) {
   const int n = lane >> 2, t = lane & 3;
   const int n_chan = chunks * 8;
 #pragma unroll
@@ -77,7 +77,7 @@ __device__ __forceinline__ void load_score_b(ScoreFrag<KB>& f, const uint16_t* _
       uint32_t w = 0u;
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        const int ci = kb * 16 + half * 8 + 2 * t + e;
+        const int ci = (kb0 + kb) * 16 + half * 8 + 2 * t + e;
         uint32_t v = 0u;
         if (ci < n_chan && n < group) {
           const int ch = chan_h[ci];
@@ -105,20 +105,21 @@ __device__ __forceinline__ uint2 ld_proxy_u2(const void* p) {
   return r;
 }
 
-// The A fragments of one tile (this lane's share).  `tile` points at the tile's first byte;
-// when `ok` is false nothing is read.  Loads go through the coherent path: in the
+// The A fragments of blocks kb0 .. kb0 + KB - 1 of one tile (this lane's share).  `tile` points
+// at the tile's first byte; when `ok` is false nothing is read.  Loads go through the coherent path: in the
 // append-then-step form the last row of the cache is written earlier in the same launch.
 template <int KB>
 __device__ __forceinline__ void load_tile(uint4 (&a)[KB], const unsigned char* tile, const ProxyGeom& pg,
-                                          int lane, bool ok) {
+                                          int lane, bool ok, int kb0 = 0) {
 #pragma unroll
-  for (int kb = 0; kb < KB; ++kb) {
-    a[kb] = make_uint4(0u, 0u, 0u, 0u);
+  for (int i = 0; i < KB; ++i) {
+    const int kb = kb0 + i;
+    a[i] = make_uint4(0u, 0u, 0u, 0u);
     if (ok && kb < pg.n16) {
-      a[kb] = ld_proxy_u4(tile + kb * 512 + lane * 16);
+      a[i] = ld_proxy_u4(tile + kb * 512 + lane * 16);
     } else if (ok && kb == pg.n16 && pg.n8) {
       const uint2 w = ld_proxy_u2(tile + pg.n16 * 512 + lane * 8);
-      a[kb] = make_uint4(w.x, w.y, 0u, 0u);
+      a[i] = make_uint4(w.x, w.y, 0u, 0u);
     }
   }
 }
@@ -131,16 +132,19 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint4& a, co
       : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b[0]), "r"(b[1]));
 }
 
-// Scores of the 16 tokens of one tile.  Every lane of quad g (lanes 4g .. 4g+3) returns the
-// score of row g in s_lo and of row g + 8 in s_hi.  MAXRED reduces the group by max instead
-// of by sum.  -0 is turned into +0 so that equal scores have equal bit patterns.
-template <int KB, bool MAXRED>
-__device__ __forceinline__ void score_tile(const uint4 (&a)[KB], const ScoreFrag<KB>& f, int n_blocks,
-                                           int group, int lane, float& s_lo, float& s_hi) {
-  float c[4] = {0.f, 0.f, 0.f, 0.f};
+// Adds the products of up to KB blocks (n_left of them exist) of one tile to c.
+template <int KB>
+__device__ __forceinline__ void mma_tile(float (&c)[4], const uint4 (&a)[KB], const ScoreFrag<KB>& f, int n_left) {
 #pragma unroll
   for (int kb = 0; kb < KB; ++kb)
-    if (kb < n_blocks) mma_bf16_16816(c, a[kb], f.b[kb]);   // uniform over the warp
+    if (kb < n_left) mma_bf16_16816(c, a[kb], f.b[kb]);     // uniform over the warp
+}
+
+// Reduces the head columns of a tile's accumulators: every lane of quad g (lanes 4g .. 4g+3)
+// returns the score of row g in s_lo and of row g + 8 in s_hi.  MAXRED reduces the group by
+// max instead of by sum.  -0 is turned into +0 so that equal scores have equal bit patterns.
+template <bool MAXRED>
+__device__ __forceinline__ void reduce_heads(const float (&c)[4], int group, int lane, float& s_lo, float& s_hi) {
   if (!MAXRED) {
     s_lo = c[0] + c[1];                                     // heads 2t and 2t+1; absent heads are exact zeros
     s_hi = c[2] + c[3];
@@ -162,6 +166,17 @@ __device__ __forceinline__ void score_tile(const uint4 (&a)[KB], const ScoreFrag
   }
   s_lo += 0.0f;
   s_hi += 0.0f;
+}
+
+// Scores of the 16 tokens of one tile.  Every lane of quad g (lanes 4g .. 4g+3) returns the
+// score of row g in s_lo and of row g + 8 in s_hi.  MAXRED reduces the group by max instead
+// of by sum.  -0 is turned into +0 so that equal scores have equal bit patterns.
+template <int KB, bool MAXRED>
+__device__ __forceinline__ void score_tile(const uint4 (&a)[KB], const ScoreFrag<KB>& f, int n_blocks,
+                                           int group, int lane, float& s_lo, float& s_hi) {
+  float c[4] = {0.f, 0.f, 0.f, 0.f};
+  mma_tile<KB>(c, a, f, n_blocks);
+  reduce_heads<MAXRED>(c, group, lane, s_lo, s_hi);
 }
 
 // After two tiles (A, B) every lane takes one of the 32 rows: t = lane % 4 picks
