@@ -129,14 +129,27 @@ fused_decode_kernel(const FusedParams p) {
   // Append-then-step: one thread reads the length for the whole CTA, so that the CTA's arrival
   // (below) certifies that it no longer needs the old value; the last CTA of the sequence to
   // arrive stores the new length.  Nothing waits on the counter.
+  // Loads that depend on nothing are issued first, so their (cold) latencies overlap: the
+  // length, this thread's share of the query for the attention phase, and the channel table
+  // with the query values of the scoring operand.
   const bool append = p.k_new != nullptr;
+  int len_raw = 0;
+  if (!append || tid == 0) len_raw = p.seq_lens[b];
+  uint4 q_stage = make_uint4(0u, 0u, 0u, 0u);
+  if (tid < FASA_MAX_GROUP * (FASA_HEAD_DIM / 8) && tid / (FASA_HEAD_DIM / 8) < p.group)
+    q_stage = *reinterpret_cast<const uint4*>(p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM + tid * 8);
+  ScoreFrag<KB> f[NG];
+#pragma unroll
+  for (int grp = 0; grp < NG; ++grp)
+    load_score_b<KB>(f[grp], p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM,
+                     p.chan + h * p.chunks * 8, p.chunks, p.group, lane, grp * KB);
   int len_old;
   if (append) {
-    if (tid == 0) s_len_old = clamp_len(p.seq_lens[b], p.max_len, p.status);
+    if (tid == 0) s_len_old = clamp_len(len_raw, p.max_len, p.status);
     __syncthreads();
     len_old = s_len_old;
   } else {
-    len_old = clamp_len(p.seq_lens[b], p.max_len, p.status);
+    len_old = clamp_len(len_raw, p.max_len, p.status);
   }
   const bool grows = append && len_old < p.max_len;
   const int len = len_old + (grows ? 1 : 0);
@@ -169,7 +182,28 @@ fused_decode_kernel(const FusedParams p) {
   }
   const uint32_t ktot = (uint32_t)ktot_ll;
 
-  if (grows && c0 <= len_old && len_old < c1) {
+  // The first proxy loads leave before the rest of the set-up (histogram clearing, query
+  // staging, its barrier), whose latency they then hide.  A warp keeps about four 16-byte
+  // loads per lane in flight (more do not raise what a warp can pull); the SM's bandwidth
+  // comes from its 32 resident warps.  Only the CTA that is about to write the new token's
+  // rows has to wait for them.
+  constexpr int TPI = KB == 1 ? 4 : 2;                        // tiles per warp iteration (even)
+  const ProxyGeom pg = proxy_geom(p.chunks);
+  const int n_blocks = pg.n16 + pg.n8;
+  const unsigned char* unit = p.proxy + (int64_t)u * ((p.max_len + 15) >> 4) * pg.tile_bytes;
+  float* srow = p.scores ? p.scores + (int64_t)u * p.max_len : nullptr;
+  auto fetch = [&](uint4 (&a)[TPI][KB], int T, int grp) {
+#pragma unroll
+    for (int j = 0; j < TPI; ++j)
+      load_tile<KB>(a[j], unit + (int64_t)(T + j) * pg.tile_bytes, pg, lane, (T + j) * 16 < c1, grp * KB);
+  };
+  const int step = kFW * TPI;
+  int T = ((crank * per) >> 4) + warp * TPI;                  // slices start on a tile boundary
+  const bool own_new = grows && c0 <= len_old && len_old < c1;
+  uint4 a[TPI][KB];
+  if (!own_new) fetch(a, T, 0);
+
+  if (own_new) {
     // this CTA's slice holds the new row: K and V copies (16 lanes each) and the packed
     // dominant-FC pairs of the key (one lane per 16-byte chunk), as in fasa_kv_append
     const uint16_t* ksrc = p.k_new + (int64_t)u * FASA_HEAD_DIM;
@@ -193,11 +227,9 @@ fused_decode_kernel(const FusedParams p) {
   }
   for (int i = tid; i < 2 * kFBins; i += kFT) hist0[i] = 0u;
   // query, scaled into the base-2 logit domain, for the attention phase
-  for (int i = tid; i < GP * (FASA_HEAD_DIM / 8); i += kFT) {
-    const int g = i / (FASA_HEAD_DIM / 8), c = (i % (FASA_HEAD_DIM / 8)) * 8;
-    uint4 w = make_uint4(0u, 0u, 0u, 0u);
-    if (g < p.group)
-      w = *reinterpret_cast<const uint4*>(p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group + g) * FASA_HEAD_DIM + c);
+  if (tid < GP * (FASA_HEAD_DIM / 8)) {
+    const int g = tid / (FASA_HEAD_DIM / 8), c = (tid % (FASA_HEAD_DIM / 8)) * 8;
+    const uint4 w = q_stage;
     const float2 f0 = bf16x2_to_f32x2(w.x), f1 = bf16x2_to_f32x2(w.y), f2 = bf16x2_to_f32x2(w.z), f3 = bf16x2_to_f32x2(w.w);
     const float sc = p.scale_log2;
     *reinterpret_cast<float4*>(&s_q[g][c]) = make_float4(f0.x * sc, f0.y * sc, f1.x * sc, f1.y * sc);
@@ -207,28 +239,7 @@ fused_decode_kernel(const FusedParams p) {
 
   // ---- 1. scoring stream -> keys + first histogram ------------------------------------------
   {
-    // A warp keeps about four 16-byte loads per lane in flight (more do not raise what a warp
-    // can pull); the SM's bandwidth comes from its 32 resident warps.
-    constexpr int TPI = KB == 1 ? 4 : 2;                      // tiles per warp iteration (even)
-    const ProxyGeom pg = proxy_geom(p.chunks);
-    const int n_blocks = pg.n16 + pg.n8;
-    const unsigned char* unit = p.proxy + (int64_t)u * ((p.max_len + 15) >> 4) * pg.tile_bytes;
-    float* srow = p.scores ? p.scores + (int64_t)u * p.max_len : nullptr;
-
-    auto fetch = [&](uint4 (&a)[TPI][KB], int T, int grp) {
-#pragma unroll
-      for (int j = 0; j < TPI; ++j)
-        load_tile<KB>(a[j], unit + (int64_t)(T + j) * pg.tile_bytes, pg, lane, (T + j) * 16 < c1, grp * KB);
-    };
-    const int step = kFW * TPI;
-    int T = ((crank * per) >> 4) + warp * TPI;                // slices start on a tile boundary
-    uint4 a[TPI][KB];
-    fetch(a, T, 0);
-    ScoreFrag<KB> f[NG];
-#pragma unroll
-    for (int grp = 0; grp < NG; ++grp)
-      load_score_b<KB>(f[grp], p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM,
-                       p.chan + h * p.chunks * 8, p.chunks, p.group, lane, grp * KB);
+    if (own_new) fetch(a, T, 0);                              // (the new row is in place now)
     while (T * 16 < c1) {       // uniform over the warp
       float c[TPI][4];
 #pragma unroll
