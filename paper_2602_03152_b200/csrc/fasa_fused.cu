@@ -1,22 +1,29 @@
-// One decode step in one launch: TIP scoring -> TopK-I -> FAC (Sec. 4.1-4.2, Eq. 6-7).
+// One decode step in one launch: UpdateCache -> TIP scoring -> TopK-I -> FAC (Algorithm 2's
+// order; Sec. 4.1-4.2, Eq. 6-7).
 //
 // One thread-block cluster per (batch, KV head) unit.  The CTAs of the cluster cut the unit's
 // cached tokens into contiguous slices and
+//   0. (append form) the CTA whose slice ends the sequence writes the new K, V and proxy rows;
 //   1. stream their slice of the tiled proxy-K buffer once (16-byte loads in tensor-core
 //      fragment order, scored with mma.sync), keep every token's selection key in shared
 //      memory and histogram its top 11 bits;
 //   2. find the budget-th largest key by an MSB-first radix select (11 + 11 + 10 bits): each
 //      pass needs one cluster barrier, after which every CTA reads the other CTAs' coarse and
 //      fine bin counts through distributed shared memory and locates the bin redundantly;
-//   3. write the selected positions in ascending order (ballot / prefix-sum compaction, equal
-//      keys lowest index first, so the result equals a stable sort);
-//   4. share the selected rows evenly, gather K/V rows by index with an online softmax, and
-//   5. merge the per-CTA partial results through distributed shared memory.
+//   3. write the selected positions in ascending order (ballot masks + prefix sums, equal keys
+//      lowest index first, so the result equals a stable sort; one more barrier for the
+//      cluster-wide prefix);
+//   4. attend, each CTA over the tokens it selected itself: K/V rows gathered by index with an
+//      online softmax;
+//   5. push their partial results into the shared memory of the CTA that finishes each output
+//      (one last barrier), which merges them locally.
 // Scores, histograms and split-K partials never travel through HBM: the launch moves the
 // proxy rows of every token, the K/V rows of the selected tokens, q and the outputs.
 //
-// Every cluster barrier sits at the top level of the kernel and is reached by all threads of
-// all CTAs the same number of times, whatever the data; no thread waits on anything else.
+// Every cluster barrier (at most five) is reached by all threads of all CTAs of a cluster the
+// same number of times: the only data-dependent decision around one, leaving the radix loop
+// early, is taken from cluster-wide sums that are identical in every CTA.  No thread spins on
+// anything.
 #include <cooperative_groups.h>
 
 #include "fasa_common.cuh"
@@ -114,12 +121,14 @@ fused_decode_kernel(const FusedParams p) {
   __shared__ unsigned long long s_tot;
   __shared__ uint32_t s_bin, s_kth, s_cnt;
   __shared__ int s_len_old;
-  __shared__ uint32_t s_mg[kCapMax / 32], s_me[kCapMax / 32];   // per 32 keys: above / equal masks
-  __shared__ unsigned long long s_roff[kCapMax / 32];           // per 32 keys: (gt, eq) selected before
+  __shared__ __align__(16) uint32_t s_mask[kCapMax / 128 * 8];  // per 128 keys: 4 above + 4 equal masks
+  __shared__ unsigned long long s_boff[kCapMax / 128];          // per 128 keys: (gt, eq) selected before
   constexpr int GP = FASA_MAX_GROUP;     // query heads a KV head can serve
   constexpr int HP = 4;                  // heads per attention pass
   __shared__ __align__(16) float s_q[GP][FASA_HEAD_DIM];
   __shared__ __align__(16) float s_part[GP][kPartStride + 2];
+  __shared__ float s_racc[FASA_MAX_GROUP * FASA_HEAD_DIM + 16];   // pushed by the cluster: accumulators of this CTA's outputs
+  __shared__ float s_rml[16][FASA_MAX_GROUP][2];                  // ... and every CTA's (m, l) per head
   __shared__ __align__(16) float s_p[kFW][16];
   __shared__ __align__(16) float s_al[kFW][HP];
   __shared__ float s_m[kFW][HP];
@@ -272,8 +281,8 @@ fused_decode_kernel(const FusedParams p) {
 
   // ---- 2. radix select of the ktot-th largest key ------------------------------------------
   // `done` (the bin that holds the kth key is needed whole, so its remaining bits do not
-  // matter) is computed from cluster-wide sums and is the same in every CTA; the barrier is
-  // taken in every pass regardless.
+  // matter) is computed from the same cluster-wide integer sums in every CTA, hence identical
+  // in all of them: the loop, barrier included, ends for the whole cluster at once.
   uint32_t prefix = 0, kth = ktot, thr = 0, tie_quota = 0;
   bool done = false;
 #pragma unroll 1
@@ -284,7 +293,8 @@ fused_decode_kernel(const FusedParams p) {
     const int ng = nb / 32;
     uint32_t* buf = (pass & 1) ? hist1 : hist0;
     uint32_t* coarse = s_coarse[pass & 1];
-    if (pass > 0 && !done) {
+    if (done) break;
+    if (pass > 0) {
       if (pass == 2) {
         for (int i = tid; i < nb; i += kFT) buf[i] = 0u;
         __syncthreads();
@@ -300,7 +310,7 @@ fused_decode_kernel(const FusedParams p) {
       }
       __syncthreads();
     }
-    if (!done) {
+    {
       // group sums: each warp reduces its kFBins/32/kFW groups side by side
       constexpr int GPW = kFBins / 32 / kFW;
       uint32_t v[GPW];
@@ -320,7 +330,6 @@ fused_decode_kernel(const FusedParams p) {
       }
     }
     cluster.sync();   // barrier 1..3
-    if (done) continue;
 
     // Every thread fetches a few of the other CTAs' coarse counts (all loads in flight at
     // once); warp 0 adds them up and finds the group of 32 bins that holds the kth key.
@@ -380,36 +389,37 @@ fused_decode_kernel(const FusedParams p) {
   }
 
   // ---- 3. ascending compaction ---------------------------------------------------------------
-  // Rows of 32 consecutive keys.  (a) every warp turns its rows into two bit masks (key above
-  // the threshold / equal to it) with independent ballots; (b) a block scan over the rows'
-  // bit counts gives each row its offsets; (c) after the cluster-wide prefix, set bits become
-  // positions.  No step carries a running counter through a loop, so the loops pipeline.
-  const int n_rows = (nloc + 31) >> 5;
-  for (int r0 = warp * 32; r0 < n_rows; r0 += kFW * 32) {   // 32 rows per warp step
-    uint32_t my_g = 0, my_e = 0;
-#pragma unroll 8
-    for (int j = 0; j < 32; ++j) {
-      const int i = (r0 + j) * 32 + lane;
-      const bool ok = i < nloc;
-      const uint32_t key = ok ? keys[i] : 0u;
-      const uint32_t mg = __ballot_sync(0xffffffffu, ok && key > thr);
-      const uint32_t me = __ballot_sync(0xffffffffu, ok && key == thr);
-      if (lane == j) { my_g = mg; my_e = me; }
+  // Blocks of 128 consecutive keys, four per lane.  (a) every warp turns its blocks into
+  // eight bit masks (key e of lane l above the threshold / equal to it) with independent
+  // ballots; (b) a block scan over the blocks' bit counts gives each block its offsets;
+  // (c) after the cluster-wide prefix, set bits become positions.  No step carries a running
+  // counter through a loop, so the loops pipeline.
+  const int n_blk = (nloc + 127) >> 7;
+  for (int bk = warp; bk < n_blk; bk += kFW) {
+    const int i = bk * 128 + lane * 4;
+    const uint4 kq = *reinterpret_cast<const uint4*>(&keys[i]);
+    const uint32_t kv[4] = {kq.x, kq.y, kq.z, kq.w};
+    uint32_t m[8];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const bool ok = i + e < nloc;
+      m[e] = __ballot_sync(0xffffffffu, ok && kv[e] > thr);
+      m[4 + e] = __ballot_sync(0xffffffffu, ok && kv[e] == thr);
     }
-    if (r0 + lane < n_rows) {
-      s_mg[r0 + lane] = my_g;
-      s_me[r0 + lane] = my_e;
+    if (lane == 0) {
+      *reinterpret_cast<uint4*>(&s_mask[bk * 8]) = make_uint4(m[0], m[1], m[2], m[3]);
+      *reinterpret_cast<uint4*>(&s_mask[bk * 8 + 4]) = make_uint4(m[4], m[5], m[6], m[7]);
     }
   }
   __syncthreads();
-  // block scan of the per-row counts (gt in the high half, eq in the low half)
-  constexpr int RPT = (kCapMax / 32 + kFT - 1) / kFT;       // rows per thread
-  unsigned long long row_cnt[RPT], mine = 0;
-#pragma unroll
-  for (int j = 0; j < RPT; ++j) {
-    const int r = tid * RPT + j;
-    row_cnt[j] = r < n_rows ? (((unsigned long long)__popc(s_mg[r]) << 32) | (unsigned)__popc(s_me[r])) : 0ull;
-    mine += row_cnt[j];
+  // block scan of the per-block counts (gt in the high half, eq in the low half); one block
+  // per thread (at most kCapMax / 128 <= kFT of them)
+  unsigned long long mine = 0;
+  if (tid < n_blk) {
+    const uint4 g4 = *reinterpret_cast<const uint4*>(&s_mask[tid * 8]);
+    const uint4 e4 = *reinterpret_cast<const uint4*>(&s_mask[tid * 8 + 4]);
+    mine = ((unsigned long long)(__popc(g4.x) + __popc(g4.y) + __popc(g4.z) + __popc(g4.w)) << 32) |
+           (unsigned)(__popc(e4.x) + __popc(e4.y) + __popc(e4.z) + __popc(e4.w));
   }
   unsigned long long incl = mine;
 #pragma unroll
@@ -430,39 +440,51 @@ fused_decode_kernel(const FusedParams p) {
     if (tid == 0) s_tot = all;
   }
   cluster.sync();   // barrier 4
+  uint32_t own_first, own_count;
   {
     // totals of the lower-ranked CTAs, one per lane, fetched side by side
     unsigned long long t = lane < crank ? *cluster.map_shared_rank(&s_tot, lane) : 0ull;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
     before += t;
+    // this CTA's selected tokens occupy a contiguous run of the index list
+    const uint32_t gb = (uint32_t)(t >> 32), eb = (uint32_t)t;
+    const unsigned long long mine_all = s_tot;
+    const uint32_t gl = (uint32_t)(mine_all >> 32), el = (uint32_t)mine_all;
+    own_first = gb + min(eb, tie_quota);
+    own_count = gl + (eb < tie_quota ? min(tie_quota - eb, el) : 0u);
   }
-#pragma unroll
-  for (int j = 0; j < RPT; ++j) {            // offsets of this thread's rows
-    const int r = tid * RPT + j;
-    if (r < n_rows) s_roff[r] = before;
-    before += row_cnt[j];
-  }
+  if (tid < n_blk) s_boff[tid] = before;     // offsets of this thread's block
   __syncthreads();
   {
     int32_t* out_idx = p.idx + (int64_t)u * p.n_sel_max;
     const uint32_t lt = (1u << lane) - 1u;
-    for (int r = warp; r < n_rows; r += kFW) {
-      const uint32_t mg = s_mg[r], me = s_me[r];
-      if ((mg | me) == 0u) continue;                         // uniform over the warp
-      const unsigned long long off = s_roff[r];
-      const uint32_t g_before = (uint32_t)(off >> 32) + __popc(mg & lt);
-      const uint32_t e_before = (uint32_t)off + __popc(me & lt);
-      // (positions are < ktot by construction; the comparison keeps a write inside the list
-      // whatever the scores hold)
-      uint32_t pos = 0xffffffffu;
-      if ((mg >> lane) & 1u) pos = g_before + min(e_before, tie_quota);
-      else if (((me >> lane) & 1u) && e_before < tie_quota) pos = g_before + e_before;
-      if (pos < ktot) out_idx[pos] = c0 + r * 32 + lane;
+    for (int bk = warp; bk < n_blk; bk += kFW) {
+      const uint4 g4 = *reinterpret_cast<const uint4*>(&s_mask[bk * 8]);
+      const uint4 e4 = *reinterpret_cast<const uint4*>(&s_mask[bk * 8 + 4]);
+      if ((g4.x | g4.y | g4.z | g4.w | e4.x | e4.y | e4.z | e4.w) == 0u) continue;   // uniform over the warp
+      const uint32_t mg[4] = {g4.x, g4.y, g4.z, g4.w}, me[4] = {e4.x, e4.y, e4.z, e4.w};
+      const unsigned long long off = s_boff[bk];
+      // selected keys of lower lanes come first, then this lane's own keys in order
+      uint32_t g_before = (uint32_t)(off >> 32), e_before = (uint32_t)off;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        g_before += __popc(mg[e] & lt);
+        e_before += __popc(me[e] & lt);
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        // (positions are < ktot by construction; the comparison keeps a write inside the
+        // list whatever the scores hold)
+        uint32_t pos = 0xffffffffu;
+        if ((mg[e] >> lane) & 1u) { pos = g_before + min(e_before, tie_quota); ++g_before; }
+        else if ((me[e] >> lane) & 1u) { if (e_before < tie_quota) pos = g_before + e_before; ++e_before; }
+        if (pos < ktot) out_idx[pos] = c0 + bk * 128 + lane * 4 + e;
+      }
     }
     if (crank == 0 && tid == 0) p.n_sel[u] = (int32_t)ktot;
   }
-  cluster.sync();   // barrier 5: the index list is complete and visible to the whole cluster
+  __syncthreads();   // this CTA's part of the index list is written: it attends to its own rows
 
   // ---- 4. attention over this CTA's share of the selected rows -----------------------------
   // Register-lean form (64 registers per thread): four query heads per pass (two passes for
@@ -470,9 +492,10 @@ fused_decode_kernel(const FusedParams p) {
   // lane owning 4 channels of every row.  The 16 partial logits (4 rows x 4 heads) of a step
   // are completed by a transposing xor-shuffle reduction, one shuffle per value.
   constexpr int R = 4;
-  const int m_per = ((((int)ktot + cs - 1) / cs) + R - 1) / R * R;
-  const int a0 = min((int)ktot, crank * m_per);
-  const int a1 = min((int)ktot, a0 + m_per);
+  // Every CTA attends to the tokens it selected itself (a contiguous run of the index list
+  // that it has just written), so no cluster barrier separates selection from attention.
+  const int a0 = (int)min(own_first, ktot);
+  const int a1 = (int)min(own_first + own_count, ktot);
   float* s_acc = reinterpret_cast<float*>(smem_raw);           // [kFW][HP][128]; the key / histogram
                                                                // area is free: all reads of it, local
                                                                // or remote, happened before barrier 4
@@ -612,46 +635,51 @@ fused_decode_kernel(const FusedParams p) {
     }
     __syncthreads();                                           // s_acc / s_m are reused by the next pass
   }
-  cluster.sync();   // barrier 6: every CTA's partial result is in its shared memory
-
+  // ---- 5b. merge across the cluster ------------------------------------------------------------
+  // CTA r finishes outputs [r * per_o, (r + 1) * per_o).  Every CTA PUSHES its partial values
+  // for those outputs into r's shared memory; after the barrier r combines from local memory
+  // only, so no CTA reads a peer afterwards and none has to wait for the others to leave.
   {
-    // This CTA finishes a contiguous share of the unit's outputs.  cs neighbouring lanes take
-    // one output together, each fetching one CTA's (m, l, acc) from its shared memory, and
-    // combine with xor-shuffles: one round of remote loads whatever the cluster size.
     const int n_out = p.group * FASA_HEAD_DIM;
     const int per_o = (n_out + cs - 1) / cs;
+    for (int o = tid; o < n_out; o += kFT) {
+      const int r = o / per_o, ol = o % per_o;
+      float* dst = cluster.map_shared_rank(&s_racc[0], r);
+      dst[crank * per_o + ol] = s_part[o / FASA_HEAD_DIM][2 + o % FASA_HEAD_DIM];
+    }
+    for (int i = tid; i < cs * GP; i += kFT) {
+      const int r = i / GP, g = i % GP;
+      float* dst = cluster.map_shared_rank(&s_rml[0][0][0], r);
+      dst[(crank * GP + g) * 2 + 0] = s_part[g][0];
+      dst[(crank * GP + g) * 2 + 1] = s_part[g][1];
+    }
+    cluster.sync();   // barrier 5: every CTA's partial results have arrived
     const int opp = kFT / cs;                // outputs per pass (cs is a power of two <= 16)
     const int r = tid % cs, tl = tid / cs;
     for (int t0 = 0; t0 < per_o; t0 += opp) {   // uniform trip count
       const int t = t0 + tl;
       const int o = crank * per_o + t;
       const bool ok = t < per_o && o < n_out;
-      const int g = ok ? o / FASA_HEAD_DIM : 0, c = ok ? o % FASA_HEAD_DIM : 0;
-      const float* pr = cluster.map_shared_rank(&s_part[g][0], r);
-      const float ms = pr[0], ls = pr[1], as = pr[2 + c];
+      const int g = ok ? o / FASA_HEAD_DIM : 0;
+      const float ms = s_rml[r][g][0], ls = s_rml[r][g][1];
+      const float as = ok ? s_racc[r * per_o + t] : 0.f;
       float mx = ms;
       for (int off = cs >> 1; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
       const float wt = ms == -INFINITY ? 0.f : exp2f(ms - mx);
-      float a = wt * as, l = wt * ls;
+      float av = wt * as, l = wt * ls;
       for (int off = cs >> 1; off > 0; off >>= 1) {
-        a += __shfl_xor_sync(0xffffffffu, a, off);
+        av += __shfl_xor_sync(0xffffffffu, av, off);
         l += __shfl_xor_sync(0xffffffffu, l, off);
       }
       if (ok && r == 0) {
+        const int c = o % FASA_HEAD_DIM;
         const int64_t hq = (int64_t)b * p.n_q_heads + (int64_t)h * p.group + g;
-        p.out[hq * FASA_HEAD_DIM + c] = l > 0.f ? a / l : 0.f;
+        p.out[hq * FASA_HEAD_DIM + c] = l > 0.f ? av / l : 0.f;
         if (p.lse && c == 0) p.lse[hq] = l > 0.f ? (mx + log2f(l)) * 0.6931471805599453f : -INFINITY;
       }
     }
   }
-  cluster.sync();   // barrier 7: no CTA leaves while a peer can still read its shared memory
 }
-
-struct FusedPlan {
-  int cs;        // cluster size, 0 = the fused kernel cannot take this configuration
-  int cap;       // keys per CTA
-  size_t smem;   // dynamic shared memory
-};
 
 size_t fused_smem_bytes(int cap) {
   const size_t sel = (size_t)cap * 4 + 2 * kFBins * 4;
