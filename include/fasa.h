@@ -210,6 +210,8 @@ int32_t fasa_sparse_decode_attn_static(fasa_ctx_t* ctx, const void* q, const voi
  * fasa_sparse_decode_attn; scores and workspace are then required (INVALID_ARG if NULL).
  * Both modes select identical index sets; outputs agree to fp32 rounding. */
 int32_t fasa_set_step_mode(fasa_ctx_t* ctx, int32_t mode);
+/* (The mode also selects the kernel behind fasa_topk: the cluster kernel's selection phases
+ * in mode 1, a register-resident cluster kernel in mode 0; the results are identical.) */
 /* Cluster size mode 1 runs with for this context; 0 = fasa_decode_step uses mode 0. */
 int32_t fasa_step_cluster_size(const fasa_ctx_t* ctx);
 int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_cache,

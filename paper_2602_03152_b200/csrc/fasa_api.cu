@@ -150,7 +150,7 @@ extern "C" int32_t fasa_set_step_mode(fasa_ctx_t* ctx, int32_t mode) {
 }
 
 extern "C" int32_t fasa_step_cluster_size(const fasa_ctx_t* ctx) {
-  return ctx && ctx->use_fused ? ctx->fused_cs : 0;
+  return ctx && ctx->use_fused && ctx->fused_step_ok ? ctx->fused_cs : 0;
 }
 
 extern "C" int64_t fasa_launch_count(const fasa_ctx_t* ctx) { return ctx ? ctx->launches : 0; }
@@ -201,7 +201,7 @@ extern "C" int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* 
   if (!ctx || !q || !k_cache || !v_cache || !proxy_k || !seq_lens || !idx || !n_sel || !out ||
       budget == 0 || budget < -1000 || n_sel_max <= 0)
     return FASA_ERR_INVALID_ARG;
-  if (ctx->use_fused && ctx->fused_cs > 0) {
+  if (ctx->use_fused && ctx->fused_step_ok && ctx->fused_cs > 0) {
     if (((uintptr_t)proxy_k & 15) || ((uintptr_t)q & 15) || ((uintptr_t)k_cache & 15) ||
         ((uintptr_t)v_cache & 15) || (scores && ((uintptr_t)scores & 3)))
       return FASA_ERR_INVALID_ARG;
@@ -226,7 +226,7 @@ extern "C" int32_t fasa_append_decode_step(fasa_ctx_t* ctx, const void* q, const
   if (!ctx || !q || !k_new || !v_new || !k_cache || !v_cache || !proxy_k || !seq_lens || !idx ||
       !n_sel || !out || budget == 0 || budget < -1000 || n_sel_max <= 0)
     return FASA_ERR_INVALID_ARG;
-  if (ctx->use_fused && ctx->fused_cs > 0) {
+  if (ctx->use_fused && ctx->fused_step_ok && ctx->fused_cs > 0) {
     if (((uintptr_t)proxy_k & 15) || ((uintptr_t)q & 15) || ((uintptr_t)k_cache & 15) ||
         ((uintptr_t)v_cache & 15) || ((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15) ||
         (scores && ((uintptr_t)scores & 3)))

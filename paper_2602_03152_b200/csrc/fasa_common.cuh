@@ -23,7 +23,8 @@ struct fasa_ctx {
   int16_t* d_chan;        // device [n_kv_heads][row_elems]: K channel of each proxy element, -1 = padding
   int32_t* d_status;      // device status word (FASA_DEV_* bits)
   int32_t* d_arrive;      // device [batch]: CTAs of a sequence that have read its length (append-then-step)
-  int fused_cs;           // cluster size of the one-launch decode step, 0 = not available
+  int fused_cs;           // cluster size of the cluster kernel (step and top-k), 0 = not available
+  int fused_step_ok;      // the one-launch step supports this configuration
   size_t fused_smem;      // its dynamic shared memory
   int use_fused;          // fasa_decode_step takes the one-launch kernel when it is available
   long long launches;     // kernels launched through this context
@@ -61,6 +62,10 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
                           int32_t n_sel_max, float* scores, int32_t* idx, int32_t* n_sel,
                           float* out, float* lse, const void* k_new, const void* v_new,
                           cudaStream_t stream);
+
+int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
+                               int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
+                               cudaStream_t stream);
 
 static inline size_t fasa_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

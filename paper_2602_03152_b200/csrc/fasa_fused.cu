@@ -101,7 +101,9 @@ __device__ __forceinline__ bool warp_find_kth(uint32_t v, uint32_t kth, int lane
 
 // A tile's 16-channel blocks are taken NG groups of KB at a time (KB = 1, 2, 4; NG = 2 only with
 // KB = 4, for more than 4 blocks), which bounds the registers the loads in flight need.
-template <int KB, int NG>
+// MODE 0: the whole step.  MODE 1: TopK-I alone (fasa_topk): the keys come from a score buffer
+// instead of the proxy stream, and the kernel ends after the index list is written.
+template <int KB, int NG, int MODE>
 __global__ void __launch_bounds__(kFT, 2)
 fused_decode_kernel(const FusedParams p) {
   cg::cluster_group cluster = cg::this_cluster();
@@ -141,13 +143,14 @@ fused_decode_kernel(const FusedParams p) {
   // Loads that depend on nothing are issued first, so their (cold) latencies overlap: the
   // length, this thread's share of the query for the attention phase, and the channel table
   // with the query values of the scoring operand.
-  const bool append = p.k_new != nullptr;
+  const bool append = MODE == 0 && p.k_new != nullptr;
   int len_raw = 0;
   if (!append || tid == 0) len_raw = p.seq_lens[b];
   uint4 q_stage = make_uint4(0u, 0u, 0u, 0u);
-  if (tid < FASA_MAX_GROUP * (FASA_HEAD_DIM / 8) && tid / (FASA_HEAD_DIM / 8) < p.group)
+  if (MODE == 0 && tid < FASA_MAX_GROUP * (FASA_HEAD_DIM / 8) && tid / (FASA_HEAD_DIM / 8) < p.group)
     q_stage = *reinterpret_cast<const uint4*>(p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM + tid * 8);
   ScoreFrag<KB> f[NG];
+  if constexpr (MODE == 0)
 #pragma unroll
   for (int grp = 0; grp < NG; ++grp)
     load_score_b<KB>(f[grp], p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM,
@@ -210,7 +213,7 @@ fused_decode_kernel(const FusedParams p) {
   int T = ((crank * per) >> 4) + warp * TPI;                  // slices start on a tile boundary
   const bool own_new = grows && c0 <= len_old && len_old < c1;
   uint4 a[TPI][KB];
-  if (!own_new) fetch(a, T, 0);
+  if (MODE == 0 && !own_new) fetch(a, T, 0);
 
   if (own_new) {
     // this CTA's slice holds the new row: K and V copies (16 lanes each) and the packed
@@ -236,7 +239,7 @@ fused_decode_kernel(const FusedParams p) {
   }
   for (int i = tid; i < 2 * kFBins; i += kFT) hist0[i] = 0u;
   // query, scaled into the base-2 logit domain, for the attention phase
-  if (tid < GP * (FASA_HEAD_DIM / 8)) {
+  if (MODE == 0 && tid < GP * (FASA_HEAD_DIM / 8)) {
     const int g = tid / (FASA_HEAD_DIM / 8), c = (tid % (FASA_HEAD_DIM / 8)) * 8;
     const uint4 w = q_stage;
     const float2 f0 = bf16x2_to_f32x2(w.x), f1 = bf16x2_to_f32x2(w.y), f2 = bf16x2_to_f32x2(w.z), f3 = bf16x2_to_f32x2(w.w);
@@ -247,7 +250,30 @@ fused_decode_kernel(const FusedParams p) {
   __syncthreads();
 
   // ---- 1. scoring stream -> keys + first histogram ------------------------------------------
-  {
+  if constexpr (MODE == 1) {
+    // keys from the caller's score buffer, four consecutive tokens per thread
+    const float* sin = p.scores + (int64_t)u * p.max_len;
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(sin) & 15) == 0);
+    for (int i = c0 + tid * 4; i < c1; i += kFT * 4) {
+      float sv[4] = {0.f, 0.f, 0.f, 0.f};
+      if (vec_ok && i + 3 < c1) {
+        const float4 v4 = *reinterpret_cast<const float4*>(sin + i);
+        sv[0] = v4.x; sv[1] = v4.y; sv[2] = v4.z; sv[3] = v4.w;
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (i + e < c1) sv[e] = sin[i + e];
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (i + e < c1) {
+          const uint32_t key = fasa_item_key(sv[e], i + e, len, p.n_sink, p.n_recent);
+          atomicAdd(&hist0[key >> 21], 1u);
+          keys[i + e - c0] = key;
+        }
+      }
+    }
+  } else {
     if (own_new) fetch(a, T, 0);                              // (the new row is in place now)
     while (T * 16 < c1) {       // uniform over the warp
       float c[TPI][4];
@@ -484,6 +510,10 @@ fused_decode_kernel(const FusedParams p) {
     }
     if (crank == 0 && tid == 0) p.n_sel[u] = (int32_t)ktot;
   }
+  if constexpr (MODE == 1) {
+    cluster.sync();   // no CTA leaves while a peer may still read its totals
+    return;
+  }
   __syncthreads();   // this CTA's part of the index list is written: it attends to its own rows
 
   // ---- 4. attention over this CTA's share of the selected rows -----------------------------
@@ -691,11 +721,13 @@ using FusedFn = void (*)(const FusedParams);
 
 FusedFn fused_fn(int chunks) {
   const int nb = (chunks + 1) / 2;      // 16-channel blocks per tile, the 8-channel one included
-  if (nb <= 1) return fused_decode_kernel<1, 1>;
-  if (nb <= 2) return fused_decode_kernel<2, 1>;
-  if (nb <= 4) return fused_decode_kernel<4, 1>;
-  return fused_decode_kernel<4, 2>;
+  if (nb <= 1) return fused_decode_kernel<1, 1, 0>;
+  if (nb <= 2) return fused_decode_kernel<2, 1, 0>;
+  if (nb <= 4) return fused_decode_kernel<4, 1, 0>;
+  return fused_decode_kernel<4, 2, 0>;
 }
+
+FusedFn topk_fn() { return fused_decode_kernel<1, 1, 1>; }
 
 }  // namespace
 
@@ -706,7 +738,7 @@ int fasa_fused_plan(fasa_ctx* ctx) {
   const fasa_config_t& c = ctx->cfg;
   ctx->fused_cs = 0;
   ctx->fused_smem = 0;
-  if (c.group_reduce != 0) return 0;          // the max reduction takes the three-kernel path
+  ctx->fused_step_ok = c.group_reduce == 0;   // the max reduction takes the three-kernel step
   const int units = c.batch * c.n_kv_heads;
   FusedFn fn = fused_fn(ctx->chunks);
   auto cap_of = [&](int cs) { return (((c.max_len + cs - 1) / cs) + 31) & ~31; };
@@ -742,6 +774,12 @@ int fasa_fused_plan(fasa_ctx* ctx) {
     cfg.numAttrs = 1;
     int n_clusters = 0;
     if (cudaOccupancyMaxActiveClusters(&n_clusters, (const void*)fn, &cfg) != cudaSuccess || n_clusters < 1) {
+      cudaGetLastError();
+      continue;
+    }
+    // the select-only form of the kernel (fasa_topk) runs with the same cluster shape
+    if (cudaFuncSetAttribute((const void*)topk_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        (cs > 8 && cudaFuncSetAttribute((const void*)topk_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)) {
       cudaGetLastError();
       continue;
     }
@@ -787,6 +825,37 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, fn, p);
+  ctx->launches += 1;
+  FASA_CUDA_TRY(ctx, e);
+  return FASA_OK;
+}
+
+// TopK-I alone with the cluster kernel's selection phases (fasa_topk).
+int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
+                               int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
+                               cudaStream_t stream) {
+  const fasa_config_t& c = ctx->cfg;
+  FusedParams p;
+  memset(&p, 0, sizeof(p));
+  p.seq_lens = seq_lens; p.scores = const_cast<float*>(scores); p.idx = idx; p.n_sel = n_sel;
+  p.status = ctx->d_status;
+  p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group; p.max_len = c.max_len;
+  p.chunks = ctx->chunks; p.n_sink = c.n_sink; p.n_recent = c.n_recent; p.budget = budget;
+  p.n_sel_max = n_sel_max;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)ctx->fused_cs, (unsigned)(c.batch * c.n_kv_heads), 1);
+  cfg.blockDim = dim3(kFT, 1, 1);
+  cfg.dynamicSmemBytes = ctx->fused_smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)ctx->fused_cs;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, topk_fn(), p);
   ctx->launches += 1;
   FASA_CUDA_TRY(ctx, e);
   return FASA_OK;

@@ -215,6 +215,11 @@ extern "C" int32_t fasa_topk(fasa_ctx_t* ctx, const float* scores, const int32_t
   if (budget < -1000) return FASA_ERR_INVALID_ARG;
   const fasa_config_t& c = ctx->cfg;
   const int units = c.batch * c.n_kv_heads;
+  // The cluster kernel's selection phases (keys in shared memory, one barrier per radix pass,
+  // mask compaction) serve wherever a cluster shape exists for this context; the
+  // register-resident kernel below remains for the rest (max_len beyond 16 x 22528).
+  if (ctx->use_fused && ctx->fused_cs > 0)
+    return fasa_fused_topk_launch(ctx, scores, seq_lens, budget, n_sel_max, idx, n_sel, (cudaStream_t)stream);
 
   // Cluster size: enough CTAs to hold max_len scores in registers, more when few units
   // would leave SMs idle (down to 2048 scores per CTA).

@@ -389,10 +389,12 @@ def test_device_status_bits_instead_of_faults():
 
 # ------------------------------------------------------------------ top-k alone ----
 
-def _topk_only(scores_cpu, lens, budget, n_sink, n_recent, n_sel_max):
+def _topk_only(scores_cpu, lens, budget, n_sink, n_recent, n_sel_max, mode=1):
+    """mode 1: the cluster kernel's selection phases; mode 0: the register-resident kernel."""
     B, H, Lm = scores_cpu.shape
     dom = torch.arange(4, dtype=torch.int32).repeat(H, 1)
     f = binding.Fasa(B, H, H, Lm, dom, n_sink=n_sink, n_recent=n_recent)
+    f.set_step_mode(mode)
     sc = scores_cpu.cuda()
     ln = torch.tensor(lens, dtype=torch.int32, device="cuda")
     idx = torch.full((B, H, n_sel_max), -7, dtype=torch.int32, device="cuda")
@@ -407,7 +409,9 @@ def _assert_topk_exact(scores_cpu, lens, budget, n_sink=0, n_recent=0, n_sel_max
     """Given the same fp32 scores, the GPU set equals the oracle's bit for bit, ties included."""
     B, H, Lm = scores_cpu.shape
     n_sel_max = n_sel_max or Lm
-    idx, ns = _topk_only(scores_cpu, lens, budget, n_sink, n_recent, n_sel_max)
+    idx, ns = _topk_only(scores_cpu, lens, budget, n_sink, n_recent, n_sel_max, 1)
+    idx0, ns0 = _topk_only(scores_cpu, lens, budget, n_sink, n_recent, n_sel_max, 0)
+    assert np.array_equal(idx, idx0) and np.array_equal(ns, ns0)      # both kernels, bit for bit
     for b in range(B):
         L = lens[b]
         k = budget if budget > 0 else (-budget * L + 999) // 1000
