@@ -205,7 +205,8 @@ int32_t fasa_sparse_decode_attn_static(fasa_ctx_t* ctx, const void* q, const voi
  * Mode 1 (default where available): ONE kernel, one thread-block cluster per (batch, KV
  * head); scores, histograms and split partials stay in (distributed) shared memory, so
  * `workspace` may be NULL and `scores` may be NULL (they are then not written).  Available
- * when group_reduce == 0 and ceil(max_len / 16) <= 45056; fasa_step_cluster_size tells.
+ * when ceil(max_len / 16) <= 22528 and the device can co-schedule such a cluster;
+ * fasa_step_cluster_size tells.
  * Mode 0, and every configuration mode 1 cannot take: fasa_fc_score -> fasa_topk ->
  * fasa_sparse_decode_attn; scores and workspace are then required (INVALID_ARG if NULL).
  * Both modes select identical index sets; outputs agree to fp32 rounding. */

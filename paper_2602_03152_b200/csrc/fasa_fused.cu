@@ -64,6 +64,7 @@ struct FusedParams {
   float* lse;              // nullable
   int32_t* status;
   int n_q_heads, n_kv_heads, group, max_len, chunks, n_sink, n_recent, budget, n_sel_max;
+  int max_reduce;          // score of a KV head = max over its query heads instead of their sum
   int64_t ksb, ksh, kst, vsb, vsh, vst;
   float scale_log2;        // softmax_scale * log2(e)
 };
@@ -290,8 +291,13 @@ fused_decode_kernel(const FusedParams p) {
 #pragma unroll
       for (int pr = 0; pr < TPI / 2; ++pr) {
         float a_lo, a_hi, b_lo, b_hi, sc;
-        reduce_heads<false>(c[2 * pr], p.group, lane, a_lo, a_hi);
-        reduce_heads<false>(c[2 * pr + 1], p.group, lane, b_lo, b_hi);
+        if (p.max_reduce) {     // uniform
+          reduce_heads<true>(c[2 * pr], p.group, lane, a_lo, a_hi);
+          reduce_heads<true>(c[2 * pr + 1], p.group, lane, b_lo, b_hi);
+        } else {
+          reduce_heads<false>(c[2 * pr], p.group, lane, a_lo, a_hi);
+          reduce_heads<false>(c[2 * pr + 1], p.group, lane, b_lo, b_hi);
+        }
         const int row = (T + 2 * pr) * 16 + pick_row_of_pair(lane, a_lo, a_hi, b_lo, b_hi, sc);
         if (row < c1) {
           const uint32_t key = fasa_item_key(sc, row, len, p.n_sink, p.n_recent);
@@ -738,7 +744,7 @@ int fasa_fused_plan(fasa_ctx* ctx) {
   const fasa_config_t& c = ctx->cfg;
   ctx->fused_cs = 0;
   ctx->fused_smem = 0;
-  ctx->fused_step_ok = c.group_reduce == 0;   // the max reduction takes the three-kernel step
+  ctx->fused_step_ok = 1;
   const int units = c.batch * c.n_kv_heads;
   FusedFn fn = fused_fn(ctx->chunks);
   auto cap_of = [&](int cs) { return (((c.max_len + cs - 1) / cs) + 31) & ~31; };
@@ -806,6 +812,7 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
   p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group; p.max_len = c.max_len;
   p.chunks = ctx->chunks; p.n_sink = c.n_sink; p.n_recent = c.n_recent; p.budget = budget;
   p.n_sel_max = n_sel_max;
+  p.max_reduce = c.group_reduce;
   p.ksb = c.k_stride_b; p.ksh = c.k_stride_h; p.kst = c.k_stride_t;
   p.vsb = c.v_stride_b; p.vsh = c.v_stride_h; p.vst = c.v_stride_t;
   p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
