@@ -149,15 +149,22 @@ def run_reference(args, w):
 
 # ---------------------------------------------------------------- our arm ----
 
-def measure(w, K, W, dev, world, step_mode=None, sampler_factory=None, want_e2e=True):
+def measure(w, K, W, dev, world, step_mode=None, sampler_factory=None, want_e2e=True, t=None, lens=None):
     """Times one workload on this rank's GPU; returns a dict of measurements (durations are
-    max over ranks where that matters)."""
+    max over ranks where that matters).  `t` reuses inputs drawn earlier (their dominant-FC
+    list is redrawn for w.n_dom); `lens` overrides the sequence lengths."""
     import torch
     import torch.distributed as dist
 
     from paper_2602_03152_b200 import binding, synth
 
-    t = synth.make_inputs(w, dev)
+    if t is None:
+        t = synth.make_inputs(w, dev)
+    else:
+        t = dict(t)
+        t["dom"] = synth.dominant_fcs(w)
+    if lens is not None:
+        t["seq_lens"] = torch.as_tensor(lens, dtype=torch.int32, device=dev)
     lens_full = t["seq_lens"].clone()
     # The cache has one spare row so each step appends at row L-1 and scores L rows.
     lens_start = (lens_full - 1).clamp_(min=0)
@@ -177,6 +184,7 @@ def measure(w, K, W, dev, world, step_mode=None, sampler_factory=None, want_e2e=
     dense_out = torch.zeros_like(out)
     lens = lens_full.clone()
     f.proxy_build(k, proxy, lens)
+    torch.cuda.synchronize()
     # the token appended each step: the cache's own last row, so the cache content never changes
     bi = torch.arange(B, device=dev)
     last = lens_start.long()
@@ -384,6 +392,82 @@ def run_fasa(args, w):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """BASELINE config 4: budget x dominant-FC-count grid at the Llama-3-8B shape, batch 8,
+    context 65536.  One JSON object with a row per point."""
+    import torch
+
+    from paper_2602_03152_b200 import build, synth
+
+    build.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    base = synth.CONFIGS["c4"]
+    if args.batch is not None:
+        base = base.replace(batch=args.batch)
+    t = synth.make_inputs(base, dev)
+    peak, peak_src = _peaks()
+    rows = []
+    for F in (4, 8, 16, 32, 64):
+        for k in (64, 128, 256, 512, 1024, 2048, 4096):
+            w = base.replace(n_dom=F, budget=k)
+            m = measure(w, args.sweep_steps, 3, dev, 1, args.step_mode, None, want_e2e=False, t=t)
+            sm = summarize(m, peak)
+            rows.append({k_: sm[k_] for k_ in ("n_dom", "budget", "us_per_step", "step_bytes", "step_gbs", "step_frac_of_peak",
+                                               "dense_us_per_step", "speedup_vs_dense", "byte_ratio_dense_over_fasa",
+                                               "standalone_us", "standalone_frac_of_peak", "step_mode", "device_status")})
+            del m
+    print(json.dumps({"sweep": base.name, "batch": base.batch, "context": base.max_len, "peak_gbs": peak,
+                      "peak_source": peak_src, "steps_per_point": args.sweep_steps, "rows": rows}), flush=True)
+
+
+def run_longcot(args):
+    """BASELINE config 3 (long-CoT shape, Qwen2.5-7B-like attention): 28 layers, batch 32, prompt
+    1024 then 15360 decode steps, budget 18.9 % of the current length, 16 dominant FCs.  One
+    layer's step is timed at sampled cache lengths (FASA and dense); the whole run's decode time
+    is the sum over steps of 28 x the step time, linearly interpolated between the samples."""
+    import torch
+
+    from paper_2602_03152_b200 import build, synth
+
+    build.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    w = synth.CONFIGS["c3"]
+    t = synth.make_inputs(w.replace(len_lo=w.max_len, len_hi=w.max_len), dev)
+    peak, _ = _peaks()
+    samples = [1025, 2048, 4096, 6144, 8192, 10240, 12288, 14336, 16384]
+    pts = []
+    for L in samples:
+        m = measure(w, args.sweep_steps, 3, dev, 1, args.step_mode, None, want_e2e=False, t=t, lens=[L] * w.batch)
+        sm = summarize(m, peak)
+        pts.append({"context": L, "n_sel_per_unit": sm["n_sel_per_unit"], "us_per_step": sm["us_per_step"],
+                    "dense_us_per_step": sm["dense_us_per_step"], "step_frac_of_peak": sm["step_frac_of_peak"],
+                    "dense_frac_of_peak": sm["dense_frac_of_peak"], "speedup_vs_dense": sm["speedup_vs_dense"],
+                    "device_status": sm["device_status"]})
+        del m
+
+    def total(key):
+        acc, n_layers = 0.0, 28
+        for L in range(1025, 16385):              # cache length after each of the 15360 appends
+            j = max(i for i, s_ in enumerate(samples) if s_ <= L)
+            if j == len(samples) - 1:
+                v = pts[j][key]
+            else:
+                a, b = samples[j], samples[j + 1]
+                v = pts[j][key] + (pts[j + 1][key] - pts[j][key]) * (L - a) / (b - a)
+            acc += v * n_layers
+        return acc * 1e-6
+
+    tf, td = total("us_per_step"), total("dense_us_per_step")
+    print(json.dumps({"longcot": w.name, "layers": 28, "batch": w.batch, "prompt": 1024, "decode_steps": 15360,
+                      "budget_permille": -w.budget, "n_dom": w.n_dom, "steps_per_sample": args.sweep_steps,
+                      "fasa_decode_attention_seconds": tf, "dense_decode_attention_seconds": td,
+                      "speedup_vs_dense": td / tf, "theory_byte_ratio": 1.0 / (w.n_dom / 128.0 + 0.189),
+                      "method": "one layer timed at the sampled contexts, linear interpolation, x 28 layers",
+                      "samples": pts}), flush=True)
+
+
 def cpu_baseline(w, t, by):
     """The fp64 oracle, as it stands, timed on the host cores on a bounded sample: the units
     of the first sequence, one whole pass (score -> select -> attention)."""
@@ -423,10 +507,17 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--extras", default="c4,c2", help="other workloads reported under other_workloads (30 steps each)")
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="config 4 grid (budget x dominant FCs) instead of the bench line")
+    ap.add_argument("--longcot", action="store_true", help="config 3 (long-CoT decode) instead of the bench line")
+    ap.add_argument("--sweep-steps", type=int, default=20)
     ap.add_argument("--step-mode", type=int, default=None, choices=[0, 1],
                     help="0: fasa_decode_step as three kernels; 1 (default): one cluster kernel where available")
     args = ap.parse_args()
 
+    if args.sweep:
+        return run_sweep(args)
+    if args.longcot:
+        return run_longcot(args)
     from paper_2602_03152_b200 import synth
     w = synth.CONFIGS[args.config]
     if args.budget is not None:
