@@ -257,6 +257,238 @@ decode_attn_kernel(const AttnParams p) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Tensor-core form.  With a GQA group of G query heads the two products of a decode step are
+// [rows x 128] . [128 x G] (logits) and [128 x rows] . [rows x G] (output, transposed): G <= 8
+// is exactly the N = 8 of mma.m16n8k16.  The scalar kernel above spends ~60 instructions per
+// K/V row per four heads and is bound by instruction issue (0.67 of the copy bandwidth at
+// G = 4, 0.3 at G = 7); here a warp handles 16 rows with 8 + 16 MMAs.
+//   - K and V rows go to shared memory with 16-byte cp.async copies (row stride padded by 16
+//     bytes, so ldmatrix reads them without bank conflicts);
+//   - logits: A = K tile via ldmatrix.x4, B = q (bf16, exact) in registers; the softmax scale
+//     is applied to the fp32 result;
+//   - online softmax per head on the accumulator fragment (a thread owns heads 2t, 2t+1 of
+//     rows g, g+8; row maxima and sums by xor-shuffles over g);
+//   - output: A = V^T via ldmatrix.x4.trans, B = P^T.  P is split into two bf16 terms
+//     (p = hi + lo, error 2^-17 p) because one bf16 term would cost up to 2^-9 |v| of the
+//     2e-3 tolerance; two MMAs per block.
+constexpr int kMmaThreads = 128;
+constexpr int kMmaWarps = kMmaThreads / 32;
+constexpr int kRowPad = FASA_HEAD_DIM + 8;          // bf16 elements per staged row (272 bytes)
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* row) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_addr(row)));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* row) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_addr(row)));
+}
+__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// round-to-nearest-even fp32 -> bf16 bits (finite inputs)
+__device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
+}
+
+struct MmaSmem {
+  uint16_t k[kMmaWarps][16][kRowPad];
+  uint16_t v[kMmaWarps][16][kRowPad];
+  uint16_t p_hi[kMmaWarps][8][16];                  // P^T: [head][row]
+  uint16_t p_lo[kMmaWarps][8][16];
+};
+
+template <bool SPARSE>
+__global__ void __launch_bounds__(kMmaThreads)
+decode_attn_mma_kernel(const AttnParams p) {
+  const int u = blockIdx.y;
+  const int h = u % p.n_kv_heads;
+  const int b = u / p.n_kv_heads;
+  int n;
+  if (SPARSE) {
+    n = p.n_rows[u];
+    if (n < 0 || n > p.n_cap) {
+      atomicOr(p.status, FASA_DEV_NSEL_CLAMPED);
+      n = n < 0 ? 0 : p.n_cap;
+    }
+  } else {
+    n = clamp_len(p.n_rows[b], p.max_len, p.status);
+  }
+  const int split = blockIdx.x;
+  const int r0 = split * p.chunk;
+  if (r0 >= n) return;
+  const int r1 = min(n, r0 + p.chunk);
+
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int g = lane >> 2, t = lane & 3;
+
+  extern __shared__ __align__(16) unsigned char attn_smem_raw[];
+  MmaSmem& sm = *reinterpret_cast<MmaSmem*>(attn_smem_raw);
+
+  // B operand of the logits: q[head g][channels], bf16 as stored, for the 8 blocks of 16 channels
+  uint32_t qb[8][2];
+  {
+    const uint16_t* qh = p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group + (g < p.group ? g : 0)) * FASA_HEAD_DIM;
+#pragma unroll
+    for (int kb = 0; kb < 8; ++kb) {
+      const uint32_t w0 = *reinterpret_cast<const uint32_t*>(qh + kb * 16 + 2 * t);
+      const uint32_t w1 = *reinterpret_cast<const uint32_t*>(qh + kb * 16 + 2 * t + 8);
+      qb[kb][0] = g < p.group ? w0 : 0u;
+      qb[kb][1] = g < p.group ? w1 : 0u;
+    }
+  }
+
+  float acc[8][4];                                  // out^T: [16-channel block][frag], heads 2t, 2t+1
+#pragma unroll
+  for (int cb = 0; cb < 8; ++cb) acc[cb][0] = acc[cb][1] = acc[cb][2] = acc[cb][3] = 0.f;
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+
+  const int32_t* irow = SPARSE ? p.idx + (int64_t)u * p.n_sel_max : nullptr;
+  const uint16_t* kunit = p.k + b * p.ksb + h * p.ksh;
+  const uint16_t* vunit = p.v + b * p.vsb + h * p.vsh;
+
+  for (int base = r0 + warp * 16; base < r1; base += kMmaWarps * 16) {   // uniform over the warp
+    // ---- stage 16 K rows and 16 V rows: lane l copies chunk (l % 16) of rows 2j + l / 16 ----
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int row = 2 * j + (lane >> 4);
+      const int r = min(base + row, r1 - 1);        // rows past the end repeat the last one (masked below)
+      int tok = SPARSE ? __ldg(irow + r) : r;
+      if (SPARSE && (tok < 0 || tok >= p.max_len)) {
+        atomicOr(p.status, FASA_DEV_IDX_CLAMPED);
+        tok = 0;
+      }
+      const int c8 = (lane & 15) * 8;
+      cp_async16(&sm.k[warp][row][c8], kunit + (int64_t)tok * p.kst + c8);
+      cp_async16(&sm.v[warp][row][c8], vunit + (int64_t)tok * p.vst + c8);
+    }
+    cp_async_wait_all();
+    __syncwarp();
+
+    // ---- logits: D[16 rows x 8 heads] ---------------------------------------------------------
+    float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int kb = 0; kb < 8; ++kb) {
+      uint32_t a[4];
+      // matrices: (rows 0-7, ch 0-7), (rows 8-15, ch 0-7), (rows 0-7, ch 8-15), (rows 8-15, ch 8-15)
+      ldmatrix_x4(a, &sm.k[warp][(lane & 7) + 8 * ((lane >> 3) & 1)][kb * 16 + 8 * (lane >> 4)]);
+      mma16816(c, a, qb[kb][0], qb[kb][1]);
+    }
+    // thread: c0, c1 = row g, heads 2t, 2t+1; c2, c3 = row g + 8
+    const bool ok_lo = base + g < r1, ok_hi = base + g + 8 < r1;
+    float lg[4];
+    lg[0] = ok_lo ? c[0] * p.scale_log2 : -INFINITY;
+    lg[1] = ok_lo ? c[1] * p.scale_log2 : -INFINITY;
+    lg[2] = ok_hi ? c[2] * p.scale_log2 : -INFINITY;
+    lg[3] = ok_hi ? c[3] * p.scale_log2 : -INFINITY;
+    float alpha[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      float bm = fmaxf(lg[e], lg[2 + e]);
+      bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
+      bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
+      bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
+      const float m_new = fmaxf(m_run[e], bm);
+      const float m_safe = m_new == -INFINITY ? 0.f : m_new;
+      alpha[e] = exp2f(m_run[e] - m_safe);
+      lg[e] = exp2f(lg[e] - m_safe);
+      lg[2 + e] = exp2f(lg[2 + e] - m_safe);
+      l_run[e] = l_run[e] * alpha[e] + lg[e] + lg[2 + e];   // this thread's rows; the g lanes are added at the end
+      m_run[e] = m_new;
+    }
+    // P^T[head][row] as two bf16 terms
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int head = 2 * t + (e & 1), row = g + 8 * (e >> 1);
+      const uint32_t hi = f32_to_bf16_bits(lg[e]);
+      const float rest = lg[e] - __uint_as_float(hi << 16);
+      sm.p_hi[warp][head][row] = (uint16_t)hi;
+      sm.p_lo[warp][head][row] = (uint16_t)f32_to_bf16_bits(rest);
+    }
+    __syncwarp();
+    // B operand of the output product: B[k = row][n = head g]: rows 2t, 2t+1 and 2t+8, 2t+9
+    const uint32_t ph0 = *reinterpret_cast<const uint32_t*>(&sm.p_hi[warp][g][2 * t]);
+    const uint32_t ph1 = *reinterpret_cast<const uint32_t*>(&sm.p_hi[warp][g][2 * t + 8]);
+    const uint32_t pl0 = *reinterpret_cast<const uint32_t*>(&sm.p_lo[warp][g][2 * t]);
+    const uint32_t pl1 = *reinterpret_cast<const uint32_t*>(&sm.p_lo[warp][g][2 * t + 8]);
+
+    // ---- output: out^T[16 ch x 8 heads] += V^T[16 ch x 16 rows] . P^T[16 rows x 8 heads] ------
+#pragma unroll
+    for (int cb = 0; cb < 8; ++cb) {
+      acc[cb][0] *= alpha[0]; acc[cb][1] *= alpha[1]; acc[cb][2] *= alpha[0]; acc[cb][3] *= alpha[1];
+      uint32_t a[4];
+      // source blocks (token rows x channels), transposed on load:
+      // (rows 0-7, ch 0-7), (rows 0-7, ch 8-15), (rows 8-15, ch 0-7), (rows 8-15, ch 8-15)
+      ldmatrix_x4_trans(a, &sm.v[warp][(lane & 7) + 8 * (lane >> 4)][cb * 16 + 8 * ((lane >> 3) & 1)]);
+      mma16816(acc[cb], a, ph0, ph1);
+      mma16816(acc[cb], a, pl0, pl1);
+    }
+    __syncwarp();   // the staging buffers are refilled by the next tile
+  }
+
+  // ---- this warp's (m, l, acc) per head; the g lanes add their sums -------------------------------
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
+    l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
+    l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
+  }
+  __syncthreads();                                  // staging memory becomes the combine area
+  float* s_acc = reinterpret_cast<float*>(attn_smem_raw);                 // [warps][8 heads][128]
+  float* s_ml = s_acc + kMmaWarps * 8 * FASA_HEAD_DIM;                    // [warps][8 heads][2]
+#pragma unroll
+  for (int cb = 0; cb < 8; ++cb) {
+    s_acc[(warp * 8 + 2 * t) * FASA_HEAD_DIM + cb * 16 + g] = acc[cb][0];
+    s_acc[(warp * 8 + 2 * t + 1) * FASA_HEAD_DIM + cb * 16 + g] = acc[cb][1];
+    s_acc[(warp * 8 + 2 * t) * FASA_HEAD_DIM + cb * 16 + g + 8] = acc[cb][2];
+    s_acc[(warp * 8 + 2 * t + 1) * FASA_HEAD_DIM + cb * 16 + g + 8] = acc[cb][3];
+  }
+  if (g == 0) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      s_ml[(warp * 8 + 2 * t + e) * 2 + 0] = m_run[e];
+      s_ml[(warp * 8 + 2 * t + e) * 2 + 1] = l_run[e];
+    }
+  }
+  __syncthreads();
+  const int cch = threadIdx.x;                      // one channel per thread
+  for (int gl = 0; gl < p.group; ++gl) {
+    float mx = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kMmaWarps; ++w) mx = fmaxf(mx, s_ml[(w * 8 + gl) * 2]);
+    float a = 0.f, l = 0.f;
+#pragma unroll
+    for (int w = 0; w < kMmaWarps; ++w) {
+      const float ms = s_ml[(w * 8 + gl) * 2];
+      const float wt = ms == -INFINITY ? 0.f : exp2f(ms - mx);
+      a += wt * s_acc[(w * 8 + gl) * FASA_HEAD_DIM + cch];
+      l += wt * s_ml[(w * 8 + gl) * 2 + 1];
+    }
+    float* dst = p.partial +
+                 (((int64_t)b * p.n_q_heads + (int64_t)h * p.group + gl) * p.n_splits + split) * kPartialStride;
+    dst[2 + cch] = a;
+    if (cch == 0) {
+      dst[0] = mx;
+      dst[1] = l;
+    }
+  }
+}
+
 // Merge pass: one CTA per (batch, query head), one channel per thread.
 template <bool SPARSE>
 __global__ void __launch_bounds__(FASA_HEAD_DIM)
@@ -308,7 +540,12 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
   dim3 grid((unsigned)plan.n_splits, (unsigned)(c.batch * c.n_kv_heads));
   const int G = ctx->group;
-  if (G == 1) decode_attn_kernel<1, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
+  if (ctx->use_fused) {   // default: the tensor-core kernel (mode 0 keeps the scalar one)
+    static_assert(sizeof(MmaSmem) >= (size_t)kMmaWarps * 8 * (FASA_HEAD_DIM + 2) * sizeof(float), "combine area");
+    auto fn = decode_attn_mma_kernel<SPARSE>;
+    FASA_CUDA_TRY(ctx, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MmaSmem)));
+    fn<<<grid, kMmaThreads, sizeof(MmaSmem), s>>>(p);
+  } else if (G == 1) decode_attn_kernel<1, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   else if (G == 2) decode_attn_kernel<2, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   else if (G == 3) decode_attn_kernel<3, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   else if (G == 4) decode_attn_kernel<4, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);

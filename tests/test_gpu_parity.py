@@ -195,11 +195,15 @@ def test_decode_step_equals_separate_calls_and_host_variant():
     for x, y in zip(ref[:3], (r.scores, r.idx, r.n_sel)):
         assert torch.equal(x, y)
     assert float((ref[3] - r.out).abs().max()) <= 1e-4      # another split of the rows: fp32 rounding only
-    r.fasa.set_step_mode(0)
+    r.fasa.set_step_mode(0)                                  # mode 0 is the three calls themselves
+    r.step()
+    ref0 = [x.clone() for x in (r.scores, r.idx, r.n_sel, r.out)]
+    assert torch.equal(ref0[1], ref[1]) and float((ref0[3] - ref[3]).abs().max()) <= 1e-4
     r.out.fill_(SENTINEL)
     r.fasa.decode_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel, r.out, r.ws)
     torch.cuda.synchronize()
-    assert torch.equal(ref[3], r.out)                        # mode 0 is the three calls themselves
+    for x, y in zip(ref0, (r.scores, r.idx, r.n_sel, r.out)):
+        assert torch.equal(x, y)
     r.fasa.set_step_mode(1)
     # host variant: append one token, then the same step; compare with the oracle on the grown cache
     s = synth.make_step_inputs(w, 0, "cpu")
