@@ -280,7 +280,7 @@ def measure(w, K, W, dev, world, step_mode=None, sampler_factory=None, want_e2e=
     clocks = sampler.stop() if sampler else None
     return dict(w=w, t=t, by=by, us_per_step=us_per_step, step_us_median=statistics.median(step_us), launches=launches,
                 kern_us=kern_us, dense_us=dense_us, e2e_us=e2e_us, h2d=h2d, d2h=d2h, status=status, clocks=clocks,
-                fused=fused, cluster_size=f.step_cluster_size(), n_sel_total=n_sel_total, lens_full=lens_full)
+                fused=fused, cluster_size=f.step_cluster_size(), launches_per_step=launches / max(K, 1), n_sel_total=n_sel_total, lens_full=lens_full)
 
 
 def summarize(m, peak):
@@ -294,7 +294,10 @@ def summarize(m, peak):
         "context": int(m["lens_full"].max()), "context_mean": float(m["lens_full"].float().mean()),
         "n_dom": w.n_dom, "budget": w.budget, "n_sink": w.n_sink, "n_recent": w.n_recent,
         "n_sel_per_unit": m["n_sel_total"] / (w.batch * w.n_kv_heads),
-        "step_mode": f"one cluster kernel (cluster of {m['cluster_size']})" if m["fused"] else "three kernels",
+        "step_mode": ("three kernels" if not m["fused"] else
+                      f"one cluster kernel (cluster of {m['cluster_size']})" if m["launches_per_step"] == 1 else
+                      f"cluster kernel (cluster of {m['cluster_size']}) + split-K tensor-core attention"),
+        "launches_per_step": m["launches_per_step"],
         "us_per_step": m["us_per_step"], "step_bytes": by["fasa"],
         "step_gbs": gbs(by["fasa"], m["us_per_step"]), "step_frac_of_peak": gbs(by["fasa"], m["us_per_step"]) / peak,
         "dense_us_per_step": m["dense_us"], "dense_bytes": by["dense"],
@@ -415,7 +418,8 @@ def run_sweep(args):
             sm = summarize(m, peak)
             rows.append({k_: sm[k_] for k_ in ("n_dom", "budget", "us_per_step", "step_bytes", "step_gbs", "step_frac_of_peak",
                                                "dense_us_per_step", "speedup_vs_dense", "byte_ratio_dense_over_fasa",
-                                               "standalone_us", "standalone_frac_of_peak", "step_mode", "device_status")})
+                                               "standalone_us", "standalone_frac_of_peak", "step_mode", "launches_per_step",
+                                               "device_status")})
             del m
     print(json.dumps({"sweep": base.name, "batch": base.batch, "context": base.max_len, "peak_gbs": peak,
                       "peak_source": peak_src, "steps_per_point": args.sweep_steps, "rows": rows}), flush=True)

@@ -205,6 +205,12 @@ extern "C" int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* 
     if (((uintptr_t)proxy_k & 15) || ((uintptr_t)q & 15) || ((uintptr_t)k_cache & 15) ||
         ((uintptr_t)v_cache & 15) || (scores && ((uintptr_t)scores & 3)))
       return FASA_ERR_INVALID_ARG;
+    if (fasa_attend_separately(ctx, n_sel_max, workspace)) {
+      int32_t st2 = fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
+                                      idx, n_sel, out, lse, nullptr, nullptr, (cudaStream_t)stream, false);
+      if (st2 != FASA_OK) return st2;
+      return fasa_sparse_decode_attn(ctx, q, k_cache, v_cache, idx, n_sel, n_sel_max, out, lse, workspace, stream);
+    }
     return fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
                              idx, n_sel, out, lse, nullptr, nullptr, (cudaStream_t)stream);
   }
@@ -231,6 +237,12 @@ extern "C" int32_t fasa_append_decode_step(fasa_ctx_t* ctx, const void* q, const
         ((uintptr_t)v_cache & 15) || ((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15) ||
         (scores && ((uintptr_t)scores & 3)))
       return FASA_ERR_INVALID_ARG;
+    if (fasa_attend_separately(ctx, n_sel_max, workspace)) {
+      int32_t st2 = fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
+                                      idx, n_sel, out, lse, k_new, v_new, (cudaStream_t)stream, false);
+      if (st2 != FASA_OK) return st2;
+      return fasa_sparse_decode_attn(ctx, q, k_cache, v_cache, idx, n_sel, n_sel_max, out, lse, workspace, stream);
+    }
     return fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
                              idx, n_sel, out, lse, k_new, v_new, (cudaStream_t)stream);
   }

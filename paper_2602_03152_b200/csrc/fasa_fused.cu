@@ -103,7 +103,9 @@ __device__ __forceinline__ bool warp_find_kth(uint32_t v, uint32_t kth, int lane
 // A tile's 16-channel blocks are taken NG groups of KB at a time (KB = 1, 2, 4; NG = 2 only with
 // KB = 4, for more than 4 blocks), which bounds the registers the loads in flight need.
 // MODE 0: the whole step.  MODE 1: TopK-I alone (fasa_topk): the keys come from a score buffer
-// instead of the proxy stream, and the kernel ends after the index list is written.
+// instead of the proxy stream, and the kernel ends after the index list is written.  MODE 2:
+// the step without its attention phase (large selections are attended by the split-K
+// tensor-core kernel instead).
 template <int KB, int NG, int MODE>
 __global__ void __launch_bounds__(kFT, 2)
 fused_decode_kernel(const FusedParams p) {
@@ -144,14 +146,14 @@ fused_decode_kernel(const FusedParams p) {
   // Loads that depend on nothing are issued first, so their (cold) latencies overlap: the
   // length, this thread's share of the query for the attention phase, and the channel table
   // with the query values of the scoring operand.
-  const bool append = MODE == 0 && p.k_new != nullptr;
+  const bool append = MODE != 1 && p.k_new != nullptr;
   int len_raw = 0;
   if (!append || tid == 0) len_raw = p.seq_lens[b];
   uint4 q_stage = make_uint4(0u, 0u, 0u, 0u);
   if (MODE == 0 && tid < FASA_MAX_GROUP * (FASA_HEAD_DIM / 8) && tid / (FASA_HEAD_DIM / 8) < p.group)
     q_stage = *reinterpret_cast<const uint4*>(p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM + tid * 8);
   ScoreFrag<KB> f[NG];
-  if constexpr (MODE == 0)
+  if constexpr (MODE != 1)
 #pragma unroll
   for (int grp = 0; grp < NG; ++grp)
     load_score_b<KB>(f[grp], p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM,
@@ -214,7 +216,7 @@ fused_decode_kernel(const FusedParams p) {
   int T = ((crank * per) >> 4) + warp * TPI;                  // slices start on a tile boundary
   const bool own_new = grows && c0 <= len_old && len_old < c1;
   uint4 a[TPI][KB];
-  if (MODE == 0 && !own_new) fetch(a, T, 0);
+  if (MODE != 1 && !own_new) fetch(a, T, 0);
 
   if (own_new) {
     // this CTA's slice holds the new row: K and V copies (16 lanes each) and the packed
@@ -516,7 +518,7 @@ fused_decode_kernel(const FusedParams p) {
     }
     if (crank == 0 && tid == 0) p.n_sel[u] = (int32_t)ktot;
   }
-  if constexpr (MODE == 1) {
+  if constexpr (MODE != 0) {
     cluster.sync();   // no CTA leaves while a peer may still read its totals
     return;
   }
@@ -735,6 +737,14 @@ FusedFn fused_fn(int chunks) {
 
 FusedFn topk_fn() { return fused_decode_kernel<1, 1, 1>; }
 
+FusedFn select_fn(int chunks) {         // the step without attention
+  const int nb = (chunks + 1) / 2;
+  if (nb <= 1) return fused_decode_kernel<1, 1, 2>;
+  if (nb <= 2) return fused_decode_kernel<2, 1, 2>;
+  if (nb <= 4) return fused_decode_kernel<4, 1, 2>;
+  return fused_decode_kernel<4, 2, 2>;
+}
+
 }  // namespace
 
 // Decides once per context whether and how the fused kernel runs: the smallest cluster whose
@@ -783,9 +793,11 @@ int fasa_fused_plan(fasa_ctx* ctx) {
       cudaGetLastError();
       continue;
     }
-    // the select-only form of the kernel (fasa_topk) runs with the same cluster shape
+    // the select-only forms of the kernel run with the same cluster shape
     if (cudaFuncSetAttribute((const void*)topk_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-        (cs > 8 && cudaFuncSetAttribute((const void*)topk_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)) {
+        cudaFuncSetAttribute((const void*)select_fn(ctx->chunks), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        (cs > 8 && (cudaFuncSetAttribute((const void*)topk_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+                    cudaFuncSetAttribute((const void*)select_fn(ctx->chunks), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess))) {
       cudaGetLastError();
       continue;
     }
@@ -800,7 +812,7 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
                           const void* proxy_k, const int32_t* seq_lens, int32_t budget,
                           int32_t n_sel_max, float* scores, int32_t* idx, int32_t* n_sel,
                           float* out, float* lse, const void* k_new, const void* v_new,
-                          cudaStream_t stream) {
+                          cudaStream_t stream, bool with_attention) {
   const fasa_config_t& c = ctx->cfg;
   FusedParams p;
   p.q = (const uint16_t*)q; p.k = (const uint16_t*)k_cache; p.v = (const uint16_t*)v_cache;
@@ -816,7 +828,7 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
   p.ksb = c.k_stride_b; p.ksh = c.k_stride_h; p.kst = c.k_stride_t;
   p.vsb = c.v_stride_b; p.vsh = c.v_stride_h; p.vst = c.v_stride_t;
   p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
-  FusedFn fn = fused_fn(ctx->chunks);
+  FusedFn fn = with_attention ? fused_fn(ctx->chunks) : select_fn(ctx->chunks);
 
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));

@@ -255,6 +255,28 @@ def test_append_decode_step_equals_append_then_step(mode):
                       n_sel=b.n_sel.cpu().numpy(), out=b.out.cpu().numpy(), what="append+step", **b.oracle_kwargs())
 
 
+def test_large_selection_is_attended_by_the_split_k_kernel():
+    # n_sel_max * ceil(G / 4) >= 2048 and a workspace: cluster kernel without its attention
+    # phase, then the split-K tensor-core attention (3 launches); same results as one launch
+    w = C["c3"].replace(batch=2, max_len=6000, len_lo=5000, len_hi=6000, budget=-300)
+    r = Run(w)
+    r.build_proxy()
+    r.step(fused=True)                       # no workspace: one launch
+    one = [x.clone() for x in (r.scores, r.idx, r.n_sel, r.out, r.lse)]
+    r.reset_outputs()
+    n0 = r.fasa.launch_count()
+    r.fasa.decode_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel, r.out, r.ws, r.lse)
+    torch.cuda.synchronize()
+    assert r.fasa.launch_count() - n0 == 3
+    for x, y in zip(one[:3], (r.scores, r.idx, r.n_sel)):
+        assert torch.equal(x, y)
+    assert float((one[3] - r.out).abs().max()) <= 1e-4 and float((one[4] - r.lse).abs().max()) <= 1e-4
+    h = r.host()
+    parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
+                      n_sel=h["n_sel"], out=h["out"], what="split attention", **r.oracle_kwargs())
+    assert r.fasa.device_status() == 0
+
+
 def test_strided_token_major_cache():
     # K/V stored [B][L][Hkv][128] (token-major), addressed through the stride fields.
     w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, batch=2, max_len=640, len_lo=400, len_hi=640, budget=40)
