@@ -40,6 +40,28 @@ UNIT = "GB/s"
 L2_FLUSH_BYTES = 256 << 20
 
 
+# DRAM traffic of the dominant kernel, from the ncu capture summarised in
+# profiles/fused_decode_kernel_c4.md: read + write bytes per launch over the launch's algorithmic
+# bytes.  Traffic follows the tokens processed, so the ratio carries over to other workloads of
+# the same kernel; it is reported only while the kernel sources are the captured ones.
+TRAFFIC_CAPTURE = {"kernel": "fused_decode_kernel", "workload": "c4", "dram_bytes": 280.64e6, "algorithmic_bytes": 277.02e6,
+                   "sources": ("paper_2602_03152_b200/csrc/fasa_fused.cu", "paper_2602_03152_b200/csrc/fasa_score_core.cuh"),
+                   "sha1": "e811772c9d0f9b9377398b2691ad92c574a265af"}
+
+
+def _traffic(bytes_per_launch):
+    import hashlib
+    h = hashlib.sha1()
+    try:
+        for f in TRAFFIC_CAPTURE["sources"]:
+            h.update(open(os.path.join(ROOT, f), "rb").read())
+    except OSError:
+        return None
+    if h.hexdigest() != TRAFFIC_CAPTURE["sha1"]:
+        return None     # the kernel changed since the counters were taken
+    return bytes_per_launch * TRAFFIC_CAPTURE["dram_bytes"] / TRAFFIC_CAPTURE["algorithmic_bytes"]
+
+
 def _peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -360,7 +382,9 @@ def run_fasa(args, w):
     if m["fused"]:
         # dominant kernel = the whole step in one launch: its algorithmic bytes are the step's
         roofline = {"kernel": "fused_decode_kernel", "bound": "hbm", "achieved": head["step_gbs"], "peak": peak,
-                    "unit": "GB/s", "frac": head["step_frac_of_peak"], "traffic": None,
+                    "unit": "GB/s", "frac": head["step_frac_of_peak"],
+                    "traffic": _traffic(by["fasa"]) if m["launches_per_step"] == 1 else None,
+                    "traffic_source": "ncu capture at workload c4 scaled by algorithmic bytes (profiles/fused_decode_kernel_c4.md)",
                     "bytes_per_launch": by["fasa"], "us_per_launch": us_per_step, "peak_source": peak_src,
                     "cluster_size": m["cluster_size"]}
     else:
