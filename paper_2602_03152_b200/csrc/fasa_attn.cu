@@ -489,9 +489,12 @@ decode_attn_mma_kernel(const AttnParams p) {
   }
 }
 
-// Merge pass: one CTA per (batch, query head), one channel per thread.
+// Merge pass: one CTA per (batch, query head); thread (c, j) takes channel c of the splits
+// s = j, j + 4, ... so that four chains of dependent loads run side by side, then the four
+// partial merges are merged.
+constexpr int kMergeWays = 4;
 template <bool SPARSE>
-__global__ void __launch_bounds__(FASA_HEAD_DIM)
+__global__ void __launch_bounds__(FASA_HEAD_DIM * kMergeWays)
 decode_attn_merge_kernel(const float* __restrict__ partial, const int32_t* __restrict__ n_rows,
                          float* __restrict__ out, float* __restrict__ lse,
                          int32_t* __restrict__ status, int n_q_heads, int n_kv_heads, int group,
@@ -508,20 +511,40 @@ decode_attn_merge_kernel(const float* __restrict__ partial, const int32_t* __res
     n = n < 0 ? 0 : (n > max_len ? max_len : n);
   }
   const int ns = min(n_splits, (n + chunk - 1) / chunk);
-  const int c = threadIdx.x;
+  const int c = threadIdx.x % FASA_HEAD_DIM;
+  const int j = threadIdx.x / FASA_HEAD_DIM;
   const float* src = partial + (int64_t)bh * n_splits * kPartialStride;
+  __shared__ float s_m[kMergeWays], s_l[kMergeWays];
+  __shared__ float s_a[kMergeWays][FASA_HEAD_DIM];
   float mx = -INFINITY;
-  for (int s = 0; s < ns; ++s) mx = fmaxf(mx, src[s * kPartialStride]);
+  for (int s = j; s < ns; s += kMergeWays) mx = fmaxf(mx, src[s * kPartialStride]);
   float a = 0.f, l = 0.f;
-  for (int s = 0; s < ns; ++s) {
+  for (int s = j; s < ns; s += kMergeWays) {
     const float ms = src[s * kPartialStride];
     const float w = ms == -INFINITY ? 0.f : exp2f(ms - mx);
     a += w * src[s * kPartialStride + 2 + c];
     l += w * src[s * kPartialStride + 1];
   }
-  out[(int64_t)bh * FASA_HEAD_DIM + c] = (ns > 0 && l > 0.f) ? a / l : 0.f;
+  s_a[j][c] = a;
+  if (c == 0) {
+    s_m[j] = mx;
+    s_l[j] = l;
+  }
+  __syncthreads();
+  if (j != 0) return;
+  float m_all = -INFINITY;
+#pragma unroll
+  for (int k = 0; k < kMergeWays; ++k) m_all = fmaxf(m_all, s_m[k]);
+  float a_all = 0.f, l_all = 0.f;
+#pragma unroll
+  for (int k = 0; k < kMergeWays; ++k) {
+    const float w = s_m[k] == -INFINITY ? 0.f : exp2f(s_m[k] - m_all);
+    a_all += w * s_a[k][c];
+    l_all += w * s_l[k];
+  }
+  out[(int64_t)bh * FASA_HEAD_DIM + c] = (ns > 0 && l_all > 0.f) ? a_all / l_all : 0.f;
   if (lse && c == 0)
-    lse[bh] = (ns > 0 && l > 0.f) ? (mx + log2f(l)) * 0.6931471805599453f : -INFINITY;
+    lse[bh] = (ns > 0 && l_all > 0.f) ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
 }
 
 template <bool SPARSE>
@@ -552,7 +575,7 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   else if (G <= 6) decode_attn_kernel<3, 2, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   else decode_attn_kernel<4, 2, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   FASA_LAUNCH_CHECK(ctx);
-  decode_attn_merge_kernel<SPARSE><<<c.batch * c.n_q_heads, FASA_HEAD_DIM, 0, s>>>(
+  decode_attn_merge_kernel<SPARSE><<<c.batch * c.n_q_heads, FASA_HEAD_DIM * kMergeWays, 0, s>>>(
       (const float*)workspace, n_rows, out, lse, ctx->d_status, c.n_q_heads, c.n_kv_heads,
       ctx->group, c.max_len, n_upper, plan.chunk, plan.n_splits);
   FASA_LAUNCH_CHECK(ctx);
