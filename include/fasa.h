@@ -236,10 +236,11 @@ int32_t fasa_append_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_ne
                                 float* scores, int32_t* idx, int32_t* n_sel, float* out,
                                 float* lse, void* workspace, void* stream);
 
-/* End-to-end step from HOST buffers (pinned memory recommended): copies q_host,
- * k_new_host, v_new_host (layouts as fasa_kv_append with n_new = 1) to the device
- * staging area dev_stage (>= fasa_stage_bytes), appends, runs fasa_decode_step,
- * copies out to out_host (fp32 [batch][n_q_heads][128]) and synchronises the stream. */
+/* End-to-end step from HOST buffers: q_host, k_new_host, v_new_host (layouts as
+ * fasa_kv_append with n_new = 1) -> fasa_append_decode_step -> out copied to out_host
+ * (fp32 [batch][n_q_heads][128]); synchronises the stream.  Inputs in pinned (page-locked,
+ * mapped) host memory are read by the kernels in place, across the host link; pageable
+ * inputs are first copied to the device staging area dev_stage (>= fasa_stage_bytes). */
 int32_t fasa_stage_bytes(const fasa_ctx_t* ctx, size_t* out_bytes);
 int32_t fasa_decode_step_host(fasa_ctx_t* ctx, const void* q_host, const void* k_new_host,
                               const void* v_new_host, void* dev_stage, void* k_cache,

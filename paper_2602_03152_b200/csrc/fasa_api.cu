@@ -223,12 +223,15 @@ extern "C" int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* 
                                  workspace, stream);
 }
 
-extern "C" int32_t fasa_append_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_new,
-                                           const void* v_new, void* k_cache, void* v_cache,
-                                           void* proxy_k, int32_t* seq_lens, int32_t budget,
-                                           int32_t n_sel_max, float* scores, int32_t* idx,
-                                           int32_t* n_sel, float* out, float* lse, void* workspace,
-                                           void* stream) {
+// out_mirror (nullable): device-accessible second destination of `out`; *mirrored tells whether
+// the path taken wrote it.
+static int32_t append_decode_step_impl(fasa_ctx_t* ctx, const void* q, const void* k_new,
+                                       const void* v_new, void* k_cache, void* v_cache,
+                                       void* proxy_k, int32_t* seq_lens, int32_t budget,
+                                       int32_t n_sel_max, float* scores, int32_t* idx,
+                                       int32_t* n_sel, float* out, float* lse, void* workspace,
+                                       void* stream, float* out_mirror, bool* mirrored) {
+  *mirrored = false;
   if (!ctx || !q || !k_new || !v_new || !k_cache || !v_cache || !proxy_k || !seq_lens || !idx ||
       !n_sel || !out || budget == 0 || budget < -1000 || n_sel_max <= 0)
     return FASA_ERR_INVALID_ARG;
@@ -243,13 +246,25 @@ extern "C" int32_t fasa_append_decode_step(fasa_ctx_t* ctx, const void* q, const
       if (st2 != FASA_OK) return st2;
       return fasa_sparse_decode_attn(ctx, q, k_cache, v_cache, idx, n_sel, n_sel_max, out, lse, workspace, stream);
     }
+    *mirrored = out_mirror != nullptr;
     return fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
-                             idx, n_sel, out, lse, k_new, v_new, (cudaStream_t)stream);
+                             idx, n_sel, out, lse, k_new, v_new, (cudaStream_t)stream, true, out_mirror);
   }
   int32_t st = fasa_kv_append(ctx, k_cache, v_cache, proxy_k, seq_lens, k_new, v_new, 1, stream);
   if (st != FASA_OK) return st;
   return fasa_decode_step(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores, idx,
                           n_sel, out, lse, workspace, stream);
+}
+
+extern "C" int32_t fasa_append_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_new,
+                                           const void* v_new, void* k_cache, void* v_cache,
+                                           void* proxy_k, int32_t* seq_lens, int32_t budget,
+                                           int32_t n_sel_max, float* scores, int32_t* idx,
+                                           int32_t* n_sel, float* out, float* lse, void* workspace,
+                                           void* stream) {
+  bool mirrored;
+  return append_decode_step_impl(ctx, q, k_new, v_new, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max,
+                                 scores, idx, n_sel, out, lse, workspace, stream, nullptr, &mirrored);
 }
 
 extern "C" int32_t fasa_stage_bytes(const fasa_ctx_t* ctx, size_t* out_bytes) {
@@ -277,14 +292,37 @@ extern "C" int32_t fasa_decode_step_host(fasa_ctx_t* ctx, const void* q_host,
   char* dq = (char*)dev_stage;
   char* dk = dq + fasa_align_up(q_bytes, 256);
   char* dv = dk + fasa_align_up(kv_bytes, 256);
-  FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
-  FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
-  FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
-  int32_t st = fasa_append_decode_step(ctx, dq, dk, dv, k_cache, v_cache, proxy_k, seq_lens, budget,
-                                       n_sel_max, scores, idx, n_sel, out, nullptr, workspace, stream);
+  // Pinned (page-locked, mapped) host buffers are read by the kernels in place: the few KB of
+  // a step cross the host link inside the step's only launch instead of in three copies that
+  // each cost more than the transfer.  Anything else is copied to the staging area first.
+  auto mapped = [](const void* hp) -> const void* {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, hp) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+  };
+  const void* mq = mapped(q_host);
+  const void* mk = mapped(k_new_host);
+  const void* mv = mapped(v_new_host);
+  if (mq && mk && mv && !((uintptr_t)mq & 15) && !((uintptr_t)mk & 15) && !((uintptr_t)mv & 15)) {
+    dq = (char*)mq; dk = (char*)mk; dv = (char*)mv;
+  } else {
+    FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
+    FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
+    FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
+  }
+  // A pinned out_host is written by the step's kernel itself (next to `out`), where the path
+  // taken has a single kernel to do it; otherwise `out` is copied back.
+  float* mo = (float*)mapped(out_host);
+  if ((uintptr_t)mo & 3) mo = nullptr;
+  bool mirrored = false;
+  int32_t st = append_decode_step_impl(ctx, dq, dk, dv, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max,
+                                       scores, idx, n_sel, out, nullptr, workspace, stream, mo, &mirrored);
   if (st != FASA_OK) return st;
   size_t o_bytes = (size_t)c.batch * c.n_q_heads * FASA_HEAD_DIM * sizeof(float);
-  FASA_CUDA_TRY(ctx, cudaMemcpyAsync(out_host, out, o_bytes, cudaMemcpyDeviceToHost, s));
+  if (!mirrored) FASA_CUDA_TRY(ctx, cudaMemcpyAsync(out_host, out, o_bytes, cudaMemcpyDeviceToHost, s));
   FASA_CUDA_TRY(ctx, cudaStreamSynchronize(s));
   return FASA_OK;
 }

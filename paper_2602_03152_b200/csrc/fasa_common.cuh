@@ -61,7 +61,7 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
                           const void* proxy_k, const int32_t* seq_lens, int32_t budget,
                           int32_t n_sel_max, float* scores, int32_t* idx, int32_t* n_sel,
                           float* out, float* lse, const void* k_new, const void* v_new,
-                          cudaStream_t stream, bool with_attention = true);
+                          cudaStream_t stream, bool with_attention = true, float* out_mirror = nullptr);
 // Large selections are attended by the split-K tensor-core kernel rather than inside the
 // cluster kernel (whose attention phase runs on CUDA cores at 64 registers per thread).
 static inline bool fasa_attend_separately(const fasa_ctx* ctx, int n_sel_max, const void* workspace) {

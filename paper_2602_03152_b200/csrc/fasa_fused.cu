@@ -61,6 +61,7 @@ struct FusedParams {
   int32_t* idx;
   int32_t* n_sel;
   float* out;
+  float* out_mirror;       // nullable: a second copy of out (mapped host memory of the host-buffer step)
   float* lse;              // nullable
   int32_t* status;
   int n_q_heads, n_kv_heads, group, max_len, chunks, n_sink, n_recent, budget, n_sel_max;
@@ -712,7 +713,9 @@ fused_decode_kernel(const FusedParams p) {
       if (ok && r == 0) {
         const int c = o % FASA_HEAD_DIM;
         const int64_t hq = (int64_t)b * p.n_q_heads + (int64_t)h * p.group + g;
-        p.out[hq * FASA_HEAD_DIM + c] = l > 0.f ? av / l : 0.f;
+        const float ov = l > 0.f ? av / l : 0.f;
+        p.out[hq * FASA_HEAD_DIM + c] = ov;
+        if (p.out_mirror) p.out_mirror[hq * FASA_HEAD_DIM + c] = ov;
         if (p.lse && c == 0) p.lse[hq] = l > 0.f ? (mx + log2f(l)) * 0.6931471805599453f : -INFINITY;
       }
     }
@@ -812,9 +815,10 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
                           const void* proxy_k, const int32_t* seq_lens, int32_t budget,
                           int32_t n_sel_max, float* scores, int32_t* idx, int32_t* n_sel,
                           float* out, float* lse, const void* k_new, const void* v_new,
-                          cudaStream_t stream, bool with_attention) {
+                          cudaStream_t stream, bool with_attention, float* out_mirror) {
   const fasa_config_t& c = ctx->cfg;
   FusedParams p;
+  p.out_mirror = out_mirror;
   p.q = (const uint16_t*)q; p.k = (const uint16_t*)k_cache; p.v = (const uint16_t*)v_cache;
   p.proxy = (const unsigned char*)proxy_k; p.seq_lens = seq_lens; p.chan = ctx->d_chan;
   p.k_new = (const uint16_t*)k_new; p.v_new = (const uint16_t*)v_new;

@@ -219,6 +219,17 @@ def test_decode_step_equals_separate_calls_and_host_variant():
                             n_sel=r.n_sel.cpu().numpy(), out=out_host.numpy(), what="host step", **r.oracle_kwargs())
     assert rep["units"] == 8
     assert torch.equal(out_host, r.out.cpu())
+    # pageable inputs take the staging copies instead of being read in place: same contract
+    s2 = synth.make_step_inputs(w, 1, "cpu")
+    out2 = torch.empty((w.batch, w.n_q_heads, 128), dtype=torch.float32)
+    r.fasa.decode_step_host(s2["q"], s2["k_new"], s2["v_new"], stage, r.k, r.v, r.proxy, r.seq_lens, w.budget,
+                            r.scores, r.idx, r.n_sel, r.out, out2, r.ws)
+    assert r.seq_lens.cpu().tolist() == [1502]
+    kc, vc = r.k.cpu(), r.v.cpu()
+    assert torch.equal(kc[:, :, 1501], s2["k_new"][:, :, 0])
+    parity.check_step(s2["q"].double().numpy(), kc.double().numpy(), vc.double().numpy(), [1502],
+                      np.sort(r.dom.numpy(), axis=1), scores=r.scores.cpu().numpy(), idx=r.idx.cpu().numpy(),
+                      n_sel=r.n_sel.cpu().numpy(), out=out2.numpy(), what="host step, pageable", **r.oracle_kwargs())
 
 
 @pytest.mark.parametrize("mode", [1, 0])
