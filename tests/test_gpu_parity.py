@@ -510,3 +510,62 @@ def test_config4_point_full_length_sampled_units():
         parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
                           n_sel=h["n_sel"], out=h["out"], dense_out=h["dense"], units=[(0, 0), (1, 3), (1, 1)],
                           what="c4", **r.oracle_kwargs())
+
+
+def _full_size_sampled(w, units, budget=None, append=False):
+    """A BASELINE configuration at its full size, inputs drawn on the device, run as bench.py runs
+    it (one fasa_append_decode_step / fasa_decode_step call) and checked against the oracle on
+    a few (batch, KV head) units whose K/V are copied to the host."""
+    from gpu_harness import ensure_built
+    ensure_built()
+    t = synth.make_inputs(w, "cuda")
+    f = binding.Fasa.from_workload(w, t["dom"])
+    B, Hq, Hkv, Lm = w.batch, w.n_q_heads, w.n_kv_heads, w.max_len
+    n_sel_max = w.n_sel_max()
+    proxy = f.alloc_proxy()
+    ws = f.alloc_workspace(n_sel_max)
+    idx = torch.full((B, Hkv, n_sel_max), -7, dtype=torch.int32, device="cuda")
+    n_sel = torch.full((B, Hkv), -7, dtype=torch.int32, device="cuda")
+    out = torch.full((B, Hq, 128), SENTINEL, dtype=torch.float32, device="cuda")
+    scores = torch.full((B, Hkv, Lm), SENTINEL, dtype=torch.float32, device="cuda")
+    lens = t["seq_lens"].clone()
+    q, k, v = t["q"], t["k"], t["v"]
+    if append:
+        lens -= 1                                    # the step appends the cache's own last row again
+        bi = torch.arange(B, device="cuda")
+        k_new = k[bi, :, lens.long()].unsqueeze(2).contiguous()
+        v_new = v[bi, :, lens.long()].unsqueeze(2).contiguous()
+        f.proxy_build(k, proxy, lens)
+        f.append_decode_step(q, k_new, v_new, k, v, proxy, lens, w.budget, scores, idx, n_sel, out, ws)
+    else:
+        f.proxy_build(k, proxy, lens)
+        f.decode_step(q, k, v, proxy, lens, w.budget, scores, idx, n_sel, out, ws)
+    torch.cuda.synchronize()
+    assert f.device_status() == 0
+    assert torch.equal(lens, t["seq_lens"])
+    G = w.group
+    dom = np.sort(t["dom"].numpy(), axis=1)
+    for (b, h) in units:
+        L = int(t["seq_lens"][b])
+        # one-unit views in the layouts check_step expects: [1][G][d], [1][1][L][d]
+        rep = parity.check_step(q[b:b + 1, h * G:(h + 1) * G].cpu().double().numpy(), k[b:b + 1, h:h + 1, :L].cpu().double().numpy(),
+                                v[b:b + 1, h:h + 1, :L].cpu().double().numpy(), [L], dom[h:h + 1], pairing=w.pairing,
+                                group_reduce=w.group_reduce, n_sink=w.n_sink, n_recent=w.n_recent, budget=w.budget,
+                                scale=1.0 / math.sqrt(128.0), scores=scores[b:b + 1, h:h + 1, :L].cpu().numpy(),
+                                idx=idx[b:b + 1, h:h + 1].cpu().numpy(), n_sel=n_sel[b:b + 1, h:h + 1].cpu().numpy(),
+                                out=out[b:b + 1, h * G:(h + 1) * G].cpu().numpy(), what=f"{w.name} unit ({b},{h})")
+        assert rep["units"] == 1
+    return f
+
+
+def test_config2_full_size_sampled_units():
+    # batch 16, ragged 64K-128K contexts, 8 GiB of K/V on the device: the cluster kernel in clusters of 8
+    f = _full_size_sampled(C["c2"], [(0, 0), (7, 5), (15, 7)])
+    assert f.step_cluster_size() == 8
+
+
+def test_config3_full_size_sampled_units_with_append():
+    # long-CoT shape at its last step: batch 32, G = 7, 16384 rows, budget 18.9 %; the selection is
+    # large, so the step is the cluster kernel without attention + the split-K tensor-core kernel
+    w = C["c3"].replace(len_lo=16384, len_hi=16384)
+    _full_size_sampled(w, [(0, 0), (31, 3), (13, 2)], append=True)
