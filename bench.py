@@ -420,7 +420,7 @@ def run_fasa(args, w):
 
 
 def run_sweep(args):
-    """BASELINE config 4: budget x dominant-FC-count grid at the Llama-3-8B shape, batch 8,
+    """Workload c4 as a grid: budget x dominant-FC count at the Llama-3-8B shape, batch 8,
     context 65536.  One JSON object with a row per point."""
     import torch
 
@@ -450,7 +450,7 @@ def run_sweep(args):
 
 
 def run_longcot(args):
-    """BASELINE config 3 (long-CoT shape, Qwen2.5-7B-like attention): 28 layers, batch 32, prompt
+    """Workload c3 (long-CoT shape, Qwen2.5-7B-like attention): 28 layers, batch 32, prompt
     1024 then 15360 decode steps, budget 18.9 % of the current length, 16 dominant FCs.  One
     layer's step is timed at sampled cache lengths (FASA and dense); the whole run's decode time
     is the sum over steps of 28 x the step time, linearly interpolated between the samples."""

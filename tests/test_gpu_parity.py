@@ -513,7 +513,7 @@ def test_config4_point_full_length_sampled_units():
 
 
 def _full_size_sampled(w, units, budget=None, append=False):
-    """A BASELINE configuration at its full size, inputs drawn on the device, run as bench.py runs
+    """A benchmark workload at its full size, inputs drawn on the device, run as bench.py runs
     it (one fasa_append_decode_step / fasa_decode_step call) and checked against the oracle on
     a few (batch, KV head) units whose K/V are copied to the host."""
     from gpu_harness import ensure_built
