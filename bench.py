@@ -94,7 +94,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", gpu_id, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -103,6 +103,10 @@ class ClockSampler:
     def _read(self):
         for line in self.proc.stdout:
             self.rows.append([x.strip() for x in line.split(",")])
+
+    def mark(self):
+        """Forget the samples taken so far (set-up time)."""
+        self.first = len(self.rows)
 
     def stop(self):
         if self.proc is None:
@@ -114,7 +118,7 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], None, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for r in self.rows[getattr(self, "first", 0):]:
             try:
                 sm.append(float(r[0])); mx = float(r[1])
             except (ValueError, IndexError):
@@ -248,7 +252,11 @@ def measure(w, K, W, dev, world, step_mode=None, sampler_factory=None, want_e2e=
         f.kv_append(k, v, proxy, lens, k_new, v_new)
         f.full_decode_attn(q, k, v, lens, dense_out, ws)
 
+    # nvidia-smi needs a moment before its first sample: the sampler was started by the caller
+    # before the inputs were drawn; only samples taken from here on are kept
     sampler = sampler_factory() if sampler_factory else None
+    if sampler is not None:
+        sampler.mark()
 
     # ---- timed region: K whole steps ------------------------------------------------
     timed(fasa_step, 0, W)
@@ -358,7 +366,8 @@ def run_fasa(args, w):
     K, W = args.steps, max(3, args.warmup)
     # Weak scaling: every rank holds its own batch of independent (batch, KV head) units.
     wl = w.replace(index=w.index + 100 * rank)
-    m = measure(wl, K, W, dev, world, args.step_mode, (lambda: ClockSampler(gpu_id)) if rank == 0 else None)
+    sampler = ClockSampler(gpu_id) if rank == 0 else None     # started early, marked at the timed region
+    m = measure(wl, K, W, dev, world, args.step_mode, (lambda: sampler) if rank == 0 else None)
 
     # Other configurations of the same path, a few steps each (single GPU only): the large
     # batched shapes, where the stream is long enough to approach the HBM roofline.
@@ -512,7 +521,7 @@ def cpu_baseline(w, t, by):
               budget=w.budget, n_sel_max=w.n_sel_max(), n_threads=cores, want_scores=False, want_dense=False)
     r = O.decode_bf16(qb, kb, vb, lens, t["dom"].numpy(), **kw)      # warm-up, page in
     reps, t0 = 0, time.perf_counter()
-    while reps < 3 or (time.perf_counter() - t0 < 10.0 and reps < 50):
+    while reps < 3 or (time.perf_counter() - t0 < 10.0 and reps < 2000):
         r = O.decode_bf16(qb, kb, vb, lens, t["dom"].numpy(), **kw)
         reps += 1
     dt = (time.perf_counter() - t0) / reps
