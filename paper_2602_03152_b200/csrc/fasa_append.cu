@@ -10,19 +10,33 @@ namespace {
 // the tiled proxy layout.
 __global__ void __launch_bounds__(256)
 kv_append_kernel(uint16_t* __restrict__ k_cache, uint16_t* __restrict__ v_cache,
-                 unsigned char* __restrict__ proxy, const int32_t* __restrict__ seq_lens,
+                 unsigned char* __restrict__ proxy, const int32_t* seq_lens /* same memory as seq_lens_w */,
                  const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
                  const int16_t* __restrict__ chan, int32_t* __restrict__ status, int n_rows,
                  int n_new, int n_kv_heads, int max_len, int chunks, int64_t ksb, int64_t ksh,
-                 int64_t kst, int64_t vsb, int64_t vsh, int64_t vst) {
+                 int64_t kst, int64_t vsb, int64_t vsh, int64_t vst, int32_t* seq_lens_w,
+                 int32_t* arrive) {
   const int row = blockIdx.x * 2 + (threadIdx.x >> 7);
-  if (row >= n_rows) return;
+  const bool live = row < n_rows;
   const int t = threadIdx.x & 127;
-  const int n = row % n_new;
-  const int u = row / n_new;  // unit = b * n_kv_heads + h
+  const int n = live ? row % n_new : 0;
+  const int u = live ? row / n_new : 0;  // unit = b * n_kv_heads + h
   const int h = u % n_kv_heads;
   const int b = u / n_kv_heads;
-  const int len = clamp_len(seq_lens[b], max_len, status);
+  const int len = live ? clamp_len(seq_lens[b], max_len, status) : 0;
+  // The length is updated here too: once every thread of the CTA has read the old value
+  // (barrier), one thread per row reports in; the last of the sequence's n_kv_heads * n_new
+  // rows to do so stores the new length.  Nobody waits on the counter.
+  __syncthreads();
+  if (live && t == 0) {
+    __threadfence();
+    if (atomicAdd(&arrive[b], 1) == n_kv_heads * n_new - 1) {
+      const int grown = len + n_new;
+      seq_lens_w[b] = grown > max_len ? max_len : grown;
+      arrive[b] = 0;
+    }
+  }
+  if (!live) return;
   const int pos = len + n;
   if (pos >= max_len) {
     if (t == 0) atomicOr(status, FASA_DEV_APPEND_FULL);
@@ -46,15 +60,6 @@ kv_append_kernel(uint16_t* __restrict__ k_cache, uint16_t* __restrict__ v_cache,
     unsigned char* unit = proxy + (int64_t)u * ((max_len + 15) >> 4) * pg.tile_bytes;
     *reinterpret_cast<uint32_t*>(unit + proxy_word_offset(pg, pos, w)) = lo | (hi << 16);
   }
-}
-
-__global__ void seq_len_bump_kernel(int32_t* __restrict__ seq_lens, int batch, int n_new,
-                                    int max_len, int32_t* __restrict__ status) {
-  int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= batch) return;
-  int len = clamp_len(seq_lens[b], max_len, status);
-  len += n_new;
-  seq_lens[b] = len > max_len ? max_len : len;
 }
 
 // One thread per proxy word of rows 0 .. seq_lens[b]-1.
@@ -102,10 +107,7 @@ extern "C" int32_t fasa_kv_append(fasa_ctx_t* ctx, void* k_cache, void* v_cache,
       (uint16_t*)k_cache, (uint16_t*)v_cache, (unsigned char*)proxy_k, seq_lens, (const uint16_t*)k_new,
       (const uint16_t*)v_new, ctx->d_chan, ctx->d_status, (int)n_rows, n_new, c.n_kv_heads,
       c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h, c.k_stride_t, c.v_stride_b,
-      c.v_stride_h, c.v_stride_t);
-  FASA_LAUNCH_CHECK(ctx);
-  seq_len_bump_kernel<<<(c.batch + 127) / 128, 128, 0, s>>>(seq_lens, c.batch, n_new, c.max_len,
-                                                            ctx->d_status);
+      c.v_stride_h, c.v_stride_t, seq_lens, ctx->d_arrive);
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
 }

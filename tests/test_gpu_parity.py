@@ -251,7 +251,7 @@ def test_append_decode_step_equals_append_then_step(mode):
         b.fasa.append_decode_step(s["q"], s["k_new"], s["v_new"], b.k, b.v, b.proxy, b.seq_lens, w.budget, b.scores,
                                   b.idx, b.n_sel, b.out, b.ws)
         torch.cuda.synchronize()
-        assert b.fasa.launch_count() - n0 == (1 if mode == 1 else 6)
+        assert b.fasa.launch_count() - n0 == (1 if mode == 1 else 5)
         for x, y in ((a.k, b.k), (a.v, b.v), (a.proxy, b.proxy), (a.seq_lens, b.seq_lens), (a.scores, b.scores),
                      (a.idx, b.idx), (a.n_sel, b.n_sel)):
             assert torch.equal(x, y)
