@@ -312,9 +312,35 @@ struct MmaSmem {
   uint16_t p_lo[kMmaWarps][8][16];
 };
 
+// Programmatic dependent launch: these kernels may be scheduled while the kernel before them
+// on the stream is still draining (their launch latency then overlaps its tail).  They wait
+// here until that kernel has completed and its writes are visible, and let their own
+// successor be scheduled early in turn.  Launched the ordinary way, both are no-ops.
+__device__ __forceinline__ void pdl_wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_release_successor() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename Kernel, typename... Args>
+cudaError_t launch_after_predecessor(Kernel kernel, dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                     Args... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 template <bool SPARSE>
 __global__ void __launch_bounds__(kMmaThreads)
 decode_attn_mma_kernel(const AttnParams p) {
+  pdl_wait_for_predecessor();
+  pdl_release_successor();
   const int u = blockIdx.y;
   const int h = u % p.n_kv_heads;
   const int b = u / p.n_kv_heads;
@@ -499,6 +525,7 @@ decode_attn_merge_kernel(const float* __restrict__ partial, const int32_t* __res
                          float* __restrict__ out, float* __restrict__ lse,
                          int32_t* __restrict__ status, int n_q_heads, int n_kv_heads, int group,
                          int max_len, int n_cap, int chunk, int n_splits) {
+  pdl_wait_for_predecessor();
   const int bh = blockIdx.x;
   const int b = bh / n_q_heads;
   const int hq = bh % n_q_heads;
@@ -567,7 +594,7 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
     static_assert(sizeof(MmaSmem) >= (size_t)kMmaWarps * 8 * (FASA_HEAD_DIM + 2) * sizeof(float), "combine area");
     auto fn = decode_attn_mma_kernel<SPARSE>;
     FASA_CUDA_TRY(ctx, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MmaSmem)));
-    fn<<<grid, kMmaThreads, sizeof(MmaSmem), s>>>(p);
+    FASA_CUDA_TRY(ctx, launch_after_predecessor(fn, grid, dim3(kMmaThreads), sizeof(MmaSmem), s, p));
   } else if (G == 1) decode_attn_kernel<1, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   else if (G == 2) decode_attn_kernel<2, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   else if (G == 3) decode_attn_kernel<3, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
@@ -575,9 +602,10 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   else if (G <= 6) decode_attn_kernel<3, 2, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   else decode_attn_kernel<4, 2, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   FASA_LAUNCH_CHECK(ctx);
-  decode_attn_merge_kernel<SPARSE><<<c.batch * c.n_q_heads, FASA_HEAD_DIM * kMergeWays, 0, s>>>(
-      (const float*)workspace, n_rows, out, lse, ctx->d_status, c.n_q_heads, c.n_kv_heads,
-      ctx->group, c.max_len, n_upper, plan.chunk, plan.n_splits);
+  FASA_CUDA_TRY(ctx, launch_after_predecessor(
+      decode_attn_merge_kernel<SPARSE>, dim3((unsigned)(c.batch * c.n_q_heads)), dim3(FASA_HEAD_DIM * kMergeWays),
+      (size_t)0, s, (const float*)workspace, n_rows, out, lse, ctx->d_status, (int)c.n_q_heads, (int)c.n_kv_heads,
+      (int)ctx->group, (int)c.max_len, (int)n_upper, (int)plan.chunk, (int)plan.n_splits));
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
 }
