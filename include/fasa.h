@@ -128,8 +128,8 @@ int32_t fasa_proxy_build(fasa_ctx_t* ctx, const void* k_cache, void* proxy_k,
 
 /* scores[b][h][j] = reduce_{g in group(h)} sum_{i in I_dom(h)}
  *                   (q[b][g][c0(i)] K[j][c0(i)] + q[b][g][c1(i)] K[j][c1(i)])
- * for j < seq_lens[b], read from proxy_k; fp32 accumulation of exact bf16
- * products; no scaling.  scores: fp32 [batch][n_kv_heads][max_len]; entries at
+ * for j < seq_lens[b], read from proxy_k; exact bf16 products accumulated in fp32 per
+ * query head on tensor cores, the heads then reduced in fp32; no scaling.  scores: fp32 [batch][n_kv_heads][max_len]; entries at
  * j >= seq_lens[b] are left untouched.  -0 is stored as +0. */
 int32_t fasa_fc_score(fasa_ctx_t* ctx, const void* q, const void* proxy_k,
                       const int32_t* seq_lens, float* scores, void* stream);
