@@ -775,7 +775,10 @@ int fasa_fused_plan(fasa_ctx* ctx) {
     const int cap = cap_of(cs);
     if (cap > kCapMax) break;
     const size_t smem = fused_smem_bytes(cap);
-    if (cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    // The opt-in limit is a property of the kernel, shared by every context of the process:
+    // it is set to the most any context can ask for, not to what this one needs.
+    const int smem_limit = (int)fused_smem_bytes(kCapMax);
+    if (cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit) != cudaSuccess) {
       cudaGetLastError();
       continue;
     }
@@ -797,8 +800,8 @@ int fasa_fused_plan(fasa_ctx* ctx) {
       continue;
     }
     // the select-only forms of the kernel run with the same cluster shape
-    if (cudaFuncSetAttribute((const void*)topk_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-        cudaFuncSetAttribute((const void*)select_fn(ctx->chunks), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+    if (cudaFuncSetAttribute((const void*)topk_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit) != cudaSuccess ||
+        cudaFuncSetAttribute((const void*)select_fn(ctx->chunks), cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit) != cudaSuccess ||
         (cs > 8 && (cudaFuncSetAttribute((const void*)topk_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
                     cudaFuncSetAttribute((const void*)select_fn(ctx->chunks), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess))) {
       cudaGetLastError();

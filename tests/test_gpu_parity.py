@@ -569,3 +569,18 @@ def test_config3_full_size_sampled_units_with_append():
     # large, so the step is the cluster kernel without attention + the split-K tensor-core kernel
     w = C["c3"].replace(len_lo=16384, len_hi=16384)
     _full_size_sampled(w, [(0, 0), (31, 3), (13, 2)], append=True)
+
+
+def test_contexts_of_different_sizes_coexist():
+    # a large context, then a small one, then the large one again: per-kernel launch limits are
+    # process-wide and must cover every live context
+    big = Run(C["c4"].replace(batch=1, n_q_heads=8, n_kv_heads=2, max_len=30000, len_lo=30000, len_hi=30000, budget=64))
+    small = Run(C["c1"].replace(n_q_heads=8, n_kv_heads=2, max_len=600, len_lo=600, len_hi=600, budget=32))
+    for r in (big, small, big):
+        r.build_proxy()
+        r.reset_outputs()
+        r.step(fused=True)
+        h = r.host()
+        parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], idx=h["idx"], n_sel=h["n_sel"], out=h["out"],
+                          what=r.w.name, **r.oracle_kwargs())
+        assert r.fasa.device_status() == 0
