@@ -18,7 +18,10 @@
  *   (2i, 2i+1, the paper's literal Eq. 1).  With grouped-query attention the
  *   score of a KV head is the sum (or max) over its query heads of the raw
  *   partial logits.  Ties rank the lower index first.  Sink / recent positions
- *   are kept in addition to the budget.
+ *   are kept in addition to the budget.  The paper keeps one index set per
+ *   (layer, head) (Sec. 4.1); how many query heads share a set is a parameter
+ *   here: all heads of a KV head (the default, one gathered set per K/V head),
+ *   one (the per-head reading), or any divisor of the group in between.
  *
  * Pins (tests/test_oracle_*.py): sum over all FCs of alpha^(i) equals q.k;
  * the relative-position identity; F = d/2 reproduces the dense top-k; budget >=
@@ -216,35 +219,46 @@ void fasa_oracle_attn_dense(const double* q, int G, const double* K, const doubl
 
 /* ------------------------------------------------- whole step on bf16 bits */
 
-/* One decode step over a batch, the steps in the paper's order per (b, KV head):
- * widen the bf16 bits -> TIP score -> TopK-I (+ forced) -> FAC, and optionally
- * the dense FKV output.  Layouts (row-major, the same bits the GPU path reads):
+/* One decode step over a batch, the steps in the paper's order per selection
+ * unit: widen the bf16 bits -> TIP score -> TopK-I (+ forced) -> FAC, and
+ * optionally the dense FKV output.  A selection unit is sel_heads consecutive
+ * query heads that share one index set (sel_heads = 0 means the whole group
+ * Hq / Hkv; it must divide the group); unit hs of a sequence covers query heads
+ * hs * sel_heads .. and reads the cache of KV head (hs * sel_heads) / (Hq / Hkv).
+ * With Hs = Hq / sel_heads units per sequence, layouts (row-major, the same bits
+ * the GPU path reads):
  *   q_bits  [B][Hq][d]           K_bits, V_bits  [B][Hkv][Lmax][d]
  *   seq_lens[B]                  dom [Hkv][F]
- * Outputs (any may be NULL): scores [B][Hkv][Lmax] (rows >= L untouched),
- *   idx [B][Hkv][n_sel_max] ascending, n_sel [B][Hkv], band [B][Hkv][4],
+ * Outputs (any may be NULL): scores [B][Hs][Lmax] (rows >= L untouched),
+ *   idx [B][Hs][n_sel_max] ascending, n_sel [B][Hs], band [B][Hs][4],
  *   out [B][Hq][d], lse [B][Hq], dense_out [B][Hq][d], dense_lse [B][Hq].
  * budget > 0 is absolute; budget < 0 means ceil(-budget/1000 * L) in integers.
  * Units are independent; with OpenMP they are spread over n_threads threads.
- * Returns the number of threads used. */
+ * Returns the number of threads used, or -1 for a sel_heads that does not divide
+ * the group. */
 int fasa_oracle_decode_bf16(const uint16_t* q_bits, const uint16_t* K_bits,
                             const uint16_t* V_bits, const int32_t* seq_lens,
                             const int32_t* dom, int B, int Hq, int Hkv, int d, int Lmax,
                             int F, int pairing, int group_reduce, int n_sink, int n_recent,
                             int budget, int n_sel_max, double scale, double tie_rel,
-                            int n_threads, double* scores, int32_t* idx, int32_t* n_sel,
-                            double* band, double* out, double* lse, double* dense_out,
-                            double* dense_lse) {
-  int G = Hq / Hkv;
+                            int n_threads, int sel_heads, double* scores, int32_t* idx,
+                            int32_t* n_sel, double* band, double* out, double* lse,
+                            double* dense_out, double* dense_lse) {
+  int group = Hq / Hkv;
+  int G = sel_heads > 0 ? sel_heads : group;   /* query heads per selection unit */
+  if (group % G != 0) return -1;
+  int Hs = Hq / G;
   int used = 1;
 #ifdef _OPENMP
   if (n_threads > 0) omp_set_num_threads(n_threads);
   used = n_threads > 0 ? n_threads : omp_get_max_threads();
-  if (used > B * Hkv) used = B * Hkv;
+  if (used > B * Hs) used = B * Hs;
 #pragma omp parallel for schedule(dynamic, 1)
 #endif
-  for (int u = 0; u < B * Hkv; ++u) {
-    int b = u / Hkv, h = u % Hkv;
+  for (int u = 0; u < B * Hs; ++u) {
+    int b = u / Hs, hs = u % Hs;
+    int q0 = hs * G;          /* first query head of the unit */
+    int h = q0 / group;       /* the KV head it attends */
     int L = seq_lens[b];
     if (L > Lmax) L = Lmax;
     if (L < 0) L = 0;
@@ -258,7 +272,7 @@ int fasa_oracle_decode_bf16(const uint16_t* q_bits, const uint16_t* K_bits,
     const uint16_t* Vb = V_bits + ((int64_t)b * Hkv + h) * (int64_t)Lmax * d;
     fasa_oracle_widen_bf16(Kb, (int64_t)L * d, Kd);
     fasa_oracle_widen_bf16(Vb, (int64_t)L * d, Vd);
-    fasa_oracle_widen_bf16(q_bits + ((int64_t)b * Hq + (int64_t)h * G) * d, (int64_t)G * d, qd);
+    fasa_oracle_widen_bf16(q_bits + ((int64_t)b * Hq + q0) * d, (int64_t)G * d, qd);
 
     fasa_oracle_fc_score(qd, G, Kd, L, d, pairing, dom + (int64_t)h * F, F, group_reduce, S);
     if (scores) memcpy(scores + (int64_t)u * Lmax, S, sizeof(double) * (size_t)L);
@@ -275,12 +289,12 @@ int fasa_oracle_decode_bf16(const uint16_t* q_bits, const uint16_t* K_bits,
     }
     if (out)
       fasa_oracle_attn_subset(qd, G, Kd, Vd, d, sel, n, scale,
-                              out + ((int64_t)b * Hq + (int64_t)h * G) * d,
-                              lse ? lse + (int64_t)b * Hq + (int64_t)h * G : NULL);
+                              out + ((int64_t)b * Hq + q0) * d,
+                              lse ? lse + (int64_t)b * Hq + q0 : NULL);
     if (dense_out)
       fasa_oracle_attn_dense(qd, G, Kd, Vd, d, L, scale,
-                             dense_out + ((int64_t)b * Hq + (int64_t)h * G) * d,
-                             dense_lse ? dense_lse + (int64_t)b * Hq + (int64_t)h * G : NULL);
+                             dense_out + ((int64_t)b * Hq + q0) * d,
+                             dense_lse ? dense_lse + (int64_t)b * Hq + q0 : NULL);
     free(Kd); free(Vd); free(qd); free(S); free(sel);
   }
   return used;

@@ -160,10 +160,13 @@ def attn_dense(q, K, V, L: int, scale: float):
 
 def decode_bf16(q_bits, K_bits, V_bits, seq_lens, dom, *, pairing=0, group_reduce=0, n_sink=0,
                 n_recent=0, budget=256, n_sel_max=None, scale=None, tie_rel=1e-3, n_threads=0,
-                want_scores=True, want_sparse=True, want_dense=True):
+                sel_heads=0, want_scores=True, want_sparse=True, want_dense=True):
     """One whole decode step on bf16 bit patterns, unit by unit in the paper's order.
 
     q_bits [B,Hq,d], K_bits/V_bits [B,Hkv,Lmax,d] (uint16), seq_lens [B], dom [Hkv,F].
+    sel_heads query heads share one index set (0 = all heads of a KV head, 1 = one set per
+    query head, the per-head reading of Sec. 4.1); scores, idx, n_sel and band then have
+    Hs = Hq / sel_heads rows per sequence instead of Hkv.
     Returns a dict with scores, idx, n_sel, band, out, lse, dense_out, dense_lse, threads.
     """
     q_bits = np.ascontiguousarray(q_bits, dtype=np.uint16)
@@ -178,11 +181,15 @@ def decode_bf16(q_bits, K_bits, V_bits, seq_lens, dom, *, pairing=0, group_reduc
         scale = 1.0 / np.sqrt(float(d))
     if n_sel_max is None:
         n_sel_max = Lmax
-    U = B * Hkv
-    scores = np.full((B, Hkv, Lmax), np.nan, dtype=np.float64) if want_scores else None
-    idx = np.full((B, Hkv, n_sel_max), -1, dtype=np.int32)
-    n_sel = np.zeros((B, Hkv), dtype=np.int32)
-    band = np.zeros((B, Hkv, 4), dtype=np.float64)
+    group = Hq // Hkv
+    per = sel_heads if sel_heads > 0 else group
+    if per <= 0 or group % per != 0:
+        raise ValueError("sel_heads must divide the group")
+    Hs = Hq // per
+    scores = np.full((B, Hs, Lmax), np.nan, dtype=np.float64) if want_scores else None
+    idx = np.full((B, Hs, n_sel_max), -1, dtype=np.int32)
+    n_sel = np.zeros((B, Hs), dtype=np.int32)
+    band = np.zeros((B, Hs, 4), dtype=np.float64)
     out = np.zeros((B, Hq, d), dtype=np.float64) if want_sparse else None
     lse = np.zeros((B, Hq), dtype=np.float64) if want_sparse else None
     dout = np.zeros((B, Hq, d), dtype=np.float64) if want_dense else None
@@ -193,8 +200,9 @@ def decode_bf16(q_bits, K_bits, V_bits, seq_lens, dom, *, pairing=0, group_reduc
         ctypes.c_int(Lmax), ctypes.c_int(F), ctypes.c_int(pairing), ctypes.c_int(group_reduce),
         ctypes.c_int(n_sink), ctypes.c_int(n_recent), ctypes.c_int(budget),
         ctypes.c_int(n_sel_max), ctypes.c_double(scale), ctypes.c_double(tie_rel),
-        ctypes.c_int(n_threads), _ptr(scores, _f64p), _ptr(idx, _i32p), _ptr(n_sel, _i32p),
+        ctypes.c_int(n_threads), ctypes.c_int(sel_heads), _ptr(scores, _f64p), _ptr(idx, _i32p), _ptr(n_sel, _i32p),
         _ptr(band, _f64p), _ptr(out, _f64p), _ptr(lse, _f64p), _ptr(dout, _f64p), _ptr(dlse, _f64p))
-    assert U >= 0
+    if used < 0:
+        raise ValueError("sel_heads must divide the group")
     return {"scores": scores, "idx": idx, "n_sel": n_sel, "band": band, "out": out, "lse": lse,
             "dense_out": dout, "dense_lse": dlse, "threads": int(used)}

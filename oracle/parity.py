@@ -68,36 +68,40 @@ def check_attention(out_gpu, out_or, what="", tol=ATTN_ABS):
 
 
 def check_step(q, k, v, seq_lens, dom, *, pairing, group_reduce, n_sink, n_recent, budget, scale,
-               scores=None, idx=None, n_sel=None, out=None, dense_out=None, units=None, what=""):
+               scores=None, idx=None, n_sel=None, out=None, dense_out=None, units=None, sel_heads=0, what=""):
     """Checks whatever parts of one decode step are given (numpy arrays in the library's
     layouts; q/k/v as float64 widenings of the bf16 inputs) against the oracle, unit by unit.
-    `units` limits the check to some (b, h) pairs.  Returns a small report dict."""
+    A unit is (b, hs): sel_heads query heads sharing one index set (0 = all heads of a KV
+    head).  `units` limits the check to some (b, hs) pairs.  Returns a small report dict."""
     B, Hq, d = q.shape
     Hkv = k.shape[1]
-    G = Hq // Hkv
+    group = Hq // Hkv
+    G = sel_heads if sel_heads > 0 else group
+    Hs = Hq // G
     rep = {"units": 0, "sets_identical": 0, "attn_err": 0.0, "dense_err": 0.0}
-    todo = units if units is not None else [(b, h) for b in range(B) for h in range(Hkv)]
-    for (b, h) in todo:
+    todo = units if units is not None else [(b, hs) for b in range(B) for hs in range(Hs)]
+    for (b, hs) in todo:
+        h = hs * G // group                      # the KV head this unit attends
         L = int(min(max(int(seq_lens[b]), 0), k.shape[2]))
-        tag = f"{what}[b={b},h={h},L={L}]"
-        qs, ks, vs = q[b, h * G:(h + 1) * G], k[b, h, :L], v[b, h, :L]
+        tag = f"{what}[b={b},unit={hs},kv={h},L={L}]"
+        qs, ks, vs = q[b, hs * G:(hs + 1) * G], k[b, h, :L], v[b, h, :L]
         s_or = O.fc_score(qs, ks, dom[h], pairing, group_reduce) if L > 0 else np.zeros(0)
         kk = budget if budget > 0 else (-budget * L + 999) // 1000
         rep["units"] += 1
         if scores is not None and L > 0:
             bound = score_bound(qs, ks, dominant_channels(dom[h], pairing, d))
-            check_scores(scores[b, h, :L], s_or, bound, tag)
+            check_scores(scores[b, hs, :L], s_or, bound, tag)
         sel = None
         if idx is not None:
-            n = int(n_sel[b, h])
-            sel = np.asarray(idx[b, h, :n])
+            n = int(n_sel[b, hs])
+            sel = np.asarray(idx[b, hs, :n])
             rep["sets_identical"] += bool(check_selection(sel, s_or, L, kk, n_sink, n_recent, tag))
         if out is not None:
             if sel is None:
                 sel, _ = O.select(s_or, kk, n_sink, n_recent, TIE_REL)
             o_or, _ = O.attn_subset(qs, ks, vs, sel, scale)
-            rep["attn_err"] = max(rep["attn_err"], check_attention(out[b, h * G:(h + 1) * G], o_or, tag + " sparse"))
+            rep["attn_err"] = max(rep["attn_err"], check_attention(out[b, hs * G:(hs + 1) * G], o_or, tag + " sparse"))
         if dense_out is not None:
             o_or, _ = O.attn_dense(qs, ks, vs, L, scale)
-            rep["dense_err"] = max(rep["dense_err"], check_attention(dense_out[b, h * G:(h + 1) * G], o_or, tag + " dense"))
+            rep["dense_err"] = max(rep["dense_err"], check_attention(dense_out[b, hs * G:(hs + 1) * G], o_or, tag + " dense"))
     return rep

@@ -53,10 +53,20 @@ class Workload:
     rope: bool = True
     dom_bias: bool = True      # weight (i+1)^2 when True, uniform otherwise
     group_reduce: int = 0
+    sel_heads: int = 0         # query heads sharing one index set; 0 = all heads of a KV head
 
     @property
     def group(self) -> int:
         return self.n_q_heads // self.n_kv_heads
+
+    @property
+    def heads_per_set(self) -> int:
+        return self.sel_heads if self.sel_heads > 0 else self.group
+
+    @property
+    def n_sets(self) -> int:
+        """Index sets (selection units) per sequence."""
+        return self.n_q_heads // self.heads_per_set
 
     def replace(self, **kw) -> "Workload":
         return dataclasses.replace(self, **kw)

@@ -280,7 +280,8 @@ def test_lse_merge_identity():
 # ----------------------------------------------------------- whole step ----
 
 def _small_workload(**kw):
-    w = synth.CONFIGS["c1"].replace(batch=2, max_len=600, len_lo=300, len_hi=600, budget=40, **kw)
+    kw.setdefault("budget", 40)
+    w = synth.CONFIGS["c1"].replace(batch=2, max_len=600, len_lo=300, len_hi=600, **kw)
     return w, synth.make_inputs(w, "cpu")
 
 
@@ -338,6 +339,64 @@ def test_budget_covering_context_reproduces_dense():
     for b in range(w.batch):
         L = int(t["seq_lens"][b])
         assert int(r2["n_sel"][b, 0]) == math.ceil(189 * L / 1000)
+
+
+# --------------------------------------------- index sets per query head ----
+
+def _decode(w, t, **kw):
+    return O.decode_bf16(synth.bf16_bits(t["q"]), synth.bf16_bits(t["k"]), synth.bf16_bits(t["v"]),
+                         t["seq_lens"].numpy(), t["dom"].numpy(), n_sink=w.n_sink, n_recent=w.n_recent,
+                         budget=w.budget, **kw)
+
+
+@pytest.mark.parametrize("sel_heads", [1, 2])
+def test_sets_per_query_head_equal_the_model_with_repeated_kv_heads(sel_heads):
+    # Sec. 4.1 keeps one index set per head.  Sets shared by sel_heads query heads of a
+    # grouped-query model must be what the default path (one set per KV head, pinned above)
+    # gives on the same model with every K/V head repeated once per set: this fixes which
+    # cache a unit reads, which query heads it covers and where its rows land.
+    w, t = _small_workload()
+    rep = w.group // sel_heads
+    r = _decode(w, t, sel_heads=sel_heads)
+    x = O.decode_bf16(synth.bf16_bits(t["q"]), np.repeat(synth.bf16_bits(t["k"]), rep, axis=1),
+                      np.repeat(synth.bf16_bits(t["v"]), rep, axis=1), t["seq_lens"].numpy(),
+                      np.repeat(t["dom"].numpy(), rep, axis=0), n_sink=w.n_sink, n_recent=w.n_recent,
+                      budget=w.budget)
+    assert r["idx"].shape == (w.batch, w.n_q_heads // sel_heads, w.max_len)
+    for key in ("scores", "idx", "n_sel", "band", "out", "lse", "dense_out", "dense_lse"):
+        assert np.array_equal(r[key], x[key], equal_nan=True), key
+    # the dense output does not depend on how sets are shared; the sparse one does
+    d = _decode(w, t)
+    assert np.array_equal(r["dense_out"], d["dense_out"])
+    assert not np.array_equal(r["out"], d["out"])
+
+
+def test_sets_per_query_head_all_fcs_reproduce_each_heads_dense_topk():
+    w, t = _small_workload(n_dom=64, n_sink=0, n_recent=0)
+    r = _decode(w, t, sel_heads=1, want_dense=False)
+    G = w.group
+    for b in range(w.batch):
+        L = int(t["seq_lens"][b])
+        for g in range(w.n_q_heads):
+            full = t["k"][b, g // G, :L].double() @ t["q"][b, g].double()
+            ref = torch.topk(full, w.budget).indices.sort().values.numpy()
+            assert np.array_equal(r["idx"][b, g, :w.budget], ref)
+            p = torch.softmax(full[ref] / math.sqrt(128), 0)
+            assert np.allclose(r["out"][b, g], (p[:, None] * t["v"][b, g // G, ref].double()).sum(0).numpy(), atol=1e-12)
+
+
+def test_sets_per_query_head_budget_covering_context_reproduces_dense():
+    w, t = _small_workload(budget=600)
+    r = _decode(w, t, sel_heads=1)
+    assert np.array_equal(r["n_sel"], np.repeat(t["seq_lens"].numpy()[:, None], w.n_q_heads, 1))
+    assert np.allclose(r["out"], r["dense_out"], atol=1e-14)
+
+
+def test_set_sharing_must_divide_the_group():
+    w, t = _small_workload()
+    with pytest.raises(ValueError):
+        _decode(w, t, sel_heads=3)
+    assert np.array_equal(_decode(w, t, sel_heads=w.group)["idx"], _decode(w, t)["idx"])
 
 
 def test_byte_model_fraction():
