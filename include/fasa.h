@@ -2,7 +2,8 @@
  * fasa.h - C ABI of the B200 (sm_100a) decode-time hot path of FASA,
  * Frequency-Aware Sparse Attention (arxiv 2602.03152).
  *
- * One decode step per (batch b, KV head h), in the paper's order:
+ * One decode step per (batch b, KV head h) - or per smaller set of query heads, see
+ * "Index sets" below - in the paper's order:
  *   fasa_kv_append          cache update, incl. the dominant part of the key cache
  *                           (C_key^dom of Algorithm 2, kept here as a packed
  *                           "proxy-K" side buffer)
@@ -36,6 +37,15 @@
  *     P[g+8][2t+8..2t+9]}; a trailing block of 8 channels, 256 bytes, when
  *     ceil(n_dom / 4) is odd).  Only fasa_kv_append, fasa_proxy_build and
  *     fasa_append_decode_step write it; treat it as opaque.
+ *   - Index sets.  The paper keeps one index set T_t per (layer, head) (Sec. 4.1).  With
+ *     grouped-query attention the default here is one set per KV head, scored by all its
+ *     query heads together, so that each selected K/V row is gathered once per KV head.
+ *     select_heads = s makes every s consecutive query heads share a set instead (s = 1:
+ *     a set per query head, the paper's literal reading; s must divide n_q_heads /
+ *     n_kv_heads).  With n_sets = n_q_heads / s sets per sequence, set hs covers query
+ *     heads hs*s .. hs*s+s-1 and reads the cache of their KV head; scores, idx and n_sel
+ *     have n_sets rows per sequence wherever the text below says n_kv_heads (I_dom, K, V
+ *     and the proxy stay per KV head).  Gathered K/V traffic grows by the group size / s.
  *   - Data-dependent problems (a sequence longer than max_len, an index out of
  *     range) never fault: the kernel clamps and ORs a bit into a device status
  *     word read by fasa_get_device_status.
@@ -70,7 +80,9 @@ typedef struct {
   int32_t max_len;        /* rows allocated per (b, kv head) in K, V, proxy and scores     */
   int32_t n_dom;          /* F = N_tip: dominant FCs per KV head, 1..64                    */
   int32_t rope_pairing;   /* 0: FC i = (i, i+64); 1: FC i = (2i, 2i+1)                     */
-  int32_t group_reduce;   /* score of a KV head over its query heads: 0 sum, 1 max         */
+  int32_t group_reduce;   /* score of an index set over its query heads: 0 sum, 1 max      */
+  int32_t select_heads;   /* query heads that share one index set: 0 => all heads of a KV  */
+                          /* head; 1 => a set per query head; else a divisor of the group  */
   int32_t n_sink;         /* first n_sink positions are always selected                    */
   int32_t n_recent;       /* last n_recent positions are always selected                   */
   float   softmax_scale;  /* 0 => 1/sqrt(head_dim)                                         */

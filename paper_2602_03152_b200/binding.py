@@ -40,7 +40,7 @@ class FasaConfig(ctypes.Structure):
     _fields_ = [
         ("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
         ("head_dim", ctypes.c_int32), ("max_len", ctypes.c_int32), ("n_dom", ctypes.c_int32),
-        ("rope_pairing", ctypes.c_int32), ("group_reduce", ctypes.c_int32),
+        ("rope_pairing", ctypes.c_int32), ("group_reduce", ctypes.c_int32), ("select_heads", ctypes.c_int32),
         ("n_sink", ctypes.c_int32), ("n_recent", ctypes.c_int32), ("softmax_scale", ctypes.c_float),
         ("k_stride_b", ctypes.c_int64), ("k_stride_h", ctypes.c_int64), ("k_stride_t", ctypes.c_int64),
         ("v_stride_b", ctypes.c_int64), ("v_stride_h", ctypes.c_int64), ("v_stride_t", ctypes.c_int64),
@@ -118,13 +118,13 @@ class Fasa:
 
     def __init__(self, batch, n_q_heads, n_kv_heads, max_len, dom, *, head_dim=128, rope_pairing=0,
                  group_reduce=0, n_sink=0, n_recent=0, softmax_scale=0.0, k_strides=(0, 0, 0),
-                 v_strides=(0, 0, 0)):
+                 v_strides=(0, 0, 0), select_heads=0):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         dom = torch.as_tensor(dom, dtype=torch.int32).contiguous().cpu()
         n_dom = dom.shape[-1] if dom.dim() == 2 else 0
         self.cfg = FasaConfig(batch, n_q_heads, n_kv_heads, head_dim, max_len, n_dom, rope_pairing,
-                              group_reduce, n_sink, n_recent, softmax_scale, *k_strides, *v_strides)
+                              group_reduce, select_heads, n_sink, n_recent, softmax_scale, *k_strides, *v_strides)
         if dom.dim() != 2 or dom.shape[0] != n_kv_heads:
             raise FasaError(ERR_INVALID_ARG, "fasa_create", "dom must be [n_kv_heads, n_dom]")
         st = self._lib.fasa_create(ctypes.byref(self.cfg), dom.data_ptr(), ctypes.byref(self._h))
@@ -133,12 +133,15 @@ class Fasa:
             raise FasaError(st, "fasa_create", self._lib.fasa_status_string(st).decode())
         self.batch, self.n_q_heads, self.n_kv_heads, self.max_len = batch, n_q_heads, n_kv_heads, max_len
         self.n_dom = n_dom
+        group = n_q_heads // n_kv_heads
+        self.select_heads = select_heads if select_heads > 0 else group    # query heads per index set
+        self.n_sets = n_q_heads // self.select_heads                       # rows of scores / idx / n_sel per sequence
         self.row_elems = proxy_row_elems(n_dom)
 
     @classmethod
     def from_workload(cls, w, dom) -> "Fasa":
         return cls(w.batch, w.n_q_heads, w.n_kv_heads, w.max_len, dom, rope_pairing=w.pairing,
-                   group_reduce=w.group_reduce, n_sink=w.n_sink, n_recent=w.n_recent)
+                   group_reduce=w.group_reduce, n_sink=w.n_sink, n_recent=w.n_recent, select_heads=w.sel_heads)
 
     def close(self):
         if getattr(self, "_h", None) is not None and self._h.value:

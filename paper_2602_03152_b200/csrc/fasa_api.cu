@@ -19,7 +19,11 @@ bool valid_cfg(const fasa_config_t& c, int32_t* why) {
   if (c.n_q_heads / c.n_kv_heads > FASA_MAX_GROUP) return false;
   if (c.rope_pairing != 0 && c.rope_pairing != 1) return false;
   if (c.group_reduce != 0 && c.group_reduce != 1) return false;
-  if ((long long)c.batch * c.n_kv_heads > 65535) return false;  // grid.y
+  if (c.select_heads < 0) return false;
+  const int group = c.n_q_heads / c.n_kv_heads;
+  const int per_set = c.select_heads > 0 ? c.select_heads : group;
+  if (group % per_set != 0) return false;
+  if ((long long)c.batch * (c.n_q_heads / per_set) > 65535) return false;  // grid.y
   return true;
 }
 
@@ -68,6 +72,8 @@ extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_h
   }
   if (c.softmax_scale == 0.f) c.softmax_scale = 0.08838834764831845f;  // 1/sqrt(128)
   ctx->group = c.n_q_heads / c.n_kv_heads;
+  ctx->sel_heads = c.select_heads > 0 ? c.select_heads : ctx->group;
+  ctx->n_sets = c.n_q_heads / ctx->sel_heads;
   ctx->chunks = (c.n_dom + 3) / 4;
   ctx->row_elems = 8 * ctx->chunks;
 
@@ -165,16 +171,15 @@ extern "C" int32_t fasa_get_device_status(fasa_ctx_t* ctx, void* stream, int32_t
 }
 
 // Splits: enough CTAs to fill the GPU a few times over, between 64 and 2048 rows each.
-static int split_count_bound(const fasa_ctx* ctx, int n_upper) {
-  const int units = ctx->cfg.batch * ctx->cfg.n_kv_heads;
+static int split_count_bound(const fasa_ctx* ctx, int n_upper, int units) {
   const int target = 4 * (ctx->n_sm > 0 ? ctx->n_sm : 148);
   const int want = std::max((target + units - 1) / units, (n_upper + 2047) / 2048);
   const int most = (n_upper + 63) / 64;
-  return std::max(1, std::min(want, most));   // non-decreasing in n_upper
+  return std::max(1, std::min(want, most));   // non-decreasing in n_upper, non-increasing in units
 }
 
-fasa_split_plan fasa_plan_splits(const fasa_ctx* ctx, int n_upper) {
-  const int n = split_count_bound(ctx, n_upper);
+fasa_split_plan fasa_plan_splits(const fasa_ctx* ctx, int n_upper, int units) {
+  const int n = split_count_bound(ctx, n_upper, units);
   int chunk = (n_upper + n - 1) / n;
   chunk = (chunk + 31) / 32 * 32;
   fasa_split_plan p;
@@ -184,10 +189,11 @@ fasa_split_plan fasa_plan_splits(const fasa_ctx* ctx, int n_upper) {
 }
 
 // The partial-result area is sized for the largest split count any call can use
-// (the bound at max_len), so it does not depend on the selection size.
+// (the bound at max_len for the fewest units a launch can have, one per KV head), so it does
+// not depend on the selection size.
 extern "C" int32_t fasa_workspace_bytes(const fasa_ctx_t* ctx, int32_t n_sel_max, size_t* out_bytes) {
   if (!ctx || !out_bytes || n_sel_max < 0) return FASA_ERR_INVALID_ARG;
-  const int n = split_count_bound(ctx, ctx->cfg.max_len);
+  const int n = split_count_bound(ctx, ctx->cfg.max_len, ctx->cfg.batch * ctx->cfg.n_kv_heads);
   size_t per_split = (size_t)ctx->cfg.batch * ctx->cfg.n_q_heads * (FASA_HEAD_DIM + 2) * sizeof(float);
   *out_bytes = fasa_align_up(per_split * (size_t)n, 256) + 256;
   return FASA_OK;

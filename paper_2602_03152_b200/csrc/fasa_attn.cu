@@ -33,7 +33,7 @@ struct AttnParams {
   const int32_t* n_rows;   // sparse: n_sel [units]; dense: seq_lens [batch]
   float* partial;          // [batch][n_q_heads][n_splits][kPartialStride]
   int32_t* status;
-  int n_q_heads, n_kv_heads, group, max_len, n_sel_max, n_cap, chunk, n_splits;
+  int n_q_heads, n_kv_heads, n_sets, group, max_len, n_sel_max, n_cap, chunk, n_splits;   // a unit = `group` query heads; n_sets units per sequence
   int64_t ksb, ksh, kst, vsb, vsh, vst;
   float scale_log2;        // softmax_scale * log2(e)
 };
@@ -43,8 +43,9 @@ template <int GP, int HWS, bool SPARSE>
 __global__ void __launch_bounds__(kAttnThreads)
 decode_attn_kernel(const AttnParams p) {
   const int u = blockIdx.y;
-  const int h = u % p.n_kv_heads;
-  const int b = u / p.n_kv_heads;
+  const SelUnit su = sel_unit(u, p.n_sets, p.group, p.n_q_heads, p.n_kv_heads);
+  const int h = su.h;
+  const int b = su.b;
   int n;
   if (SPARSE) {
     n = p.n_rows[u];
@@ -80,7 +81,7 @@ decode_attn_kernel(const AttnParams p) {
   for (int g = 0; g < GP; ++g) {
     const bool head_ok = g0 + g < p.group;
     const uint16_t* qp =
-        p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group + (head_ok ? g0 + g : 0)) * FASA_HEAD_DIM + l16 * 8;
+        p.q + (su.q0 + (head_ok ? g0 + g : 0)) * FASA_HEAD_DIM + l16 * 8;
     uint4 w = *reinterpret_cast<const uint4*>(qp);
     const float sc = head_ok ? p.scale_log2 : 0.f;
     float2 t;
@@ -248,7 +249,7 @@ decode_attn_kernel(const AttnParams p) {
       l += w * s_l[hwi][gi];
     }
     float* dst = p.partial +
-                 (((int64_t)b * p.n_q_heads + (int64_t)h * p.group + gl) * p.n_splits + split) * kPartialStride;
+                 ((su.q0 + gl) * p.n_splits + split) * kPartialStride;
     dst[2 + c] = a;
     if (c == 0) {
       dst[0] = mx;
@@ -342,8 +343,9 @@ decode_attn_mma_kernel(const AttnParams p) {
   pdl_wait_for_predecessor();
   pdl_release_successor();
   const int u = blockIdx.y;
-  const int h = u % p.n_kv_heads;
-  const int b = u / p.n_kv_heads;
+  const SelUnit su = sel_unit(u, p.n_sets, p.group, p.n_q_heads, p.n_kv_heads);
+  const int h = su.h;
+  const int b = su.b;
   int n;
   if (SPARSE) {
     n = p.n_rows[u];
@@ -369,7 +371,7 @@ decode_attn_mma_kernel(const AttnParams p) {
   // B operand of the logits: q[head g][channels], bf16 as stored, for the 8 blocks of 16 channels
   uint32_t qb[8][2];
   {
-    const uint16_t* qh = p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group + (g < p.group ? g : 0)) * FASA_HEAD_DIM;
+    const uint16_t* qh = p.q + (su.q0 + (g < p.group ? g : 0)) * FASA_HEAD_DIM;
 #pragma unroll
     for (int kb = 0; kb < 8; ++kb) {
       const uint32_t w0 = *reinterpret_cast<const uint32_t*>(qh + kb * 16 + 2 * t);
@@ -506,7 +508,7 @@ decode_attn_mma_kernel(const AttnParams p) {
       l += wt * s_ml[(w * 8 + gl) * 2 + 1];
     }
     float* dst = p.partial +
-                 (((int64_t)b * p.n_q_heads + (int64_t)h * p.group + gl) * p.n_splits + split) * kPartialStride;
+                 ((su.q0 + gl) * p.n_splits + split) * kPartialStride;
     dst[2 + cch] = a;
     if (cch == 0) {
       dst[0] = mx;
@@ -523,7 +525,7 @@ template <bool SPARSE>
 __global__ void __launch_bounds__(FASA_HEAD_DIM * kMergeWays)
 decode_attn_merge_kernel(const float* __restrict__ partial, const int32_t* __restrict__ n_rows,
                          float* __restrict__ out, float* __restrict__ lse,
-                         int32_t* __restrict__ status, int n_q_heads, int n_kv_heads, int group,
+                         int32_t* __restrict__ status, int n_q_heads, int n_sets, int group,
                          int max_len, int n_cap, int chunk, int n_splits) {
   pdl_wait_for_predecessor();
   const int bh = blockIdx.x;
@@ -531,7 +533,7 @@ decode_attn_merge_kernel(const float* __restrict__ partial, const int32_t* __res
   const int hq = bh % n_q_heads;
   int n;
   if (SPARSE) {
-    n = n_rows[b * n_kv_heads + hq / group];
+    n = n_rows[b * n_sets + hq / group];
     n = n < 0 ? 0 : (n > n_cap ? n_cap : n);
   } else {
     n = n_rows[b];
@@ -579,17 +581,19 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
                     const int32_t* idx, const int32_t* n_rows, int n_upper, int n_sel_max,
                     float* out, float* lse, void* workspace, cudaStream_t s) {
   const fasa_config_t& c = ctx->cfg;
-  const fasa_split_plan plan = fasa_plan_splits(ctx, n_upper);
+  // the dense pass treats a KV head with all its query heads as the unit
+  const int n_sets = SPARSE ? ctx->n_sets : c.n_kv_heads;
+  const int G = SPARSE ? ctx->sel_heads : ctx->group;
+  const fasa_split_plan plan = fasa_plan_splits(ctx, n_upper, c.batch * n_sets);
   AttnParams p;
   p.q = (const uint16_t*)q; p.k = (const uint16_t*)k; p.v = (const uint16_t*)v;
   p.idx = idx; p.n_rows = n_rows; p.partial = (float*)workspace; p.status = ctx->d_status;
-  p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group;
+  p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.n_sets = n_sets; p.group = G;
   p.max_len = c.max_len; p.n_sel_max = n_sel_max; p.n_cap = n_upper; p.chunk = plan.chunk; p.n_splits = plan.n_splits;
   p.ksb = c.k_stride_b; p.ksh = c.k_stride_h; p.kst = c.k_stride_t;
   p.vsb = c.v_stride_b; p.vsh = c.v_stride_h; p.vst = c.v_stride_t;
   p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
-  dim3 grid((unsigned)plan.n_splits, (unsigned)(c.batch * c.n_kv_heads));
-  const int G = ctx->group;
+  dim3 grid((unsigned)plan.n_splits, (unsigned)(c.batch * n_sets));
   if (ctx->use_fused) {   // default: the tensor-core kernel (mode 0 keeps the scalar one)
     static_assert(sizeof(MmaSmem) >= (size_t)kMmaWarps * 8 * (FASA_HEAD_DIM + 2) * sizeof(float), "combine area");
     auto fn = decode_attn_mma_kernel<SPARSE>;
@@ -604,8 +608,8 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   FASA_LAUNCH_CHECK(ctx);
   FASA_CUDA_TRY(ctx, launch_after_predecessor(
       decode_attn_merge_kernel<SPARSE>, dim3((unsigned)(c.batch * c.n_q_heads)), dim3(FASA_HEAD_DIM * kMergeWays),
-      (size_t)0, s, (const float*)workspace, n_rows, out, lse, ctx->d_status, (int)c.n_q_heads, (int)c.n_kv_heads,
-      (int)ctx->group, (int)c.max_len, (int)n_upper, (int)plan.chunk, (int)plan.n_splits));
+      (size_t)0, s, (const float*)workspace, n_rows, out, lse, ctx->d_status, (int)c.n_q_heads, (int)n_sets,
+      (int)G, (int)c.max_len, (int)n_upper, (int)plan.chunk, (int)plan.n_splits));
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
 }
@@ -656,7 +660,7 @@ extern "C" int32_t fasa_sparse_decode_attn_static(fasa_ctx_t* ctx, const void* q
   if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16)) return FASA_ERR_INVALID_ARG;
   const fasa_config_t& c = ctx->cfg;
   const int n_upper = n_sel_max < c.max_len ? n_sel_max : c.max_len;
-  const fasa_split_plan plan = fasa_plan_splits(ctx, n_upper);
+  const fasa_split_plan plan = fasa_plan_splits(ctx, n_upper, c.batch * ctx->n_sets);
   const size_t need = (size_t)c.batch * c.n_q_heads * (size_t)plan.n_splits * kPartialStride * sizeof(float);
   if (need > kStaticScratchBytes) return FASA_ERR_WORKSPACE;
 

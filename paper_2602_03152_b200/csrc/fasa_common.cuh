@@ -16,6 +16,8 @@
 struct fasa_ctx {
   fasa_config_t cfg;      // strides and softmax_scale filled in
   int group;              // query heads per KV head
+  int sel_heads;          // query heads that share one index set (a divisor of group)
+  int n_sets;             // index sets (selection units) per sequence = n_q_heads / sel_heads
   int chunks;             // 16-byte chunks per proxy row = ceil(n_dom / 4)
   int row_elems;          // bf16 elements per proxy row = 8 * chunks
   int device;
@@ -48,12 +50,13 @@ struct fasa_ctx {
     FASA_CUDA_TRY(ctx, cudaGetLastError());                                            \
   } while (0)
 
-// How the attention kernels cut a list of at most n_upper rows into splits.
+// How the attention kernels cut a list of at most n_upper rows per unit into splits, given
+// the number of units (grid.y) of the launch.
 struct fasa_split_plan {
   int n_splits;   // grid.x
   int chunk;      // rows per split (multiple of 32)
 };
-fasa_split_plan fasa_plan_splits(const fasa_ctx* ctx, int n_upper);
+fasa_split_plan fasa_plan_splits(const fasa_ctx* ctx, int n_upper, int units);
 
 // One-launch decode step (fasa_fused.cu): plan at context creation, launch per step.
 int fasa_fused_plan(fasa_ctx* ctx);
@@ -65,7 +68,7 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
 // Large selections are attended by the split-K tensor-core kernel rather than inside the
 // cluster kernel (whose attention phase runs on CUDA cores at 64 registers per thread).
 static inline bool fasa_attend_separately(const fasa_ctx* ctx, int n_sel_max, const void* workspace) {
-  return workspace != nullptr && (long long)n_sel_max * ((ctx->group + 3) / 4) >= 2048;
+  return workspace != nullptr && (long long)n_sel_max * ((ctx->sel_heads + 3) / 4) >= 2048;
 }
 
 int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
@@ -102,6 +105,25 @@ __device__ __forceinline__ float dot8(const float2 (&q)[4], const uint4& k) {
   a = __ffma2_rn(q[2], bf16x2_to_f32x2(k.z), a);
   a = __ffma2_rn(q[3], bf16x2_to_f32x2(k.w), a);
   return a.x + a.y;
+}
+
+// A selection unit: `heads` consecutive query heads of one sequence that share an index set
+// (Sec. 4.1 keeps a set per head; by default all heads of a KV head share one).  Unit u of
+// the grid is set hs = u % n_sets of sequence b = u / n_sets.
+struct SelUnit {
+  int b;        // sequence
+  int h;        // KV head whose cache the unit reads
+  int kv;       // b * n_kv_heads + h: index of that cache (K, V, proxy, appended rows)
+  int64_t q0;   // b * n_q_heads + first query head of the unit: row of q, out and lse
+};
+__device__ __forceinline__ SelUnit sel_unit(int u, int n_sets, int heads, int n_q_heads, int n_kv_heads) {
+  SelUnit s;
+  const int hs = u % n_sets;
+  s.b = u / n_sets;
+  s.h = hs / (n_sets / n_kv_heads);
+  s.kv = s.b * n_kv_heads + s.h;
+  s.q0 = (int64_t)s.b * n_q_heads + (int64_t)hs * heads;
+  return s;
 }
 
 __device__ __forceinline__ int clamp_len(int len, int max_len, int32_t* status) {

@@ -64,7 +64,7 @@ struct FusedParams {
   float* out_mirror;       // nullable: a second copy of out (mapped host memory of the host-buffer step)
   float* lse;              // nullable
   int32_t* status;
-  int n_q_heads, n_kv_heads, group, max_len, chunks, n_sink, n_recent, budget, n_sel_max;
+  int n_q_heads, n_kv_heads, n_sets, group, max_len, chunks, n_sink, n_recent, budget, n_sel_max;   // group: query heads of a unit
   int max_reduce;          // score of a KV head = max over its query heads instead of their sum
   int64_t ksb, ksh, kst, vsb, vsh, vst;
   float scale_log2;        // softmax_scale * log2(e)
@@ -117,8 +117,9 @@ fused_decode_kernel(const FusedParams p) {
   const int lane = tid & 31;
   const int warp = tid >> 5;
   const int u = blockIdx.y;
-  const int h = u % p.n_kv_heads;
-  const int b = u / p.n_kv_heads;
+  const SelUnit su = sel_unit(u, p.n_sets, p.group, p.n_q_heads, p.n_kv_heads);
+  const int h = su.h;
+  const int b = su.b;
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ uint32_t s_coarse[2][kFBins / 32];
@@ -152,12 +153,12 @@ fused_decode_kernel(const FusedParams p) {
   if (!append || tid == 0) len_raw = p.seq_lens[b];
   uint4 q_stage = make_uint4(0u, 0u, 0u, 0u);
   if (MODE == 0 && tid < FASA_MAX_GROUP * (FASA_HEAD_DIM / 8) && tid / (FASA_HEAD_DIM / 8) < p.group)
-    q_stage = *reinterpret_cast<const uint4*>(p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM + tid * 8);
+    q_stage = *reinterpret_cast<const uint4*>(p.q + su.q0 * FASA_HEAD_DIM + tid * 8);
   ScoreFrag<KB> f[NG];
   if constexpr (MODE != 1)
 #pragma unroll
   for (int grp = 0; grp < NG; ++grp)
-    load_score_b<KB>(f[grp], p.q + ((int64_t)b * p.n_q_heads + (int64_t)h * p.group) * FASA_HEAD_DIM,
+    load_score_b<KB>(f[grp], p.q + su.q0 * FASA_HEAD_DIM,
                      p.chan + h * p.chunks * 8, p.chunks, p.group, lane, grp * KB);
   int len_old;
   if (append) {
@@ -172,7 +173,7 @@ fused_decode_kernel(const FusedParams p) {
   if (append && tid == 0) {
     if (!grows && crank == 0) atomicOr(p.status, FASA_DEV_APPEND_FULL);
     __threadfence();
-    const int total = p.n_kv_heads * cs;
+    const int total = p.n_sets * cs;
     if (atomicAdd(&p.arrive[b], 1) == total - 1) {
       p.seq_lens_w[b] = len;
       p.arrive[b] = 0;
@@ -206,7 +207,7 @@ fused_decode_kernel(const FusedParams p) {
   constexpr int TPI = KB == 1 ? 4 : 2;                        // tiles per warp iteration (even)
   const ProxyGeom pg = proxy_geom(p.chunks);
   const int n_blocks = pg.n16 + pg.n8;
-  const unsigned char* unit = p.proxy + (int64_t)u * ((p.max_len + 15) >> 4) * pg.tile_bytes;
+  const unsigned char* unit = p.proxy + (int64_t)su.kv * ((p.max_len + 15) >> 4) * pg.tile_bytes;
   float* srow = p.scores ? p.scores + (int64_t)u * p.max_len : nullptr;
   auto fetch = [&](uint4 (&a)[TPI][KB], int T, int grp) {
 #pragma unroll
@@ -221,15 +222,16 @@ fused_decode_kernel(const FusedParams p) {
 
   if (own_new) {
     // this CTA's slice holds the new row: K and V copies (16 lanes each) and the packed
-    // dominant-FC pairs of the key (one lane per 16-byte chunk), as in fasa_kv_append
-    const uint16_t* ksrc = p.k_new + (int64_t)u * FASA_HEAD_DIM;
+    // dominant-FC pairs of the key (one lane per 16-byte chunk), as in fasa_kv_append.  When
+    // several units share a KV head each writes the same values, and reads back its own.
+    const uint16_t* ksrc = p.k_new + (int64_t)su.kv * FASA_HEAD_DIM;
     if (tid < 16) {
       *reinterpret_cast<uint4*>(p.k_w + b * p.ksb + h * p.ksh + (int64_t)len_old * p.kst + tid * 8) =
           *reinterpret_cast<const uint4*>(ksrc + tid * 8);
     } else if (tid < 32) {
       const int c = tid - 16;
       *reinterpret_cast<uint4*>(p.v_w + b * p.vsb + h * p.vsh + (int64_t)len_old * p.vst + c * 8) =
-          *reinterpret_cast<const uint4*>(p.v_new + (int64_t)u * FASA_HEAD_DIM + c * 8);
+          *reinterpret_cast<const uint4*>(p.v_new + (int64_t)su.kv * FASA_HEAD_DIM + c * 8);
     } else if (tid - 32 < 4 * p.chunks) {
       const int w = tid - 32;                       // one dominant FC = one 4-byte channel pair
       const ProxyGeom pg = proxy_geom(p.chunks);
@@ -237,7 +239,7 @@ fused_decode_kernel(const FusedParams p) {
       const int ch0 = ch[0], ch1 = ch[1];
       const uint32_t lo = ch0 >= 0 ? ksrc[ch0] : 0u;
       const uint32_t hi = ch1 >= 0 ? ksrc[ch1] : 0u;
-      unsigned char* unit = p.proxy_w + (int64_t)u * ((p.max_len + 15) >> 4) * pg.tile_bytes;
+      unsigned char* unit = p.proxy_w + (int64_t)su.kv * ((p.max_len + 15) >> 4) * pg.tile_bytes;
       *reinterpret_cast<uint32_t*>(unit + proxy_word_offset(pg, len_old, w)) = lo | (hi << 16);
     }
   }
@@ -712,7 +714,7 @@ fused_decode_kernel(const FusedParams p) {
       }
       if (ok && r == 0) {
         const int c = o % FASA_HEAD_DIM;
-        const int64_t hq = (int64_t)b * p.n_q_heads + (int64_t)h * p.group + g;
+        const int64_t hq = su.q0 + g;
         const float ov = l > 0.f ? av / l : 0.f;
         p.out[hq * FASA_HEAD_DIM + c] = ov;
         if (p.out_mirror) p.out_mirror[hq * FASA_HEAD_DIM + c] = ov;
@@ -758,7 +760,7 @@ int fasa_fused_plan(fasa_ctx* ctx) {
   ctx->fused_cs = 0;
   ctx->fused_smem = 0;
   ctx->fused_step_ok = 1;
-  const int units = c.batch * c.n_kv_heads;
+  const int units = c.batch * ctx->n_sets;
   FusedFn fn = fused_fn(ctx->chunks);
   auto cap_of = [&](int cs) { return (((c.max_len + cs - 1) / cs) + 31) & ~31; };
   // Two CTAs per SM can be resident; a cluster is doubled while the whole grid still fits
@@ -828,7 +830,7 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
   p.k_w = (uint16_t*)k_cache; p.v_w = (uint16_t*)v_cache; p.proxy_w = (unsigned char*)proxy_k;
   p.seq_lens_w = (int32_t*)seq_lens; p.arrive = ctx->d_arrive;
   p.scores = scores; p.idx = idx; p.n_sel = n_sel; p.out = out; p.lse = lse; p.status = ctx->d_status;
-  p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group; p.max_len = c.max_len;
+  p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.n_sets = ctx->n_sets; p.group = ctx->sel_heads; p.max_len = c.max_len;
   p.chunks = ctx->chunks; p.n_sink = c.n_sink; p.n_recent = c.n_recent; p.budget = budget;
   p.n_sel_max = n_sel_max;
   p.max_reduce = c.group_reduce;
@@ -839,7 +841,7 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
 
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3((unsigned)ctx->fused_cs, (unsigned)(c.batch * c.n_kv_heads), 1);
+  cfg.gridDim = dim3((unsigned)ctx->fused_cs, (unsigned)(c.batch * ctx->n_sets), 1);
   cfg.blockDim = dim3(kFT, 1, 1);
   cfg.dynamicSmemBytes = ctx->fused_smem;
   cfg.stream = stream;
@@ -865,12 +867,12 @@ int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t
   memset(&p, 0, sizeof(p));
   p.seq_lens = seq_lens; p.scores = const_cast<float*>(scores); p.idx = idx; p.n_sel = n_sel;
   p.status = ctx->d_status;
-  p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group; p.max_len = c.max_len;
+  p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.n_sets = ctx->n_sets; p.group = ctx->sel_heads; p.max_len = c.max_len;
   p.chunks = ctx->chunks; p.n_sink = c.n_sink; p.n_recent = c.n_recent; p.budget = budget;
   p.n_sel_max = n_sel_max;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3((unsigned)ctx->fused_cs, (unsigned)(c.batch * c.n_kv_heads), 1);
+  cfg.gridDim = dim3((unsigned)ctx->fused_cs, (unsigned)(c.batch * ctx->n_sets), 1);
   cfg.blockDim = dim3(kFT, 1, 1);
   cfg.dynamicSmemBytes = ctx->fused_smem;
   cfg.stream = stream;

@@ -24,11 +24,12 @@ __global__ void __launch_bounds__(kScoreThreads)
 fc_score_kernel(const uint16_t* __restrict__ q, const unsigned char* __restrict__ proxy,
                 const int32_t* __restrict__ seq_lens, const int16_t* __restrict__ chan,
                 float* __restrict__ scores, int32_t* __restrict__ status, int n_q_heads,
-                int n_kv_heads, int group, int max_len, int chunks, int tiles_per_cta) {
+                int n_kv_heads, int n_sets, int group, int max_len, int chunks, int tiles_per_cta) {
   constexpr int TPI = TilesPerIter<KB>::value;
   const int u = blockIdx.y;
-  const int h = u % n_kv_heads;
-  const int b = u / n_kv_heads;
+  const SelUnit su = sel_unit(u, n_sets, group, n_q_heads, n_kv_heads);
+  const int h = su.h;
+  const int b = su.b;
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const ProxyGeom pg = proxy_geom(chunks);
@@ -36,7 +37,7 @@ fc_score_kernel(const uint16_t* __restrict__ q, const unsigned char* __restrict_
   const int tiles_alloc = (max_len + 15) >> 4;
   const int cta_tile0 = blockIdx.x * tiles_per_cta;
   const int cta_tile1 = min(tiles_alloc, cta_tile0 + tiles_per_cta);
-  const unsigned char* unit = proxy + (int64_t)u * tiles_alloc * pg.tile_bytes;
+  const unsigned char* unit = proxy + (int64_t)su.kv * tiles_alloc * pg.tile_bytes;
 
   // First batch of loads: every tile up to max_len is allocated, so reading past the
   // sequence length is harmless and overlaps with the loads of the length and the query.
@@ -51,7 +52,7 @@ fc_score_kernel(const uint16_t* __restrict__ q, const unsigned char* __restrict_
   const int row1 = min(len, cta_tile1 * 16);
 
   ScoreFrag<KB> f;
-  load_score_b<KB>(f, q + ((int64_t)b * n_q_heads + (int64_t)h * group) * FASA_HEAD_DIM,
+  load_score_b<KB>(f, q + su.q0 * FASA_HEAD_DIM,
                    chan + h * chunks * 8, chunks, group, lane);
   float* srow = scores + (int64_t)u * max_len;
 
@@ -79,7 +80,7 @@ template <int KB>
 void launch_score(fasa_ctx* ctx, const void* q, const void* proxy, const int32_t* seq_lens,
                   float* scores, cudaStream_t s) {
   const fasa_config_t& c = ctx->cfg;
-  const int units = c.batch * c.n_kv_heads;
+  const int units = c.batch * ctx->n_sets;
   // Enough CTAs to cover the SMs several times, at least one warp iteration each.
   constexpr int kStep = TilesPerIter<KB>::value * kScoreWarps;
   const int tiles = (c.max_len + 15) / 16;
@@ -90,11 +91,11 @@ void launch_score(fasa_ctx* ctx, const void* q, const void* proxy, const int32_t
   if (c.group_reduce == 0)
     fc_score_kernel<KB, false><<<grid, kScoreThreads, 0, s>>>(
         (const uint16_t*)q, (const unsigned char*)proxy, seq_lens, ctx->d_chan, scores, ctx->d_status,
-        c.n_q_heads, c.n_kv_heads, ctx->group, c.max_len, ctx->chunks, per);
+        c.n_q_heads, c.n_kv_heads, ctx->n_sets, ctx->sel_heads, c.max_len, ctx->chunks, per);
   else
     fc_score_kernel<KB, true><<<grid, kScoreThreads, 0, s>>>(
         (const uint16_t*)q, (const unsigned char*)proxy, seq_lens, ctx->d_chan, scores, ctx->d_status,
-        c.n_q_heads, c.n_kv_heads, ctx->group, c.max_len, ctx->chunks, per);
+        c.n_q_heads, c.n_kv_heads, ctx->n_sets, ctx->sel_heads, c.max_len, ctx->chunks, per);
 }
 
 }  // namespace

@@ -53,13 +53,13 @@ template <bool CACHED>
 __global__ void __launch_bounds__(kTopkThreads, 1)
 topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ seq_lens, int budget,
             int n_sel_max, int32_t* __restrict__ idx, int32_t* __restrict__ n_sel,
-            int32_t* __restrict__ status, int n_kv_heads, int max_len, int n_sink, int n_recent) {
+            int32_t* __restrict__ status, int n_sets, int max_len, int n_sink, int n_recent) {
   cg::cluster_group cluster = cg::this_cluster();
   const int cs = (int)cluster.num_blocks();
   const int crank = (int)cluster.block_rank();
   const int tid = threadIdx.x;
   const int u = blockIdx.y;
-  const int b = u / n_kv_heads;
+  const int b = u / n_sets;
   const int len = clamp_len(seq_lens[b], max_len, status);
 
   // Selection size: forced positions come on top of the budget.
@@ -214,7 +214,7 @@ extern "C" int32_t fasa_topk(fasa_ctx_t* ctx, const float* scores, const int32_t
     return FASA_ERR_INVALID_ARG;
   if (budget < -1000) return FASA_ERR_INVALID_ARG;
   const fasa_config_t& c = ctx->cfg;
-  const int units = c.batch * c.n_kv_heads;
+  const int units = c.batch * ctx->n_sets;
   // The cluster kernel's selection phases (keys in shared memory, one barrier per radix pass,
   // mask compaction) serve wherever a cluster shape exists for this context; the
   // register-resident kernel below remains for the rest (max_len beyond 16 x 22528).
@@ -244,11 +244,11 @@ extern "C" int32_t fasa_topk(fasa_ctx_t* ctx, const float* scores, const int32_t
   cudaError_t e;
   if (cached)
     e = cudaLaunchKernelEx(&cfg, topk_kernel<true>, scores, seq_lens, (int)budget, (int)n_sel_max,
-                           idx, n_sel, ctx->d_status, (int)c.n_kv_heads, (int)c.max_len,
+                           idx, n_sel, ctx->d_status, (int)ctx->n_sets, (int)c.max_len,
                            (int)c.n_sink, (int)c.n_recent);
   else
     e = cudaLaunchKernelEx(&cfg, topk_kernel<false>, scores, seq_lens, (int)budget, (int)n_sel_max,
-                           idx, n_sel, ctx->d_status, (int)c.n_kv_heads, (int)c.max_len,
+                           idx, n_sel, ctx->d_status, (int)ctx->n_sets, (int)c.max_len,
                            (int)c.n_sink, (int)c.n_recent);
   ctx->launches += 1;
   FASA_CUDA_TRY(ctx, e);

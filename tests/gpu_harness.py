@@ -29,11 +29,12 @@ class Run:
         self.dom = self.t["dom"]
         self.fasa = binding.Fasa.from_workload(w, self.dom)
         self.n_sel_max = n_sel_max if n_sel_max is not None else w.n_sel_max()
-        B, Hq, Hkv, Lm = w.batch, w.n_q_heads, w.n_kv_heads, w.max_len
+        B, Hq, Hs, Lm = w.batch, w.n_q_heads, w.n_sets, w.max_len      # Hs index sets per sequence
+        assert self.fasa.n_sets == Hs
         self.proxy = self.fasa.alloc_proxy(dev)
-        self.scores = torch.full((B, Hkv, Lm), SENTINEL, dtype=torch.float32, device=dev)
-        self.idx = torch.full((B, Hkv, self.n_sel_max), -7, dtype=torch.int32, device=dev)
-        self.n_sel = torch.full((B, Hkv), -7, dtype=torch.int32, device=dev)
+        self.scores = torch.full((B, Hs, Lm), SENTINEL, dtype=torch.float32, device=dev)
+        self.idx = torch.full((B, Hs, self.n_sel_max), -7, dtype=torch.int32, device=dev)
+        self.n_sel = torch.full((B, Hs), -7, dtype=torch.int32, device=dev)
         self.out = torch.full((B, Hq, 128), SENTINEL, dtype=torch.float32, device=dev)
         self.lse = torch.full((B, Hq), SENTINEL, dtype=torch.float32, device=dev)
         self.dense = torch.full((B, Hq, 128), SENTINEL, dtype=torch.float32, device=dev)
@@ -82,4 +83,5 @@ class Run:
     def oracle_kwargs(self, budget=None):
         w = self.w
         return dict(pairing=w.pairing, group_reduce=w.group_reduce, n_sink=w.n_sink, n_recent=w.n_recent,
-                    budget=w.budget if budget is None else budget, scale=1.0 / math.sqrt(128.0))
+                    budget=w.budget if budget is None else budget, scale=1.0 / math.sqrt(128.0),
+                    sel_heads=w.sel_heads)

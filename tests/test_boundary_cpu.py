@@ -37,11 +37,11 @@ def test_status_strings_and_row_elems(lib):
 
 def _cfg(**kw):
     base = dict(batch=1, n_q_heads=4, n_kv_heads=1, head_dim=128, max_len=64, n_dom=2, rope_pairing=0,
-                group_reduce=0, n_sink=0, n_recent=0, softmax_scale=0.0)
+                group_reduce=0, select_heads=0, n_sink=0, n_recent=0, softmax_scale=0.0)
     base.update(kw)
     return binding.FasaConfig(base["batch"], base["n_q_heads"], base["n_kv_heads"], base["head_dim"],
                               base["max_len"], base["n_dom"], base["rope_pairing"], base["group_reduce"],
-                              base["n_sink"], base["n_recent"], base["softmax_scale"], 0, 0, 0, 0, 0, 0)
+                              base["select_heads"], base["n_sink"], base["n_recent"], base["softmax_scale"], 0, 0, 0, 0, 0, 0)
 
 
 @pytest.mark.parametrize("kw,expect", [
@@ -55,6 +55,8 @@ def _cfg(**kw):
     (dict(n_q_heads=9, n_kv_heads=1), binding.ERR_UNSUPPORTED),
     (dict(rope_pairing=2), binding.ERR_UNSUPPORTED),
     (dict(group_reduce=3), binding.ERR_UNSUPPORTED),
+    (dict(select_heads=3), binding.ERR_UNSUPPORTED),      # does not divide the group of 4
+    (dict(select_heads=-1), binding.ERR_UNSUPPORTED),
 ])
 def test_create_rejects_bad_config_without_a_gpu(lib, kw, expect):
     cfg = _cfg(**kw)

@@ -37,7 +37,7 @@ def _full_check(r: Run, budget=None, dense=True):
         for b in range(r.w.batch):
             L = int(h["seq_lens"][b])
             assert np.all(h["scores"][b, :, L:] == SENTINEL)
-            for hh in range(r.w.n_kv_heads):
+            for hh in range(r.w.n_sets):
                 assert np.all(h["idx"][b, hh, int(h["n_sel"][b, hh]):] == -7)
         assert r.fasa.device_status() == 0
         if not fused:
@@ -285,6 +285,89 @@ def test_large_selection_is_attended_by_the_split_k_kernel():
     h = r.host()
     parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
                       n_sel=h["n_sel"], out=h["out"], what="split attention", **r.oracle_kwargs())
+    assert r.fasa.device_status() == 0
+
+
+# ---- index sets shared by fewer query heads than a KV head serves (Sec. 4.1: a set per head) ----
+
+@pytest.mark.parametrize("cfg,sel,kw", [
+    ("c1", 1, dict(max_len=3001, len_lo=2999, len_hi=2999)),                        # 32 sets of one head
+    ("c1", 2, dict(batch=2, max_len=2100, len_lo=900, len_hi=2100)),                # 16 sets of two heads
+    ("c3", 1, dict(batch=2, max_len=1500, len_lo=900, len_hi=1400)),                # group of 7, permille budget
+    ("c0", 1, dict()),                                                              # config 0 at full size
+    ("c1", 1, dict(max_len=1200, len_lo=1100, len_hi=1200, group_reduce=1, pairing=1, n_dom=5)),
+])
+def test_index_sets_per_query_head(cfg, sel, kw):
+    w = C[cfg].replace(sel_heads=sel, **kw)
+    rep, h = _full_check(Run(w))
+    assert rep["units"] == w.batch * w.n_q_heads // sel
+    assert h["idx"].shape[1] == w.n_q_heads // sel
+
+
+def test_index_sets_per_query_head_equal_the_model_with_repeated_kv_heads():
+    # the same statement as the oracle's pin, on the GPU: bit-exact scores and sets, both routes
+    w = C["c1"].replace(batch=2, max_len=2000, len_lo=1500, len_hi=2000, sel_heads=1)
+    t = synth.make_inputs(w, "cpu")
+    x = dict(t)
+    x["k"], x["v"] = t["k"].repeat_interleave(w.group, dim=1), t["v"].repeat_interleave(w.group, dim=1)
+    x["dom"] = t["dom"].repeat_interleave(w.group, dim=0)
+    a, b = Run(w, t), Run(w.replace(n_kv_heads=w.n_q_heads, sel_heads=0), x)
+    for fused in (False, True):
+        for r in (a, b):
+            r.build_proxy()
+            r.reset_outputs()
+            r.step(fused=fused)
+        for u, v in ((a.scores, b.scores), (a.idx, b.idx), (a.n_sel, b.n_sel), (a.out, b.out), (a.lse, b.lse)):
+            assert torch.equal(u, v)
+
+
+@pytest.mark.parametrize("mode", [1, 0])
+def test_index_sets_per_query_head_append_form(mode):
+    # several sets share a KV head: each cluster of the one-launch form writes the new rows itself
+    w = C["c3"].replace(batch=3, max_len=1300, len_lo=700, len_hi=1297, sel_heads=1)
+    t = synth.make_inputs(w, "cpu")
+    t["seq_lens"] = torch.tensor([700, 1299, 1001], dtype=torch.int32)
+    a, b = Run(w, t), Run(w, {k_: (v_.clone() if torch.is_tensor(v_) else v_) for k_, v_ in t.items()})
+    for r in (a, b):
+        r.fasa.set_step_mode(mode)
+        r.build_proxy()
+    for step in range(3):
+        s = synth.make_step_inputs(w, step, "cuda")
+        a.fasa.kv_append(a.k, a.v, a.proxy, a.seq_lens, s["k_new"], s["v_new"])
+        a.fasa.decode_step(s["q"], a.k, a.v, a.proxy, a.seq_lens, w.budget, a.scores, a.idx, a.n_sel, a.out, a.ws)
+        n0 = b.fasa.launch_count()
+        b.fasa.append_decode_step(s["q"], s["k_new"], s["v_new"], b.k, b.v, b.proxy, b.seq_lens, w.budget, b.scores,
+                                  b.idx, b.n_sel, b.out, b.ws)
+        torch.cuda.synchronize()
+        assert b.fasa.launch_count() - n0 == (1 if mode == 1 else 5)
+        for u, v in ((a.k, b.k), (a.v, b.v), (a.proxy, b.proxy), (a.seq_lens, b.seq_lens), (a.scores, b.scores),
+                     (a.idx, b.idx), (a.n_sel, b.n_sel)):
+            assert torch.equal(u, v)
+        assert float((a.out - b.out).abs().max()) <= 1e-5
+    assert a.seq_lens.cpu().tolist() == [703, 1300, 1004]
+    parity.check_step(s["q"].cpu().double().numpy(), b.k.cpu().double().numpy(), b.v.cpu().double().numpy(),
+                      [703, 1300, 1004], np.sort(b.dom.numpy(), axis=1), scores=b.scores.cpu().numpy(),
+                      idx=b.idx.cpu().numpy(), n_sel=b.n_sel.cpu().numpy(), out=b.out.cpu().numpy(),
+                      what="append+step, sets per head", **b.oracle_kwargs())
+
+
+def test_index_sets_per_query_head_large_selection_and_static_scratch():
+    # one head per set: the split route starts at n_sel_max >= 2048; the no-workspace variant agrees
+    w = C["c1"].replace(batch=1, n_q_heads=8, n_kv_heads=2, max_len=6000, len_lo=5000, len_hi=6000, budget=2500,
+                        sel_heads=1)
+    r = Run(w)
+    r.build_proxy()
+    n0 = r.fasa.launch_count()
+    r.fasa.decode_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel, r.out, r.ws, r.lse)
+    torch.cuda.synchronize()
+    assert r.fasa.launch_count() - n0 == 3
+    h = r.host()
+    parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
+                      n_sel=h["n_sel"], out=h["out"], what="split attention, sets per head", **r.oracle_kwargs())
+    out2 = torch.full_like(r.out, SENTINEL)
+    r.fasa.sparse_decode_attn_static(r.q, r.k, r.v, r.idx, r.n_sel, out2)
+    torch.cuda.synchronize()
+    assert torch.equal(out2, r.out)
     assert r.fasa.device_status() == 0
 
 
