@@ -73,7 +73,8 @@ def _peaks():
 
 def step_bytes(w, lens, n_sel):
     """Algorithmic bytes of one FASA step and of one dense step (Sec. 4.4 byte model).
-    lens: per-sequence context at scoring time; n_sel: tokens attended per unit."""
+    lens: per-sequence context at scoring time; n_sel: tokens attended, summed over the index
+    sets.  The proxy counts once per KV head however many index sets share it."""
     units_len = sum(int(l) for l in lens) * w.n_kv_heads
     qo = w.batch * w.n_q_heads * 128 * (2 + 4)
     proxy = units_len * 4 * w.n_dom
@@ -200,12 +201,12 @@ def measure(w, K, W, dev, world, step_mode=None, sampler_factory=None, want_e2e=
     fused = f.step_cluster_size() > 0
     q, k, v = t["q"], t["k"], t["v"]
     n_sel_max = w.n_sel_max()
-    B, Hq, Hkv, Lm = w.batch, w.n_q_heads, w.n_kv_heads, w.max_len
+    B, Hq, Hs, Lm = w.batch, w.n_q_heads, w.n_sets, w.max_len        # Hs index sets per sequence
     proxy = f.alloc_proxy(dev)
     ws = f.alloc_workspace(n_sel_max, dev)
-    scores = torch.zeros((B, Hkv, Lm), dtype=torch.float32, device=dev)
-    idx = torch.zeros((B, Hkv, n_sel_max), dtype=torch.int32, device=dev)
-    n_sel = torch.zeros((B, Hkv), dtype=torch.int32, device=dev)
+    scores = torch.zeros((B, Hs, Lm), dtype=torch.float32, device=dev)
+    idx = torch.zeros((B, Hs, n_sel_max), dtype=torch.int32, device=dev)
+    n_sel = torch.zeros((B, Hs), dtype=torch.int32, device=dev)
     out = torch.zeros((B, Hq, 128), dtype=torch.float32, device=dev)
     dense_out = torch.zeros_like(out)
     lens = lens_full.clone()
@@ -323,7 +324,7 @@ def summarize(m, peak):
         "workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
         "context": int(m["lens_full"].max()), "context_mean": float(m["lens_full"].float().mean()),
         "n_dom": w.n_dom, "budget": w.budget, "n_sink": w.n_sink, "n_recent": w.n_recent,
-        "n_sel_per_unit": m["n_sel_total"] / (w.batch * w.n_kv_heads),
+        "n_sel_per_unit": m["n_sel_total"] / (w.batch * w.n_sets), "heads_per_index_set": w.heads_per_set,
         "step_mode": ("three kernels" if not m["fused"] else
                       f"one cluster kernel (cluster of {m['cluster_size']})" if m["launches_per_step"] == 1 else
                       f"cluster kernel (cluster of {m['cluster_size']}) + split-K tensor-core attention"),
@@ -441,10 +442,12 @@ def run_sweep(args):
     base = synth.CONFIGS["c4"]
     if args.batch is not None:
         base = base.replace(batch=args.batch)
+    if args.select_heads is not None:
+        base = base.replace(sel_heads=args.select_heads)
     t = synth.make_inputs(base, dev)
     peak, peak_src = _peaks()
     rows = []
-    for F in (4, 8, 16, 32, 64):
+    for F in ((4, 8, 16, 32, 64) if args.n_dom is None else (args.n_dom,)):
         for k in (64, 128, 256, 512, 1024, 2048, 4096):
             w = base.replace(n_dom=F, budget=k)
             m = measure(w, args.sweep_steps, 3, dev, 1, args.step_mode, None, want_e2e=False, t=t)
@@ -454,7 +457,8 @@ def run_sweep(args):
                                                "standalone_us", "standalone_frac_of_peak", "step_mode", "launches_per_step",
                                                "device_status")})
             del m
-    print(json.dumps({"sweep": base.name, "batch": base.batch, "context": base.max_len, "peak_gbs": peak,
+    print(json.dumps({"sweep": base.name, "batch": base.batch, "context": base.max_len,
+                      "heads_per_index_set": base.heads_per_set, "peak_gbs": peak,
                       "peak_source": peak_src, "steps_per_point": args.sweep_steps, "rows": rows}), flush=True)
 
 
@@ -541,6 +545,8 @@ def main():
     ap.add_argument("--budget", type=int, default=None)
     ap.add_argument("--n-dom", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (profiling)")
+    ap.add_argument("--select-heads", type=int, default=None,
+                    help="query heads sharing one index set (default: all heads of a KV head; 1 = a set per head)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--extras", default="c4,c2", help="other workloads reported under other_workloads (30 steps each)")
     ap.add_argument("--no-extras", action="store_true")
@@ -563,6 +569,8 @@ def main():
         w = w.replace(n_dom=args.n_dom)
     if args.batch is not None:
         w = w.replace(batch=args.batch)
+    if args.select_heads is not None:
+        w = w.replace(sel_heads=args.select_heads)
     if args.impl == "reference":
         run_reference(args, w)
     else:

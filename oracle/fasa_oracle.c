@@ -12,6 +12,8 @@
  *   - T_t = TopK-I(S_t, N_fac)                                       (Sec. 4.1)
  *   - Gather + Softmax(q K_T^T / sqrt(d)) V_T                         (Sec. 4.2, Eq. 6-7)
  *   - full-KV attention (the FKV baseline)                            (Sec. 5.1)
+ *   - contextual agreement CA of a single FC with the full head, and the
+ *     offline choice of the dominant FCs from its mean          (Sec. 3.3, Eq. 4; Algorithm 1)
  *
  * Readings taken where the paper is silent (each is listed in the design notes):
  *   FC channel pairing is selectable: 0 = rotate-half (i, i+d/2), 1 = interleaved
@@ -215,6 +217,132 @@ void fasa_oracle_attn_dense(const double* q, int G, const double* K, const doubl
   for (int j = 0; j < L; ++j) idx[j] = j;
   fasa_oracle_attn_subset(q, G, K, V, d, idx, L, scale, O, lse);
   free(idx);
+}
+
+/* ------------------------------------------------------------ calibration */
+
+/* CA (Sec. 3.3, Eq. 4) of every FC for one query head: counts[i] =
+ * | TopK-I(alpha, top_k)  intersected with  TopK-I(alpha^(i), top_k) |, i.e. CA times top_k.
+ * alpha^(i) are the single-FC raw scores (Eq. 3) and alpha their sum over all FCs, the
+ * full-head raw scores (Eq. 2).  TopK-I ranks as everywhere here: higher score first,
+ * then lower index.
+ * Which index enters a top-k set is an integer decided by floating point, so it is
+ * taken in the precision of the path being checked when f32 != 0: each product in
+ * binary32 (exact for bf16 inputs), alpha^(i) = their binary32 sum, alpha = the
+ * binary32 sum of alpha^(0), alpha^(1), ... in this order.  f32 == 0 is the plain
+ * fp64 statement. */
+void fasa_oracle_ca_counts(const double* q, const double* K, int L, int d, int pairing,
+                           int top_k, int f32, int* counts) {
+  int n_fc = d / 2;
+  size_t rows = (size_t)(L > 0 ? L : 1);
+  double* a = (double*)malloc(sizeof(double) * (size_t)n_fc * rows);
+  double* full = (double*)malloc(sizeof(double) * rows);
+  int* t_full = (int*)malloc(sizeof(int) * rows);
+  int* t_fc = (int*)malloc(sizeof(int) * rows);
+  double band[4];
+  for (int j = 0; j < L; ++j) {
+    double acc = 0.0;
+    float acc32 = 0.0f;
+    for (int i = 0; i < n_fc; ++i) {
+      int c0, c1;
+      fc_channels(i, d, pairing, &c0, &c1);
+      double p0 = q[c0] * K[(int64_t)j * d + c0], p1 = q[c1] * K[(int64_t)j * d + c1];
+      if (f32) {
+        volatile float s32 = (float)p0 + (float)p1;   /* one binary32 rounding */
+        volatile float t32 = acc32 + s32;
+        acc32 = t32;
+        a[(int64_t)i * L + j] = (double)s32;
+      } else {
+        a[(int64_t)i * L + j] = p0 + p1;
+        acc += p0 + p1;
+      }
+    }
+    full[j] = f32 ? (double)acc32 : acc;
+  }
+  int n_full = fasa_oracle_select(full, L, top_k, 0, 0, 0.0, t_full, band);
+  for (int i = 0; i < n_fc; ++i) {
+    int n_i = fasa_oracle_select(a + (int64_t)i * L, L, top_k, 0, 0, 0.0, t_fc, band);
+    int x = 0, y = 0, common = 0;          /* both lists ascending */
+    while (x < n_full && y < n_i) {
+      if (t_full[x] == t_fc[y]) { ++common; ++x; ++y; }
+      else if (t_full[x] < t_fc[y]) ++x;
+      else ++y;
+    }
+    counts[i] = common;
+  }
+  free(a); free(full); free(t_full); free(t_fc);
+}
+
+/* Stage 1 of Algorithm 1 over a batch of bf16 tensors laid out as in the decode
+ * step: a sample is a (sequence b, query head g) pair whose sequence is longer
+ * than top_k (a shorter one selects every position and says nothing).  Adds each
+ * sample's counts to counts[g][i] ([Hq][d/2]) and 1 to n_used[g] ([Hq]).
+ * Returns the number of threads used. */
+int fasa_oracle_calibrate_bf16(const uint16_t* q_bits, const uint16_t* K_bits,
+                               const int32_t* seq_lens, int B, int Hq, int Hkv, int d,
+                               int Lmax, int pairing, int top_k, int f32, int n_threads,
+                               int64_t* counts, int64_t* n_used) {
+  int group = Hq / Hkv, n_fc = d / 2;
+  int used = 1;
+#ifdef _OPENMP
+  if (n_threads > 0) omp_set_num_threads(n_threads);
+  used = n_threads > 0 ? n_threads : omp_get_max_threads();
+  if (used > B * Hq) used = B * Hq;
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+  for (int u = 0; u < B * Hq; ++u) {
+    int b = u / Hq, g = u % Hq, h = g / group;
+    int L = seq_lens[b];
+    if (L > Lmax) L = Lmax;
+    if (L <= top_k) continue;
+    double* Kd = (double*)malloc(sizeof(double) * (size_t)L * (size_t)d);
+    double* qd = (double*)malloc(sizeof(double) * (size_t)d);
+    int* c = (int*)malloc(sizeof(int) * (size_t)n_fc);
+    fasa_oracle_widen_bf16(K_bits + ((int64_t)b * Hkv + h) * (int64_t)Lmax * d, (int64_t)L * d, Kd);
+    fasa_oracle_widen_bf16(q_bits + ((int64_t)b * Hq + g) * d, d, qd);
+    fasa_oracle_ca_counts(qd, Kd, L, d, pairing, top_k, f32, c);
+    for (int i = 0; i < n_fc; ++i) {
+#ifdef _OPENMP
+#pragma omp atomic
+#endif
+      counts[(int64_t)g * n_fc + i] += c[i];
+    }
+#ifdef _OPENMP
+#pragma omp atomic
+#endif
+    n_used[g] += 1;
+    free(Kd); free(qd); free(c);
+  }
+  return used;
+}
+
+/* Stage 2 of Algorithm 1: the mean CA of FC i for KV head h is taken over every
+ * sample of the query heads that share h (they read the same keys, and the
+ * dominant part of the key cache is kept per KV head); I_dom(h) = the F FCs with
+ * the highest mean, a lower index first among equal means, returned ascending.
+ * mean_ca ([Hkv][n_fc], may be NULL) receives the means (0 where no sample). */
+void fasa_oracle_select_dominant(const int64_t* counts, const int64_t* n_used, int Hq,
+                                 int Hkv, int n_fc, int top_k, int F, int32_t* dom,
+                                 double* mean_ca) {
+  int group = Hq / Hkv;
+  for (int h = 0; h < Hkv; ++h) {
+    ranked_t* r = (ranked_t*)malloc(sizeof(ranked_t) * (size_t)n_fc);
+    int64_t samples = 0;
+    for (int g = h * group; g < (h + 1) * group; ++g) samples += n_used[g];
+    for (int i = 0; i < n_fc; ++i) {
+      int64_t sum = 0;
+      for (int g = h * group; g < (h + 1) * group; ++g) sum += counts[(int64_t)g * n_fc + i];
+      r[i].s = samples > 0 ? (double)sum / ((double)samples * (double)top_k) : 0.0;
+      r[i].j = i;
+      if (mean_ca) mean_ca[(int64_t)h * n_fc + i] = r[i].s;
+    }
+    qsort(r, (size_t)n_fc, sizeof(ranked_t), rank_cmp);
+    int* pick = (int*)malloc(sizeof(int) * (size_t)F);
+    for (int t = 0; t < F; ++t) pick[t] = r[t].j;
+    qsort(pick, (size_t)F, sizeof(int), int_cmp);
+    for (int t = 0; t < F; ++t) dom[(int64_t)h * F + t] = pick[t];
+    free(pick); free(r);
+  }
 }
 
 /* ------------------------------------------------- whole step on bf16 bits */

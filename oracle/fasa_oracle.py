@@ -34,7 +34,7 @@ def build(force: bool = False) -> str:
         if force or stale:
             tmp = _LIB + ".tmp.%d" % os.getpid()
             subprocess.check_call(
-                ["gcc", "-O2", "-std=c99", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"]
+                ["gcc", "-O2", "-std=c99", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"]
             )
             os.replace(tmp, _LIB)
     return _LIB
@@ -156,6 +156,51 @@ def attn_dense(q, K, V, L: int, scale: float):
                                    ctypes.c_int(d), ctypes.c_int(L), ctypes.c_double(scale),
                                    _ptr(O, _f64p), _ptr(lse, _f64p))
     return O, lse
+
+
+def ca_counts(q, K, top_k: int, pairing: int = 0, f32: bool = False) -> np.ndarray:
+    """top_k * CA of every FC for one query head (Sec. 3.3, Eq. 4): sizes of the
+    intersections of the full-head and single-FC top-k index sets."""
+    q, K = _f64(q), _f64(K)
+    L, d = K.shape
+    c = np.zeros(d // 2, dtype=np.int32)
+    _load().fasa_oracle_ca_counts(_ptr(q, _f64p), _ptr(K, _f64p), ctypes.c_int(L), ctypes.c_int(d),
+                                  ctypes.c_int(pairing), ctypes.c_int(top_k), ctypes.c_int(int(f32)),
+                                  _ptr(c, _i32p))
+    return c
+
+
+def calibrate_bf16(q_bits, K_bits, seq_lens, top_k: int, *, pairing=0, f32=True, n_threads=0,
+                   counts=None, n_used=None):
+    """Stage 1 of Algorithm 1 on bf16 bit patterns: adds every (sequence, query head) sample's
+    intersection counts to counts [Hq, d/2] and the sample count to n_used [Hq] (int64)."""
+    q_bits = np.ascontiguousarray(q_bits, dtype=np.uint16)
+    K_bits = np.ascontiguousarray(K_bits, dtype=np.uint16)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    B, Hq, d = q_bits.shape
+    _, Hkv, Lmax, _ = K_bits.shape
+    counts = np.zeros((Hq, d // 2), dtype=np.int64) if counts is None else counts
+    n_used = np.zeros(Hq, dtype=np.int64) if n_used is None else n_used
+    i64p = ctypes.POINTER(ctypes.c_int64)
+    _load().fasa_oracle_calibrate_bf16(
+        _ptr(q_bits, _u16p), _ptr(K_bits, _u16p), _ptr(seq_lens, _i32p), ctypes.c_int(B), ctypes.c_int(Hq),
+        ctypes.c_int(Hkv), ctypes.c_int(d), ctypes.c_int(Lmax), ctypes.c_int(pairing), ctypes.c_int(top_k),
+        ctypes.c_int(int(f32)), ctypes.c_int(n_threads), _ptr(counts, i64p), _ptr(n_used, i64p))
+    return counts, n_used
+
+
+def select_dominant(counts, n_used, n_kv_heads: int, top_k: int, n_dom: int):
+    """Stage 2 of Algorithm 1: (I_dom [Hkv, n_dom] ascending, mean CA [Hkv, d/2])."""
+    counts = np.ascontiguousarray(counts, dtype=np.int64)
+    n_used = np.ascontiguousarray(n_used, dtype=np.int64)
+    Hq, n_fc = counts.shape
+    dom = np.zeros((n_kv_heads, n_dom), dtype=np.int32)
+    mean = np.zeros((n_kv_heads, n_fc), dtype=np.float64)
+    i64p = ctypes.POINTER(ctypes.c_int64)
+    _load().fasa_oracle_select_dominant(_ptr(counts, i64p), _ptr(n_used, i64p), ctypes.c_int(Hq),
+                                        ctypes.c_int(n_kv_heads), ctypes.c_int(n_fc), ctypes.c_int(top_k),
+                                        ctypes.c_int(n_dom), _ptr(dom, _i32p), _ptr(mean, _f64p))
+    return dom, mean
 
 
 def decode_bf16(q_bits, K_bits, V_bits, seq_lens, dom, *, pairing=0, group_reduce=0, n_sink=0,

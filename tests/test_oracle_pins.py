@@ -399,6 +399,101 @@ def test_set_sharing_must_divide_the_group():
     assert np.array_equal(_decode(w, t, sel_heads=w.group)["idx"], _decode(w, t)["idx"])
 
 
+# --------------------------------- offline calibration (Algorithm 1, Eq. 4) ----
+
+def test_ca_hand_worked():
+    g = GOLD["scores"]
+    q, K = np.array(g["q"]), np.array(g["K"])
+    for f32 in (False, True):
+        assert O.ca_counts(q, K, 2, f32=f32).tolist() == GOLD["ca"]["top2_common"]
+        assert O.ca_counts(q, K, 1, f32=f32).tolist() == GOLD["ca"]["top1_common"]
+
+
+@pytest.mark.parametrize("pairing", [0, 1])
+def test_ca_matches_library_topk_and_python_sets(pairing):
+    rng = np.random.default_rng(77 + pairing)
+    L, d, k = 300, 128, 24
+    q, K = rng.standard_normal(d), rng.standard_normal((L, d))
+    got = O.ca_counts(q, K, k, pairing)
+    full = set(torch.topk(torch.from_numpy(K @ q), k).indices.tolist())
+    for i in range(d // 2):
+        c0, c1 = (i, i + d // 2) if pairing == 0 else (2 * i, 2 * i + 1)
+        a_i = torch.from_numpy(q[c0] * K[:, c0] + q[c1] * K[:, c1])
+        assert got[i] == len(full & set(torch.topk(a_i, k).indices.tolist())), i
+
+
+def test_ca_of_a_query_living_in_one_fc():
+    # q is zero outside FC 5: alpha equals alpha^(5) (CA = 1), every other alpha^(i) is all
+    # zeros, whose top-k is the first k positions by the tie rule
+    rng = np.random.default_rng(5)
+    L, d, k = 200, 128, 16
+    K = rng.standard_normal((L, d))
+    q = np.zeros(d)
+    q[5], q[5 + 64] = 1.5, -0.75
+    got = O.ca_counts(q, K, k)
+    assert got[5] == k
+    first = set(range(k))
+    top = set(torch.topk(torch.from_numpy(K @ q), k).indices.tolist())
+    assert all(got[i] == len(first & top) for i in range(64) if i != 5)
+
+
+def test_ca_binary32_path_equals_fp64_where_binary32_is_exact():
+    # small integers: every product and sum is exact in binary32, so both paths rank alike;
+    # many equal scores exercise the tie rule in both
+    rng = np.random.default_rng(9)
+    q = rng.integers(-3, 4, 128).astype(np.float64)
+    K = rng.integers(-3, 4, (150, 128)).astype(np.float64)
+    assert np.array_equal(O.ca_counts(q, K, 20, f32=True), O.ca_counts(q, K, 20, f32=False))
+
+
+def test_calibration_batch_accumulates_samples_and_skips_short_sequences():
+    w = synth.CONFIGS["c1"].replace(batch=3, max_len=400, len_lo=100, len_hi=400)
+    t = synth.make_inputs(w, "cpu")
+    t["seq_lens"] = torch.tensor([400, 32, 257], dtype=torch.int32)          # the middle one is too short for top-32
+    qb, kb = synth.bf16_bits(t["q"]), synth.bf16_bits(t["k"])
+    counts, used = O.calibrate_bf16(qb, kb, t["seq_lens"].numpy(), 32, f32=False, n_threads=2)
+    assert used.tolist() == [2] * w.n_q_heads
+    q64, k64 = t["q"].double().numpy(), t["k"].double().numpy()
+    for g in (0, 13, 31):
+        want = sum(O.ca_counts(q64[b, g], k64[b, g // w.group, :L], 32) for b, L in ((0, 400), (2, 257)))
+        assert np.array_equal(counts[g], want)
+    # a second call adds to the same arrays
+    O.calibrate_bf16(qb, kb, t["seq_lens"].numpy(), 32, f32=False, counts=counts, n_used=used)
+    assert used.tolist() == [4] * w.n_q_heads and np.array_equal(counts[13] // 2, counts[13] - counts[13] // 2)
+    assert counts.max() <= 4 * 32 and counts.min() >= 0
+
+
+def test_select_dominant_ranks_group_means_with_lower_index_first():
+    counts = np.zeros((4, 64), dtype=np.int64)                # 2 KV heads x 2 query heads
+    used = np.array([3, 1, 2, 2], dtype=np.int64)
+    counts[0, [7, 9, 20]] = [30, 10, 12]
+    counts[1, [9, 20, 40]] = [20, 18, 5]                      # KV head 0 sums: FC 7: 30, 9: 30, 20: 30, 40: 5
+    counts[2, 63] = 8
+    counts[3, [0, 63]] = [8, 1]                               # KV head 1 sums: FC 63: 9, 0: 8
+    dom, mean = O.select_dominant(counts, used, 2, top_k=10, n_dom=2)
+    assert dom.tolist() == [[7, 9], [0, 63]]                  # three-way tie keeps the two lowest indices
+    assert math.isclose(mean[0, 7], 30 / (4 * 10)) and math.isclose(mean[1, 63], 9 / (4 * 10)) and mean[0, 1] == 0.0
+    order = np.argsort(-counts[:2].sum(0), kind="stable")[:3]
+    assert sorted(order.tolist()) == O.select_dominant(counts, used, 2, 10, 3)[0][0].tolist()
+
+
+def test_calibration_recovers_planted_dominant_fcs():
+    # keys and queries whose energy sits in three FCs: those FCs decide the ranking, so their
+    # CA is the highest and Algorithm 1 returns exactly them
+    rng = np.random.default_rng(11)
+    B, Hq, Hkv, L, d = 2, 4, 2, 500, 128
+    planted = [3, 17, 40]
+    scale = np.ones(d)
+    for i in planted:
+        scale[[i, i + 64]] = 12.0
+    q = torch.from_numpy(rng.standard_normal((B, Hq, d)) * scale).to(torch.bfloat16)
+    K = torch.from_numpy(rng.standard_normal((B, Hkv, L, d)) * scale).to(torch.bfloat16)
+    counts, used = O.calibrate_bf16(synth.bf16_bits(q), synth.bf16_bits(K), np.array([L, L - 37], dtype=np.int32), 50)
+    dom, mean = O.select_dominant(counts, used, Hkv, 50, 3)
+    assert dom.tolist() == [planted, planted]
+    assert mean[:, planted].min() > 1.5 * np.delete(mean, planted, axis=1).max()
+
+
 def test_byte_model_fraction():
     # Sec. 4.4: fraction of KV bytes loaded = N_tip/d + N_fac/t.
     for F, k, L in ((16, 256, 32768), (8, 256, 4096), (64, 4096, 65536)):
