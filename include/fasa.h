@@ -260,6 +260,39 @@ int32_t fasa_decode_step_host(fasa_ctx_t* ctx, const void* q_host, const void* k
                               int32_t n_sel_max, float* scores, int32_t* idx, int32_t* n_sel,
                               float* out, float* out_host, void* workspace, void* stream);
 
+/* ---- offline calibration of the dominant FCs (Algorithm 1) ---------------- */
+
+/* Contextual agreement (Sec. 3.3, Eq. 4) of each FC i with the full head, for a batch laid
+ * out as for a decode step: a sample is a (sequence b, query head g) pair with
+ * seq_lens[b] > top_k (shorter sequences select every position and are skipped).  For each
+ * sample and each FC i the call adds
+ *     | TopK-I(alpha, top_k)  n  TopK-I(alpha^(i), top_k) |          ( = top_k * CA )
+ * to ca_counts[g][i] and 1 to n_used[g], where alpha^(i)[j] = q[c0(i)] K[j][c0(i)] +
+ * q[c1(i)] K[j][c1(i)] are the single-FC raw scores (Eq. 3) and alpha their sum over the
+ * 64 FCs, both in fp32 (alpha^(i) rounded once, alpha accumulated in ascending i); TopK-I
+ * ranks higher scores first and lower indices first among equal scores.
+ * q: bf16 [batch][n_q_heads][128]; k_cache as everywhere; ca_counts: int64
+ * [n_q_heads][64] and n_used: int64 [n_q_heads], device, 8-byte aligned, zeroed by the
+ * caller before the first call and carried from call to call (Stage 1 of Algorithm 1).
+ * workspace: fasa_calib_workspace_bytes(ctx, top_k) bytes = batch * n_q_heads * 65 *
+ * (max_len + top_k + 1) * 4 plus padding, 256-byte aligned.  The context's n_dom, sinks,
+ * budget and select_heads play no part.  Three kernels on `stream`, no synchronisation.
+ * UNSUPPORTED: top_k outside 1..min(max_len, 8192), batch * n_q_heads * 65 > 65535, or a
+ * max_len the cluster kernel cannot take (fasa_step_cluster_size() == 0). */
+int32_t fasa_calib_workspace_bytes(const fasa_ctx_t* ctx, int32_t top_k, size_t* out_bytes);
+int32_t fasa_calib_accumulate(fasa_ctx_t* ctx, const void* q, const void* k_cache,
+                              const int32_t* seq_lens, int32_t top_k, int64_t* ca_counts,
+                              int64_t* n_used, void* workspace, void* stream);
+
+/* Stage 2 of Algorithm 1, on the host (no GPU work): from counts and sample numbers copied
+ * back by the caller, the mean CA of FC i for KV head h over all samples of the query
+ * heads that share h, and I_dom(h) = the n_dom FCs with the highest mean (a lower index
+ * first among equal means), written ascending to dom_fc_host [n_kv_heads][n_dom] - the
+ * table fasa_create takes.  mean_ca_host (nullable): double [n_kv_heads][64]. */
+int32_t fasa_calib_select(int32_t n_q_heads, int32_t n_kv_heads, const int64_t* ca_counts_host,
+                          const int64_t* n_used_host, int32_t top_k, int32_t n_dom,
+                          int32_t* dom_fc_host, double* mean_ca_host);
+
 #ifdef __cplusplus
 }
 #endif

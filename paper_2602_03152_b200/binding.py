@@ -27,6 +27,7 @@ SYMBOLS = [
     "fasa_full_decode_attn", "fasa_decode_step", "fasa_stage_bytes", "fasa_decode_step_host",
     "fasa_sparse_decode_attn_static", "fasa_set_step_mode", "fasa_step_cluster_size",
     "fasa_append_decode_step", "fasa_proxy_bytes",
+    "fasa_calib_workspace_bytes", "fasa_calib_accumulate", "fasa_calib_select",
 ]
 
 
@@ -84,6 +85,9 @@ def load_library() -> ctypes.CDLL:
         "fasa_append_decode_step": (i32, [vp] * 8 + [i32, i32] + [vp] * 7),
         "fasa_stage_bytes": (i32, [vp, ctypes.POINTER(ctypes.c_size_t)]),
         "fasa_decode_step_host": (i32, [vp] * 9 + [i32, i32] + [vp] * 7),
+        "fasa_calib_workspace_bytes": (i32, [vp, i32, ctypes.POINTER(ctypes.c_size_t)]),
+        "fasa_calib_accumulate": (i32, [vp, vp, vp, vp, i32, vp, vp, vp, vp]),
+        "fasa_calib_select": (i32, [i32, i32, vp, vp, i32, i32, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -268,6 +272,20 @@ class Fasa:
             _dp(scores, torch.float32), _dp(idx, torch.int32), _dp(n_sel, torch.int32), _dp(out, torch.float32),
             _dp(lse), _dp(workspace), _stream()), "fasa_append_decode_step")
 
+    # -- offline calibration (Algorithm 1) ---------------------------------------
+    def calib_workspace_bytes(self, top_k: int) -> int:
+        out = ctypes.c_size_t()
+        self._check(self._lib.fasa_calib_workspace_bytes(self._h, top_k, ctypes.byref(out)), "fasa_calib_workspace_bytes")
+        return int(out.value)
+
+    def calib_accumulate(self, q, k_cache, seq_lens, top_k, ca_counts, n_used, workspace):
+        """Adds this batch's top_k * CA sums (Eq. 4) to ca_counts [n_q_heads, 64] and the sample
+        numbers to n_used [n_q_heads] (int64 CUDA tensors carried from call to call)."""
+        self._check(self._lib.fasa_calib_accumulate(self._h, _dp(q, torch.bfloat16), k_cache.data_ptr(),
+                                                    _dp(seq_lens, torch.int32), top_k, _dp(ca_counts, torch.int64),
+                                                    _dp(n_used, torch.int64), _dp(workspace), _stream()),
+                    "fasa_calib_accumulate")
+
     def decode_step_host(self, q_host, k_new_host, v_new_host, dev_stage, k_cache, v_cache, proxy_k, seq_lens,
                          budget, scores, idx, n_sel, out, out_host, workspace):
         """Host tensors in (pinned recommended), host tensor out; synchronises the stream."""
@@ -280,3 +298,19 @@ class Fasa:
             k_cache.data_ptr(), v_cache.data_ptr(), _dp(proxy_k), _dp(seq_lens, torch.int32), budget, n_sel_max,
             _dp(scores, torch.float32), _dp(idx, torch.int32), _dp(n_sel, torch.int32), _dp(out, torch.float32),
             out_host.data_ptr(), _dp(workspace), _stream()), "fasa_decode_step_host")
+
+
+def calib_select(ca_counts, n_used, n_kv_heads: int, top_k: int, n_dom: int):
+    """Stage 2 of Algorithm 1 on the host: (I_dom int32 [n_kv_heads, n_dom] ascending, mean CA
+    float64 [n_kv_heads, 64]) from the accumulated counts (any device; copied to the host)."""
+    lib = load_library()
+    counts = ca_counts.detach().to("cpu", torch.int64).contiguous()
+    used = n_used.detach().to("cpu", torch.int64).contiguous()
+    n_q_heads = counts.shape[0]
+    dom = torch.zeros((n_kv_heads, n_dom), dtype=torch.int32)
+    mean = torch.zeros((n_kv_heads, 64), dtype=torch.float64)
+    st = lib.fasa_calib_select(n_q_heads, n_kv_heads, counts.data_ptr(), used.data_ptr(), top_k, n_dom,
+                               dom.data_ptr(), mean.data_ptr())
+    if st != OK:
+        raise FasaError(st, "fasa_calib_select", lib.fasa_status_string(st).decode())
+    return dom, mean

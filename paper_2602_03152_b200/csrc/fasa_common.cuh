@@ -75,6 +75,10 @@ int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t
                                int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
                                cudaStream_t stream);
 
+int32_t fasa_fused_topk_rows(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
+                             int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
+                             int rows_per_seq, int n_sink, int n_recent, cudaStream_t stream);
+
 static inline size_t fasa_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 #ifdef __CUDACC__

@@ -862,17 +862,27 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
 int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
                                int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
                                cudaStream_t stream) {
+  return fasa_fused_topk_rows(ctx, scores, seq_lens, budget, n_sel_max, idx, n_sel, ctx->n_sets,
+                              ctx->cfg.n_sink, ctx->cfg.n_recent, stream);
+}
+
+// TopK-I over rows_per_seq score rows per sequence (row r of the buffer belongs to sequence
+// r / rows_per_seq), with the given forced positions instead of the context's.
+int32_t fasa_fused_topk_rows(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
+                             int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
+                             int rows_per_seq, int n_sink, int n_recent, cudaStream_t stream) {
   const fasa_config_t& c = ctx->cfg;
   FusedParams p;
   memset(&p, 0, sizeof(p));
   p.seq_lens = seq_lens; p.scores = const_cast<float*>(scores); p.idx = idx; p.n_sel = n_sel;
   p.status = ctx->d_status;
-  p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.n_sets = ctx->n_sets; p.group = ctx->sel_heads; p.max_len = c.max_len;
-  p.chunks = ctx->chunks; p.n_sink = c.n_sink; p.n_recent = c.n_recent; p.budget = budget;
+  // (the select-only form uses the unit index for its score row and its sequence alone)
+  p.n_q_heads = rows_per_seq; p.n_kv_heads = 1; p.n_sets = rows_per_seq; p.group = 1; p.max_len = c.max_len;
+  p.chunks = ctx->chunks; p.n_sink = n_sink; p.n_recent = n_recent; p.budget = budget;
   p.n_sel_max = n_sel_max;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3((unsigned)ctx->fused_cs, (unsigned)(c.batch * ctx->n_sets), 1);
+  cfg.gridDim = dim3((unsigned)ctx->fused_cs, (unsigned)(c.batch * rows_per_seq), 1);
   cfg.blockDim = dim3(kFT, 1, 1);
   cfg.dynamicSmemBytes = ctx->fused_smem;
   cfg.stream = stream;

@@ -77,3 +77,24 @@ def test_create_rejects_bad_fc_lists_and_nulls(lib):
     assert lib.fasa_fc_score(None, None, None, None, None, None) == binding.ERR_INVALID_ARG
     assert lib.fasa_topk(None, None, None, 1, 1, None, None, None, None) == binding.ERR_INVALID_ARG
     assert lib.fasa_launch_count(None) == 0
+
+
+def test_calib_select_is_host_only_and_agrees_with_the_oracle(lib):
+    # Stage 2 of Algorithm 1 runs on the host: random counts with many equal sums (ties keep
+    # the lower FC), compared with the oracle's separate statement of the same rule
+    import numpy as np
+    import torch
+    from oracle import fasa_oracle as O
+    rng = np.random.default_rng(3)
+    Hq, Hkv, top_k = 28, 4, 64
+    counts = rng.integers(0, 6, (Hq, 64)).astype(np.int64) * 10
+    used = rng.integers(1, 5, Hq).astype(np.int64)
+    for n_dom in (1, 16, 63, 64):
+        dom, mean = binding.calib_select(torch.from_numpy(counts), torch.from_numpy(used), Hkv, top_k, n_dom)
+        dom_or, mean_or = O.select_dominant(counts, used, Hkv, top_k, n_dom)
+        assert np.array_equal(dom.numpy(), dom_or)
+        assert np.allclose(mean.numpy(), mean_or, rtol=1e-15, atol=0)
+    with pytest.raises(binding.FasaError):
+        binding.calib_select(torch.from_numpy(counts), torch.from_numpy(used), Hkv, top_k, 65)
+    with pytest.raises(binding.FasaError):
+        binding.calib_select(torch.from_numpy(counts), torch.from_numpy(used), 5, top_k, 4)

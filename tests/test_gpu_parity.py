@@ -371,6 +371,80 @@ def test_index_sets_per_query_head_large_selection_and_static_scratch():
     assert r.fasa.device_status() == 0
 
 
+# ---- offline calibration (Algorithm 1; CA of Eq. 4): integer counts, bit-exact ----
+
+def _calib(w, t, top_k, calls=1):
+    f = binding.Fasa.from_workload(w, t["dom"])
+    q, k, lens = t["q"].cuda(), t["k"].cuda(), t["seq_lens"].cuda()
+    counts = torch.zeros((w.n_q_heads, 64), dtype=torch.int64, device="cuda")
+    used = torch.zeros(w.n_q_heads, dtype=torch.int64, device="cuda")
+    ws = torch.empty(f.calib_workspace_bytes(top_k), dtype=torch.uint8, device="cuda")
+    for _ in range(calls):
+        n0 = f.launch_count()
+        f.calib_accumulate(q, k, lens, top_k, counts, used, ws)
+        assert f.launch_count() == n0 + 3
+    torch.cuda.synchronize()
+    assert f.device_status() == 0
+    c_or, u_or = O.calibrate_bf16(synth.bf16_bits(t["q"]), synth.bf16_bits(t["k"]), t["seq_lens"].numpy(), top_k,
+                                  pairing=w.pairing, f32=True)
+    return counts.cpu().numpy(), used.cpu().numpy(), c_or, u_or
+
+
+@pytest.mark.parametrize("cfg,kw,top_k", [
+    ("c0", dict(), 256),                                                            # config 0 at full size
+    ("c1", dict(batch=2, max_len=3001, len_lo=1500, len_hi=3001), 100),            # ragged, tail tile
+    ("c3", dict(batch=2, max_len=1500, len_lo=900, len_hi=1400), 33),              # group of 7, no RoPE
+    ("c1", dict(batch=1, max_len=2048, len_lo=2048, len_hi=2048, pairing=1), 1),   # interleaved pairing, top-1
+    ("c1", dict(batch=1, n_q_heads=4, n_kv_heads=1, max_len=20000, len_lo=20000, len_hi=20000), 4096),
+])
+def test_calibration_counts_match_the_oracle(cfg, kw, top_k):
+    w = C[cfg].replace(**kw)
+    t = synth.make_inputs(w, "cpu")
+    counts, used, c_or, u_or = _calib(w, t, top_k)
+    assert np.array_equal(used, u_or) and used.min() >= 1
+    assert np.array_equal(counts, c_or)
+    assert counts.max() <= used.max() * top_k
+
+
+def test_calibration_accumulates_and_skips_short_sequences():
+    w = C["c1"].replace(batch=3, n_q_heads=8, n_kv_heads=2, max_len=700, len_lo=100, len_hi=700)
+    t = synth.make_inputs(w, "cpu")
+    t["seq_lens"] = torch.tensor([700, 64, 0], dtype=torch.int32)      # 64 == top_k and 0: not samples
+    counts, used, c_or, u_or = _calib(w, t, 64, calls=2)
+    assert used.tolist() == [2] * 8 and np.array_equal(counts, 2 * c_or) and np.array_equal(u_or, [1] * 8)
+
+
+def test_calibration_end_to_end_recovers_planted_fcs_and_feeds_create():
+    # the planted-energy case of the oracle's pin, on the GPU, through Stage 2 into fasa_create
+    rng = np.random.default_rng(11)
+    w = C["c1"].replace(batch=2, n_q_heads=4, n_kv_heads=2, max_len=500, len_lo=500, len_hi=500, n_dom=3)
+    planted = [3, 17, 40]
+    scale = np.ones(128)
+    for i in planted:
+        scale[[i, i + 64]] = 12.0
+    t = {"q": torch.from_numpy(rng.standard_normal((2, 4, 128)) * scale).to(torch.bfloat16),
+         "k": torch.from_numpy(rng.standard_normal((2, 2, 500, 128)) * scale).to(torch.bfloat16),
+         "seq_lens": torch.tensor([500, 463], dtype=torch.int32), "dom": torch.tensor([[0, 1, 2], [0, 1, 2]], dtype=torch.int32)}
+    counts, used, c_or, u_or = _calib(w, t, 50)
+    assert np.array_equal(counts, c_or) and np.array_equal(used, u_or)
+    dom, mean = binding.calib_select(torch.from_numpy(counts), torch.from_numpy(used), 2, 50, 3)
+    assert dom.tolist() == [planted, planted]
+    assert np.array_equal(dom.numpy(), O.select_dominant(c_or, u_or, 2, 50, 3)[0])
+    binding.Fasa.from_workload(w, dom).close()
+
+
+def test_calibration_rejects_what_it_cannot_take():
+    w = C["c1"].replace(batch=32, max_len=512, len_lo=512, len_hi=512)           # 32 * 32 * 65 > 65535 grid rows
+    f = binding.Fasa.from_workload(w, synth.dominant_fcs(w))
+    with pytest.raises(binding.FasaError) as e:
+        f.calib_workspace_bytes(16)
+    assert e.value.status == binding.ERR_UNSUPPORTED
+    g = binding.Fasa.from_workload(w.replace(batch=1), synth.dominant_fcs(w))
+    for bad in (0, 513, -3):
+        with pytest.raises(binding.FasaError):
+            g.calib_workspace_bytes(bad)
+
+
 def test_strided_token_major_cache():
     # K/V stored [B][L][Hkv][128] (token-major), addressed through the stride fields.
     w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, batch=2, max_len=640, len_lo=400, len_hi=640, budget=40)
