@@ -462,6 +462,65 @@ def run_sweep(args):
                       "peak_source": peak_src, "steps_per_point": args.sweep_steps, "rows": rows}), flush=True)
 
 
+def run_calib(args):
+    """Offline calibration (Algorithm 1) on the Llama-3-8B shape of workload c1: one call =
+    batch x query heads samples (per-FC and full raw scores, 65 top-k selections each,
+    intersection counts).  One JSON object: time per call, samples per second, the bytes the
+    three kernels move and the oracle's time for one sample on the host."""
+    import time
+
+    import numpy as np
+    import torch
+
+    from oracle import fasa_oracle as O
+    from paper_2602_03152_b200 import binding, build, synth
+
+    build.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    w = synth.CONFIGS[args.config]
+    if args.batch is not None:
+        w = w.replace(batch=args.batch)
+    top_k = args.budget if args.budget is not None else 256
+    t = synth.make_inputs(w, dev)
+    f = binding.Fasa.from_workload(w, t["dom"])
+    counts = torch.zeros((w.n_q_heads, 64), dtype=torch.int64, device=dev)
+    used = torch.zeros(w.n_q_heads, dtype=torch.int64, device=dev)
+    ws = torch.empty(f.calib_workspace_bytes(top_k), dtype=torch.uint8, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    ts = []
+    for i in range(args.warmup + args.steps):
+        flush.fill_(i & 1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        f.calib_accumulate(t["q"], t["k"], t["seq_lens"], top_k, counts, used, ws)
+        b.record()
+        b.synchronize()
+        if i >= args.warmup:
+            ts.append(a.elapsed_time(b) * 1e3)
+    us = float(np.mean(ts))
+    samples = int(sum(1 for l in t["seq_lens"].tolist() if l > top_k)) * w.n_q_heads
+    tokens = int(sum(t["seq_lens"].tolist()))
+    # K rows once per KV head (query heads of a group re-read them from L2), 65 fp32 score rows
+    # per sample written and read once, 65 index lists written and read once
+    by = tokens * w.n_kv_heads * 256 + 2 * tokens * w.n_q_heads * 65 * 4 + 2 * samples * 65 * top_k * 4
+    peak, peak_src = _peaks()
+    # the oracle on one sample (sequence 0, query head 0), as it stands
+    q0 = t["q"][0, 0].double().cpu().numpy()
+    k0 = t["k"][0, 0, :int(t["seq_lens"][0])].double().cpu().numpy()
+    t0 = time.perf_counter()
+    c_or = O.ca_counts(q0, k0, top_k, w.pairing, f32=True)
+    cpu_s = time.perf_counter() - t0
+    got = (counts[0].cpu().numpy() // max(1, args.warmup + args.steps)) if w.batch == 1 else None
+    print(json.dumps({"calibration": w.name, "top_k": top_k, "samples_per_call": samples, "us_per_call": us,
+                      "samples_per_s": samples / us * 1e6, "bytes_per_call": by, "gbs": by / us / 1e3,
+                      "frac_of_peak": by / us / 1e3 / peak, "peak_source": peak_src,
+                      "workspace_bytes": int(ws.numel()), "launches_per_call": 3, "steps": args.steps,
+                      "oracle_s_per_sample": cpu_s, "oracle_samples_per_s": 1.0 / cpu_s,
+                      "counts_match_oracle_sample": None if got is None else bool(np.array_equal(got, c_or)),
+                      "device_status": f.device_status()}), flush=True)
+
+
 def run_longcot(args):
     """Workload c3 (long-CoT shape, Qwen2.5-7B-like attention): 28 layers, batch 32, prompt
     1024 then 15360 decode steps, budget 18.9 % of the current length, 16 dominant FCs.  One
@@ -552,6 +611,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="config 4 grid (budget x dominant FCs) instead of the bench line")
     ap.add_argument("--longcot", action="store_true", help="config 3 (long-CoT decode) instead of the bench line")
+    ap.add_argument("--calib", action="store_true",
+                    help="offline calibration (Algorithm 1) on --config's shape instead of the bench line; --budget = top-k")
     ap.add_argument("--sweep-steps", type=int, default=20)
     ap.add_argument("--step-mode", type=int, default=None, choices=[0, 1],
                     help="0: fasa_decode_step as three kernels; 1 (default): one cluster kernel where available")
@@ -561,6 +622,8 @@ def main():
         return run_sweep(args)
     if args.longcot:
         return run_longcot(args)
+    if args.calib:
+        return run_calib(args)
     from paper_2602_03152_b200 import synth
     w = synth.CONFIGS[args.config]
     if args.budget is not None:

@@ -880,15 +880,24 @@ int32_t fasa_fused_topk_rows(fasa_ctx* ctx, const float* scores, const int32_t* 
   p.n_q_heads = rows_per_seq; p.n_kv_heads = 1; p.n_sets = rows_per_seq; p.group = 1; p.max_len = c.max_len;
   p.chunks = ctx->chunks; p.n_sink = n_sink; p.n_recent = n_recent; p.budget = budget;
   p.n_sel_max = n_sel_max;
+  // The context's cluster size suits its own number of rows (few rows: wide clusters, so the
+  // whole GPU works on them).  A launch with many more rows takes the narrowest cluster that
+  // holds a row's keys: more rows are then resident at once.
+  int cs = ctx->fused_cs;
+  auto cap_of = [&](int n) { return (((c.max_len + n - 1) / n) + 31) & ~31; };
+  if (rows_per_seq > ctx->n_sets) {
+    cs = 1;
+    while (cs < ctx->fused_cs && cap_of(cs) > kCapPair) cs *= 2;
+  }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3((unsigned)ctx->fused_cs, (unsigned)(c.batch * rows_per_seq), 1);
+  cfg.gridDim = dim3((unsigned)cs, (unsigned)(c.batch * rows_per_seq), 1);
   cfg.blockDim = dim3(kFT, 1, 1);
-  cfg.dynamicSmemBytes = ctx->fused_smem;
+  cfg.dynamicSmemBytes = cs == ctx->fused_cs ? ctx->fused_smem : fused_smem_bytes(cap_of(cs));
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)ctx->fused_cs;
+  attr[0].val.clusterDim.x = (unsigned)cs;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
