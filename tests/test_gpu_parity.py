@@ -445,6 +445,45 @@ def test_calibration_rejects_what_it_cannot_take():
             g.calib_workspace_bytes(bad)
 
 
+def test_decode_loop_replays_from_a_cuda_graph():
+    # a serving loop captures its steps once and replays them: three append+step calls (one
+    # launch each) and a dense call in one graph; nothing in a call allocates or synchronises,
+    # and the lengths advance on the device, so a replay continues where the last one ended
+    w = C["c1"].replace(batch=2, max_len=1200, len_lo=700, len_hi=1100)
+    t = synth.make_inputs(w, "cpu")
+    eager, graphed = Run(w, t), Run(w, {k_: (v_.clone() if torch.is_tensor(v_) else v_) for k_, v_ in t.items()})
+    steps = [synth.make_step_inputs(w, i, "cuda") for i in range(3)]
+    outs_e = [torch.zeros_like(eager.out) for _ in steps]
+    outs_g = [torch.zeros_like(eager.out) for _ in steps]
+    for r in (eager, graphed):
+        r.build_proxy()
+    torch.cuda.synchronize()
+
+    def run(r, outs):
+        for s_, o in zip(steps, outs):
+            r.fasa.append_decode_step(s_["q"], s_["k_new"], s_["v_new"], r.k, r.v, r.proxy, r.seq_lens, w.budget,
+                                      None, r.idx, r.n_sel, o, None)
+        r.fasa.full_decode_attn(steps[-1]["q"], r.k, r.v, r.seq_lens, r.dense, r.ws)
+
+    g = torch.cuda.CUDAGraph()
+    n0 = graphed.fasa.launch_count()
+    with torch.cuda.graph(g):
+        run(graphed, outs_g)
+    assert graphed.fasa.launch_count() - n0 == 3 + 2
+    for rounds in range(2):
+        g.replay()
+        run(eager, outs_e)
+        torch.cuda.synchronize()
+        for x, y in ((eager.k, graphed.k), (eager.v, graphed.v), (eager.proxy, graphed.proxy),
+                     (eager.seq_lens, graphed.seq_lens), (eager.idx, graphed.idx), (eager.n_sel, graphed.n_sel),
+                     (eager.dense, graphed.dense)):
+            assert torch.equal(x, y)
+        for x, y in zip(outs_e, outs_g):
+            assert torch.equal(x, y)
+    assert graphed.seq_lens.cpu().tolist() == [int(l) + 6 for l in t["seq_lens"].tolist()]
+    assert graphed.fasa.device_status() == 0
+
+
 def test_strided_token_major_cache():
     # K/V stored [B][L][Hkv][128] (token-major), addressed through the stride fields.
     w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, batch=2, max_len=640, len_lo=400, len_hi=640, budget=40)
