@@ -521,6 +521,84 @@ def run_calib(args):
                       "device_status": f.device_status()}), flush=True)
 
 
+def _longcot_resident(w, samples, reps, dev, n_layers=28):
+    """All 28 layers of workload c3 resident at once (their own random bf16 K/V caches, proxies and
+    dominant-FC tables, about 32 GB), one decode step of the whole stack = 28 append+step
+    calls captured in a CUDA graph, a second graph for the dense stack; both replayed at the
+    sampled cache lengths.  The lengths are device data, so one capture could serve them all;
+    a serving loop knows its step count, though, and passes the selection bound of the current
+    length (n_sel_max = ceil(0.189 L)), which lets the library attend inside the cluster kernel
+    while selections are small: one capture per sampled length, as a loop with length buckets
+    would hold.  No L2 flush: 28 layers of cache stream through L2 between two visits of a layer."""
+    import torch
+
+    from paper_2602_03152_b200 import binding, synth
+
+    B, Hq, Hkv, Lm = w.batch, w.n_q_heads, w.n_kv_heads, w.max_len
+    n_sel_max = w.n_sel_max()
+    lens_all = torch.zeros((n_layers, B), dtype=torch.int32, device=dev)
+    full = torch.full((B,), Lm, dtype=torch.int32, device=dev)
+    layers = []
+    for l in range(n_layers):
+        wl = w.replace(index=w.index + 1000 * (l + 1))              # every layer its own seed
+        t = synth.make_inputs(wl.replace(len_lo=Lm, len_hi=Lm), dev)
+        s = synth.make_step_inputs(wl, 0, dev)
+        f = binding.Fasa.from_workload(wl, t["dom"])
+        proxy = f.alloc_proxy(dev)
+        f.proxy_build(t["k"], proxy, full)
+        layers.append(dict(f=f, k=t["k"], v=t["v"], proxy=proxy, lens=lens_all[l], q=s["q"], kn=s["k_new"], vn=s["v_new"],
+                           idx=torch.zeros(B * w.n_sets * n_sel_max, dtype=torch.int32, device=dev),
+                           n_sel=torch.zeros((B, w.n_sets), dtype=torch.int32, device=dev),
+                           out=torch.zeros((B, Hq, 128), dtype=torch.float32, device=dev),
+                           ws=f.alloc_workspace(n_sel_max, dev)))
+    torch.cuda.synchronize()
+
+    def fasa_stack(n_bound):
+        for y in layers:
+            idx = y["idx"][:B * w.n_sets * n_bound].view(B, w.n_sets, n_bound)
+            y["f"].append_decode_step(y["q"], y["kn"], y["vn"], y["k"], y["v"], y["proxy"], y["lens"], w.budget, None,
+                                      idx, y["n_sel"], y["out"], y["ws"])
+
+    def dense_stack():
+        for y in layers:
+            y["f"].kv_append(y["k"], y["v"], y["proxy"], y["lens"], y["kn"], y["vn"])
+            y["f"].full_decode_attn(y["q"], y["k"], y["v"], y["lens"], y["out"], y["ws"])
+
+    def capture(fn):
+        lens_all.fill_(1024)
+        n0 = sum(y["f"].launch_count() for y in layers)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        return g, sum(y["f"].launch_count() for y in layers) - n0
+
+    dense_graph = capture(dense_stack)
+    pts = []
+    for L in samples:
+        n_bound = min(n_sel_max, (-w.budget * L + 999) // 1000 + w.n_sink + w.n_recent) if w.budget < 0 else n_sel_max
+        row = {"context": L, "n_sel_max_passed": n_bound}
+        for name, (g, launches) in (("fasa", capture(lambda: fasa_stack(n_bound))), ("dense", dense_graph)):
+            ts = []
+            for i in range(reps + 2):
+                lens_all.fill_(L - 1)                               # every step appends at row L-1
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                g.replay()
+                b.record()
+                b.synchronize()
+                if i >= 2:
+                    ts.append(a.elapsed_time(b) * 1e3)
+            row[name + "_us_per_token_step"] = sum(ts) / len(ts)
+            row[name + "_launches"] = launches
+        row["n_sel_per_unit"] = float(layers[0]["n_sel"].float().mean().item())
+        row["speedup_vs_dense"] = row["dense_us_per_token_step"] / row["fasa_us_per_token_step"]
+        pts.append(row)
+    status = 0
+    for y in layers:
+        status |= y["f"].device_status()
+    return pts, status
+
+
 def run_longcot(args):
     """Workload c3 (long-CoT shape, Qwen2.5-7B-like attention): 28 layers, batch 32, prompt
     1024 then 15360 decode steps, budget 18.9 % of the current length, 16 dominant FCs.  One
@@ -547,25 +625,36 @@ def run_longcot(args):
                     "device_status": sm["device_status"]})
         del m
 
-    def total(key):
-        acc, n_layers = 0.0, 28
+    def total(points, key, n_layers):
+        acc = 0.0
         for L in range(1025, 16385):              # cache length after each of the 15360 appends
             j = max(i for i, s_ in enumerate(samples) if s_ <= L)
             if j == len(samples) - 1:
-                v = pts[j][key]
+                v = points[j][key]
             else:
                 a, b = samples[j], samples[j + 1]
-                v = pts[j][key] + (pts[j + 1][key] - pts[j][key]) * (L - a) / (b - a)
+                v = points[j][key] + (points[j + 1][key] - points[j][key]) * (L - a) / (b - a)
             acc += v * n_layers
         return acc * 1e-6
 
-    tf, td = total("us_per_step"), total("dense_us_per_step")
-    print(json.dumps({"longcot": w.name, "layers": 28, "batch": w.batch, "prompt": 1024, "decode_steps": 15360,
-                      "budget_permille": -w.budget, "n_dom": w.n_dom, "steps_per_sample": args.sweep_steps,
-                      "fasa_decode_attention_seconds": tf, "dense_decode_attention_seconds": td,
-                      "speedup_vs_dense": td / tf, "theory_byte_ratio": 1.0 / (w.n_dom / 128.0 + 0.189),
-                      "method": "one layer timed at the sampled contexts, linear interpolation, x 28 layers",
-                      "samples": pts}), flush=True)
+    tf, td = total(pts, "us_per_step", 28), total(pts, "dense_us_per_step", 28)
+    res = {"longcot": w.name, "layers": 28, "batch": w.batch, "prompt": 1024, "decode_steps": 15360,
+           "budget_permille": -w.budget, "n_dom": w.n_dom, "steps_per_sample": args.sweep_steps,
+           "fasa_decode_attention_seconds": tf, "dense_decode_attention_seconds": td,
+           "speedup_vs_dense": td / tf, "theory_byte_ratio": 1.0 / (w.n_dom / 128.0 + 0.189),
+           "method": "one layer timed at the sampled contexts (L2 flushed before each step), linear interpolation, x 28 layers",
+           "samples": pts}
+    del t
+    free, _ = torch.cuda.mem_get_info()
+    if free > (48 << 30) and not args.no_resident:
+        rp, status = _longcot_resident(w, samples, max(3, args.sweep_steps // 2), dev)
+        rf, rd = total(rp, "fasa_us_per_token_step", 1), total(rp, "dense_us_per_token_step", 1)
+        res["resident_stack"] = {
+            "method": "28 layers resident (own caches, ~32 GB), one token step of the whole stack replayed from a CUDA "
+                      "graph at the sampled contexts, no L2 flush, linear interpolation over the 15360 steps",
+            "fasa_decode_attention_seconds": rf, "dense_decode_attention_seconds": rd, "speedup_vs_dense": rd / rf,
+            "device_status": status, "samples": rp}
+    print(json.dumps(res), flush=True)
 
 
 def cpu_baseline(w, t, by):
@@ -613,6 +702,7 @@ def main():
     ap.add_argument("--longcot", action="store_true", help="config 3 (long-CoT decode) instead of the bench line")
     ap.add_argument("--calib", action="store_true",
                     help="offline calibration (Algorithm 1) on --config's shape instead of the bench line; --budget = top-k")
+    ap.add_argument("--no-resident", action="store_true", help="--longcot: skip the 28-layer resident measurement")
     ap.add_argument("--sweep-steps", type=int, default=20)
     ap.add_argument("--step-mode", type=int, default=None, choices=[0, 1],
                     help="0: fasa_decode_step as three kernels; 1 (default): one cluster kernel where available")

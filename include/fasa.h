@@ -224,7 +224,11 @@ int32_t fasa_sparse_decode_attn_static(fasa_ctx_t* ctx, const void* q, const voi
  * tensor-core kernel of fasa_sparse_decode_attn (three launches instead of one).
  * Mode 0, and every configuration mode 1 cannot take: fasa_fc_score -> fasa_topk ->
  * fasa_sparse_decode_attn; scores and workspace are then required (INVALID_ARG if NULL).
- * Both modes select identical index sets; outputs agree to fp32 rounding. */
+ * Both modes select identical index sets; outputs agree to fp32 rounding.
+ * n_sel_max is also the bound the launch shapes are planned with (route, split count): a
+ * caller that knows the current lengths should pass the tightest bound it can (e.g.
+ * ceil(0.189 * L) + n_sink + n_recent for a permille budget) rather than the bound at
+ * max_len; idx is addressed with whatever n_sel_max is passed as its row stride. */
 int32_t fasa_set_step_mode(fasa_ctx_t* ctx, int32_t mode);
 /* (The mode also selects the kernel behind fasa_topk: the cluster kernel's selection phases
  * in mode 1, a register-resident cluster kernel in mode 0; the results are identical.) */
