@@ -24,6 +24,17 @@
  *     (or the strides in fasa_config_t), keys stored post-RoPE at their
  *     absolute positions.  q: [batch][n_q_heads][128] bf16, post-RoPE; query
  *     head g belongs to KV head g / (n_q_heads / n_kv_heads).
+ *   - Where the caches live.  k_cache and v_cache (not proxy_k) may instead be page-locked
+ *     host memory that the device can address (cudaHostAlloc / cudaHostRegister under
+ *     unified addressing): this is the memory-optimised variant of the method (FASA-M,
+ *     Algorithm 2), which keeps only the dominant part of the key cache - here the proxy-K
+ *     buffer - on the GPU.  Every call works unchanged: scoring and selection run on the
+ *     GPU-resident proxy, the attention kernels fetch just the selected K/V rows across
+ *     the host link by index (no host-side gather, no staging copy), and the append calls
+ *     store the new rows there.  GPU memory per cached token drops from 512 bytes to
+ *     proxy_row_elems * 2 (64 at n_dom = 16); a step then moves n_sel * 512 bytes per
+ *     (batch, KV head) over the link, which bounds it.  The dense path over host-resident
+ *     caches streams the whole cache over the link and is only useful as a reference.
  *   - Frequency chunk (FC) i, 0 <= i < 64, is the channel pair (i, i+64) with
  *     rope_pairing 0 (rotate-half layout) or (2i, 2i+1) with rope_pairing 1
  *     (the paper's Eq. 1 layout).  An FC is never split (Appendix, design choices).

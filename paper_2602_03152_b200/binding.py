@@ -208,6 +208,12 @@ class Fasa:
     def alloc_workspace(self, n_sel_max: int, device="cuda") -> torch.Tensor:
         return torch.empty(self.workspace_bytes(n_sel_max), dtype=torch.uint8, device=device)
 
+    def alloc_host_cache(self) -> torch.Tensor:
+        """A K or V cache [batch, n_kv_heads, max_len, 128] (bf16) in page-locked host memory
+        that the kernels address directly: the cache placement of FASA-M (Algorithm 2).  Pass it
+        wherever a call takes k_cache / v_cache."""
+        return torch.zeros((self.batch, self.n_kv_heads, self.max_len, 128), dtype=torch.bfloat16).pin_memory()
+
     # -- the calls of include/fasa.h --------------------------------------------
     def kv_append(self, k_cache, v_cache, proxy_k, seq_lens, k_new, v_new):
         n_new = k_new.shape[2]

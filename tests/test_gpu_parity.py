@@ -484,6 +484,48 @@ def test_decode_loop_replays_from_a_cuda_graph():
     assert graphed.fasa.device_status() == 0
 
 
+def test_fasa_m_caches_in_pinned_host_memory():
+    # Algorithm 2 (the memory-optimised variant): only the dominant part of the key cache - the
+    # proxy - lives on the GPU; K and V sit in page-locked host memory, the attention kernels
+    # fetch the selected rows over the host link and the append calls store new rows there.
+    # Same kernels, same bits: every result must equal the device-resident run exactly.
+    w = C["c3"].replace(batch=2, max_len=3000, len_lo=1400, len_hi=2900)
+    t = synth.make_inputs(w, "cpu")
+    dev = Run(w, t, n_sel_max=1300)
+    host = Run(w, {k_: (v_.clone() if torch.is_tensor(v_) else v_) for k_, v_ in t.items()}, n_sel_max=1300)
+    kh, vh = host.fasa.alloc_host_cache(), host.fasa.alloc_host_cache()
+    assert kh.is_pinned() and not kh.is_cuda
+    kh.copy_(t["k"]); vh.copy_(t["v"])
+    host.k, host.v = kh, vh
+    for r in (dev, host):
+        r.build_proxy()                                        # Split of the whole cache, read over the link
+    assert torch.equal(dev.proxy, host.proxy)
+    bulk = synth.make_step_inputs(w.replace(index=w.index + 5), 0, "cuda")
+    kb, vb = bulk["k_new"].repeat(1, 1, 3, 1).contiguous(), bulk["v_new"].repeat(1, 1, 3, 1).contiguous()
+    for r in (dev, host):
+        r.fasa.kv_append(r.k, r.v, r.proxy, r.seq_lens, kb, vb)           # three rows at once
+    for step, ws in enumerate((None, "ws", None)):             # one launch / split-K route / one launch
+        s = synth.make_step_inputs(w, step, "cuda")
+        for r in (dev, host):
+            r.fasa.append_decode_step(s["q"], s["k_new"], s["v_new"], r.k, r.v, r.proxy, r.seq_lens, -400 if ws else w.budget,
+                                      r.scores, r.idx, r.n_sel, r.out, r.ws if ws else None, r.lse)
+        torch.cuda.synchronize()
+        for x, y in ((dev.proxy, host.proxy), (dev.seq_lens, host.seq_lens), (dev.scores, host.scores),
+                     (dev.idx, host.idx), (dev.n_sel, host.n_sel), (dev.out, host.out), (dev.lse, host.lse)):
+            assert torch.equal(x, y)
+    host.dense_step(); dev.dense_step()
+    assert torch.equal(dev.dense, host.dense)
+    # the host tensors themselves now hold the appended rows
+    assert torch.equal(dev.k.cpu(), kh) and torch.equal(dev.v.cpu(), vh)
+    lens = dev.seq_lens.cpu().tolist()
+    assert lens == [int(l) + 6 for l in t["seq_lens"].tolist()]
+    parity.check_step(s["q"].cpu().double().numpy(), kh.double().numpy(), vh.double().numpy(), lens,
+                      np.sort(host.dom.numpy(), axis=1), scores=host.scores.cpu().numpy(), idx=host.idx.cpu().numpy(),
+                      n_sel=host.n_sel.cpu().numpy(), out=host.out.cpu().numpy(),
+                      what="caches in host memory", **host.oracle_kwargs())
+    assert host.fasa.device_status() == 0
+
+
 def test_strided_token_major_cache():
     # K/V stored [B][L][Hkv][128] (token-major), addressed through the stride fields.
     w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, batch=2, max_len=640, len_lo=400, len_hi=640, budget=40)
