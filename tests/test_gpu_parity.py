@@ -2,6 +2,7 @@
 element on the same seeded bf16 inputs.  Index sets are bit-exact outside a 1e-3-relative
 tie band; attention is within max-abs 2e-3; scores within 1e-5 of sum |q_c k_c|."""
 import math
+import os
 
 import numpy as np
 import pytest
@@ -524,6 +525,33 @@ def test_fasa_m_caches_in_pinned_host_memory():
                       n_sel=host.n_sel.cpu().numpy(), out=host.out.cpu().numpy(),
                       what="caches in host memory", **host.oracle_kwargs())
     assert host.fasa.device_status() == 0
+
+
+def _random_workloads(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        hkv = int(rng.integers(1, 4))
+        g = int(rng.choice([1, 2, 3, 4, 6, 7, 8]))
+        sel = int(rng.choice([d for d in range(1, g + 1) if g % d == 0]))
+        lm = int(rng.integers(40, 5000))
+        lo = int(rng.integers(1, lm + 1))
+        budget = int(rng.integers(1, lm + 50)) if rng.random() < 0.7 else -int(rng.integers(1, 1001))
+        out.append(C["c1"].replace(index=100 + i, batch=int(rng.integers(1, 4)), n_q_heads=hkv * g, n_kv_heads=hkv,
+                                   max_len=lm, len_lo=lo, len_hi=lm, n_dom=int(rng.integers(1, 65)), budget=budget,
+                                   n_sink=int(rng.integers(0, 9)), n_recent=int(rng.integers(0, 70)),
+                                   pairing=int(rng.integers(0, 2)), group_reduce=int(rng.integers(0, 2)),
+                                   sel_heads=0 if sel == g else sel, rope=bool(rng.integers(0, 2))))
+    return out
+
+
+@pytest.mark.parametrize("w", _random_workloads(int(os.environ.get("FASA_RANDOM_CASES", "24")), 20260203),
+                         ids=lambda w: f"i{w.index}")
+def test_seeded_random_configurations(w):
+    # shapes nobody picked by hand: heads, group, set sharing, lengths, F, budget form, forced
+    # positions, pairing and reduction all drawn at random (seeded)
+    rep, h = _full_check(Run(w))
+    assert rep["units"] == w.batch * w.n_sets
 
 
 def test_strided_token_major_cache():
