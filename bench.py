@@ -402,6 +402,7 @@ def run_fasa(args, w):
         roofline = {"kernel": "fc_score_kernel", "bound": "hbm", "achieved": by["proxy"] / (fc_us * 1e-6) / 1e9,
                     "peak": peak, "unit": "GB/s", "frac": by["proxy"] / (fc_us * 1e-6) / 1e9 / peak, "traffic": None,
                     "bytes_per_launch": by["proxy"], "us_per_launch": fc_us, "peak_source": peak_src}
+    roofline["frac_of_nominal_8tbs"] = roofline["achieved"] / 8000.0      # context: the DGX figure for HBM3e
     cfg = {k_: head[k_] for k_ in ("workload", "batch", "n_q_heads", "n_kv_heads", "context", "context_mean", "n_dom",
                                    "budget", "n_sink", "n_recent", "n_sel_per_unit", "step_mode")}
     cfg["l2"] = f"flushed before every step ({L2_FLUSH_BYTES >> 20} MiB write)"
@@ -730,13 +731,37 @@ def run_longcot(args):
             acc += v * n_layers
         return acc * 1e-6
 
+    # the prompt's cache update: 1024 rows per (sequence, KV head) in one fasa_kv_append call
+    # (K, V and the dominant slices), against the bytes it must move
+    from paper_2602_03152_b200 import binding
+    fpre = binding.Fasa.from_workload(w, t["dom"])
+    ppre = fpre.alloc_proxy(dev)
+    lens0 = torch.zeros(w.batch, dtype=torch.int32, device=dev)
+    kn, vn = t["k"][:, :, :1024].contiguous(), t["v"][:, :, :1024].contiguous()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    tsp = []
+    for i in range(8):
+        flush.fill_(i & 1)
+        lens0.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fpre.kv_append(t["k"], t["v"], ppre, lens0, kn, vn)
+        b.record()
+        b.synchronize()
+        if i >= 3:
+            tsp.append(a.elapsed_time(b) * 1e3)
+    pre_bytes = w.batch * w.n_kv_heads * 1024 * (2 * 512 + 4 * w.n_dom)          # K, V read + written, proxy written
+    prefill = {"rows_per_unit": 1024, "us_per_layer": sum(tsp) / len(tsp), "bytes": pre_bytes,
+               "gbs": pre_bytes / (sum(tsp) / len(tsp)) / 1e3, "frac_of_peak": pre_bytes / (sum(tsp) / len(tsp)) / 1e3 / peak}
+    del fpre, ppre, flush, kn, vn
+
     tf, td = total(pts, "us_per_step", 28), total(pts, "dense_us_per_step", 28)
     res = {"longcot": w.name, "layers": 28, "batch": w.batch, "prompt": 1024, "decode_steps": 15360,
            "budget_permille": -w.budget, "n_dom": w.n_dom, "steps_per_sample": args.sweep_steps,
            "fasa_decode_attention_seconds": tf, "dense_decode_attention_seconds": td,
            "speedup_vs_dense": td / tf, "theory_byte_ratio": 1.0 / (w.n_dom / 128.0 + 0.189),
            "method": "one layer timed at the sampled contexts (L2 flushed before each step), linear interpolation, x 28 layers",
-           "samples": pts}
+           "prefill_kv_append": prefill, "samples": pts}
     del t
     free, _ = torch.cuda.mem_get_info()
     if free > (48 << 30) and not args.no_resident:

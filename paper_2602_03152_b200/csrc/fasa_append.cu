@@ -62,29 +62,71 @@ kv_append_kernel(uint16_t* __restrict__ k_cache, uint16_t* __restrict__ v_cache,
   }
 }
 
-// One thread per proxy word of rows 0 .. seq_lens[b]-1.
+// Many rows at once (a prompt's cache update, or the proxy build of a cache written by other
+// means): a CTA takes 16 consecutive rows of one (batch, KV head) unit.  The 16 key rows go
+// through shared memory once: from there they are copied to the cache with 16-byte stores and
+// their dominant-FC pairs are picked for the proxy, so the keys are read from HBM a single time
+// with full-width loads.  APPEND: source = the new rows, destination row = old length + n, and
+// the CTA reports in on the sequence's arrival counter (the last one stores the new length).
+// Otherwise: source = the cache rows themselves, j < seq_lens[b].
+constexpr int kBulkRows = 16;
+template <bool APPEND>
 __global__ void __launch_bounds__(256)
-proxy_build_kernel(const uint16_t* __restrict__ k_cache, unsigned char* __restrict__ proxy,
-                   const int32_t* __restrict__ seq_lens, const int16_t* __restrict__ chan,
-                   int32_t* __restrict__ status, int n_kv_heads, int max_len, int chunks,
-                   int64_t ksb, int64_t ksh, int64_t kst) {
+bulk_rows_kernel(uint16_t* k_cache, uint16_t* __restrict__ v_cache, unsigned char* __restrict__ proxy,
+                 const int32_t* seq_lens /* same memory as seq_lens_w */, const uint16_t* __restrict__ k_new,
+                 const uint16_t* __restrict__ v_new, const int16_t* __restrict__ chan,
+                 int32_t* __restrict__ status, int n_new, int n_kv_heads, int max_len, int chunks,
+                 int64_t ksb, int64_t ksh, int64_t kst, int64_t vsb, int64_t vsh, int64_t vst,
+                 int32_t* seq_lens_w, int32_t* arrive) {
+  __shared__ __align__(16) uint16_t s_k[kBulkRows][FASA_HEAD_DIM];
   const int u = blockIdx.y;
   const int h = u % n_kv_heads;
   const int b = u / n_kv_heads;
+  const int tid = threadIdx.x;
   const int len = clamp_len(seq_lens[b], max_len, status);
-  const int words = 4 * chunks;
-  const int64_t item = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int j = (int)(item / words);
-  const int w = (int)(item % words);
-  if (j >= len) return;
+  const int n0 = blockIdx.x * kBulkRows;                 // first row of this CTA (new-row index, or cache row)
+  if (APPEND) {
+    __syncthreads();                                     // every thread has read the old length
+    if (tid == 0) {
+      const int total = n_kv_heads * (int)gridDim.x;
+      if (atomicAdd(&arrive[b], 1) == total - 1) {
+        const int grown = len + n_new;
+        seq_lens_w[b] = grown > max_len ? max_len : grown;
+        arrive[b] = 0;
+      }
+    }
+  }
+  const int n_src = APPEND ? n_new : len;                // rows that exist at the source
+  const int first = APPEND ? len + n0 : n0;              // destination row of source row n0
+  if (n0 >= n_src) return;
+  if (APPEND && first + min(kBulkRows, n_src - n0) > max_len && tid == 0) atomicOr(status, FASA_DEV_APPEND_FULL);
+  const int r = tid >> 4, c8 = (tid & 15) * 8;
+  const bool row_ok = n0 + r < n_src && first + r < max_len;
+  uint4 kx = make_uint4(0u, 0u, 0u, 0u);
+  if (row_ok) {
+    const uint16_t* ksrc = APPEND ? k_new + ((int64_t)u * n_new + n0 + r) * FASA_HEAD_DIM
+                                  : k_cache + b * ksb + h * ksh + (int64_t)(n0 + r) * kst;
+    kx = *reinterpret_cast<const uint4*>(ksrc + c8);
+    if (APPEND) {
+      *reinterpret_cast<uint4*>(k_cache + b * ksb + h * ksh + (int64_t)(first + r) * kst + c8) = kx;
+      *reinterpret_cast<uint4*>(v_cache + b * vsb + h * vsh + (int64_t)(first + r) * vst + c8) =
+          *reinterpret_cast<const uint4*>(v_new + ((int64_t)u * n_new + n0 + r) * FASA_HEAD_DIM + c8);
+    }
+  }
+  *reinterpret_cast<uint4*>(&s_k[r][c8]) = kx;
+  __syncthreads();
   const ProxyGeom pg = proxy_geom(chunks);
-  const int16_t* ch = chan + h * chunks * 8 + 2 * w;
-  const uint16_t* ksrc = k_cache + b * ksb + h * ksh + (int64_t)j * kst;
-  const int c0 = ch[0], c1 = ch[1];
-  const uint32_t lo = c0 >= 0 ? ksrc[c0] : 0u;
-  const uint32_t hi = c1 >= 0 ? ksrc[c1] : 0u;
+  const int words = 4 * chunks;
   unsigned char* unit = proxy + (int64_t)u * ((max_len + 15) >> 4) * pg.tile_bytes;
-  *reinterpret_cast<uint32_t*>(unit + proxy_word_offset(pg, j, w)) = lo | (hi << 16);
+  const int16_t* ch = chan + h * chunks * 8;
+  for (int i = tid; i < kBulkRows * words; i += 256) {
+    const int rr = i / words, w = i % words;
+    if (n0 + rr >= n_src || first + rr >= max_len) continue;
+    const int c0 = ch[2 * w], c1 = ch[2 * w + 1];
+    const uint32_t lo = c0 >= 0 ? s_k[rr][c0] : 0u;
+    const uint32_t hi = c1 >= 0 ? s_k[rr][c1] : 0u;
+    *reinterpret_cast<uint32_t*>(unit + proxy_word_offset(pg, first + rr, w)) = lo | (hi << 16);
+  }
 }
 
 bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
@@ -103,11 +145,19 @@ extern "C" int32_t fasa_kv_append(fasa_ctx_t* ctx, void* k_cache, void* v_cache,
   long long n_rows = (long long)c.batch * c.n_kv_heads * n_new;
   if (n_rows > (1ll << 30)) return FASA_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  kv_append_kernel<<<(unsigned)((n_rows + 1) / 2), 256, 0, s>>>(
-      (uint16_t*)k_cache, (uint16_t*)v_cache, (unsigned char*)proxy_k, seq_lens, (const uint16_t*)k_new,
-      (const uint16_t*)v_new, ctx->d_chan, ctx->d_status, (int)n_rows, n_new, c.n_kv_heads,
-      c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h, c.k_stride_t, c.v_stride_b,
-      c.v_stride_h, c.v_stride_t, seq_lens, ctx->d_arrive);
+  if (n_new >= kBulkRows) {
+    dim3 grid((unsigned)((n_new + kBulkRows - 1) / kBulkRows), (unsigned)(c.batch * c.n_kv_heads));
+    bulk_rows_kernel<true><<<grid, 256, 0, s>>>(
+        (uint16_t*)k_cache, (uint16_t*)v_cache, (unsigned char*)proxy_k, seq_lens, (const uint16_t*)k_new,
+        (const uint16_t*)v_new, ctx->d_chan, ctx->d_status, n_new, c.n_kv_heads, c.max_len, ctx->chunks,
+        c.k_stride_b, c.k_stride_h, c.k_stride_t, c.v_stride_b, c.v_stride_h, c.v_stride_t, seq_lens, ctx->d_arrive);
+  } else {
+    kv_append_kernel<<<(unsigned)((n_rows + 1) / 2), 256, 0, s>>>(
+        (uint16_t*)k_cache, (uint16_t*)v_cache, (unsigned char*)proxy_k, seq_lens, (const uint16_t*)k_new,
+        (const uint16_t*)v_new, ctx->d_chan, ctx->d_status, (int)n_rows, n_new, c.n_kv_heads,
+        c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h, c.k_stride_t, c.v_stride_b,
+        c.v_stride_h, c.v_stride_t, seq_lens, ctx->d_arrive);
+  }
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
 }
@@ -117,11 +167,11 @@ extern "C" int32_t fasa_proxy_build(fasa_ctx_t* ctx, const void* k_cache, void* 
   if (!ctx || !k_cache || !proxy_k || !seq_lens) return FASA_ERR_INVALID_ARG;
   if (!aligned16(k_cache) || !aligned16(proxy_k)) return FASA_ERR_INVALID_ARG;
   const fasa_config_t& c = ctx->cfg;
-  long long items = (long long)c.max_len * ctx->chunks * 4;
-  dim3 grid((unsigned)((items + 255) / 256), (unsigned)(c.batch * c.n_kv_heads));
-  proxy_build_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(
-      (const uint16_t*)k_cache, (unsigned char*)proxy_k, seq_lens, ctx->d_chan, ctx->d_status,
-      c.n_kv_heads, c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h, c.k_stride_t);
+  dim3 grid((unsigned)((c.max_len + kBulkRows - 1) / kBulkRows), (unsigned)(c.batch * c.n_kv_heads));
+  bulk_rows_kernel<false><<<grid, 256, 0, (cudaStream_t)stream>>>(
+      const_cast<uint16_t*>((const uint16_t*)k_cache), nullptr, (unsigned char*)proxy_k, seq_lens, nullptr, nullptr,
+      ctx->d_chan, ctx->d_status, 0, c.n_kv_heads, c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h,
+      c.k_stride_t, 0, 0, 0, nullptr, nullptr);
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
 }

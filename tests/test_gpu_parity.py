@@ -653,6 +653,34 @@ def test_kv_append_bulk_then_stepwise():
                       n_sel=h["n_sel"], out=h["out"], dense_out=h["dense"], what="appended", **r.oracle_kwargs())
 
 
+def test_kv_append_bulk_from_ragged_lengths_and_into_a_full_cache():
+    # 40 rows at once onto sequences of different, unaligned lengths; one of them runs out of rows
+    w = C["c1"].replace(batch=3, n_q_heads=8, n_kv_heads=2, max_len=120, len_lo=0, len_hi=0, n_dom=13)
+    t = synth.make_inputs(w.replace(len_lo=120, len_hi=120), "cpu")
+    r = Run(w, t)
+    start = [7, 95, 50]
+    lens = torch.tensor(start, dtype=torch.int32, device="cuda")
+    r.fasa.proxy_build(r.k, r.proxy, lens)
+    g = torch.Generator().manual_seed(3)
+    kn = torch.randn((3, 2, 40, 128), generator=g).to(torch.bfloat16).cuda()
+    vn = torch.randn((3, 2, 40, 128), generator=g).to(torch.bfloat16).cuda()
+    k_ref, v_ref = r.k.clone(), r.v.clone()
+    r.fasa.kv_append(r.k, r.v, r.proxy, lens, kn, vn)
+    torch.cuda.synchronize()
+    assert lens.cpu().tolist() == [47, 120, 90]
+    assert r.fasa.device_status() == binding.DEV_APPEND_FULL
+    for b, (l0, l1) in enumerate(zip(start, [47, 120, 90])):
+        k_ref[b, :, l0:l1] = kn[b, :, :l1 - l0]
+        v_ref[b, :, l0:l1] = vn[b, :, :l1 - l0]
+    assert torch.equal(r.k, k_ref) and torch.equal(r.v, v_ref)
+    exp = _expected_proxy(k_ref.cpu().view(torch.int16), torch.sort(r.dom, dim=1).values, 0, r.fasa.row_elems, [47, 120, 90])
+    got = r.proxy.cpu().view(torch.int16)
+    # rows past the new lengths may hold what the first build left there: compare the live rows
+    live = _expected_proxy(torch.ones_like(k_ref.cpu().view(torch.int16)), torch.sort(r.dom, dim=1).values, 0,
+                           r.fasa.row_elems, [47, 120, 90]) != 0
+    assert torch.equal(got[live], exp[live])
+
+
 def test_device_status_bits_instead_of_faults():
     w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, max_len=128, len_lo=128, len_hi=128, budget=16)
     r = Run(w)
