@@ -282,9 +282,10 @@ __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)
 __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst)), "l"(src) : "memory");
 }
-__device__ __forceinline__ void cp_async_wait_all() {
-  asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
-}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// waits until at most N of this thread's committed groups are still in flight
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* row) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_addr(row)));
@@ -390,22 +391,47 @@ decode_attn_mma_kernel(const AttnParams p) {
   const uint16_t* kunit = p.k + b * p.ksb + h * p.ksh;
   const uint16_t* vunit = p.v + b * p.vsb + h * p.vsh;
 
-  for (int base = r0 + warp * 16; base < r1; base += kMmaWarps * 16) {   // uniform over the warp
-    // ---- stage 16 K rows and 16 V rows: lane l copies chunk (l % 16) of rows 2j + l / 16 ----
+  // The CTA's slice of the index list goes to shared memory in one coalesced read (checked
+  // once): a tile then costs one memory round trip (its rows), not two (its indices first).
+  int32_t* s_idx = reinterpret_cast<int32_t*>(attn_smem_raw + sizeof(MmaSmem));
+  if (SPARSE) {
+    for (int i = threadIdx.x; i < r1 - r0; i += kMmaThreads) {
+      int tok = __ldg(irow + r0 + i);
+      if (tok < 0 || tok >= p.max_len) {
+        atomicOr(p.status, FASA_DEV_IDX_CLAMPED);
+        tok = 0;
+      }
+      s_idx[i] = tok;
+    }
+    __syncthreads();
+  }
+
+  // Staging of a tile's 16 K rows (or V rows): lane l copies chunk (l % 16) of rows 2j + l / 16.
+  // The K and the V buffer of a warp are two pipeline stages: the next tile's K rows are
+  // requested as soon as this tile's logits are done (they travel during the output
+  // product), its V rows as soon as the output product is done (they travel during the next
+  // logits), so memory stays busy while the warp computes.  One cp.async group per buffer
+  // fill, an empty group when there is no next tile, so "all but the newest group" always
+  // names the buffer that is needed next.
+  auto stage = [&](uint16_t (*dst)[kRowPad], const uint16_t* src_unit, int64_t stride, int base) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int row = 2 * j + (lane >> 4);
       const int r = min(base + row, r1 - 1);        // rows past the end repeat the last one (masked below)
-      int tok = SPARSE ? __ldg(irow + r) : r;
-      if (SPARSE && (tok < 0 || tok >= p.max_len)) {
-        atomicOr(p.status, FASA_DEV_IDX_CLAMPED);
-        tok = 0;
-      }
+      const int tok = SPARSE ? s_idx[r - r0] : r;
       const int c8 = (lane & 15) * 8;
-      cp_async16(&sm.k[warp][row][c8], kunit + (int64_t)tok * p.kst + c8);
-      cp_async16(&sm.v[warp][row][c8], vunit + (int64_t)tok * p.vst + c8);
+      cp_async16(&dst[row][c8], src_unit + (int64_t)tok * stride + c8);
     }
-    cp_async_wait_all();
+  };
+  constexpr int kTileStep = kMmaWarps * 16;
+  if (r0 + warp * 16 < r1) stage(sm.k[warp], kunit, p.kst, r0 + warp * 16);
+  cp_async_commit();
+  if (r0 + warp * 16 < r1) stage(sm.v[warp], vunit, p.vst, r0 + warp * 16);
+  cp_async_commit();
+
+  for (int base = r0 + warp * 16; base < r1; base += kTileStep) {   // uniform over the warp
+    const bool more = base + kTileStep < r1;
+    cp_async_wait<1>();                             // this tile's K rows have landed
     __syncwarp();
 
     // ---- logits: D[16 rows x 8 heads] ---------------------------------------------------------
@@ -448,6 +474,10 @@ decode_attn_mma_kernel(const AttnParams p) {
       sm.p_hi[warp][head][row] = (uint16_t)hi;
       sm.p_lo[warp][head][row] = (uint16_t)f32_to_bf16_bits(rest);
     }
+    __syncwarp();                                   // P is visible; every lane is done with the K buffer
+    if (more) stage(sm.k[warp], kunit, p.kst, base + kTileStep);
+    cp_async_commit();
+    cp_async_wait<1>();                             // this tile's V rows have landed
     __syncwarp();
     // B operand of the output product: B[k = row][n = head g]: rows 2t, 2t+1 and 2t+8, 2t+9
     const uint32_t ph0 = *reinterpret_cast<const uint32_t*>(&sm.p_hi[warp][g][2 * t]);
@@ -466,8 +496,11 @@ decode_attn_mma_kernel(const AttnParams p) {
       mma16816(acc[cb], a, ph0, ph1);
       mma16816(acc[cb], a, pl0, pl1);
     }
-    __syncwarp();   // the staging buffers are refilled by the next tile
+    __syncwarp();                                   // every lane is done with the V buffer
+    if (more) stage(sm.v[warp], vunit, p.vst, base + kTileStep);
+    cp_async_commit();
   }
+  cp_async_wait<0>();
 
   // ---- this warp's (m, l, acc) per head; the g lanes add their sums -------------------------------
 #pragma unroll
@@ -597,8 +630,11 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   if (ctx->use_fused) {   // default: the tensor-core kernel (mode 0 keeps the scalar one)
     static_assert(sizeof(MmaSmem) >= (size_t)kMmaWarps * 8 * (FASA_HEAD_DIM + 2) * sizeof(float), "combine area");
     auto fn = decode_attn_mma_kernel<SPARSE>;
-    FASA_CUDA_TRY(ctx, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(MmaSmem)));
-    FASA_CUDA_TRY(ctx, launch_after_predecessor(fn, grid, dim3(kMmaThreads), sizeof(MmaSmem), s, p));
+    // (+ the slice of the index list: chunk <= 2048 rows)
+    const size_t smem = sizeof(MmaSmem) + (SPARSE ? (size_t)plan.chunk * sizeof(int32_t) : 0);
+    FASA_CUDA_TRY(ctx, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)(sizeof(MmaSmem) + 2080 * sizeof(int32_t))));
+    FASA_CUDA_TRY(ctx, launch_after_predecessor(fn, grid, dim3(kMmaThreads), smem, s, p));
   } else if (G == 1) decode_attn_kernel<1, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   else if (G == 2) decode_attn_kernel<2, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   else if (G == 3) decode_attn_kernel<3, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
