@@ -35,6 +35,17 @@
  *     proxy_row_elems * 2 (64 at n_dom = 16); a step then moves n_sel * 512 bytes per
  *     (batch, KV head) over the link, which bounds it.  The dense path over host-resident
  *     caches streams the whole cache over the link and is only useful as a reference.
+ *   - Paged caches (page_size > 0).  K, V and the proxy are pools of n_pages pages of
+ *     page_size tokens, shared by the sequences; a block table, int32
+ *     [batch][ceil(max_len / page_size)] on the device, names the physical page of every
+ *     logical page of a sequence (fasa_set_block_table; the caller owns it and may rewrite
+ *     it between calls, in stream order).  K and V: [n_pages][n_kv_heads][page_size][128],
+ *     or any layout the stride fields describe with stride_b read as the PAGE stride;
+ *     proxy: [n_pages][n_kv_heads][page_size / 16 tiles], fasa_proxy_bytes() in all.
+ *     Token positions everywhere else (seq_lens, idx, scores) stay logical.  Reads through
+ *     an entry outside [0, n_pages) use page 0 and set FASA_DEV_PAGE_CLAMPED, writes through
+ *     one are dropped.  Paged contexts run the step as separate kernels (scoring, TopK-I,
+ *     attention): fasa_step_cluster_size() is 0 for them.
  *   - Frequency chunk (FC) i, 0 <= i < 64, is the channel pair (i, i+64) with
  *     rope_pairing 0 (rotate-half layout) or (2i, 2i+1) with rope_pairing 1
  *     (the paper's Eq. 1 layout).  An FC is never split (Appendix, design choices).
@@ -83,6 +94,7 @@ extern "C" {
 #define FASA_DEV_APPEND_FULL    2   /* kv_append ran out of rows; the excess was dropped   */
 #define FASA_DEV_IDX_CLAMPED    4   /* sparse attention met an index outside [0, max_len)  */
 #define FASA_DEV_NSEL_CLAMPED   8   /* n_sel exceeded n_sel_max                            */
+#define FASA_DEV_PAGE_CLAMPED  16   /* a block-table entry was < 0 or >= n_pages           */
 
 typedef struct fasa_ctx fasa_ctx_t;
 
@@ -99,6 +111,9 @@ typedef struct {
   float   softmax_scale;  /* 0 => 1/sqrt(head_dim)                                         */
   int64_t k_stride_b, k_stride_h, k_stride_t; /* in elements; all 0 => dense layout above  */
   int64_t v_stride_b, v_stride_h, v_stride_t; /* stride_t must be a multiple of 8          */
+  int32_t page_size;      /* 0: one contiguous cache per sequence; else tokens per page    */
+                          /* (a power of two >= 16) of a paged cache, see "Paged caches"   */
+  int32_t n_pages;        /* pages in the pool (paged caches only)                         */
 } fasa_config_t;
 
 /* ---- context (off the hot path) ----------------------------------------- */
@@ -111,10 +126,16 @@ typedef struct {
 int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_host, fasa_ctx_t** out);
 int32_t fasa_destroy(fasa_ctx_t* ctx);
 
+/* Paged caches: the block table the calls after this one translate token positions with
+ * (device pointer, int32 [batch][ceil(max_len / page_size)], kept by reference).
+ * INVALID_ARG for a context with page_size == 0 or a null table. */
+int32_t fasa_set_block_table(fasa_ctx_t* ctx, const int32_t* block_table);
+
 /* bf16 values per token in the proxy-K buffer for n_dom dominant FCs: 8 * ceil(n_dom / 4). */
 int32_t fasa_proxy_row_elems(int32_t n_dom);
 /* Size of the proxy-K buffer of this context:
- * batch * n_kv_heads * 16 * ceil(max_len / 16) * proxy_row_elems * 2 bytes. */
+ * batch * n_kv_heads * 16 * ceil(max_len / 16) * proxy_row_elems * 2 bytes, or
+ * n_pages * n_kv_heads * page_size * proxy_row_elems * 2 bytes for paged caches. */
 int32_t fasa_proxy_bytes(const fasa_ctx_t* ctx, size_t* out_bytes);
 
 /* Bytes of caller-provided scratch that fasa_topk, the two attention calls and

@@ -17,7 +17,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libfasa.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
-DEV_LEN_CLAMPED, DEV_APPEND_FULL, DEV_IDX_CLAMPED, DEV_NSEL_CLAMPED = 1, 2, 4, 8
+DEV_LEN_CLAMPED, DEV_APPEND_FULL, DEV_IDX_CLAMPED, DEV_NSEL_CLAMPED, DEV_PAGE_CLAMPED = 1, 2, 4, 8, 16
 
 # Every entry point include/fasa.h declares.
 SYMBOLS = [
@@ -27,7 +27,7 @@ SYMBOLS = [
     "fasa_full_decode_attn", "fasa_decode_step", "fasa_stage_bytes", "fasa_decode_step_host",
     "fasa_sparse_decode_attn_static", "fasa_set_step_mode", "fasa_step_cluster_size",
     "fasa_append_decode_step", "fasa_proxy_bytes",
-    "fasa_calib_workspace_bytes", "fasa_calib_accumulate", "fasa_calib_select",
+    "fasa_calib_workspace_bytes", "fasa_calib_accumulate", "fasa_calib_select", "fasa_set_block_table",
 ]
 
 
@@ -45,6 +45,7 @@ class FasaConfig(ctypes.Structure):
         ("n_sink", ctypes.c_int32), ("n_recent", ctypes.c_int32), ("softmax_scale", ctypes.c_float),
         ("k_stride_b", ctypes.c_int64), ("k_stride_h", ctypes.c_int64), ("k_stride_t", ctypes.c_int64),
         ("v_stride_b", ctypes.c_int64), ("v_stride_h", ctypes.c_int64), ("v_stride_t", ctypes.c_int64),
+        ("page_size", ctypes.c_int32), ("n_pages", ctypes.c_int32),
     ]
 
 
@@ -88,6 +89,7 @@ def load_library() -> ctypes.CDLL:
         "fasa_calib_workspace_bytes": (i32, [vp, i32, ctypes.POINTER(ctypes.c_size_t)]),
         "fasa_calib_accumulate": (i32, [vp, vp, vp, vp, i32, vp, vp, vp, vp]),
         "fasa_calib_select": (i32, [i32, i32, vp, vp, i32, i32, vp, vp]),
+        "fasa_set_block_table": (i32, [vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -122,13 +124,14 @@ class Fasa:
 
     def __init__(self, batch, n_q_heads, n_kv_heads, max_len, dom, *, head_dim=128, rope_pairing=0,
                  group_reduce=0, n_sink=0, n_recent=0, softmax_scale=0.0, k_strides=(0, 0, 0),
-                 v_strides=(0, 0, 0), select_heads=0):
+                 v_strides=(0, 0, 0), select_heads=0, page_size=0, n_pages=0):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         dom = torch.as_tensor(dom, dtype=torch.int32).contiguous().cpu()
         n_dom = dom.shape[-1] if dom.dim() == 2 else 0
         self.cfg = FasaConfig(batch, n_q_heads, n_kv_heads, head_dim, max_len, n_dom, rope_pairing,
-                              group_reduce, select_heads, n_sink, n_recent, softmax_scale, *k_strides, *v_strides)
+                              group_reduce, select_heads, n_sink, n_recent, softmax_scale, *k_strides, *v_strides,
+                              page_size, n_pages)
         if dom.dim() != 2 or dom.shape[0] != n_kv_heads:
             raise FasaError(ERR_INVALID_ARG, "fasa_create", "dom must be [n_kv_heads, n_dom]")
         st = self._lib.fasa_create(ctypes.byref(self.cfg), dom.data_ptr(), ctypes.byref(self._h))
@@ -137,6 +140,8 @@ class Fasa:
             raise FasaError(st, "fasa_create", self._lib.fasa_status_string(st).decode())
         self.batch, self.n_q_heads, self.n_kv_heads, self.max_len = batch, n_q_heads, n_kv_heads, max_len
         self.n_dom = n_dom
+        self.page_size, self.n_pages = page_size, n_pages
+        self._block_table = None
         group = n_q_heads // n_kv_heads
         self.select_heads = select_heads if select_heads > 0 else group    # query heads per index set
         self.n_sets = n_q_heads // self.select_heads                       # rows of scores / idx / n_sel per sequence
@@ -201,12 +206,23 @@ class Fasa:
         """Zero-filled proxy-K buffer: [batch, kv heads, tiles of 16 tokens, 16 * row_elems] bf16
         (opaque tile-internal order, see include/fasa.h)."""
         tiles = (self.max_len + 15) // 16
-        t = torch.zeros((self.batch, self.n_kv_heads, tiles, 16 * self.row_elems), dtype=torch.bfloat16, device=device)
+        shape = (self.n_pages, self.n_kv_heads, self.page_size // 16) if self.page_size else (self.batch, self.n_kv_heads, tiles)
+        t = torch.zeros(shape + (16 * self.row_elems,), dtype=torch.bfloat16, device=device)
         assert t.numel() * 2 == self.proxy_bytes()
         return t
 
     def alloc_workspace(self, n_sel_max: int, device="cuda") -> torch.Tensor:
         return torch.empty(self.workspace_bytes(n_sel_max), dtype=torch.uint8, device=device)
+
+    def set_block_table(self, table: torch.Tensor):
+        """Paged caches: int32 CUDA tensor [batch, ceil(max_len / page_size)] of physical pages.
+        Kept by reference: its contents may change between calls."""
+        self._check(self._lib.fasa_set_block_table(self._h, _dp(table, torch.int32)), "fasa_set_block_table")
+        self._block_table = table
+
+    def alloc_paged_cache(self, device="cuda") -> torch.Tensor:
+        """A K or V page pool [n_pages, n_kv_heads, page_size, 128] (bf16)."""
+        return torch.zeros((self.n_pages, self.n_kv_heads, self.page_size, 128), dtype=torch.bfloat16, device=device)
 
     def alloc_host_cache(self) -> torch.Tensor:
         """A K or V cache [batch, n_kv_heads, max_len, 128] (bf16) in page-locked host memory

@@ -19,6 +19,9 @@ bool valid_cfg(const fasa_config_t& c, int32_t* why) {
   if (c.n_q_heads / c.n_kv_heads > FASA_MAX_GROUP) return false;
   if (c.rope_pairing != 0 && c.rope_pairing != 1) return false;
   if (c.group_reduce != 0 && c.group_reduce != 1) return false;
+  if (c.page_size != 0) {
+    if (c.page_size < 16 || (c.page_size & (c.page_size - 1)) != 0 || c.n_pages < 1) return false;
+  }
   if (c.select_heads < 0) return false;
   const int group = c.n_q_heads / c.n_kv_heads;
   const int per_set = c.select_heads > 0 ? c.select_heads : group;
@@ -30,7 +33,7 @@ bool valid_cfg(const fasa_config_t& c, int32_t* why) {
 bool fill_strides(int64_t& sb, int64_t& sh, int64_t& st, const fasa_config_t& c) {
   if (sb == 0 && sh == 0 && st == 0) {
     st = FASA_HEAD_DIM;
-    sh = (int64_t)c.max_len * FASA_HEAD_DIM;
+    sh = (int64_t)(c.page_size > 0 ? c.page_size : c.max_len) * FASA_HEAD_DIM;   // rows per head of a page / a sequence
     sb = sh * c.n_kv_heads;
     return true;
   }
@@ -49,7 +52,8 @@ extern "C" int32_t fasa_proxy_bytes(const fasa_ctx_t* ctx, size_t* out_bytes) {
   if (!ctx || !out_bytes) return FASA_ERR_INVALID_ARG;
   const fasa_config_t& c = ctx->cfg;
   const size_t rows = (size_t)((c.max_len + 15) / 16) * 16;
-  *out_bytes = (size_t)c.batch * c.n_kv_heads * rows * ctx->row_elems * 2;
+  *out_bytes = c.page_size > 0 ? (size_t)c.n_pages * c.n_kv_heads * c.page_size * ctx->row_elems * 2
+                               : (size_t)c.batch * c.n_kv_heads * rows * ctx->row_elems * 2;
   return FASA_OK;
 }
 
@@ -74,6 +78,10 @@ extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_h
   ctx->group = c.n_q_heads / c.n_kv_heads;
   ctx->sel_heads = c.select_heads > 0 ? c.select_heads : ctx->group;
   ctx->n_sets = c.n_q_heads / ctx->sel_heads;
+  if (c.page_size > 0) {
+    while ((1 << ctx->page_shift) < c.page_size) ++ctx->page_shift;
+    ctx->pages_per_seq = (c.max_len + c.page_size - 1) / c.page_size;
+  }
   ctx->chunks = (c.n_dom + 3) / 4;
   ctx->row_elems = 8 * ctx->chunks;
 
@@ -119,8 +127,15 @@ extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_h
     return FASA_ERR_CUDA;
   }
   fasa_fused_plan(ctx);
+  if (c.page_size > 0) ctx->fused_step_ok = 0;   // the one-launch step reads contiguous caches only
   ctx->use_fused = 1;
   *out = ctx;
+  return FASA_OK;
+}
+
+extern "C" int32_t fasa_set_block_table(fasa_ctx_t* ctx, const int32_t* block_table) {
+  if (!ctx || !block_table || ctx->cfg.page_size == 0) return FASA_ERR_INVALID_ARG;
+  ctx->block_table = block_table;
   return FASA_OK;
 }
 

@@ -5,6 +5,42 @@
 
 namespace {
 
+// Where row `pos` of (sequence b, KV head h) is written.  Paged caches: a table entry outside
+// the pool drops the row (ok = false) instead of redirecting the write.
+struct RowDst {
+  int64_t k, v;          // element offsets into the K and V caches
+  int64_t proxy_unit;    // byte offset of the (page, head) or (sequence, head) proxy block
+  int proxy_row;         // row inside that block
+  bool ok;
+};
+__device__ __forceinline__ RowDst row_dst(const PageMap& m, int b, int h, int n_kv_heads, int pos, int max_len,
+                                          int tile_bytes, int64_t ksb, int64_t ksh, int64_t kst, int64_t vsb,
+                                          int64_t vsh, int64_t vst, int32_t* status) {
+  RowDst d;
+  d.ok = true;
+  if (m.table == nullptr) {
+    d.k = b * ksb + h * ksh + (int64_t)pos * kst;
+    d.v = b * vsb + h * vsh + (int64_t)pos * vst;
+    d.proxy_unit = (int64_t)(b * n_kv_heads + h) * ((max_len + 15) >> 4) * tile_bytes;
+    d.proxy_row = pos;
+    return d;
+  }
+  const int page = page_of(m, b, pos);
+  if (!page_ok(m, page)) {
+    atomicOr(status, FASA_DEV_PAGE_CLAMPED);
+    d.ok = false;
+    d.k = d.v = d.proxy_unit = 0;
+    d.proxy_row = 0;
+    return d;
+  }
+  const int in_page = pos & ((1 << m.shift) - 1);
+  d.k = page * ksb + h * ksh + (int64_t)in_page * kst;
+  d.v = page * vsb + h * vsh + (int64_t)in_page * vst;
+  d.proxy_unit = ((int64_t)page * n_kv_heads + h) * (1 << (m.shift - 4)) * tile_bytes;
+  d.proxy_row = in_page;
+  return d;
+}
+
 // 128 threads per appended row: 16 copy the K row, 16 the V row (16 bytes each), up to 64
 // write the proxy words (one dominant FC = one 4-byte channel pair each) to their places in
 // the tiled proxy layout.
@@ -15,7 +51,7 @@ kv_append_kernel(uint16_t* __restrict__ k_cache, uint16_t* __restrict__ v_cache,
                  const int16_t* __restrict__ chan, int32_t* __restrict__ status, int n_rows,
                  int n_new, int n_kv_heads, int max_len, int chunks, int64_t ksb, int64_t ksh,
                  int64_t kst, int64_t vsb, int64_t vsh, int64_t vst, int32_t* seq_lens_w,
-                 int32_t* arrive) {
+                 int32_t* arrive, const PageMap pm) {
   const int row = blockIdx.x * 2 + (threadIdx.x >> 7);
   const bool live = row < n_rows;
   const int t = threadIdx.x & 127;
@@ -43,22 +79,23 @@ kv_append_kernel(uint16_t* __restrict__ k_cache, uint16_t* __restrict__ v_cache,
     return;
   }
   const uint16_t* ksrc = k_new + (int64_t)row * FASA_HEAD_DIM;
+  const ProxyGeom pg = proxy_geom(chunks);
+  const RowDst d = row_dst(pm, b, h, n_kv_heads, pos, max_len, pg.tile_bytes, ksb, ksh, kst, vsb, vsh, vst, status);
+  if (!d.ok) return;
   if (t < 16) {
     uint4 x = *reinterpret_cast<const uint4*>(ksrc + t * 8);
-    *reinterpret_cast<uint4*>(k_cache + b * ksb + h * ksh + pos * kst + t * 8) = x;
+    *reinterpret_cast<uint4*>(k_cache + d.k + t * 8) = x;
   } else if (t < 32) {
     const int c = t - 16;
     uint4 x = *reinterpret_cast<const uint4*>(v_new + (int64_t)row * FASA_HEAD_DIM + c * 8);
-    *reinterpret_cast<uint4*>(v_cache + b * vsb + h * vsh + pos * vst + c * 8) = x;
+    *reinterpret_cast<uint4*>(v_cache + d.v + c * 8) = x;
   } else if (t - 32 < 4 * chunks) {
     const int w = t - 32;
-    const ProxyGeom pg = proxy_geom(chunks);
     const int16_t* ch = chan + h * chunks * 8 + 2 * w;
     const int c0 = ch[0], c1 = ch[1];
     const uint32_t lo = c0 >= 0 ? ksrc[c0] : 0u;
     const uint32_t hi = c1 >= 0 ? ksrc[c1] : 0u;
-    unsigned char* unit = proxy + (int64_t)u * ((max_len + 15) >> 4) * pg.tile_bytes;
-    *reinterpret_cast<uint32_t*>(unit + proxy_word_offset(pg, pos, w)) = lo | (hi << 16);
+    *reinterpret_cast<uint32_t*>(proxy + d.proxy_unit + proxy_word_offset(pg, d.proxy_row, w)) = lo | (hi << 16);
   }
 }
 
@@ -77,7 +114,7 @@ bulk_rows_kernel(uint16_t* k_cache, uint16_t* __restrict__ v_cache, unsigned cha
                  const uint16_t* __restrict__ v_new, const int16_t* __restrict__ chan,
                  int32_t* __restrict__ status, int n_new, int n_kv_heads, int max_len, int chunks,
                  int64_t ksb, int64_t ksh, int64_t kst, int64_t vsb, int64_t vsh, int64_t vst,
-                 int32_t* seq_lens_w, int32_t* arrive) {
+                 int32_t* seq_lens_w, int32_t* arrive, const PageMap pm) {
   __shared__ __align__(16) uint16_t s_k[kBulkRows][FASA_HEAD_DIM];
   const int u = blockIdx.y;
   const int h = u % n_kv_heads;
@@ -101,31 +138,34 @@ bulk_rows_kernel(uint16_t* k_cache, uint16_t* __restrict__ v_cache, unsigned cha
   if (n0 >= n_src) return;
   if (APPEND && first + min(kBulkRows, n_src - n0) > max_len && tid == 0) atomicOr(status, FASA_DEV_APPEND_FULL);
   const int r = tid >> 4, c8 = (tid & 15) * 8;
+  const ProxyGeom pg = proxy_geom(chunks);
   const bool row_ok = n0 + r < n_src && first + r < max_len;
   uint4 kx = make_uint4(0u, 0u, 0u, 0u);
   if (row_ok) {
-    const uint16_t* ksrc = APPEND ? k_new + ((int64_t)u * n_new + n0 + r) * FASA_HEAD_DIM
-                                  : k_cache + b * ksb + h * ksh + (int64_t)(n0 + r) * kst;
-    kx = *reinterpret_cast<const uint4*>(ksrc + c8);
-    if (APPEND) {
-      *reinterpret_cast<uint4*>(k_cache + b * ksb + h * ksh + (int64_t)(first + r) * kst + c8) = kx;
-      *reinterpret_cast<uint4*>(v_cache + b * vsb + h * vsh + (int64_t)(first + r) * vst + c8) =
-          *reinterpret_cast<const uint4*>(v_new + ((int64_t)u * n_new + n0 + r) * FASA_HEAD_DIM + c8);
+    const RowDst d = row_dst(pm, b, h, n_kv_heads, first + r, max_len, pg.tile_bytes, ksb, ksh, kst, vsb, vsh, vst, status);
+    if (d.ok) {
+      const uint16_t* ksrc = APPEND ? k_new + ((int64_t)u * n_new + n0 + r) * FASA_HEAD_DIM : k_cache + d.k;
+      kx = *reinterpret_cast<const uint4*>(ksrc + c8);
+      if (APPEND) {
+        *reinterpret_cast<uint4*>(k_cache + d.k + c8) = kx;
+        *reinterpret_cast<uint4*>(v_cache + d.v + c8) =
+            *reinterpret_cast<const uint4*>(v_new + ((int64_t)u * n_new + n0 + r) * FASA_HEAD_DIM + c8);
+      }
     }
   }
   *reinterpret_cast<uint4*>(&s_k[r][c8]) = kx;
   __syncthreads();
-  const ProxyGeom pg = proxy_geom(chunks);
   const int words = 4 * chunks;
-  unsigned char* unit = proxy + (int64_t)u * ((max_len + 15) >> 4) * pg.tile_bytes;
   const int16_t* ch = chan + h * chunks * 8;
   for (int i = tid; i < kBulkRows * words; i += 256) {
     const int rr = i / words, w = i % words;
     if (n0 + rr >= n_src || first + rr >= max_len) continue;
+    const RowDst d = row_dst(pm, b, h, n_kv_heads, first + rr, max_len, pg.tile_bytes, ksb, ksh, kst, vsb, vsh, vst, status);
+    if (!d.ok) continue;
     const int c0 = ch[2 * w], c1 = ch[2 * w + 1];
     const uint32_t lo = c0 >= 0 ? s_k[rr][c0] : 0u;
     const uint32_t hi = c1 >= 0 ? s_k[rr][c1] : 0u;
-    *reinterpret_cast<uint32_t*>(unit + proxy_word_offset(pg, first + rr, w)) = lo | (hi << 16);
+    *reinterpret_cast<uint32_t*>(proxy + d.proxy_unit + proxy_word_offset(pg, d.proxy_row, w)) = lo | (hi << 16);
   }
 }
 
@@ -139,7 +179,7 @@ extern "C" int32_t fasa_kv_append(fasa_ctx_t* ctx, void* k_cache, void* v_cache,
   if (!ctx || !k_cache || !v_cache || !proxy_k || !seq_lens || !k_new || !v_new || n_new <= 0)
     return FASA_ERR_INVALID_ARG;
   if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(proxy_k) || !aligned16(k_new) ||
-      !aligned16(v_new))
+      !aligned16(v_new) || !fasa_pages_ready(ctx))
     return FASA_ERR_INVALID_ARG;
   const fasa_config_t& c = ctx->cfg;
   long long n_rows = (long long)c.batch * c.n_kv_heads * n_new;
@@ -150,13 +190,14 @@ extern "C" int32_t fasa_kv_append(fasa_ctx_t* ctx, void* k_cache, void* v_cache,
     bulk_rows_kernel<true><<<grid, 256, 0, s>>>(
         (uint16_t*)k_cache, (uint16_t*)v_cache, (unsigned char*)proxy_k, seq_lens, (const uint16_t*)k_new,
         (const uint16_t*)v_new, ctx->d_chan, ctx->d_status, n_new, c.n_kv_heads, c.max_len, ctx->chunks,
-        c.k_stride_b, c.k_stride_h, c.k_stride_t, c.v_stride_b, c.v_stride_h, c.v_stride_t, seq_lens, ctx->d_arrive);
+        c.k_stride_b, c.k_stride_h, c.k_stride_t, c.v_stride_b, c.v_stride_h, c.v_stride_t, seq_lens, ctx->d_arrive,
+        fasa_page_map(ctx));
   } else {
     kv_append_kernel<<<(unsigned)((n_rows + 1) / 2), 256, 0, s>>>(
         (uint16_t*)k_cache, (uint16_t*)v_cache, (unsigned char*)proxy_k, seq_lens, (const uint16_t*)k_new,
         (const uint16_t*)v_new, ctx->d_chan, ctx->d_status, (int)n_rows, n_new, c.n_kv_heads,
         c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h, c.k_stride_t, c.v_stride_b,
-        c.v_stride_h, c.v_stride_t, seq_lens, ctx->d_arrive);
+        c.v_stride_h, c.v_stride_t, seq_lens, ctx->d_arrive, fasa_page_map(ctx));
   }
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
@@ -165,13 +206,13 @@ extern "C" int32_t fasa_kv_append(fasa_ctx_t* ctx, void* k_cache, void* v_cache,
 extern "C" int32_t fasa_proxy_build(fasa_ctx_t* ctx, const void* k_cache, void* proxy_k,
                                     const int32_t* seq_lens, void* stream) {
   if (!ctx || !k_cache || !proxy_k || !seq_lens) return FASA_ERR_INVALID_ARG;
-  if (!aligned16(k_cache) || !aligned16(proxy_k)) return FASA_ERR_INVALID_ARG;
+  if (!aligned16(k_cache) || !aligned16(proxy_k) || !fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
   const fasa_config_t& c = ctx->cfg;
   dim3 grid((unsigned)((c.max_len + kBulkRows - 1) / kBulkRows), (unsigned)(c.batch * c.n_kv_heads));
   bulk_rows_kernel<false><<<grid, 256, 0, (cudaStream_t)stream>>>(
       const_cast<uint16_t*>((const uint16_t*)k_cache), nullptr, (unsigned char*)proxy_k, seq_lens, nullptr, nullptr,
       ctx->d_chan, ctx->d_status, 0, c.n_kv_heads, c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h,
-      c.k_stride_t, 0, 0, 0, nullptr, nullptr);
+      c.k_stride_t, 0, 0, 0, nullptr, nullptr, fasa_page_map(ctx));
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
 }

@@ -35,6 +35,7 @@ struct AttnParams {
   int32_t* status;
   int n_q_heads, n_kv_heads, n_sets, group, max_len, n_sel_max, n_cap, chunk, n_splits;   // a unit = `group` query heads; n_sets units per sequence
   int64_t ksb, ksh, kst, vsb, vsh, vst;
+  PageMap pm;              // paged caches (all zero: contiguous)
   float scale_log2;        // softmax_scale * log2(e)
 };
 
@@ -101,8 +102,8 @@ decode_attn_kernel(const AttnParams p) {
     for (int e = 0; e < 4; ++e) acc[g][e] = make_float2(0.f, 0.f);
   }
 
-  const uint16_t* kbase = p.k + b * p.ksb + h * p.ksh + l16 * 8;
-  const uint16_t* vbase = p.v + b * p.vsb + h * p.vsh + l16 * 8;
+  const uint16_t* kbase = p.k + l16 * 8;
+  const uint16_t* vbase = p.v + l16 * 8;
   const int32_t* irow = SPARSE ? p.idx + (int64_t)u * p.n_sel_max : nullptr;
   // The row of the batch whose finished logit lands in this lane after the reduction.
   const int my_row = ((l16 >> 3) & 1) * 4 + ((l16 >> 2) & 1) * 2 + ((l16 >> 1) & 1);
@@ -128,8 +129,8 @@ decode_attn_kernel(const AttnParams p) {
           atomicOr(p.status, FASA_DEV_IDX_CLAMPED);
           t = 0;
         }
-        kk[i] = ld_stream_u4(kbase + (int64_t)t * p.kst);
-        vv[i] = ld_stream_u4(vbase + (int64_t)t * p.vst);
+        kk[i] = ld_stream_u4(kbase + cache_row(p.pm, b, h, t, p.ksb, p.ksh, p.kst, p.status));
+        vv[i] = ld_stream_u4(vbase + cache_row(p.pm, b, h, t, p.vsb, p.vsh, p.vst, p.status));
       } else {
         kk[i] = make_uint4(0u, 0u, 0u, 0u);
         vv[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -388,8 +389,6 @@ decode_attn_mma_kernel(const AttnParams p) {
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
 
   const int32_t* irow = SPARSE ? p.idx + (int64_t)u * p.n_sel_max : nullptr;
-  const uint16_t* kunit = p.k + b * p.ksb + h * p.ksh;
-  const uint16_t* vunit = p.v + b * p.vsb + h * p.vsh;
 
   // The CTA's slice of the index list goes to shared memory in one coalesced read (checked
   // once): a tile then costs one memory round trip (its rows), not two (its indices first).
@@ -413,20 +412,20 @@ decode_attn_mma_kernel(const AttnParams p) {
   // logits), so memory stays busy while the warp computes.  One cp.async group per buffer
   // fill, an empty group when there is no next tile, so "all but the newest group" always
   // names the buffer that is needed next.
-  auto stage = [&](uint16_t (*dst)[kRowPad], const uint16_t* src_unit, int64_t stride, int base) {
+  auto stage = [&](uint16_t (*dst)[kRowPad], const uint16_t* cache, int64_t sb, int64_t sh, int64_t st, int base) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int row = 2 * j + (lane >> 4);
       const int r = min(base + row, r1 - 1);        // rows past the end repeat the last one (masked below)
       const int tok = SPARSE ? s_idx[r - r0] : r;
       const int c8 = (lane & 15) * 8;
-      cp_async16(&dst[row][c8], src_unit + (int64_t)tok * stride + c8);
+      cp_async16(&dst[row][c8], cache + cache_row(p.pm, b, h, tok, sb, sh, st, p.status) + c8);
     }
   };
   constexpr int kTileStep = kMmaWarps * 16;
-  if (r0 + warp * 16 < r1) stage(sm.k[warp], kunit, p.kst, r0 + warp * 16);
+  if (r0 + warp * 16 < r1) stage(sm.k[warp], p.k, p.ksb, p.ksh, p.kst, r0 + warp * 16);
   cp_async_commit();
-  if (r0 + warp * 16 < r1) stage(sm.v[warp], vunit, p.vst, r0 + warp * 16);
+  if (r0 + warp * 16 < r1) stage(sm.v[warp], p.v, p.vsb, p.vsh, p.vst, r0 + warp * 16);
   cp_async_commit();
 
   for (int base = r0 + warp * 16; base < r1; base += kTileStep) {   // uniform over the warp
@@ -475,7 +474,7 @@ decode_attn_mma_kernel(const AttnParams p) {
       sm.p_lo[warp][head][row] = (uint16_t)f32_to_bf16_bits(rest);
     }
     __syncwarp();                                   // P is visible; every lane is done with the K buffer
-    if (more) stage(sm.k[warp], kunit, p.kst, base + kTileStep);
+    if (more) stage(sm.k[warp], p.k, p.ksb, p.ksh, p.kst, base + kTileStep);
     cp_async_commit();
     cp_async_wait<1>();                             // this tile's V rows have landed
     __syncwarp();
@@ -497,7 +496,7 @@ decode_attn_mma_kernel(const AttnParams p) {
       mma16816(acc[cb], a, pl0, pl1);
     }
     __syncwarp();                                   // every lane is done with the V buffer
-    if (more) stage(sm.v[warp], vunit, p.vst, base + kTileStep);
+    if (more) stage(sm.v[warp], p.v, p.vsb, p.vsh, p.vst, base + kTileStep);
     cp_async_commit();
   }
   cp_async_wait<0>();
@@ -614,6 +613,7 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
                     const int32_t* idx, const int32_t* n_rows, int n_upper, int n_sel_max,
                     float* out, float* lse, void* workspace, cudaStream_t s) {
   const fasa_config_t& c = ctx->cfg;
+  if (!fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
   // the dense pass treats a KV head with all its query heads as the unit
   const int n_sets = SPARSE ? ctx->n_sets : c.n_kv_heads;
   const int G = SPARSE ? ctx->sel_heads : ctx->group;
@@ -625,6 +625,7 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   p.max_len = c.max_len; p.n_sel_max = n_sel_max; p.n_cap = n_upper; p.chunk = plan.chunk; p.n_splits = plan.n_splits;
   p.ksb = c.k_stride_b; p.ksh = c.k_stride_h; p.kst = c.k_stride_t;
   p.vsb = c.v_stride_b; p.vsh = c.v_stride_h; p.vst = c.v_stride_t;
+  p.pm = fasa_page_map(ctx);
   p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
   dim3 grid((unsigned)plan.n_splits, (unsigned)(c.batch * n_sets));
   if (ctx->use_fused) {   // default: the tensor-core kernel (mode 0 keeps the scalar one)

@@ -33,7 +33,7 @@ __global__ void __launch_bounds__(kCalibWarps * 32)
 calib_score_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
                    const int32_t* __restrict__ seq_lens, float* __restrict__ scores,
                    int32_t* __restrict__ status, int n_q_heads, int n_kv_heads, int max_len, int pairing,
-                   int64_t ksb, int64_t ksh, int64_t kst) {
+                   int64_t ksb, int64_t ksh, int64_t kst, const PageMap pm) {
   const int u = blockIdx.y;
   const int b = u / n_q_heads, hq = u % n_q_heads;
   const int h = hq / (n_q_heads / n_kv_heads);
@@ -59,10 +59,9 @@ calib_score_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ 
     qv[e][0] = bf16_bits_to_f32(qrow[c[e][0]]);
     qv[e][1] = bf16_bits_to_f32(qrow[c[e][1]]);
   }
-  const uint16_t* kunit = k + b * ksb + h * ksh;
   const int n_tok = min(32, len - base);
   for (int tt = 0; tt < n_tok; ++tt) {
-    const uint16_t* krow = kunit + (int64_t)(base + tt) * kst;
+    const uint16_t* krow = k + cache_row(pm, b, h, base + tt, ksb, ksh, kst, status);
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
       const float p0 = qv[e][0] * bf16_bits_to_f32(krow[c[e][0]]);     // exact
@@ -154,6 +153,7 @@ extern "C" int32_t fasa_calib_accumulate(fasa_ctx_t* ctx, const void* q, const v
   if (!ctx || !q || !k_cache || !seq_lens || !ca_counts || !n_used || !workspace) return FASA_ERR_INVALID_ARG;
   if (((uintptr_t)workspace & 255) != 0 || ((uintptr_t)ca_counts & 7) != 0 || ((uintptr_t)n_used & 7) != 0)
     return FASA_ERR_INVALID_ARG;
+  if (!fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
   if (!calib_args_ok(ctx, top_k) || ctx->fused_cs <= 0) return FASA_ERR_UNSUPPORTED;
   const fasa_config_t& c = ctx->cfg;
   cudaStream_t s = (cudaStream_t)stream;
@@ -166,7 +166,7 @@ extern "C" int32_t fasa_calib_accumulate(fasa_ctx_t* ctx, const void* q, const v
   dim3 grid((unsigned)((c.max_len + 32 * kCalibWarps - 1) / (32 * kCalibWarps)), (unsigned)samples);
   calib_score_kernel<<<grid, kCalibWarps * 32, 0, s>>>(
       (const uint16_t*)q, (const uint16_t*)k_cache, seq_lens, scores, ctx->d_status, c.n_q_heads, c.n_kv_heads,
-      c.max_len, c.rope_pairing, c.k_stride_b, c.k_stride_h, c.k_stride_t);
+      c.max_len, c.rope_pairing, c.k_stride_b, c.k_stride_h, c.k_stride_t, fasa_page_map(ctx));
   FASA_LAUNCH_CHECK(ctx);
   const int32_t st = fasa_fused_topk_rows(ctx, scores, seq_lens, top_k, top_k, idx, n_sel, c.n_q_heads * kRows,
                                           0, 0, s);

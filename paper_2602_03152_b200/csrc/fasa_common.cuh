@@ -22,6 +22,9 @@ struct fasa_ctx {
   int row_elems;          // bf16 elements per proxy row = 8 * chunks
   int device;
   int n_sm;
+  const int32_t* block_table;  // paged caches: device [batch][pages_per_seq], caller-owned; null until set
+  int page_shift;         // log2(page_size), 0 for contiguous caches
+  int pages_per_seq;      // ceil(max_len / page_size)
   int16_t* d_chan;        // device [n_kv_heads][row_elems]: K channel of each proxy element, -1 = padding
   int32_t* d_status;      // device status word (FASA_DEV_* bits)
   int32_t* d_arrive;      // device [batch]: CTAs of a sequence that have read its length (append-then-step)
@@ -79,6 +82,24 @@ int32_t fasa_fused_topk_rows(fasa_ctx* ctx, const float* scores, const int32_t* 
                              int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
                              int rows_per_seq, int n_sink, int n_recent, cudaStream_t stream);
 
+// Paged caches: how a (sequence, token) pair finds its page.  All zero = contiguous caches.
+struct PageMap {
+  const int32_t* table;   // [batch][pages_per_seq]: physical page of each logical page
+  int shift;              // log2(tokens per page)
+  int pages_per_seq;
+  int n_pages;
+};
+static inline PageMap fasa_page_map(const fasa_ctx* ctx) {
+  PageMap m;
+  m.table = ctx->block_table;
+  m.shift = ctx->page_shift;
+  m.pages_per_seq = ctx->pages_per_seq;
+  m.n_pages = ctx->cfg.n_pages;
+  return m;
+}
+// Paged contexts need their block table before any call that touches a cache.
+static inline bool fasa_pages_ready(const fasa_ctx* ctx) { return ctx->cfg.page_size == 0 || ctx->block_table != nullptr; }
+
 static inline size_t fasa_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 #ifdef __CUDACC__
@@ -109,6 +130,43 @@ __device__ __forceinline__ float dot8(const float2 (&q)[4], const uint4& k) {
   a = __ffma2_rn(q[2], bf16x2_to_f32x2(k.z), a);
   a = __ffma2_rn(q[3], bf16x2_to_f32x2(k.w), a);
   return a.x + a.y;
+}
+
+__device__ __forceinline__ bool page_ok(const PageMap& m, int page) { return page >= 0 && page < m.n_pages; }
+__device__ __forceinline__ int page_of(const PageMap& m, int b, int tok) {
+  return __ldg(m.table + (int64_t)b * m.pages_per_seq + (tok >> m.shift));
+}
+// Element offset of row `tok` of (sequence b, KV head h) in a K or V cache, for reading: an
+// entry outside the pool reads page 0 and raises the status bit.
+__device__ __forceinline__ int64_t cache_row(const PageMap& m, int b, int h, int tok, int64_t sb, int64_t sh,
+                                             int64_t st, int32_t* status) {
+  if (m.table == nullptr) return b * sb + h * sh + (int64_t)tok * st;
+  int page = page_of(m, b, tok);
+  if (!page_ok(m, page)) {
+    atomicOr(status, FASA_DEV_PAGE_CLAMPED);
+    page = 0;
+  }
+  return page * sb + h * sh + (int64_t)(tok & ((1 << m.shift) - 1)) * st;
+}
+// Byte offset of the proxy tile of token tile T (tokens 16 T .. 16 T + 15) of (b, h).
+// status == nullptr: a speculative read (a tile that may lie past the sequence's end, where no
+// page need be mapped) - page 0 is read and nothing is reported.
+__device__ __forceinline__ int64_t proxy_tile_offset(const PageMap& m, int b, int h, int n_kv_heads, int T,
+                                                     int tiles_per_unit, int tile_bytes, int32_t* status) {
+  if (m.table == nullptr) return ((int64_t)(b * n_kv_heads + h) * tiles_per_unit + T) * tile_bytes;
+  int page = (T >> (m.shift - 4)) < m.pages_per_seq ? page_of(m, b, T << 4) : -1;
+  if (!page_ok(m, page)) {
+    if (status) atomicOr(status, FASA_DEV_PAGE_CLAMPED);
+    page = 0;
+  }
+  const int tpp = 1 << (m.shift - 4);           // tiles per page
+  return (((int64_t)page * n_kv_heads + h) * tpp + (T & (tpp - 1))) * tile_bytes;
+}
+
+// Reports (status bit) a token tile whose page is not in the pool; for tiles that were read
+// speculatively and turned out to be part of the sequence.
+__device__ __forceinline__ void proxy_tile_check(const PageMap& m, int b, int T, int32_t* status) {
+  if (m.table != nullptr && !page_ok(m, page_of(m, b, T << 4))) atomicOr(status, FASA_DEV_PAGE_CLAMPED);
 }
 
 // A selection unit: `heads` consecutive query heads of one sequence that share an index set

@@ -19,12 +19,13 @@ struct TilesPerIter {
 };
 
 // KB = 16-channel blocks per tile rounded up to a power of two (1, 2, 4, 8).
-template <int KB, bool MAXRED>
+template <int KB, bool MAXRED, bool PAGED>
 __global__ void __launch_bounds__(kScoreThreads)
 fc_score_kernel(const uint16_t* __restrict__ q, const unsigned char* __restrict__ proxy,
                 const int32_t* __restrict__ seq_lens, const int16_t* __restrict__ chan,
                 float* __restrict__ scores, int32_t* __restrict__ status, int n_q_heads,
-                int n_kv_heads, int n_sets, int group, int max_len, int chunks, int tiles_per_cta) {
+                int n_kv_heads, int n_sets, int group, int max_len, int chunks, int tiles_per_cta,
+                const PageMap pm) {
   constexpr int TPI = TilesPerIter<KB>::value;
   const int u = blockIdx.y;
   const SelUnit su = sel_unit(u, n_sets, group, n_q_heads, n_kv_heads);
@@ -37,7 +38,12 @@ fc_score_kernel(const uint16_t* __restrict__ q, const unsigned char* __restrict_
   const int tiles_alloc = (max_len + 15) >> 4;
   const int cta_tile0 = blockIdx.x * tiles_per_cta;
   const int cta_tile1 = min(tiles_alloc, cta_tile0 + tiles_per_cta);
+  // (contiguous caches: plain pointer arithmetic, as compiled without the page map)
   const unsigned char* unit = proxy + (int64_t)su.kv * tiles_alloc * pg.tile_bytes;
+  auto tile_at = [&](int T, int32_t* report) {
+    if constexpr (PAGED) return proxy + proxy_tile_offset(pm, b, h, n_kv_heads, T, tiles_alloc, pg.tile_bytes, report);
+    else return unit + (int64_t)T * pg.tile_bytes;
+  };
 
   // First batch of loads: every tile up to max_len is allocated, so reading past the
   // sequence length is harmless and overlaps with the loads of the length and the query.
@@ -45,11 +51,16 @@ fc_score_kernel(const uint16_t* __restrict__ q, const unsigned char* __restrict_
   uint4 a[TPI][KB];
 #pragma unroll
   for (int j = 0; j < TPI; ++j)
-    load_tile<KB>(a[j], unit + (int64_t)(T + j) * pg.tile_bytes, pg, lane, T + j < cta_tile1);
+    load_tile<KB>(a[j], tile_at(PAGED ? min(T + j, tiles_alloc - 1) : T + j, nullptr), pg, lane, T + j < cta_tile1);
 
   const int len = clamp_len(seq_lens[b], max_len, status);
   if (cta_tile0 * 16 >= len) return;
   const int row1 = min(len, cta_tile1 * 16);
+  if constexpr (PAGED) {
+#pragma unroll
+    for (int j = 0; j < TPI; ++j)
+      if ((T + j) * 16 < row1) proxy_tile_check(pm, b, T + j, status);
+  }
 
   ScoreFrag<KB> f;
   load_score_b<KB>(f, q + su.q0 * FASA_HEAD_DIM,
@@ -64,7 +75,8 @@ fc_score_kernel(const uint16_t* __restrict__ q, const unsigned char* __restrict_
     if (next * 16 < row1) {
 #pragma unroll
       for (int j = 0; j < TPI; ++j)
-        load_tile<KB>(a[j], unit + (int64_t)(next + j) * pg.tile_bytes, pg, lane, (next + j) * 16 < row1);
+        load_tile<KB>(a[j], tile_at(PAGED ? min(next + j, tiles_alloc - 1) : next + j,
+                                    (next + j) * 16 < row1 ? status : nullptr), pg, lane, (next + j) * 16 < row1);
     }
 #pragma unroll
     for (int p = 0; p < TPI / 2; ++p) {
@@ -88,21 +100,21 @@ void launch_score(fasa_ctx* ctx, const void* q, const void* proxy, const int32_t
   int per = (tiles + want_ctas - 1) / want_ctas;
   per = (per + kStep - 1) / kStep * kStep;
   dim3 grid((unsigned)((tiles + per - 1) / per), (unsigned)units);
-  if (c.group_reduce == 0)
-    fc_score_kernel<KB, false><<<grid, kScoreThreads, 0, s>>>(
+  auto go = [&](auto kernel) {
+    kernel<<<grid, kScoreThreads, 0, s>>>(
         (const uint16_t*)q, (const unsigned char*)proxy, seq_lens, ctx->d_chan, scores, ctx->d_status,
-        c.n_q_heads, c.n_kv_heads, ctx->n_sets, ctx->sel_heads, c.max_len, ctx->chunks, per);
-  else
-    fc_score_kernel<KB, true><<<grid, kScoreThreads, 0, s>>>(
-        (const uint16_t*)q, (const unsigned char*)proxy, seq_lens, ctx->d_chan, scores, ctx->d_status,
-        c.n_q_heads, c.n_kv_heads, ctx->n_sets, ctx->sel_heads, c.max_len, ctx->chunks, per);
+        c.n_q_heads, c.n_kv_heads, ctx->n_sets, ctx->sel_heads, c.max_len, ctx->chunks, per, fasa_page_map(ctx));
+  };
+  const bool paged = c.page_size > 0;
+  if (c.group_reduce == 0) paged ? go(fc_score_kernel<KB, false, true>) : go(fc_score_kernel<KB, false, false>);
+  else paged ? go(fc_score_kernel<KB, true, true>) : go(fc_score_kernel<KB, true, false>);
 }
 
 }  // namespace
 
 extern "C" int32_t fasa_fc_score(fasa_ctx_t* ctx, const void* q, const void* proxy_k,
                                  const int32_t* seq_lens, float* scores, void* stream) {
-  if (!ctx || !q || !proxy_k || !seq_lens || !scores) return FASA_ERR_INVALID_ARG;
+  if (!ctx || !q || !proxy_k || !seq_lens || !scores || !fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
   if (((uintptr_t)proxy_k & 15) != 0 || ((uintptr_t)q & 1) != 0 || ((uintptr_t)scores & 3) != 0)
     return FASA_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;

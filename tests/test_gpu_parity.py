@@ -554,6 +554,162 @@ def test_seeded_random_configurations(w):
     assert rep["units"] == w.batch * w.n_sets
 
 
+# ---- paged caches: page pools + a block table; every call must give the contiguous results ----
+
+def _paged_twin(w, t, P, spare=3, seed=0, extra_tokens=0):
+    """A contiguous Run and a paged context over the same logical caches, pages in random order;
+    logical pages past what a sequence needs (its length + extra_tokens) stay unmapped (-1)."""
+    r = Run(w, t)
+    B, Hkv, Lm = w.batch, w.n_kv_heads, w.max_len
+    pps = (Lm + P - 1) // P
+    need = [min(pps, (int(l) + extra_tokens + P - 1) // P) for l in t["seq_lens"].tolist()]
+    n_pages = sum(need) + spare
+    perm = torch.randperm(n_pages, generator=torch.Generator().manual_seed(seed)).tolist()
+    table = torch.full((B, pps), -1, dtype=torch.int32)
+    it = iter(perm)
+    for b in range(B):
+        for lp in range(need[b]):
+            table[b, lp] = next(it)
+    f = binding.Fasa(B, w.n_q_heads, Hkv, Lm, t["dom"], rope_pairing=w.pairing, group_reduce=w.group_reduce,
+                     n_sink=w.n_sink, n_recent=w.n_recent, select_heads=w.sel_heads, page_size=P, n_pages=n_pages)
+    assert f.step_cluster_size() == 0
+    kp, vp = f.alloc_paged_cache(), f.alloc_paged_cache()
+    pad = pps * P - Lm
+    kl = torch.nn.functional.pad(t["k"], (0, 0, 0, pad)).view(B, Hkv, pps, P, 128)
+    vl = torch.nn.functional.pad(t["v"], (0, 0, 0, pad)).view(B, Hkv, pps, P, 128)
+    for b in range(B):
+        for lp in range(need[b]):
+            kp[table[b, lp]] = kl[b, :, lp].cuda()
+            vp[table[b, lp]] = vl[b, :, lp].cuda()
+    tab = table.cuda()
+    f.set_block_table(tab)
+    return r, f, kp, vp, tab, table, need
+
+
+def _logical(pool, table, need, P, Lm):
+    """[B, Hkv, Lm, ...] view of a page pool through the block table (unmapped pages read as zero)."""
+    B, pps = table.shape
+    out = torch.zeros((B, pool.shape[1], pps * P) + tuple(pool.shape[3:]), dtype=pool.dtype, device=pool.device)
+    for b in range(B):
+        for lp in range(need[b]):
+            out[b, :, lp * P:(lp + 1) * P] = pool[table[b, lp]]
+    return out[:, :, :Lm]
+
+
+@pytest.mark.parametrize("P,cfg,kw", [
+    (16, "c1", dict(batch=2, max_len=1000, len_lo=300, len_hi=990)),
+    (64, "c3", dict(batch=3, max_len=2100, len_lo=500, len_hi=2000)),
+    (256, "c1", dict(batch=2, max_len=3001, len_lo=1500, len_hi=2990, n_dom=5, pairing=1, sel_heads=1)),
+])
+def test_paged_caches_give_the_contiguous_results(P, cfg, kw):
+    w = C[cfg].replace(**kw)
+    t = synth.make_inputs(w, "cpu")
+    r, f, kp, vp, tab, table, need = _paged_twin(w, t, P, extra_tokens=45)
+    Lm = w.max_len
+    proxy_p = f.alloc_proxy()
+    lens_p = r.seq_lens.clone()
+    # Split of the whole cache
+    r.build_proxy()
+    f.proxy_build(kp, proxy_p, lens_p)
+    tiles = (Lm + 15) // 16
+    lp_proxy = _logical(proxy_p.view(f.n_pages, w.n_kv_heads, P // 16, -1), table, need, P // 16, tiles)
+    assert torch.equal(lp_proxy, r.proxy)
+    # a bulk append (40 rows) and single-token appends that cross page boundaries
+    g = torch.Generator().manual_seed(9)
+    kn = torch.randn((w.batch, w.n_kv_heads, 40, 128), generator=g).to(torch.bfloat16).cuda()
+    vn = torch.randn((w.batch, w.n_kv_heads, 40, 128), generator=g).to(torch.bfloat16).cuda()
+    r.fasa.kv_append(r.k, r.v, r.proxy, r.seq_lens, kn, vn)
+    f.kv_append(kp, vp, proxy_p, lens_p, kn, vn)
+    for i in range(5):
+        r.fasa.kv_append(r.k, r.v, r.proxy, r.seq_lens, kn[:, :, i:i + 1].contiguous(), vn[:, :, i:i + 1].contiguous())
+        f.kv_append(kp, vp, proxy_p, lens_p, kn[:, :, i:i + 1].contiguous(), vn[:, :, i:i + 1].contiguous())
+    torch.cuda.synchronize()
+    assert torch.equal(lens_p, r.seq_lens)
+    lens = r.seq_lens.cpu().tolist()
+    kl, vl = _logical(kp, table, need, P, Lm), _logical(vp, table, need, P, Lm)
+    for b, L in enumerate(lens):
+        assert torch.equal(kl[b, :, :L], r.k[b, :, :L]) and torch.equal(vl[b, :, :L], r.v[b, :, :L])
+    lp_proxy = _logical(proxy_p.view(f.n_pages, w.n_kv_heads, P // 16, -1), table, need, P // 16, tiles)
+    for b, L in enumerate(lens):
+        assert torch.equal(lp_proxy[b, :, :L // 16], r.proxy[b, :, :L // 16])
+    # the three calls, the composite step, the dense path, the append form and the calibration
+    out_p, lse_p = torch.zeros_like(r.out), torch.zeros_like(r.lse)
+    scores_p, idx_p, n_sel_p = torch.full_like(r.scores, SENTINEL), torch.full_like(r.idx, -7), torch.zeros_like(r.n_sel)
+    r.step()
+    f.fc_score(r.q, proxy_p, lens_p, scores_p)
+    f.topk(scores_p, lens_p, w.budget, idx_p, n_sel_p, r.ws)
+    f.sparse_decode_attn(r.q, kp, vp, idx_p, n_sel_p, out_p, r.ws, lse_p)
+    torch.cuda.synchronize()
+    for x, y in ((scores_p, r.scores), (idx_p, r.idx), (n_sel_p, r.n_sel), (out_p, r.out), (lse_p, r.lse)):
+        assert torch.equal(x, y)
+    out2 = torch.zeros_like(out_p)
+    n0 = f.launch_count()
+    f.decode_step(r.q, kp, vp, proxy_p, lens_p, w.budget, scores_p, idx_p, n_sel_p, out2, r.ws)
+    assert f.launch_count() - n0 == 4
+    r.dense_step()
+    dense_p = torch.zeros_like(r.dense)
+    f.full_decode_attn(r.q, kp, vp, lens_p, dense_p, r.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out2, r.out) and torch.equal(dense_p, r.dense)
+    out3 = torch.zeros_like(out_p)
+    f.sparse_decode_attn_static(r.q, kp, vp, idx_p, n_sel_p, out3)
+    s_ = synth.make_step_inputs(w, 1, "cuda")
+    r.fasa.set_step_mode(0)
+    r.fasa.append_decode_step(s_["q"], s_["k_new"], s_["v_new"], r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx,
+                              r.n_sel, r.out, r.ws)
+    f.append_decode_step(s_["q"], s_["k_new"], s_["v_new"], kp, vp, proxy_p, lens_p, w.budget, scores_p, idx_p, n_sel_p,
+                         out2, r.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out3, out_p)
+    assert torch.equal(lens_p, r.seq_lens) and torch.equal(idx_p, r.idx) and torch.equal(scores_p, r.scores)
+    assert float((out2 - r.out).abs().max()) <= 1e-4          # mode 0 attends with the scalar kernel
+    if w.batch * w.n_q_heads * 65 <= 65535:
+        top_k = 64
+        cc = [torch.zeros((w.n_q_heads, 64), dtype=torch.int64, device="cuda") for _ in range(2)]
+        uu = [torch.zeros(w.n_q_heads, dtype=torch.int64, device="cuda") for _ in range(2)]
+        ws_c = torch.empty(f.calib_workspace_bytes(top_k), dtype=torch.uint8, device="cuda")
+        r.fasa.calib_accumulate(r.q, r.k, r.seq_lens, top_k, cc[0], uu[0], ws_c)
+        f.calib_accumulate(r.q, kp, lens_p, top_k, cc[1], uu[1], ws_c)
+        torch.cuda.synchronize()
+        assert torch.equal(cc[0], cc[1]) and torch.equal(uu[0], uu[1]) and int(uu[0].min()) >= 1
+    assert f.device_status() == 0 and r.fasa.device_status() == 0
+    # and against the oracle, on the logical view of the pools
+    h = r.host()
+    kl, vl = _logical(kp, table, need, P, Lm), _logical(vp, table, need, P, Lm)
+    parity.check_step(s_["q"].cpu().double().numpy(), kl.cpu().double().numpy(), vl.cpu().double().numpy(),
+                      lens_p.cpu().numpy(), h["dom"], scores=scores_p.cpu().numpy(), idx=idx_p.cpu().numpy(),
+                      n_sel=n_sel_p.cpu().numpy(), out=out2.cpu().numpy(), what="paged", **r.oracle_kwargs())
+
+
+def test_paged_cache_table_errors_are_flagged_not_followed():
+    w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, max_len=256, len_lo=200, len_hi=200, budget=32)
+    t = synth.make_inputs(w, "cpu")
+    r, f, kp, vp, tab, table, need = _paged_twin(w, t, 64)
+    proxy_p = f.alloc_proxy()
+    lens = r.seq_lens.clone()
+    f.proxy_build(kp, proxy_p, lens)
+    assert f.device_status() == 0
+    # a block table must be set before a paged context touches a cache
+    g = binding.Fasa(1, 8, 2, 256, t["dom"], page_size=64, n_pages=8)
+    with pytest.raises(binding.FasaError):
+        g.proxy_build(kp, proxy_p, lens)
+    # reads through a bad entry use page 0 and raise the bit; the result stays finite
+    tab[0, 1] = 10 ** 6
+    f.full_decode_attn(r.q, kp, vp, lens, r.dense, r.ws)
+    assert f.device_status() == binding.DEV_PAGE_CLAMPED and torch.isfinite(r.dense).all()
+    tab[0, 1] = -1
+    f.fc_score(r.q, proxy_p, lens, r.scores)
+    assert f.device_status() == binding.DEV_PAGE_CLAMPED
+    # writes through a bad entry are dropped: the pools do not change
+    lens.fill_(64)
+    before = (kp.clone(), vp.clone(), proxy_p.clone())
+    s_ = synth.make_step_inputs(w, 0, "cuda")
+    f.kv_append(kp, vp, proxy_p, lens, s_["k_new"], s_["v_new"])
+    assert f.device_status() == binding.DEV_PAGE_CLAMPED
+    assert torch.equal(kp, before[0]) and torch.equal(vp, before[1]) and torch.equal(proxy_p, before[2])
+    assert lens.cpu().tolist() == [65]
+
+
 def test_strided_token_major_cache():
     # K/V stored [B][L][Hkv][128] (token-major), addressed through the stride fields.
     w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, batch=2, max_len=640, len_lo=400, len_hi=640, budget=40)
