@@ -693,6 +693,88 @@ def run_offload(args):
         "device_status": f.device_status()}), flush=True)
 
 
+def run_paged(args):
+    """Paged caches on --config's shape (page pools in random page order behind a block table): the
+    step as the three stand-alone kernels (what a paged context runs) and the dense path, next to
+    the same three kernels and the dense path on contiguous caches.  One JSON object."""
+    import numpy as np
+    import torch
+
+    from paper_2602_03152_b200 import binding, build, synth
+
+    build.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    w = synth.CONFIGS[args.config]
+    if args.budget is not None:
+        w = w.replace(budget=args.budget)
+    if args.batch is not None:
+        w = w.replace(batch=args.batch)
+    P = args.paged
+    t = synth.make_inputs(w, dev)
+    B, Hq, Hkv, Lm = w.batch, w.n_q_heads, w.n_kv_heads, w.max_len
+    pps = (Lm + P - 1) // P
+    n_pages = B * pps
+    table = torch.randperm(n_pages, generator=torch.Generator().manual_seed(1)).to(torch.int32).view(B, pps).to(dev)
+    fc = binding.Fasa.from_workload(w, t["dom"])
+    fp = binding.Fasa(B, Hq, Hkv, Lm, t["dom"], rope_pairing=w.pairing, group_reduce=w.group_reduce, n_sink=w.n_sink,
+                      n_recent=w.n_recent, select_heads=w.sel_heads, page_size=P, n_pages=n_pages)
+    fp.set_block_table(table)
+    kp, vp = fp.alloc_paged_cache(dev), fp.alloc_paged_cache(dev)
+    pad = pps * P - Lm
+    for src, dst in ((t["k"], kp), (t["v"], vp)):
+        lv = torch.nn.functional.pad(src, (0, 0, 0, pad)).view(B, Hkv, pps, P, 128).permute(0, 2, 1, 3, 4)
+        dst[table.long().view(-1)] = lv.reshape(B * pps, Hkv, P, 128)
+    n_sel_max = w.n_sel_max()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    res = {}
+    outs = {}
+    for name, f, k, v in (("contiguous", fc, t["k"], t["v"]), ("paged", fp, kp, vp)):
+        proxy = f.alloc_proxy(dev)
+        f.proxy_build(k, proxy, t["seq_lens"])
+        scores = torch.zeros((B, w.n_sets, Lm), dtype=torch.float32, device=dev)
+        idx = torch.zeros((B, w.n_sets, n_sel_max), dtype=torch.int32, device=dev)
+        n_sel = torch.zeros((B, w.n_sets), dtype=torch.int32, device=dev)
+        out = torch.zeros((B, Hq, 128), dtype=torch.float32, device=dev)
+        ws = f.alloc_workspace(n_sel_max, dev)
+        f.set_step_mode(1)
+
+        def three():
+            f.fc_score(t["q"], proxy, t["seq_lens"], scores)
+            f.topk(scores, t["seq_lens"], w.budget, idx, n_sel, ws)
+            f.sparse_decode_attn(t["q"], k, v, idx, n_sel, out, ws)
+
+        row = {}
+        for what, fn in (("step_three_kernels_us", three),
+                         ("dense_us", lambda: f.full_decode_attn(t["q"], k, v, t["seq_lens"], out, ws))):
+            ts = []
+            for i in range(args.warmup + args.steps):
+                flush.fill_(i & 1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn()
+                b.record()
+                b.synchronize()
+                if i >= args.warmup:
+                    ts.append(a.elapsed_time(b) * 1e3)
+            row[what] = float(np.mean(ts))
+        three()
+        torch.cuda.synchronize()
+        outs[name] = (out.clone(), idx.clone())
+        row["device_status"] = f.device_status()
+        res[name] = row
+        del proxy, scores
+    by = step_bytes(w, t["seq_lens"].cpu().tolist(), int(n_sel.sum().item()))
+    peak, _ = _peaks()
+    for name in res:
+        res[name]["step_frac_of_peak"] = by["fasa"] / res[name]["step_three_kernels_us"] / 1e3 / peak
+        res[name]["dense_frac_of_peak"] = by["dense"] / res[name]["dense_us"] / 1e3 / peak
+    print(json.dumps({"paged": w.name, "page_size": P, "n_pages": n_pages, "budget": w.budget, "steps": args.steps,
+                      "results_identical": bool(torch.equal(outs["paged"][0], outs["contiguous"][0]) and
+                                                torch.equal(outs["paged"][1], outs["contiguous"][1])),
+                      **res}), flush=True)
+
+
 def run_longcot(args):
     """Workload c3 (long-CoT shape, Qwen2.5-7B-like attention): 28 layers, batch 32, prompt
     1024 then 15360 decode steps, budget 18.9 % of the current length, 16 dominant FCs.  One
@@ -822,6 +904,8 @@ def main():
                     help="offline calibration (Algorithm 1) on --config's shape instead of the bench line; --budget = top-k")
     ap.add_argument("--offload", action="store_true",
                     help="FASA-M (Algorithm 2): K/V caches in page-locked host memory, instead of the bench line")
+    ap.add_argument("--paged", type=int, default=0, metavar="PAGE_SIZE",
+                    help="paged caches with this page size (a power of two >= 16) against contiguous ones, instead of the bench line")
     ap.add_argument("--no-resident", action="store_true", help="--longcot: skip the 28-layer resident measurement")
     ap.add_argument("--sweep-steps", type=int, default=20)
     ap.add_argument("--step-mode", type=int, default=None, choices=[0, 1],
@@ -836,6 +920,8 @@ def main():
         return run_calib(args)
     if args.offload:
         return run_offload(args)
+    if args.paged:
+        return run_paged(args)
     from paper_2602_03152_b200 import synth
     w = synth.CONFIGS[args.config]
     if args.budget is not None:

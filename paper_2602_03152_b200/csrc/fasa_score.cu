@@ -66,6 +66,17 @@ fc_score_kernel(const uint16_t* __restrict__ q, const unsigned char* __restrict_
   load_score_b<KB>(f, q + su.q0 * FASA_HEAD_DIM,
                    chan + h * chunks * 8, chunks, group, lane);
   float* srow = scores + (int64_t)u * max_len;
+  // Paged caches: the pages of the batch of tiles after this one are looked up one iteration
+  // ahead, so that the table reads overlap the proxy loads in flight instead of preceding them.
+  const unsigned char* ahead[TPI];
+  auto look_ahead = [&](int Tn) {
+    if constexpr (PAGED) {
+#pragma unroll
+      for (int j = 0; j < TPI; ++j)
+        ahead[j] = tile_at(min(Tn + j, tiles_alloc - 1), (Tn + j) * 16 < row1 ? status : nullptr);
+    }
+  };
+  look_ahead(T + kScoreWarps * TPI);
 
   while (T * 16 < row1) {       // uniform over the warp
     float s_lo[TPI], s_hi[TPI];
@@ -75,8 +86,8 @@ fc_score_kernel(const uint16_t* __restrict__ q, const unsigned char* __restrict_
     if (next * 16 < row1) {
 #pragma unroll
       for (int j = 0; j < TPI; ++j)
-        load_tile<KB>(a[j], tile_at(PAGED ? min(next + j, tiles_alloc - 1) : next + j,
-                                    (next + j) * 16 < row1 ? status : nullptr), pg, lane, (next + j) * 16 < row1);
+        load_tile<KB>(a[j], PAGED ? ahead[j] : tile_at(next + j, nullptr), pg, lane, (next + j) * 16 < row1);
+      look_ahead(next + kScoreWarps * TPI);
     }
 #pragma unroll
     for (int p = 0; p < TPI / 2; ++p) {
