@@ -37,11 +37,12 @@ def test_status_strings_and_row_elems(lib):
 
 def _cfg(**kw):
     base = dict(batch=1, n_q_heads=4, n_kv_heads=1, head_dim=128, max_len=64, n_dom=2, rope_pairing=0,
-                group_reduce=0, select_heads=0, n_sink=0, n_recent=0, softmax_scale=0.0)
+                group_reduce=0, select_heads=0, n_sink=0, n_recent=0, softmax_scale=0.0, page_size=0, n_pages=0)
     base.update(kw)
     return binding.FasaConfig(base["batch"], base["n_q_heads"], base["n_kv_heads"], base["head_dim"],
                               base["max_len"], base["n_dom"], base["rope_pairing"], base["group_reduce"],
-                              base["select_heads"], base["n_sink"], base["n_recent"], base["softmax_scale"], 0, 0, 0, 0, 0, 0)
+                              base["select_heads"], base["n_sink"], base["n_recent"], base["softmax_scale"], 0, 0, 0, 0, 0, 0,
+                              base["page_size"], base["n_pages"])
 
 
 @pytest.mark.parametrize("kw,expect", [
@@ -57,6 +58,9 @@ def _cfg(**kw):
     (dict(group_reduce=3), binding.ERR_UNSUPPORTED),
     (dict(select_heads=3), binding.ERR_UNSUPPORTED),      # does not divide the group of 4
     (dict(select_heads=-1), binding.ERR_UNSUPPORTED),
+    (dict(page_size=24, n_pages=4), binding.ERR_UNSUPPORTED),   # not a power of two
+    (dict(page_size=8, n_pages=4), binding.ERR_UNSUPPORTED),    # smaller than a 16-token proxy tile
+    (dict(page_size=16, n_pages=0), binding.ERR_UNSUPPORTED),   # an empty pool
 ])
 def test_create_rejects_bad_config_without_a_gpu(lib, kw, expect):
     cfg = _cfg(**kw)
