@@ -251,9 +251,11 @@ int32_t fasa_sparse_decode_attn_static(fasa_ctx_t* ctx, const void* q, const voi
  * `workspace` may be NULL and `scores` may be NULL (they are then not written).  Available
  * when ceil(max_len / 16) <= 22528 and the device can co-schedule such a cluster;
  * fasa_step_cluster_size tells.
- * When a workspace is given and the selection is large (n_sel_max * ceil(group / 4) >= 2048),
- * mode 1 ends the cluster kernel after the selection and attends with the split-K
- * tensor-core kernel of fasa_sparse_decode_attn (three launches instead of one).
+ * When a workspace is given and the selection is large (n_sel_max * ceil(heads per set / 4)
+ * >= 2048; >= 512 when all units together reach 24576 such rows; >= 256 when the cluster
+ * kernel's grid exceeds two CTAs per SM), mode 1 ends the
+ * cluster kernel after the selection and attends with the split-K tensor-core kernel of
+ * fasa_sparse_decode_attn (three launches instead of one).
  * Mode 0, and every configuration mode 1 cannot take: fasa_fc_score -> fasa_topk ->
  * fasa_sparse_decode_attn; scores and workspace are then required (INVALID_ARG if NULL).
  * Both modes select identical index sets; outputs agree to fp32 rounding.

@@ -129,8 +129,13 @@ decode_attn_kernel(const AttnParams p) {
           atomicOr(p.status, FASA_DEV_IDX_CLAMPED);
           t = 0;
         }
-        kk[i] = ld_stream_u4(kbase + cache_row(p.pm, b, h, t, p.ksb, p.ksh, p.kst, p.status));
-        vv[i] = ld_stream_u4(vbase + cache_row(p.pm, b, h, t, p.vsb, p.vsh, p.vst, p.status));
+        if (p.pm.table != nullptr) {
+          kk[i] = ld_stream_u4(kbase + cache_row(p.pm, b, h, t, p.ksb, p.ksh, p.kst, p.status));
+          vv[i] = ld_stream_u4(vbase + cache_row(p.pm, b, h, t, p.vsb, p.vsh, p.vst, p.status));
+        } else {
+          kk[i] = ld_stream_u4(kbase + b * p.ksb + h * p.ksh + (int64_t)t * p.kst);
+          vv[i] = ld_stream_u4(vbase + b * p.vsb + h * p.vsh + (int64_t)t * p.vst);
+        }
       } else {
         kk[i] = make_uint4(0u, 0u, 0u, 0u);
         vv[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -339,7 +344,7 @@ cudaError_t launch_after_predecessor(Kernel kernel, dim3 grid, dim3 block, size_
   return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
-template <bool SPARSE>
+template <bool SPARSE, bool PAGED>
 __global__ void __launch_bounds__(kMmaThreads)
 decode_attn_mma_kernel(const AttnParams p) {
   pdl_wait_for_predecessor();
@@ -412,20 +417,24 @@ decode_attn_mma_kernel(const AttnParams p) {
   // logits), so memory stays busy while the warp computes.  One cp.async group per buffer
   // fill, an empty group when there is no next tile, so "all but the newest group" always
   // names the buffer that is needed next.
-  auto stage = [&](uint16_t (*dst)[kRowPad], const uint16_t* cache, int64_t sb, int64_t sh, int64_t st, int base) {
+  const uint16_t* kunit = PAGED ? p.k : p.k + b * p.ksb + h * p.ksh;
+  const uint16_t* vunit = PAGED ? p.v : p.v + b * p.vsb + h * p.vsh;
+  auto stage = [&](uint16_t (*dst)[kRowPad], const uint16_t* unit, int64_t sb, int64_t sh, int64_t st, int base) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int row = 2 * j + (lane >> 4);
       const int r = min(base + row, r1 - 1);        // rows past the end repeat the last one (masked below)
       const int tok = SPARSE ? s_idx[r - r0] : r;
       const int c8 = (lane & 15) * 8;
-      cp_async16(&dst[row][c8], cache + cache_row(p.pm, b, h, tok, sb, sh, st, p.status) + c8);
+      // (contiguous caches keep the plain address arithmetic: the page map costs registers)
+      if constexpr (PAGED) cp_async16(&dst[row][c8], unit + cache_row(p.pm, b, h, tok, sb, sh, st, p.status) + c8);
+      else cp_async16(&dst[row][c8], unit + (int64_t)tok * st + c8);
     }
   };
   constexpr int kTileStep = kMmaWarps * 16;
-  if (r0 + warp * 16 < r1) stage(sm.k[warp], p.k, p.ksb, p.ksh, p.kst, r0 + warp * 16);
+  if (r0 + warp * 16 < r1) stage(sm.k[warp], kunit, p.ksb, p.ksh, p.kst, r0 + warp * 16);
   cp_async_commit();
-  if (r0 + warp * 16 < r1) stage(sm.v[warp], p.v, p.vsb, p.vsh, p.vst, r0 + warp * 16);
+  if (r0 + warp * 16 < r1) stage(sm.v[warp], vunit, p.vsb, p.vsh, p.vst, r0 + warp * 16);
   cp_async_commit();
 
   for (int base = r0 + warp * 16; base < r1; base += kTileStep) {   // uniform over the warp
@@ -474,7 +483,7 @@ decode_attn_mma_kernel(const AttnParams p) {
       sm.p_lo[warp][head][row] = (uint16_t)f32_to_bf16_bits(rest);
     }
     __syncwarp();                                   // P is visible; every lane is done with the K buffer
-    if (more) stage(sm.k[warp], p.k, p.ksb, p.ksh, p.kst, base + kTileStep);
+    if (more) stage(sm.k[warp], kunit, p.ksb, p.ksh, p.kst, base + kTileStep);
     cp_async_commit();
     cp_async_wait<1>();                             // this tile's V rows have landed
     __syncwarp();
@@ -496,7 +505,7 @@ decode_attn_mma_kernel(const AttnParams p) {
       mma16816(acc[cb], a, pl0, pl1);
     }
     __syncwarp();                                   // every lane is done with the V buffer
-    if (more) stage(sm.v[warp], p.v, p.vsb, p.vsh, p.vst, base + kTileStep);
+    if (more) stage(sm.v[warp], vunit, p.vsb, p.vsh, p.vst, base + kTileStep);
     cp_async_commit();
   }
   cp_async_wait<0>();
@@ -630,7 +639,7 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   dim3 grid((unsigned)plan.n_splits, (unsigned)(c.batch * n_sets));
   if (ctx->use_fused) {   // default: the tensor-core kernel (mode 0 keeps the scalar one)
     static_assert(sizeof(MmaSmem) >= (size_t)kMmaWarps * 8 * (FASA_HEAD_DIM + 2) * sizeof(float), "combine area");
-    auto fn = decode_attn_mma_kernel<SPARSE>;
+    auto fn = c.page_size > 0 ? decode_attn_mma_kernel<SPARSE, true> : decode_attn_mma_kernel<SPARSE, false>;
     // (+ the slice of the index list: chunk <= 2048 rows)
     const size_t smem = sizeof(MmaSmem) + (SPARSE ? (size_t)plan.chunk * sizeof(int32_t) : 0);
     FASA_CUDA_TRY(ctx, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize,

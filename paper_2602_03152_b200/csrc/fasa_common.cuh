@@ -69,9 +69,22 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
                           float* out, float* lse, const void* k_new, const void* v_new,
                           cudaStream_t stream, bool with_attention = true, float* out_mirror = nullptr);
 // Large selections are attended by the split-K tensor-core kernel rather than inside the
-// cluster kernel (whose attention phase runs on CUDA cores at 64 registers per thread).
+// cluster kernel (whose attention phase runs on CUDA cores at 64 registers per thread).  When
+// the cluster kernel's grid needs several waves of CTAs, every wave pays for its attention
+// phase with idle HBM while one split-K launch covers all units at once: the hand-over then
+// starts at much smaller selections (measured at B 16 x 8 heads, 64-128 K: 202 vs 223 us at
+// budget 256, 218 vs 250 us at 1024).
 static inline bool fasa_attend_separately(const fasa_ctx* ctx, int n_sel_max, const void* workspace) {
-  return workspace != nullptr && (long long)n_sel_max * ((ctx->sel_heads + 3) / 4) >= 2048;
+  const long long rows = (long long)n_sel_max * ((ctx->sel_heads + 3) / 4);
+  const long long ctas = (long long)ctx->cfg.batch * ctx->n_sets * ctx->fused_cs;
+  const bool several_waves = ctas > 2ll * ctx->n_sm;
+  // One wave: the two extra launches pay off once a unit has ~512 rows to attend and the
+  // units together ~24 K (B 8 x 8 heads, 64 K: 82.9 vs 86.0 us at budget 512, 87.0 vs 98.3 us
+  // at 1024; B 32 x 4 heads with 7 query heads each, context 4096: 48.2 vs 63.5 us; a batch-1
+  // step with 8 units stays in one launch: 28.7 vs 33.7 us at budget 512).
+  const long long all_rows = rows * ctx->cfg.batch * ctx->n_sets;
+  return workspace != nullptr &&
+         (rows >= 2048 || (several_waves && rows >= 256) || (rows >= 512 && all_rows >= 24576));
 }
 
 int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
