@@ -107,14 +107,15 @@ kv_append_kernel(uint16_t* __restrict__ k_cache, uint16_t* __restrict__ v_cache,
 // the CTA reports in on the sequence's arrival counter (the last one stores the new length).
 // Otherwise: source = the cache rows themselves, j < seq_lens[b].
 constexpr int kBulkRows = 16;
-template <bool APPEND>
+template <bool APPEND, bool PAGED>
 __global__ void __launch_bounds__(256)
 bulk_rows_kernel(uint16_t* k_cache, uint16_t* __restrict__ v_cache, unsigned char* __restrict__ proxy,
                  const int32_t* seq_lens /* same memory as seq_lens_w */, const uint16_t* __restrict__ k_new,
                  const uint16_t* __restrict__ v_new, const int16_t* __restrict__ chan,
                  int32_t* __restrict__ status, int n_new, int n_kv_heads, int max_len, int chunks,
                  int64_t ksb, int64_t ksh, int64_t kst, int64_t vsb, int64_t vsh, int64_t vst,
-                 int32_t* seq_lens_w, int32_t* arrive, const PageMap pm) {
+                 int32_t* seq_lens_w, int32_t* arrive, const PageMap pm_arg) {
+  const PageMap pm = PAGED ? pm_arg : PageMap{nullptr, 0, 0, 0};   // contiguous: the translation folds away
   __shared__ __align__(16) uint16_t s_k[kBulkRows][FASA_HEAD_DIM];
   const int u = blockIdx.y;
   const int h = u % n_kv_heads;
@@ -187,7 +188,8 @@ extern "C" int32_t fasa_kv_append(fasa_ctx_t* ctx, void* k_cache, void* v_cache,
   cudaStream_t s = (cudaStream_t)stream;
   if (n_new >= kBulkRows) {
     dim3 grid((unsigned)((n_new + kBulkRows - 1) / kBulkRows), (unsigned)(c.batch * c.n_kv_heads));
-    bulk_rows_kernel<true><<<grid, 256, 0, s>>>(
+    auto bulk = c.page_size > 0 ? bulk_rows_kernel<true, true> : bulk_rows_kernel<true, false>;
+    bulk<<<grid, 256, 0, s>>>(
         (uint16_t*)k_cache, (uint16_t*)v_cache, (unsigned char*)proxy_k, seq_lens, (const uint16_t*)k_new,
         (const uint16_t*)v_new, ctx->d_chan, ctx->d_status, n_new, c.n_kv_heads, c.max_len, ctx->chunks,
         c.k_stride_b, c.k_stride_h, c.k_stride_t, c.v_stride_b, c.v_stride_h, c.v_stride_t, seq_lens, ctx->d_arrive,
@@ -209,7 +211,8 @@ extern "C" int32_t fasa_proxy_build(fasa_ctx_t* ctx, const void* k_cache, void* 
   if (!aligned16(k_cache) || !aligned16(proxy_k) || !fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
   const fasa_config_t& c = ctx->cfg;
   dim3 grid((unsigned)((c.max_len + kBulkRows - 1) / kBulkRows), (unsigned)(c.batch * c.n_kv_heads));
-  bulk_rows_kernel<false><<<grid, 256, 0, (cudaStream_t)stream>>>(
+  auto build = c.page_size > 0 ? bulk_rows_kernel<false, true> : bulk_rows_kernel<false, false>;
+  build<<<grid, 256, 0, (cudaStream_t)stream>>>(
       const_cast<uint16_t*>((const uint16_t*)k_cache), nullptr, (unsigned char*)proxy_k, seq_lens, nullptr, nullptr,
       ctx->d_chan, ctx->d_status, 0, c.n_kv_heads, c.max_len, ctx->chunks, c.k_stride_b, c.k_stride_h,
       c.k_stride_t, 0, 0, 0, nullptr, nullptr, fasa_page_map(ctx));

@@ -29,6 +29,7 @@ constexpr int kPad = 33;                      // row stride of the staging tile 
 // tokens: lane l evaluates FCs l and l + 32 of one token at a time (coalesced 2-byte loads of
 // the key row), the tile is transposed through shared memory and every score row is written
 // with coalesced 128-byte stores.
+template <bool PAGED>
 __global__ void __launch_bounds__(kCalibWarps * 32)
 calib_score_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
                    const int32_t* __restrict__ seq_lens, float* __restrict__ scores,
@@ -61,7 +62,8 @@ calib_score_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ 
   }
   const int n_tok = min(32, len - base);
   for (int tt = 0; tt < n_tok; ++tt) {
-    const uint16_t* krow = k + cache_row(pm, b, h, base + tt, ksb, ksh, kst, status);
+    const uint16_t* krow = PAGED ? k + cache_row(pm, b, h, base + tt, ksb, ksh, kst, status)
+                                 : k + b * ksb + h * ksh + (int64_t)(base + tt) * kst;
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
       const float p0 = qv[e][0] * bf16_bits_to_f32(krow[c[e][0]]);     // exact
@@ -164,7 +166,8 @@ extern "C" int32_t fasa_calib_accumulate(fasa_ctx_t* ctx, const void* q, const v
   const int samples = c.batch * c.n_q_heads;
 
   dim3 grid((unsigned)((c.max_len + 32 * kCalibWarps - 1) / (32 * kCalibWarps)), (unsigned)samples);
-  calib_score_kernel<<<grid, kCalibWarps * 32, 0, s>>>(
+  auto score = c.page_size > 0 ? calib_score_kernel<true> : calib_score_kernel<false>;
+  score<<<grid, kCalibWarps * 32, 0, s>>>(
       (const uint16_t*)q, (const uint16_t*)k_cache, seq_lens, scores, ctx->d_status, c.n_q_heads, c.n_kv_heads,
       c.max_len, c.rope_pairing, c.k_stride_b, c.k_stride_h, c.k_stride_t, fasa_page_map(ctx));
   FASA_LAUNCH_CHECK(ctx);
