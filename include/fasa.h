@@ -158,7 +158,9 @@ int64_t fasa_launch_count(const fasa_ctx_t* ctx);
  * seq_lens[b]+n_new-1 of the caches, the dominant-FC slices of the new keys go
  * to the same rows of proxy_k, then seq_lens[b] += n_new (on the device, in
  * stream order).  k_new, v_new: bf16 [batch][n_kv_heads][n_new][128], post-RoPE.
- * Rows that would pass max_len are dropped and FASA_DEV_APPEND_FULL is set. */
+ * Rows that would pass max_len are dropped and FASA_DEV_APPEND_FULL is set.
+ * One launch: a row per half-CTA for a few rows, 16 rows per CTA (keys staged in
+ * shared memory once) from n_new = 16 on, the size of a prompt. */
 int32_t fasa_kv_append(fasa_ctx_t* ctx, void* k_cache, void* v_cache, void* proxy_k,
                        int32_t* seq_lens, const void* k_new, const void* v_new,
                        int32_t n_new, void* stream);
@@ -173,8 +175,10 @@ int32_t fasa_proxy_build(fasa_ctx_t* ctx, const void* k_cache, void* proxy_k,
 /* scores[b][h][j] = reduce_{g in group(h)} sum_{i in I_dom(h)}
  *                   (q[b][g][c0(i)] K[j][c0(i)] + q[b][g][c1(i)] K[j][c1(i)])
  * for j < seq_lens[b], read from proxy_k; exact bf16 products accumulated in fp32 per
- * query head on tensor cores, the heads then reduced in fp32; no scaling.  scores: fp32 [batch][n_kv_heads][max_len]; entries at
- * j >= seq_lens[b] are left untouched.  -0 is stored as +0. */
+ * query head on tensor cores, the heads then reduced in fp32; no scaling.
+ * scores: fp32 [batch][n_kv_heads][max_len] (n_sets rows per sequence with select_heads,
+ * here and for idx / n_sel below; see "Index sets"); entries at j >= seq_lens[b] are left
+ * untouched.  -0 is stored as +0. */
 int32_t fasa_fc_score(fasa_ctx_t* ctx, const void* q, const void* proxy_k,
                       const int32_t* seq_lens, float* scores, void* stream);
 
