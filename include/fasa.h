@@ -44,8 +44,7 @@
  *     proxy: [n_pages][n_kv_heads][page_size / 16 tiles], fasa_proxy_bytes() in all.
  *     Token positions everywhere else (seq_lens, idx, scores) stay logical.  Reads through
  *     an entry outside [0, n_pages) use page 0 and set FASA_DEV_PAGE_CLAMPED, writes through
- *     one are dropped.  Paged contexts run the step as separate kernels (scoring, TopK-I,
- *     attention): fasa_step_cluster_size() is 0 for them.
+ *     one are dropped.  Every call takes paged caches, the one-launch step included.
  *   - Frequency chunk (FC) i, 0 <= i < 64, is the channel pair (i, i+64) with
  *     rope_pairing 0 (rotate-half layout) or (2i, 2i+1) with rope_pairing 1
  *     (the paper's Eq. 1 layout).  An FC is never split (Appendix, design choices).

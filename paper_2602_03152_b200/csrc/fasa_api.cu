@@ -127,7 +127,6 @@ extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_h
     return FASA_ERR_CUDA;
   }
   fasa_fused_plan(ctx);
-  if (c.page_size > 0) ctx->fused_step_ok = 0;   // the one-launch step reads contiguous caches only
   ctx->use_fused = 1;
   *out = ctx;
   return FASA_OK;

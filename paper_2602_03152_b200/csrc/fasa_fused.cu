@@ -68,6 +68,7 @@ struct FusedParams {
   int max_reduce;          // score of a KV head = max over its query heads instead of their sum
   int64_t ksb, ksh, kst, vsb, vsh, vst;
   float scale_log2;        // softmax_scale * log2(e)
+  PageMap pm;              // paged caches (all zero: contiguous)
 };
 
 __device__ __forceinline__ uint2 ld_stream_u2(const void* p) {
@@ -107,7 +108,9 @@ __device__ __forceinline__ bool warp_find_kth(uint32_t v, uint32_t kth, int lane
 // instead of the proxy stream, and the kernel ends after the index list is written.  MODE 2:
 // the step without its attention phase (large selections are attended by the split-K
 // tensor-core kernel instead).
-template <int KB, int NG, int MODE>
+// PAGED: K, V and the proxy are page pools behind a block table (compiled separately, so that
+// the contiguous form keeps its plain address arithmetic within 64 registers).
+template <int KB, int NG, int MODE, bool PAGED = false>
 __global__ void __launch_bounds__(kFT, 2)
 fused_decode_kernel(const FusedParams p) {
   cg::cluster_group cluster = cg::this_cluster();
@@ -209,15 +212,33 @@ fused_decode_kernel(const FusedParams p) {
   const int n_blocks = pg.n16 + pg.n8;
   const unsigned char* unit = p.proxy + (int64_t)su.kv * ((p.max_len + 15) >> 4) * pg.tile_bytes;
   float* srow = p.scores ? p.scores + (int64_t)u * p.max_len : nullptr;
-  auto fetch = [&](uint4 (&a)[TPI][KB], int T, int grp) {
+  const int tiles_alloc = (p.max_len + 15) >> 4;
+  // Paged caches: the tiles of a batch are located through the block table.  The table is read
+  // one batch ahead (tp_next) so that its latency overlaps the proxy loads in flight.
+  const unsigned char* tp[PAGED ? TPI : 1];
+  const unsigned char* tp_next[PAGED ? TPI : 1];
+  auto locate = [&](const unsigned char* (&out)[PAGED ? TPI : 1], int T) {
+    if constexpr (PAGED) {
 #pragma unroll
-    for (int j = 0; j < TPI; ++j)
-      load_tile<KB>(a[j], unit + (int64_t)(T + j) * pg.tile_bytes, pg, lane, (T + j) * 16 < c1, grp * KB);
+      for (int j = 0; j < TPI; ++j)
+        out[j] = p.proxy + proxy_tile_offset(p.pm, b, h, p.n_kv_heads, min(T + j, tiles_alloc - 1), tiles_alloc,
+                                             pg.tile_bytes, (T + j) * 16 < c1 ? p.status : nullptr);
+    }
+  };
+  auto fetch = [&](uint4 (&a)[TPI][KB], int T, int grp) {      // (paged: tp holds the tiles of batch T)
+#pragma unroll
+    for (int j = 0; j < TPI; ++j) {
+      const unsigned char* tile;
+      if constexpr (PAGED) tile = tp[j];
+      else tile = unit + (int64_t)(T + j) * pg.tile_bytes;
+      load_tile<KB>(a[j], tile, pg, lane, (T + j) * 16 < c1, grp * KB);
+    }
   };
   const int step = kFW * TPI;
   int T = ((crank * per) >> 4) + warp * TPI;                  // slices start on a tile boundary
   const bool own_new = grows && c0 <= len_old && len_old < c1;
   uint4 a[TPI][KB];
+  if (MODE != 1) locate(tp, T);
   if (MODE != 1 && !own_new) fetch(a, T, 0);
 
   if (own_new) {
@@ -225,22 +246,37 @@ fused_decode_kernel(const FusedParams p) {
     // dominant-FC pairs of the key (one lane per 16-byte chunk), as in fasa_kv_append.  When
     // several units share a KV head each writes the same values, and reads back its own.
     const uint16_t* ksrc = p.k_new + (int64_t)su.kv * FASA_HEAD_DIM;
-    if (tid < 16) {
-      *reinterpret_cast<uint4*>(p.k_w + b * p.ksb + h * p.ksh + (int64_t)len_old * p.kst + tid * 8) =
-          *reinterpret_cast<const uint4*>(ksrc + tid * 8);
+    const ProxyGeom pg = proxy_geom(p.chunks);
+    // where the row goes: the sequence's own cache, or (paged) the page of position len_old; a
+    // table entry outside the pool drops the row
+    int64_t koff = b * p.ksb + h * p.ksh + (int64_t)len_old * p.kst;
+    int64_t voff = b * p.vsb + h * p.vsh + (int64_t)len_old * p.vst;
+    int64_t poff = (int64_t)su.kv * ((p.max_len + 15) >> 4) * pg.tile_bytes;
+    int prow = len_old;
+    bool row_ok = true;
+    if constexpr (PAGED) {
+      const int page = page_of(p.pm, b, len_old);
+      row_ok = page_ok(p.pm, page);
+      if (!row_ok && tid == 0) atomicOr(p.status, FASA_DEV_PAGE_CLAMPED);
+      prow = len_old & ((1 << p.pm.shift) - 1);
+      koff = page * p.ksb + h * p.ksh + (int64_t)prow * p.kst;
+      voff = page * p.vsb + h * p.vsh + (int64_t)prow * p.vst;
+      poff = ((int64_t)page * p.n_kv_heads + h) * (1 << (p.pm.shift - 4)) * pg.tile_bytes;
+    }
+    if (!row_ok) {
+    } else if (tid < 16) {
+      *reinterpret_cast<uint4*>(p.k_w + koff + tid * 8) = *reinterpret_cast<const uint4*>(ksrc + tid * 8);
     } else if (tid < 32) {
       const int c = tid - 16;
-      *reinterpret_cast<uint4*>(p.v_w + b * p.vsb + h * p.vsh + (int64_t)len_old * p.vst + c * 8) =
+      *reinterpret_cast<uint4*>(p.v_w + voff + c * 8) =
           *reinterpret_cast<const uint4*>(p.v_new + (int64_t)su.kv * FASA_HEAD_DIM + c * 8);
     } else if (tid - 32 < 4 * p.chunks) {
       const int w = tid - 32;                       // one dominant FC = one 4-byte channel pair
-      const ProxyGeom pg = proxy_geom(p.chunks);
       const int16_t* ch = p.chan + h * p.chunks * 8 + 2 * w;
       const int ch0 = ch[0], ch1 = ch[1];
       const uint32_t lo = ch0 >= 0 ? ksrc[ch0] : 0u;
       const uint32_t hi = ch1 >= 0 ? ksrc[ch1] : 0u;
-      unsigned char* unit = p.proxy_w + (int64_t)su.kv * ((p.max_len + 15) >> 4) * pg.tile_bytes;
-      *reinterpret_cast<uint32_t*>(unit + proxy_word_offset(pg, len_old, w)) = lo | (hi << 16);
+      *reinterpret_cast<uint32_t*>(p.proxy_w + poff + proxy_word_offset(pg, prow, w)) = lo | (hi << 16);
     }
   }
   for (int i = tid; i < 2 * kFBins; i += kFT) hist0[i] = 0u;
@@ -281,6 +317,7 @@ fused_decode_kernel(const FusedParams p) {
     }
   } else {
     if (own_new) fetch(a, T, 0);                              // (the new row is in place now)
+    locate(tp_next, T + step);
     while (T * 16 < c1) {       // uniform over the warp
       float c[TPI][4];
 #pragma unroll
@@ -290,8 +327,16 @@ fused_decode_kernel(const FusedParams p) {
 #pragma unroll
         for (int j = 0; j < TPI; ++j) mma_tile<KB>(c[j], a[j], f[grp], n_blocks - grp * KB);
         // the registers are free again: the next group, or the next batch of tiles, at once
-        if (grp + 1 < NG) fetch(a, T, grp + 1);
-        else if ((T + step) * 16 < c1) fetch(a, T + step, 0);
+        if (grp + 1 < NG) {
+          fetch(a, T, grp + 1);
+        } else if ((T + step) * 16 < c1) {
+          if constexpr (PAGED) {
+#pragma unroll
+            for (int j = 0; j < TPI; ++j) tp[j] = tp_next[j];
+          }
+          fetch(a, T + step, 0);
+          locate(tp_next, T + 2 * step);
+        }
       }
 #pragma unroll
       for (int pr = 0; pr < TPI / 2; ++pr) {
@@ -561,8 +606,13 @@ fused_decode_kernel(const FusedParams p) {
 #pragma unroll
       for (int i = 0; i < R; ++i) {
         const int t = min(max(tok[i], 0), p.max_len - 1);
-        kk[i] = ld_stream_u2(kbase + (int64_t)t * p.kst);
-        vv[i] = ld_stream_u2(vbase + (int64_t)t * p.vst);
+        if constexpr (PAGED) {
+          kk[i] = ld_stream_u2(p.k + lane * 4 + cache_row(p.pm, b, h, t, p.ksb, p.ksh, p.kst, p.status));
+          vv[i] = ld_stream_u2(p.v + lane * 4 + cache_row(p.pm, b, h, t, p.vsb, p.vsh, p.vst, p.status));
+        } else {
+          kk[i] = ld_stream_u2(kbase + (int64_t)t * p.kst);
+          vv[i] = ld_stream_u2(vbase + (int64_t)t * p.vst);
+        }
       }
       float part[16];
 #pragma unroll
@@ -732,22 +782,23 @@ size_t fused_smem_bytes(int cap) {
 
 using FusedFn = void (*)(const FusedParams);
 
-FusedFn fused_fn(int chunks) {
+template <int MODE, bool PAGED>
+FusedFn fused_variant(int chunks) {
   const int nb = (chunks + 1) / 2;      // 16-channel blocks per tile, the 8-channel one included
-  if (nb <= 1) return fused_decode_kernel<1, 1, 0>;
-  if (nb <= 2) return fused_decode_kernel<2, 1, 0>;
-  if (nb <= 4) return fused_decode_kernel<4, 1, 0>;
-  return fused_decode_kernel<4, 2, 0>;
+  if (nb <= 1) return fused_decode_kernel<1, 1, MODE, PAGED>;
+  if (nb <= 2) return fused_decode_kernel<2, 1, MODE, PAGED>;
+  if (nb <= 4) return fused_decode_kernel<4, 1, MODE, PAGED>;
+  return fused_decode_kernel<4, 2, MODE, PAGED>;
+}
+
+FusedFn fused_fn(int chunks, bool paged = false) {
+  return paged ? fused_variant<0, true>(chunks) : fused_variant<0, false>(chunks);
 }
 
 FusedFn topk_fn() { return fused_decode_kernel<1, 1, 1>; }
 
-FusedFn select_fn(int chunks) {         // the step without attention
-  const int nb = (chunks + 1) / 2;
-  if (nb <= 1) return fused_decode_kernel<1, 1, 2>;
-  if (nb <= 2) return fused_decode_kernel<2, 1, 2>;
-  if (nb <= 4) return fused_decode_kernel<4, 1, 2>;
-  return fused_decode_kernel<4, 2, 2>;
+FusedFn select_fn(int chunks, bool paged = false) {         // the step without attention
+  return paged ? fused_variant<2, true>(chunks) : fused_variant<2, false>(chunks);
 }
 
 }  // namespace
@@ -761,7 +812,8 @@ int fasa_fused_plan(fasa_ctx* ctx) {
   ctx->fused_smem = 0;
   ctx->fused_step_ok = 1;
   const int units = c.batch * ctx->n_sets;
-  FusedFn fn = fused_fn(ctx->chunks);
+  const bool paged = c.page_size > 0;
+  FusedFn fn = fused_fn(ctx->chunks, paged);
   auto cap_of = [&](int cs) { return (((c.max_len + cs - 1) / cs) + 31) & ~31; };
   // Two CTAs per SM can be resident; a cluster is doubled while the whole grid still fits
   // in one wave of them and every CTA keeps at least 512 tokens.
@@ -803,9 +855,9 @@ int fasa_fused_plan(fasa_ctx* ctx) {
     }
     // the select-only forms of the kernel run with the same cluster shape
     if (cudaFuncSetAttribute((const void*)topk_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit) != cudaSuccess ||
-        cudaFuncSetAttribute((const void*)select_fn(ctx->chunks), cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit) != cudaSuccess ||
+        cudaFuncSetAttribute((const void*)select_fn(ctx->chunks, paged), cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit) != cudaSuccess ||
         (cs > 8 && (cudaFuncSetAttribute((const void*)topk_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-                    cudaFuncSetAttribute((const void*)select_fn(ctx->chunks), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess))) {
+                    cudaFuncSetAttribute((const void*)select_fn(ctx->chunks, paged), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess))) {
       cudaGetLastError();
       continue;
     }
@@ -837,7 +889,10 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
   p.ksb = c.k_stride_b; p.ksh = c.k_stride_h; p.kst = c.k_stride_t;
   p.vsb = c.v_stride_b; p.vsh = c.v_stride_h; p.vst = c.v_stride_t;
   p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
-  FusedFn fn = with_attention ? fused_fn(ctx->chunks) : select_fn(ctx->chunks);
+  p.pm = fasa_page_map(ctx);
+  if (!fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
+  const bool paged = c.page_size > 0;
+  FusedFn fn = with_attention ? fused_fn(ctx->chunks, paged) : select_fn(ctx->chunks, paged);
 
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));

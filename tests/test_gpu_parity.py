@@ -572,7 +572,7 @@ def _paged_twin(w, t, P, spare=3, seed=0, extra_tokens=0):
             table[b, lp] = next(it)
     f = binding.Fasa(B, w.n_q_heads, Hkv, Lm, t["dom"], rope_pairing=w.pairing, group_reduce=w.group_reduce,
                      n_sink=w.n_sink, n_recent=w.n_recent, select_heads=w.sel_heads, page_size=P, n_pages=n_pages)
-    assert f.step_cluster_size() == 0
+    assert f.step_cluster_size() == r.fasa.step_cluster_size() > 0
     kp, vp = f.alloc_paged_cache(), f.alloc_paged_cache()
     pad = pps * P - Lm
     kl = torch.nn.functional.pad(t["k"], (0, 0, 0, pad)).view(B, Hkv, pps, P, 128)
@@ -642,27 +642,41 @@ def test_paged_caches_give_the_contiguous_results(P, cfg, kw):
     torch.cuda.synchronize()
     for x, y in ((scores_p, r.scores), (idx_p, r.idx), (n_sel_p, r.n_sel), (out_p, r.out), (lse_p, r.lse)):
         assert torch.equal(x, y)
-    out2 = torch.zeros_like(out_p)
-    n0 = f.launch_count()
-    f.decode_step(r.q, kp, vp, proxy_p, lens_p, w.budget, scores_p, idx_p, n_sel_p, out2, r.ws)
-    assert f.launch_count() - n0 == 4
+    out3 = torch.zeros_like(out_p)
+    f.sparse_decode_attn_static(r.q, kp, vp, idx_p, n_sel_p, out3)
     r.dense_step()
     dense_p = torch.zeros_like(r.dense)
     f.full_decode_attn(r.q, kp, vp, lens_p, dense_p, r.ws)
     torch.cuda.synchronize()
-    assert torch.equal(out2, r.out) and torch.equal(dense_p, r.dense)
-    out3 = torch.zeros_like(out_p)
-    f.sparse_decode_attn_static(r.q, kp, vp, idx_p, n_sel_p, out3)
-    s_ = synth.make_step_inputs(w, 1, "cuda")
-    r.fasa.set_step_mode(0)
-    r.fasa.append_decode_step(s_["q"], s_["k_new"], s_["v_new"], r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx,
-                              r.n_sel, r.out, r.ws)
-    f.append_decode_step(s_["q"], s_["k_new"], s_["v_new"], kp, vp, proxy_p, lens_p, w.budget, scores_p, idx_p, n_sel_p,
-                         out2, r.ws)
-    torch.cuda.synchronize()
-    assert torch.equal(out3, out_p)
-    assert torch.equal(lens_p, r.seq_lens) and torch.equal(idx_p, r.idx) and torch.equal(scores_p, r.scores)
-    assert float((out2 - r.out).abs().max()) <= 1e-4          # mode 0 attends with the scalar kernel
+    assert torch.equal(out3, out_p) and torch.equal(dense_p, r.dense)
+    # the one-launch step (no workspace) and the select + split-K route (large bound, workspace)
+    out2 = torch.zeros_like(out_p)
+    for ws_, launches in ((None, 1), (r.ws, None)):
+        r.reset_outputs()
+        scores_p.fill_(SENTINEL); idx_p.fill_(-7)
+        n0, m0 = f.launch_count(), r.fasa.launch_count()
+        f.decode_step(r.q, kp, vp, proxy_p, lens_p, w.budget, scores_p, idx_p, n_sel_p, out2, ws_)
+        r.fasa.decode_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel, r.out, ws_)
+        torch.cuda.synchronize()
+        assert f.launch_count() - n0 == r.fasa.launch_count() - m0 == (launches or f.launch_count() - n0)
+        for x, y in ((scores_p, r.scores), (idx_p, r.idx), (n_sel_p, r.n_sel), (out2, r.out)):
+            assert torch.equal(x, y)
+    # the append form, one launch on both sides, then once more as separate kernels (mode 0)
+    for mode in (1, 0):
+        s_ = synth.make_step_inputs(w, 1 + mode, "cuda")
+        for ff in (r.fasa, f):
+            ff.set_step_mode(mode)
+        n0 = f.launch_count()
+        r.fasa.append_decode_step(s_["q"], s_["k_new"], s_["v_new"], r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores,
+                                  r.idx, r.n_sel, r.out, r.ws if mode == 0 else None)
+        f.append_decode_step(s_["q"], s_["k_new"], s_["v_new"], kp, vp, proxy_p, lens_p, w.budget, scores_p, idx_p,
+                             n_sel_p, out2, r.ws if mode == 0 else None)
+        torch.cuda.synchronize()
+        assert f.launch_count() - n0 == (1 if mode == 1 else 5)
+        for x, y in ((lens_p, r.seq_lens), (scores_p, r.scores), (idx_p, r.idx), (n_sel_p, r.n_sel), (out2, r.out)):
+            assert torch.equal(x, y)
+    for ff in (r.fasa, f):
+        ff.set_step_mode(1)
     if w.batch * w.n_q_heads * 65 <= 65535:
         top_k = 64
         cc = [torch.zeros((w.n_q_heads, 64), dtype=torch.int64, device="cuda") for _ in range(2)]
@@ -708,6 +722,12 @@ def test_paged_cache_table_errors_are_flagged_not_followed():
     assert f.device_status() == binding.DEV_PAGE_CLAMPED
     assert torch.equal(kp, before[0]) and torch.equal(vp, before[1]) and torch.equal(proxy_p, before[2])
     assert lens.cpu().tolist() == [65]
+    # the same through the one-launch append form
+    lens.fill_(64)
+    f.append_decode_step(s_["q"], s_["k_new"], s_["v_new"], kp, vp, proxy_p, lens, w.budget, None, r.idx, r.n_sel, r.out, None)
+    assert f.device_status() & binding.DEV_PAGE_CLAMPED
+    assert torch.equal(kp, before[0]) and torch.equal(vp, before[1]) and torch.equal(proxy_p, before[2])
+    assert lens.cpu().tolist() == [65] and torch.isfinite(r.out).all()
 
 
 def test_strided_token_major_cache():
