@@ -46,7 +46,7 @@ L2_FLUSH_BYTES = 256 << 20
 # the same kernel; it is reported only while the kernel sources are the captured ones.
 TRAFFIC_CAPTURE = {"kernel": "fused_decode_kernel", "workload": "c4", "dram_bytes": 280.93e6, "algorithmic_bytes": 277.02e6,
                    "sources": ("paper_2602_03152_b200/csrc/fasa_fused.cu", "paper_2602_03152_b200/csrc/fasa_score_core.cuh"),
-                   "sha1": "f6cddc1348a50562b578ec9b33960bb9fe814b9b"}
+                   "sha1": "136a0c564a41be4a3b7cd7b1cdedb6ef1d5d0761"}
 
 
 def _traffic(bytes_per_launch):

@@ -1,14 +1,19 @@
 // FAC (Sec. 4.2, Eq. 6-7) and the dense FKV path (Sec. 5.1): split-K flash decoding with an
 // online softmax, rows gathered by index for the sparse form, followed by a merge pass.
 //
-// Mapping.  A KV row (128 bf16 = 256 bytes) is read by a half-warp, 16 bytes per lane, so a
-// lane owns 8 channels of every row it sees and keeps, for up to 4 query heads of the GQA
-// group, its slice of q and of the output accumulator in registers.  One K/V row therefore
-// serves the whole group from a single load.  Groups of 5-8 heads use both half-warps of a
-// warp on the same row (the second load is merged by the coalescer).  Logits of a batch of
-// 8 rows are completed with a transposing xor-shuffle reduction (8 shuffles per head per
-// batch); probabilities travel back to all lanes through shared memory.  All multiply-adds
-// are packed two-wide fp32 FMAs.  No tensor cores: one query token per sequence.
+// Two kernels compute the partial results of a split.
+//   decode_attn_mma_kernel (the default): the GQA group (<= 8 query heads) is the N = 8 of
+//     mma.m16n8k16, so both products of the step run on tensor cores; described above the
+//     kernel.
+//   decode_attn_kernel (step mode 0, the first version): a KV row (128 bf16 = 256 bytes) is
+//     read by a half-warp, 16 bytes per lane; a lane owns 8 channels of every row it sees and
+//     keeps, for up to 4 query heads of the group, its slice of q and of the output
+//     accumulator in registers, so one K/V row serves the whole group from a single load.
+//     Groups of 5-8 heads use both half-warps of a warp on the same row (the second load is
+//     merged by the coalescer).  Logits of a batch of 8 rows are completed with a transposing
+//     xor-shuffle reduction (8 shuffles per head per batch); probabilities travel back to all
+//     lanes through shared memory.  All multiply-adds are packed two-wide fp32 FMAs.
+// decode_attn_merge_kernel then combines the splits of every (sequence, query head).
 #include <mutex>
 
 #include "fasa_common.cuh"

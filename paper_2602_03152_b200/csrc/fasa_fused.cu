@@ -1,8 +1,9 @@
 // One decode step in one launch: UpdateCache -> TIP scoring -> TopK-I -> FAC (Algorithm 2's
 // order; Sec. 4.1-4.2, Eq. 6-7).
 //
-// One thread-block cluster per (batch, KV head) unit.  The CTAs of the cluster cut the unit's
-// cached tokens into contiguous slices and
+// One thread-block cluster per selection unit: a (batch, KV head) pair, or the part of a KV
+// head's query heads that shares an index set.  The CTAs of the cluster cut the unit's cached
+// tokens into contiguous slices and
 //   0. (append form) the CTA whose slice ends the sequence writes the new K, V and proxy rows;
 //   1. stream their slice of the tiled proxy-K buffer once (16-byte loads in tensor-core
 //      fragment order, scored with mma.sync), keep every token's selection key in shared
