@@ -44,9 +44,9 @@ L2_FLUSH_BYTES = 256 << 20
 # profiles/fused_decode_kernel_c4.md: read + write bytes per launch over the launch's algorithmic
 # bytes.  Traffic follows the tokens processed, so the ratio carries over to other workloads of
 # the same kernel; it is reported only while the kernel sources are the captured ones.
-TRAFFIC_CAPTURE = {"kernel": "fused_decode_kernel", "workload": "c4", "dram_bytes": 280.93e6, "algorithmic_bytes": 277.02e6,
+TRAFFIC_CAPTURE = {"kernel": "fused_decode_kernel", "workload": "c4", "dram_bytes": 281.33e6, "algorithmic_bytes": 277.02e6,
                    "sources": ("paper_2602_03152_b200/csrc/fasa_fused.cu", "paper_2602_03152_b200/csrc/fasa_score_core.cuh"),
-                   "sha1": "136a0c564a41be4a3b7cd7b1cdedb6ef1d5d0761"}
+                   "sha1": "581807e7fbd2071aa25b429937d6ecd98d2c144d"}
 
 
 def _traffic(bytes_per_launch):

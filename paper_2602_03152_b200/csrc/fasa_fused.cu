@@ -137,6 +137,8 @@ fused_decode_kernel(const FusedParams p) {
   constexpr int GP = FASA_MAX_GROUP;     // query heads a KV head can serve
   constexpr int HP = 4;                  // heads per attention pass
   __shared__ __align__(16) float s_q[GP][FASA_HEAD_DIM];
+  __shared__ __align__(16) uint16_t s_qraw[GP][FASA_HEAD_DIM];   // the unit's query rows as stored (scoring operand)
+  __shared__ int16_t s_chan[8 * FASA_MAX_DOM / 4];               // the head's channel table
   __shared__ __align__(16) float s_part[GP][kPartStride + 2];
   __shared__ float s_racc[FASA_MAX_GROUP * FASA_HEAD_DIM + 16];   // pushed by the cluster: accumulators of this CTA's outputs
   __shared__ float s_rml[16][FASA_MAX_GROUP][2];                  // ... and every CTA's (m, l) per head
@@ -150,20 +152,17 @@ fused_decode_kernel(const FusedParams p) {
   // (below) certifies that it no longer needs the old value; the last CTA of the sequence to
   // arrive stores the new length.  Nothing waits on the counter.
   // Loads that depend on nothing are issued first, so their (cold) latencies overlap: the
-  // length, this thread's share of the query for the attention phase, and the channel table
-  // with the query values of the scoring operand.
+  // length, this thread's 16 bytes of the unit's query rows and its entry of the channel table.
+  // The scoring operand (query values at the dominant channels) is gathered from the staged
+  // copies in shared memory after the set-up barrier: no load waits on another load's result.
   const bool append = MODE != 1 && p.k_new != nullptr;
   int len_raw = 0;
   if (!append || tid == 0) len_raw = p.seq_lens[b];
   uint4 q_stage = make_uint4(0u, 0u, 0u, 0u);
-  if (MODE == 0 && tid < FASA_MAX_GROUP * (FASA_HEAD_DIM / 8) && tid / (FASA_HEAD_DIM / 8) < p.group)
+  if (MODE != 1 && tid < FASA_MAX_GROUP * (FASA_HEAD_DIM / 8) && tid / (FASA_HEAD_DIM / 8) < p.group)
     q_stage = *reinterpret_cast<const uint4*>(p.q + su.q0 * FASA_HEAD_DIM + tid * 8);
-  ScoreFrag<KB> f[NG];
-  if constexpr (MODE != 1)
-#pragma unroll
-  for (int grp = 0; grp < NG; ++grp)
-    load_score_b<KB>(f[grp], p.q + su.q0 * FASA_HEAD_DIM,
-                     p.chan + h * p.chunks * 8, p.chunks, p.group, lane, grp * KB);
+  int16_t chan_stage = -1;
+  if (MODE != 1 && tid < p.chunks * 8) chan_stage = p.chan[h * p.chunks * 8 + tid];
   int len_old;
   if (append) {
     if (tid == 0) s_len_old = clamp_len(len_raw, p.max_len, p.status);
@@ -281,6 +280,9 @@ fused_decode_kernel(const FusedParams p) {
     }
   }
   for (int i = tid; i < 2 * kFBins; i += kFT) hist0[i] = 0u;
+  if (MODE != 1 && tid < GP * (FASA_HEAD_DIM / 8))
+    *reinterpret_cast<uint4*>(&s_qraw[tid / (FASA_HEAD_DIM / 8)][(tid % (FASA_HEAD_DIM / 8)) * 8]) = q_stage;
+  if (MODE != 1 && tid < p.chunks * 8) s_chan[tid] = chan_stage;
   // query, scaled into the base-2 logit domain, for the attention phase
   if (MODE == 0 && tid < GP * (FASA_HEAD_DIM / 8)) {
     const int g = tid / (FASA_HEAD_DIM / 8), c = (tid % (FASA_HEAD_DIM / 8)) * 8;
@@ -291,6 +293,12 @@ fused_decode_kernel(const FusedParams p) {
     *reinterpret_cast<float4*>(&s_q[g][c + 4]) = make_float4(f2.x * sc, f2.y * sc, f3.x * sc, f3.y * sc);
   }
   __syncthreads();
+  ScoreFrag<KB> f[NG];
+  if constexpr (MODE != 1) {
+#pragma unroll
+    for (int grp = 0; grp < NG; ++grp)
+      load_score_b<KB>(f[grp], &s_qraw[0][0], s_chan, p.chunks, p.group, lane, grp * KB);
+  }
 
   // ---- 1. scoring stream -> keys + first histogram ------------------------------------------
   if constexpr (MODE == 1) {
