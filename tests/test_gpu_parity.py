@@ -695,6 +695,42 @@ def test_paged_caches_give_the_contiguous_results(P, cfg, kw):
                       n_sel=n_sel_p.cpu().numpy(), out=out2.cpu().numpy(), what="paged", **r.oracle_kwargs())
 
 
+@pytest.mark.parametrize("w", _random_workloads(int(os.environ.get("FASA_RANDOM_CASES", "24")), 777),
+                         ids=lambda w: f"i{w.index}")
+def test_seeded_random_configurations_paged(w):
+    # the random shapes again, on page pools of a random page size: the one-launch step (with
+    # and without a workspace), the three calls and the dense path must equal the contiguous run
+    P = [16, 32, 64, 128][w.index % 4]
+    t = synth.make_inputs(w, "cpu")
+    r, f, kp, vp, tab, table, need = _paged_twin(w, t, P, seed=w.index, extra_tokens=2)     # two appends below
+    proxy_p = f.alloc_proxy()
+    lens_p = r.seq_lens.clone()
+    r.build_proxy()
+    f.proxy_build(kp, proxy_p, lens_p)
+    s_ = synth.make_step_inputs(w, 0, "cuda")
+    scores_p, idx_p, n_sel_p = torch.full_like(r.scores, SENTINEL), torch.full_like(r.idx, -7), torch.zeros_like(r.n_sel)
+    out_p, dense_p = torch.zeros_like(r.out), torch.zeros_like(r.dense)
+    for ws_ in (None, r.ws):
+        r.fasa.append_decode_step(s_["q"], s_["k_new"], s_["v_new"], r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx,
+                                  r.n_sel, r.out, ws_)
+        f.append_decode_step(s_["q"], s_["k_new"], s_["v_new"], kp, vp, proxy_p, lens_p, w.budget, scores_p, idx_p, n_sel_p,
+                             out_p, ws_)
+        torch.cuda.synchronize()
+        for x, y in ((lens_p, r.seq_lens), (scores_p, r.scores), (idx_p, r.idx), (n_sel_p, r.n_sel), (out_p, r.out)):
+            assert torch.equal(x, y)
+    r.q = s_["q"]
+    r.step()
+    f.fc_score(r.q, proxy_p, lens_p, scores_p)
+    f.topk(scores_p, lens_p, w.budget, idx_p, n_sel_p, r.ws)
+    f.sparse_decode_attn(r.q, kp, vp, idx_p, n_sel_p, out_p, r.ws)
+    r.dense_step()
+    f.full_decode_attn(r.q, kp, vp, lens_p, dense_p, r.ws)
+    torch.cuda.synchronize()
+    for x, y in ((scores_p, r.scores), (idx_p, r.idx), (n_sel_p, r.n_sel), (out_p, r.out), (dense_p, r.dense)):
+        assert torch.equal(x, y)
+    assert f.device_status() == r.fasa.device_status()       # (a full cache flags the dropped token on both sides)
+
+
 def test_paged_cache_table_errors_are_flagged_not_followed():
     w = C["c1"].replace(n_q_heads=8, n_kv_heads=2, max_len=256, len_lo=200, len_hi=200, budget=32)
     t = synth.make_inputs(w, "cpu")
