@@ -41,7 +41,7 @@ struct fasa_ctx {
   do {                                                                                 \
     cudaError_t e_ = (expr);                                                           \
     if (e_ != cudaSuccess) {                                                           \
-      snprintf((ctx)->cuda_err, sizeof((ctx)->cuda_err), "%s: %s", #expr,              \
+      snprintf((ctx)->cuda_err, sizeof((ctx)->cuda_err), "%.120s: %.100s", #expr,      \
                cudaGetErrorString(e_));                                                \
       return FASA_ERR_CUDA;                                                            \
     }                                                                                  \
