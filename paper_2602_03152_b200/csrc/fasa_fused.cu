@@ -8,23 +8,32 @@
 //   1. stream their slice of the tiled proxy-K buffer once (16-byte loads in tensor-core
 //      fragment order, scored with mma.sync), keep every token's selection key in shared
 //      memory and histogram its top 11 bits;
-//   2. find the budget-th largest key by an MSB-first radix select (11 + 11 + 10 bits): each
-//      pass needs one cluster barrier, after which every CTA reads the other CTAs' coarse and
-//      fine bin counts through distributed shared memory and locates the bin redundantly;
+//   2. find the budget-th largest key by an MSB-first radix select.  A radix pass (11, 11, 10
+//      bits) costs one cluster barrier: before it every CTA PUSHES the sums of its 32-bin
+//      groups into every peer's shared memory, after it every warp locates the group from its
+//      local copy, fetches that group's 32 bins from the peers through distributed shared
+//      memory and locates the bin, redundantly and without a block barrier.  As soon as the
+//      bin that holds the budget-th key has few keys cluster-wide (normally after the first
+//      pass), every CTA pushes its keys of that bin to all peers (second barrier) and each CTA
+//      finishes the selection on its own copy with block-level passes;
 //   3. write the selected positions in ascending order (ballot masks + prefix sums, equal keys
-//      lowest index first, so the result equals a stable sort; one more barrier for the
-//      cluster-wide prefix);
-//   4. attend, each CTA over the tokens it selected itself: K/V rows gathered by index with an
-//      online softmax;
+//      lowest index first, so the result equals a stable sort).  The number of selected tokens
+//      in lower-ranked CTAs follows from what step 2 has already fetched (their bin counts and
+//      their pushed keys), so no barrier is needed here;
+//   4. attend, each CTA over an equal share of the index list (one barrier makes the peers'
+//      parts of the list visible): K/V rows gathered by index with an online softmax;
 //   5. push their partial results into the shared memory of the CTA that finishes each output
 //      (one last barrier), which merges them locally.
 // Scores, histograms and split-K partials never travel through HBM: the launch moves the
 // proxy rows of every token, the K/V rows of the selected tokens, q and the outputs.
 //
-// Every cluster barrier (at most five) is reached by all threads of all CTAs of a cluster the
-// same number of times: the only data-dependent decision around one, leaving the radix loop
-// early, is taken from cluster-wide sums that are identical in every CTA.  No thread spins on
-// anything.
+// Cluster barriers per launch: the split set-up barrier, then normally four (first histogram,
+// candidate keys, index list, merge); up to six when many keys share the leading bits of the
+// budget-th key.  Each is reached by all
+// threads of all CTAs of a cluster the same number of times: every decision around one is taken
+// from cluster-wide integer sums that are identical in every warp of every CTA.  The whole-step
+// form ends with the merge barrier; the select-only forms end with the last barrier of the
+// selection, after which no CTA touches a peer's shared memory.  No thread spins on anything.
 #include <cooperative_groups.h>
 
 #include "fasa_common.cuh"
@@ -41,6 +50,47 @@ constexpr int kFBins = 2048;           // bins of the widest radix pass
 constexpr int kPartStride = FASA_HEAD_DIM + 2;   // m, l, acc[128]
 constexpr int kCapMax = 22528;         // keys a CTA can hold (88 KB of shared memory)
 constexpr int kCapPair = 16384;        // ... and still leave room for a second CTA on the SM
+constexpr int kMaxCs = 16;             // CTAs per cluster at most
+constexpr int kGroups = kFBins / 32;   // 32-bin groups of the widest radix pass
+constexpr int kCandCap = 4096;         // keys of one bin that the cluster finishes locally
+constexpr int kFinBits = 7;            // bits per block-level pass of that local finish
+constexpr int kFinBins = 1 << kFinBits;
+constexpr int kHP = 4;                 // query heads per attention pass
+
+// Dynamic shared memory of one CTA holding `cap` keys (bytes from the start):
+//   keys[cap] | hist1 (8 KB) | sums1 (4 KB) | 4 KB | sums0 (4 KB) | hist0 (8 KB) | masks
+// hist0 / hist1: the histograms of even / odd radix passes; sums0 / sums1: the group sums that
+// every CTA of the cluster pushes here before the barrier of an even / odd pass, [rank][group].
+// The candidate keys pushed after pass 0 land in hist1 .. the spare 4 KB (nothing else uses
+// them then), those pushed after pass 1 in the spare 4 KB .. hist0 (read by peers during pass
+// 0 only).  The attention phase reuses the area from its start (keys, histograms and masks are
+// dead by then; no peer writes here after the last barrier of the selection).
+struct FusedSmem {
+  int keys, hist1, sums1, spare, sums0, hist0, mask, sel_end;
+  int acc, part, p, al, m, l, att_end;
+  int total;
+};
+__host__ __device__ inline FusedSmem fused_smem_layout(int cap) {
+  FusedSmem L;
+  L.keys = 0;
+  L.hist1 = cap * 4;
+  L.sums1 = L.hist1 + kFBins * 4;
+  L.spare = L.sums1 + kMaxCs * kGroups * 4;
+  L.sums0 = L.spare + 4096;
+  L.hist0 = L.sums0 + kMaxCs * kGroups * 4;
+  L.mask = L.hist0 + kFBins * 4;
+  L.sel_end = L.mask + 2 * (cap / 32 + 1) * 4;     // one bit per key: above / equal to the threshold
+  L.acc = 0;                                       // [kFW][kHP][128] fp32
+  L.part = L.acc + kFW * kHP * FASA_HEAD_DIM * 4;  // [8][kPartStride + 2]
+  L.p = L.part + FASA_MAX_GROUP * (kPartStride + 2) * 4;   // [kFW][16]
+  L.al = L.p + kFW * 16 * 4;                       // [kFW][kHP]
+  L.m = L.al + kFW * kHP * 4;
+  L.l = L.m + kFW * kHP * 4;
+  L.att_end = L.l + kFW * kHP * 4;
+  L.total = L.sel_end > L.att_end ? L.sel_end : L.att_end;
+  return L;
+}
+static_assert(kFBins * 4 + kMaxCs * kGroups * 4 + 4096 == kCandCap * 4, "candidate area");
 
 struct FusedParams {
   const uint16_t* q;
@@ -77,6 +127,11 @@ __device__ __forceinline__ uint2 ld_stream_u2(const void* p) {
   asm volatile("ld.global.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p) : "memory");
   return r;
 }
+
+// The two halves of a cluster barrier (cluster.sync() = arrive + wait), for all threads of all
+// CTAs alike: what a thread wrote before its arrive is visible to every thread after its wait.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
 #pragma unroll
@@ -126,26 +181,20 @@ fused_decode_kernel(const FusedParams p) {
   const int b = su.b;
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  __shared__ uint32_t s_coarse[2][kFBins / 32];
-  __shared__ uint32_t s_gather[16][kFBins / 32];   // remote counts, one row per cluster rank
   __shared__ unsigned long long s_wcnt[kFW];
-  __shared__ unsigned long long s_tot;
-  __shared__ uint32_t s_bin, s_kth, s_cnt;
+  __shared__ uint32_t s_fin[3][kFinBins];          // histograms of the local finish (one per pass)
+  __shared__ __align__(8) uint32_t s_gsum[3][2][kGroups];   // per radix pass: cluster-wide group sums, and those of the lower ranks (added by the peers)
+  __shared__ uint32_t s_fine[3][2][32];            // per radix pass: the bins of the group that holds the kth key, same two sums
+  __shared__ uint32_t s_mine[kGroups];             // this CTA's group sums of the current pass
+  __shared__ uint32_t s_ncand, s_cgt, s_ceq;       // candidates found here; pushed keys of lower ranks above / equal to the threshold
   __shared__ int s_len_old;
-  __shared__ __align__(16) uint32_t s_mask[kCapMax / 128 * 8];  // per 128 keys: 4 above + 4 equal masks
-  __shared__ unsigned long long s_boff[kCapMax / 128];          // per 128 keys: (gt, eq) selected before
   constexpr int GP = FASA_MAX_GROUP;     // query heads a KV head can serve
-  constexpr int HP = 4;                  // heads per attention pass
+  constexpr int HP = kHP;                // heads per attention pass
   __shared__ __align__(16) float s_q[GP][FASA_HEAD_DIM];
   __shared__ __align__(16) uint16_t s_qraw[GP][FASA_HEAD_DIM];   // the unit's query rows as stored (scoring operand)
   __shared__ int16_t s_chan[8 * FASA_MAX_DOM / 4];               // the head's channel table
-  __shared__ __align__(16) float s_part[GP][kPartStride + 2];
   __shared__ float s_racc[FASA_MAX_GROUP * FASA_HEAD_DIM + 16];   // pushed by the cluster: accumulators of this CTA's outputs
-  __shared__ float s_rml[16][FASA_MAX_GROUP][2];                  // ... and every CTA's (m, l) per head
-  __shared__ __align__(16) float s_p[kFW][16];
-  __shared__ __align__(16) float s_al[kFW][HP];
-  __shared__ float s_m[kFW][HP];
-  __shared__ float s_l[kFW][HP];
+  __shared__ float s_rml[kMaxCs][FASA_MAX_GROUP][2];              // ... and every CTA's (m, l) per head
 
   // ---- slices -------------------------------------------------------------------------
   // Append-then-step: one thread reads the length for the whole CTA, so that the CTA's arrival
@@ -187,9 +236,11 @@ fused_decode_kernel(const FusedParams p) {
   const int c1 = min(len, c0 + per);
   const int nloc = c1 - c0;
   const int cap = (((p.max_len + cs - 1) / cs) + 31) & ~31;
-  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw);
-  uint32_t* hist0 = keys + cap;
-  uint32_t* hist1 = hist0 + kFBins;
+  const FusedSmem sl = fused_smem_layout(cap);
+  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + sl.keys);
+  uint32_t* hist0 = reinterpret_cast<uint32_t*>(smem_raw + sl.hist0);
+  uint32_t* hist1 = reinterpret_cast<uint32_t*>(smem_raw + sl.hist1);
+  uint32_t* s_mask = reinterpret_cast<uint32_t*>(smem_raw + sl.mask);
 
   const long long k_budget =
       p.budget > 0 ? (long long)p.budget : ((long long)(-p.budget) * len + 999) / 1000;
@@ -279,7 +330,11 @@ fused_decode_kernel(const FusedParams p) {
       *reinterpret_cast<uint32_t*>(p.proxy_w + poff + proxy_word_offset(pg, prow, w)) = lo | (hi << 16);
     }
   }
-  for (int i = tid; i < 2 * kFBins; i += kFT) hist0[i] = 0u;
+  for (int i = tid; i < kFBins; i += kFT) { hist0[i] = 0u; hist1[i] = 0u; }
+  if (tid < 3 * kFinBins) (&s_fin[0][0])[tid] = 0u;
+  if (tid < 3 * 2 * kGroups) (&s_gsum[0][0][0])[tid] = 0u;
+  if (tid < 3 * 2 * 32) (&s_fine[0][0][0])[tid] = 0u;
+  if (tid == 0) { s_ncand = 0u; s_cgt = 0u; s_ceq = 0u; }
   if (MODE != 1 && tid < GP * (FASA_HEAD_DIM / 8))
     *reinterpret_cast<uint4*>(&s_qraw[tid / (FASA_HEAD_DIM / 8)][(tid % (FASA_HEAD_DIM / 8)) * 8]) = q_stage;
   if (MODE != 1 && tid < p.chunks * 8) s_chan[tid] = chan_stage;
@@ -293,6 +348,9 @@ fused_decode_kernel(const FusedParams p) {
     *reinterpret_cast<float4*>(&s_q[g][c + 4]) = make_float4(f2.x * sc, f2.y * sc, f3.x * sc, f3.y * sc);
   }
   __syncthreads();
+  // This CTA runs and its totals are cleared: the peers may add to them from now on.  Each CTA
+  // waits for the others' arrival only when it is about to touch them, after its stream.
+  cluster_arrive();
   ScoreFrag<KB> f[NG];
   if constexpr (MODE != 1) {
 #pragma unroll
@@ -371,22 +429,33 @@ fused_decode_kernel(const FusedParams p) {
   __syncthreads();
 
   // ---- 2. radix select of the ktot-th largest key ------------------------------------------
-  // `done` (the bin that holds the kth key is needed whole, so its remaining bits do not
-  // matter) is computed from the same cluster-wide integer sums in every CTA, hence identical
-  // in all of them: the loop, barrier included, ends for the whole cluster at once.
-  uint32_t prefix = 0, kth = ktot, thr = 0, tie_quota = 0;
-  bool done = false;
+  // Every value that steers this phase (the bin found, the keys still wanted from it, the
+  // number of keys it holds) is computed by every warp of every CTA from the same cluster-wide
+  // integer sums, hence identical everywhere: loops and barriers end for the whole cluster at
+  // once.  `lower_gt` / `lower_eq` count, over the lower-ranked CTAs, the keys above the
+  // threshold found so far and the keys equal to it: the compaction's cluster-wide prefix.
+  cluster_wait();               // (set-up barrier, second half: every peer has started and cleared its totals)
+  uint32_t prefix = 0, kth = ktot, thr = 0, tie_quota = 0, lower_gt = 0, lower_eq = 0;
+  bool done = false;            // thr and tie_quota are final
+  bool peers_idle = false;      // a barrier has passed since the last access to a peer's memory
+  bool have_masks = false;      // s_mask already holds (higher bins, candidates) per block of 128 keys
+  // Bit masks over the keys: word w covers keys 32 w .. 32 w + 31.  A warp owns a contiguous run
+  // of words, a lane one word of every 32 of them: after the first pass over the keys all work
+  // is per word, without ballots.
+  const int n_words = (nloc + 31) >> 5;
+  const int words_per_warp = (n_words + kFW - 1) / kFW;
+  const int w0 = min(n_words, warp * words_per_warp), w1 = min(n_words, w0 + words_per_warp);
+  uint32_t* s_mg = s_mask;                       // keys above the threshold (first: in higher bins)
+  uint32_t* s_me = s_mask + (cap / 32 + 1);      // keys equal to it (first: the candidates)
 #pragma unroll 1
-  for (int pass = 0; pass < 3; ++pass) {
+  for (int pass = 0; pass < 3 && !done; ++pass) {
     const int bits = pass == 2 ? 10 : 11;
     const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
     const int nb = 1 << bits;
     const int ng = nb / 32;
     uint32_t* buf = (pass & 1) ? hist1 : hist0;
-    uint32_t* coarse = s_coarse[pass & 1];
-    if (done) break;
     if (pass > 0) {
-      if (pass == 2) {
+      if (pass == 2) {          // (hist0: its remote readers of pass 0 are past the barrier of pass 1)
         for (int i = tid; i < nb; i += kFT) buf[i] = 0u;
         __syncthreads();
       }
@@ -402,8 +471,11 @@ fused_decode_kernel(const FusedParams p) {
       __syncthreads();
     }
     {
-      // group sums: each warp reduces its kFBins/32/kFW groups side by side
-      constexpr int GPW = kFBins / 32 / kFW;
+      // Group sums: each warp reduces its groups side by side; after a block barrier warp r
+      // ADDS them into CTA r's totals (coalesced remote atomics, zeros skipped: scores crowd
+      // into few groups), and into CTA r's totals of lower ranks if this CTA ranks below r.
+      // After the cluster barrier every CTA holds the cluster-wide sums, already reduced.
+      constexpr int GPW = kGroups / kFW;
       uint32_t v[GPW];
 #pragma unroll
       for (int j = 0; j < GPW; ++j) {
@@ -416,170 +488,271 @@ fused_decode_kernel(const FusedParams p) {
         for (int j = 0; j < GPW; ++j) v[j] += __shfl_xor_sync(0xffffffffu, v[j], o);
       if (lane == 0) {
 #pragma unroll
-        for (int j = 0; j < GPW; ++j)
-          if (warp + j * kFW < ng) coarse[warp + j * kFW] = v[j];
+        for (int j = 0; j < GPW; ++j) s_mine[warp + j * kFW] = v[j];
+      }
+      __syncthreads();
+      if (warp < cs) {
+        uint32_t* tot = cluster.map_shared_rank(&s_gsum[pass][0][0], warp);
+        uint32_t* low = cluster.map_shared_rank(&s_gsum[pass][1][0], warp);
+#pragma unroll
+        for (int j = 0; j < kGroups / 32; ++j) {
+          const uint32_t x = s_mine[lane + 32 * j];
+          if (x) {
+            atomicAdd(tot + lane + 32 * j, x);
+            if (crank < warp) atomicAdd(low + lane + 32 * j, x);
+          }
+        }
       }
     }
-    cluster.sync();   // barrier 1..3
+    cluster.sync();   // one per radix pass: all group sums have arrived, all histograms are complete
 
-    // Every thread fetches a few of the other CTAs' coarse counts (all loads in flight at
-    // once); warp 0 adds them up and finds the group of 32 bins that holds the kth key.
-    for (int i = tid; i < ng * cs; i += kFT) {
-      const int r = i / ng, g = i % ng;
-      s_gather[r][g] = cluster.map_shared_rank(coarse, r)[g];
-    }
-    __syncthreads();
-    if (warp == 0) {
-      uint32_t res = kth, tot = 0;
-      int hit = 0, group_id = -1;
-      for (int g0 = ng - 1; g0 >= 0 && group_id < 0; g0 -= 32) {   // groups, highest first
-        const int g = g0 - lane;
-        uint32_t v = 0;
-        for (int r = 0; r < cs; ++r) v += s_gather[r][g];
-        if (warp_find_kth(v, res, lane, &hit, &res, &tot)) group_id = g0 - hit;
-        else res -= tot;
+    // (a) every warp finds the group of 32 bins that holds the kth key from the local totals:
+    // lane l owns groups 63 - 2 l and 62 - 2 l (highest first)
+    uint32_t res, above_lower;                 // above_lower: keys of lower ranks in higher bins
+    int group_id;
+    {
+      const uint2 t2 = *reinterpret_cast<const uint2*>(&s_gsum[pass][0][kGroups - 2 - 2 * lane]);   // (.y, .x) = (first, second)
+      const uint2 l2 = *reinterpret_cast<const uint2*>(&s_gsum[pass][1][kGroups - 2 - 2 * lane]);
+      int hit = 31;
+      uint32_t tot = 0;
+      res = 1;
+      if (!warp_find_kth(t2.x + t2.y, kth, lane, &hit, &res, &tot)) { hit = 31; res = 1; }   // cannot fail: kth <= number of keys
+      above_lower = __reduce_add_sync(0xffffffffu, lane < hit ? l2.x + l2.y : 0u);
+      const uint32_t first = __shfl_sync(0xffffffffu, t2.y, hit), first_low = __shfl_sync(0xffffffffu, l2.y, hit);
+      group_id = kGroups - 1 - 2 * hit;
+      if (first < res) {
+        res -= first;
+        above_lower += first_low;
+        --group_id;
       }
-      if (group_id < 0) { group_id = 0; res = 1; }   // cannot happen: kth <= number of keys
-      if (lane == 0) { s_bin = (uint32_t)group_id; s_kth = res; }
     }
-    __syncthreads();
-    const int group_id = (int)s_bin;
-    const uint32_t kth_in_group = s_kth;
-    __syncthreads();
-    // the 32 bins of that group, from every CTA
-    for (int i = tid; i < 32 * cs; i += kFT) {
-      const int r = i / 32, bl = i % 32;
-      s_gather[r][bl] = cluster.map_shared_rank(buf, r)[group_id * 32 + bl];
-    }
-    __syncthreads();
-    if (warp == 0) {
-      uint32_t v = 0, res2 = kth_in_group, tot = 0;
-      int hit = 0;
-      for (int r = 0; r < cs; ++r) v += s_gather[r][31 - lane];   // lane 0 = highest bin
-      if (!warp_find_kth(v, kth_in_group, lane, &hit, &res2, &tot)) { hit = 31; res2 = 1; }
-      const uint32_t in_bin = __shfl_sync(0xffffffffu, v, hit);
-      if (lane == 0) {
-        s_bin = (uint32_t)(group_id * 32 + 31 - hit);
-        s_kth = res2;
-        s_cnt = in_bin;
+    // (b) warp r fetches the 32 bins of that group from CTA r (one transaction) and adds them to
+    // the block's totals; after a block barrier every warp locates the bin
+    if (warp < cs) {
+      const uint32_t x = cluster.map_shared_rank(buf, warp)[group_id * 32 + 31 - lane];   // lane 0 = highest bin
+      if (x) {
+        atomicAdd(&s_fine[pass][0][lane], x);
+        if (warp < crank) atomicAdd(&s_fine[pass][1][lane], x);
       }
     }
     __syncthreads();
-    prefix = (prefix << bits) | s_bin;
-    kth = s_kth;
-    if (s_cnt == kth && pass < 2) {   // every key of this bin is selected
+    uint32_t in_bin, bin_lower;                // keys in the bin: cluster-wide / in lower ranks
+    {
+      const uint32_t v = s_fine[pass][0][lane], vl = s_fine[pass][1][lane];
+      int hit = 31;
+      uint32_t tot = 0, res2 = 1;
+      if (!warp_find_kth(v, res, lane, &hit, &res2, &tot)) { hit = 31; res2 = 1; }
+      in_bin = __shfl_sync(0xffffffffu, v, hit);
+      bin_lower = __shfl_sync(0xffffffffu, vl, hit);
+      above_lower += __reduce_add_sync(0xffffffffu, lane < hit ? vl : 0u);
+      prefix = (prefix << bits) | (uint32_t)(group_id * 32 + 31 - hit);
+      kth = res2;
+    }
+    lower_gt += above_lower;
+    peers_idle = false;
+
+    if (in_bin == kth) {            // every key of this bin is selected: its other bits do not matter
       thr = prefix << shift;
       tie_quota = 0xffffffffu;
+      lower_gt += bin_lower;
       done = true;
+    } else if (pass == 2) {         // all 32 bits are fixed: the bin holds the keys equal to the threshold
+      thr = prefix;
+      tie_quota = kth;
+      lower_eq = bin_lower;
+      done = true;
+    } else if (in_bin <= (uint32_t)kCandCap) {
+      // ---- few keys share this prefix: every CTA gets all of them and finishes on its own ----
+      // CTA r's keys occupy [sum of lower ranks' counts, + its own count) of every copy.
+      uint32_t* cand = reinterpret_cast<uint32_t*>(smem_raw + (pass == 0 ? sl.hist1 : sl.spare));
+      // One pass over the keys: masks of the keys in higher bins (selected for certain) and of
+      // the keys in this bin (the candidates, decided once the threshold is known); then the
+      // candidates themselves are appended, with one counter update per warp.
+      have_masks = true;
+      {
+        uint32_t cnt = 0;
+#pragma unroll 4
+        for (int w = w0; w < w1; ++w) {
+          const int i = 32 * w + lane;
+          const uint32_t top = keys[i] >> shift;
+          const uint32_t ma = __ballot_sync(0xffffffffu, i < nloc && top > prefix);
+          const uint32_t mc = __ballot_sync(0xffffffffu, i < nloc && top == prefix);
+          if (lane == 0) { s_mg[w] = ma; s_me[w] = mc; }
+          cnt += __popc(mc);
+        }
+        uint32_t base = 0;
+        if (lane == 0 && cnt) base = atomicAdd(&s_ncand, cnt);
+        base = __shfl_sync(0xffffffffu, base, 0) + bin_lower;
+        __syncwarp();
+        for (int wb = w0; wb < w1; wb += 32) {     // uniform over the warp
+          const int w = wb + lane;
+          uint32_t m = w < w1 ? s_me[w] : 0u;
+          const uint32_t c = __popc(m), incl = warp_incl_scan(c, lane);
+          uint32_t slot = base + incl - c;
+          base += __shfl_sync(0xffffffffu, incl, 31);
+          while (m) {
+            const int j = __ffs(m) - 1;
+            m &= m - 1;
+            if (slot < (uint32_t)kCandCap) cand[slot] = keys[32 * w + j];
+            ++slot;
+          }
+        }
+      }
+      __syncthreads();
+      if (warp < cs && warp != crank) {          // this CTA's run of keys, to CTA `warp`, coalesced
+        const uint32_t n_own = min(s_ncand, (uint32_t)kCandCap - min(bin_lower, (uint32_t)kCandCap));
+        uint32_t* dst = cluster.map_shared_rank(cand, warp) + bin_lower;
+        for (uint32_t i = lane; i < n_own; i += 32) dst[i] = cand[bin_lower + i];
+      }
+      cluster.sync();   // every CTA holds every candidate; no peer is touched from here to the merge
+      peers_idle = true;
+      // block-level radix passes over the remaining `shift` bits, kFinBits at a time; every
+      // warp scans the small histogram itself, so a pass costs one block barrier
+      int rem = shift;
+#pragma unroll 1
+      for (int fp = 0; rem > 0 && !done; ++fp) {
+        const int wbits = rem < kFinBits ? rem : kFinBits;
+        const int sh = rem - wbits;
+        uint32_t* fh = s_fin[fp];
+        for (int i = tid; i < (int)in_bin; i += kFT) {
+          const uint32_t key = cand[i];
+          if ((key >> rem) == prefix) atomicAdd(&fh[(key >> sh) & (uint32_t)((1 << wbits) - 1)], 1u);
+        }
+        __syncthreads();
+        // lane l owns the four bins 127 - 4 l .. 124 - 4 l (highest first)
+        uint32_t c4[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) c4[j] = fh[kFinBins - 1 - 4 * lane - j];
+        int hit = 0;
+        uint32_t res2 = 1, tot = 0;
+        if (!warp_find_kth(c4[0] + c4[1] + c4[2] + c4[3], kth, lane, &hit, &res2, &tot)) { hit = 0; res2 = 1; }
+        uint32_t digit = 0, cnt = 0;
+        bool found = false;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t c = __shfl_sync(0xffffffffu, c4[j], hit);
+          if (!found) {
+            if (c >= res2) { digit = (uint32_t)(kFinBins - 1 - 4 * hit - j); cnt = c; found = true; }
+            else res2 -= c;
+          }
+        }
+        prefix = (prefix << wbits) | digit;
+        kth = res2;
+        rem = sh;
+        if (cnt == kth && rem > 0) {     // the rest of this bin is selected whole
+          thr = prefix << rem;
+          tie_quota = 0xffffffffu;
+          done = true;
+        }
+      }
+      if (!done) {
+        thr = prefix;
+        tie_quota = kth;
+        done = true;
+      }
+      // pushed keys of the lower-ranked CTAs against the threshold (they lie in [0, bin_lower))
+      {
+        uint32_t ngt = 0, neq = 0;
+        for (int i = tid; i < (int)bin_lower; i += kFT) {
+          const uint32_t key = cand[i];
+          ngt += key > thr ? 1u : 0u;
+          neq += key == thr ? 1u : 0u;
+        }
+        ngt = __reduce_add_sync(0xffffffffu, ngt);
+        neq = __reduce_add_sync(0xffffffffu, neq);
+        if (lane == 0 && (ngt | neq)) { atomicAdd(&s_cgt, ngt); atomicAdd(&s_ceq, neq); }
+      }
     }
-    __syncthreads();
   }
-  if (!done) {
-    thr = prefix;
-    tie_quota = kth;
-  }
+  // The attention phase reuses the histograms, and a CTA of the select-only forms may leave:
+  // both only once no peer can still be reading this CTA's bins.
+  if (!peers_idle) cluster.sync();
 
   // ---- 3. ascending compaction ---------------------------------------------------------------
-  // Blocks of 128 consecutive keys, four per lane.  (a) every warp turns its blocks into
-  // eight bit masks (key e of lane l above the threshold / equal to it) with independent
-  // ballots; (b) a block scan over the blocks' bit counts gives each block its offsets;
-  // (c) after the cluster-wide prefix, set bits become positions.  No step carries a running
-  // counter through a loop, so the loops pipeline.
-  const int n_blk = (nloc + 127) >> 7;
-  for (int bk = warp; bk < n_blk; bk += kFW) {
-    const int i = bk * 128 + lane * 4;
-    const uint4 kq = *reinterpret_cast<const uint4*>(&keys[i]);
-    const uint32_t kv[4] = {kq.x, kq.y, kq.z, kq.w};
-    uint32_t m[8];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const bool ok = i + e < nloc;
-      m[e] = __ballot_sync(0xffffffffu, ok && kv[e] > thr);
-      m[4 + e] = __ballot_sync(0xffffffffu, ok && kv[e] == thr);
-    }
-    if (lane == 0) {
-      *reinterpret_cast<uint4*>(&s_mask[bk * 8]) = make_uint4(m[0], m[1], m[2], m[3]);
-      *reinterpret_cast<uint4*>(&s_mask[bk * 8 + 4]) = make_uint4(m[4], m[5], m[6], m[7]);
-    }
-  }
-  __syncthreads();
-  // block scan of the per-block counts (gt in the high half, eq in the low half); one block
-  // per thread (at most kCapMax / 128 <= kFT of them)
-  unsigned long long mine = 0;
-  if (tid < n_blk) {
-    const uint4 g4 = *reinterpret_cast<const uint4*>(&s_mask[tid * 8]);
-    const uint4 e4 = *reinterpret_cast<const uint4*>(&s_mask[tid * 8 + 4]);
-    mine = ((unsigned long long)(__popc(g4.x) + __popc(g4.y) + __popc(g4.z) + __popc(g4.w)) << 32) |
-           (unsigned)(__popc(e4.x) + __popc(e4.y) + __popc(e4.z) + __popc(e4.w));
-  }
-  unsigned long long incl = mine;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += t;
-  }
-  if (lane == 31) s_wcnt[warp] = incl;
-  __syncthreads();
-  unsigned long long before = incl - mine;
+  // (a) the masks of the keys above / equal to the threshold: from the keys (ballots), or,
+  // where the select phase has left the masks of the higher bins and of the candidates, by
+  // looking at the candidates alone, each lane at the bits of its own words; (b) the warps'
+  // totals give each warp its offset (one block barrier); (c) every lane turns the set bits of
+  // its words into positions of the index list (prefix over the lanes by shuffles).  Equal
+  // keys are taken lowest index first, so the result equals a stable sort.
   {
-    unsigned long long all = 0;
-    for (int w = 0; w < kFW; ++w) {
-      const unsigned long long c = s_wcnt[w];
-      if (w < warp) before += c;
-      all += c;
+    uint32_t g_tot = 0, e_tot = 0;
+    if (have_masks) {
+      for (int w = w0 + lane; w < w1; w += 32) {
+        uint32_t mc = s_me[w], mg = s_mg[w], me = 0u;
+        while (mc) {
+          const int j = __ffs(mc) - 1;
+          mc &= mc - 1;
+          const uint32_t key = keys[32 * w + j];
+          if (key > thr) mg |= 1u << j;
+          else if (key == thr) me |= 1u << j;
+        }
+        s_mg[w] = mg;
+        s_me[w] = me;
+        g_tot += __popc(mg);
+        e_tot += __popc(me);
+      }
+      g_tot = __reduce_add_sync(0xffffffffu, g_tot);
+      e_tot = __reduce_add_sync(0xffffffffu, e_tot);
+    } else {
+#pragma unroll 4
+      for (int w = w0; w < w1; ++w) {
+        const int i = 32 * w + lane;
+        const uint32_t key = keys[i];
+        const uint32_t mg = __ballot_sync(0xffffffffu, i < nloc && key > thr);
+        const uint32_t me = __ballot_sync(0xffffffffu, i < nloc && key == thr);
+        if (lane == 0) { s_mg[w] = mg; s_me[w] = me; }
+        g_tot += __popc(mg);
+        e_tot += __popc(me);
+      }
     }
-    if (tid == 0) s_tot = all;
+    if (lane == 0) s_wcnt[warp] = ((unsigned long long)g_tot << 32) | e_tot;
   }
-  cluster.sync();   // barrier 4
-  uint32_t own_first, own_count;
+  __syncthreads();            // the warps' totals; the candidate counts of the select phase
+  uint32_t g_run, e_run;        // selected keys before this warp's run: above / equal to the threshold
   {
-    // totals of the lower-ranked CTAs, one per lane, fetched side by side
-    unsigned long long t = lane < crank ? *cluster.map_shared_rank(&s_tot, lane) : 0ull;
+    static_assert(kFW <= 32, "one lane per warp total");
+    const unsigned long long mine = lane < kFW ? s_wcnt[lane] : 0ull;
+    unsigned long long incl = mine;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-    before += t;
-    // this CTA's selected tokens occupy a contiguous run of the index list
-    const uint32_t gb = (uint32_t)(t >> 32), eb = (uint32_t)t;
-    const unsigned long long mine_all = s_tot;
-    const uint32_t gl = (uint32_t)(mine_all >> 32), el = (uint32_t)mine_all;
-    own_first = gb + min(eb, tie_quota);
-    own_count = gl + (eb < tie_quota ? min(tie_quota - eb, el) : 0u);
+    for (int o = 1; o < kFW; o <<= 1) {
+      const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    const unsigned long long before = __shfl_sync(0xffffffffu, incl - mine, warp);
+    const unsigned long long all = __shfl_sync(0xffffffffu, incl, kFW - 1);
+    // selected tokens of the lower-ranked CTAs: from the bin counts and the pushed keys that
+    // the select phase has seen, no barrier needed
+    const uint32_t gb = lower_gt + s_cgt, eb = lower_eq + s_ceq;
+    g_run = gb + (uint32_t)(before >> 32);
+    e_run = eb + (uint32_t)before;
   }
-  if (tid < n_blk) s_boff[tid] = before;     // offsets of this thread's block
-  __syncthreads();
   {
     int32_t* out_idx = p.idx + (int64_t)u * p.n_sel_max;
-    const uint32_t lt = (1u << lane) - 1u;
-    for (int bk = warp; bk < n_blk; bk += kFW) {
-      const uint4 g4 = *reinterpret_cast<const uint4*>(&s_mask[bk * 8]);
-      const uint4 e4 = *reinterpret_cast<const uint4*>(&s_mask[bk * 8 + 4]);
-      if ((g4.x | g4.y | g4.z | g4.w | e4.x | e4.y | e4.z | e4.w) == 0u) continue;   // uniform over the warp
-      const uint32_t mg[4] = {g4.x, g4.y, g4.z, g4.w}, me[4] = {e4.x, e4.y, e4.z, e4.w};
-      const unsigned long long off = s_boff[bk];
-      // selected keys of lower lanes come first, then this lane's own keys in order
-      uint32_t g_before = (uint32_t)(off >> 32), e_before = (uint32_t)off;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        g_before += __popc(mg[e] & lt);
-        e_before += __popc(me[e] & lt);
-      }
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
+    for (int wb = w0; wb < w1; wb += 32) {         // uniform over the warp
+      const int w = wb + lane;
+      const uint32_t mg = w < w1 ? s_mg[w] : 0u, me = w < w1 ? s_me[w] : 0u;
+      // counts of the lower lanes' words, packed (a word holds at most 32 keys, a CTA < 65536)
+      const uint32_t cnt = (__popc(mg) << 16) | __popc(me), incl = warp_incl_scan(cnt, lane);
+      uint32_t g_before = g_run + ((incl - cnt) >> 16), e_before = e_run + ((incl - cnt) & 0xffffu);
+      const uint32_t all = __shfl_sync(0xffffffffu, incl, 31);
+      g_run += all >> 16;
+      e_run += all & 0xffffu;
+      uint32_t m = mg | me;
+      while (m) {
+        const int j = __ffs(m) - 1;
+        m &= m - 1;
         // (positions are < ktot by construction; the comparison keeps a write inside the
         // list whatever the scores hold)
         uint32_t pos = 0xffffffffu;
-        if ((mg[e] >> lane) & 1u) { pos = g_before + min(e_before, tie_quota); ++g_before; }
-        else if ((me[e] >> lane) & 1u) { if (e_before < tie_quota) pos = g_before + e_before; ++e_before; }
-        if (pos < ktot) out_idx[pos] = c0 + bk * 128 + lane * 4 + e;
+        if ((mg >> j) & 1u) { pos = g_before + min(e_before, tie_quota); ++g_before; }
+        else { if (e_before < tie_quota) pos = g_before + e_before; ++e_before; }
+        if (pos < ktot) out_idx[pos] = c0 + 32 * w + j;
       }
     }
     if (crank == 0 && tid == 0) p.n_sel[u] = (int32_t)ktot;
   }
-  if constexpr (MODE != 0) {
-    cluster.sync();   // no CTA leaves while a peer may still read its totals
-    return;
-  }
-  __syncthreads();   // this CTA's part of the index list is written: it attends to its own rows
+  if constexpr (MODE != 0) return;   // (no peer reads this CTA's memory after the selection's last barrier)
 
   // ---- 4. attention over this CTA's share of the selected rows -----------------------------
   // Register-lean form (64 registers per thread): four query heads per pass (two passes for
@@ -587,13 +760,21 @@ fused_decode_kernel(const FusedParams p) {
   // lane owning 4 channels of every row.  The 16 partial logits (4 rows x 4 heads) of a step
   // are completed by a transposing xor-shuffle reduction, one shuffle per value.
   constexpr int R = 4;
-  // Every CTA attends to the tokens it selected itself (a contiguous run of the index list
-  // that it has just written), so no cluster barrier separates selection from attention.
-  const int a0 = (int)min(own_first, ktot);
-  const int a1 = (int)min(own_first + own_count, ktot);
-  float* s_acc = reinterpret_cast<float*>(smem_raw);           // [kFW][HP][128]; the key / histogram
-                                                               // area is free: all reads of it, local
-                                                               // or remote, happened before barrier 4
+  // The selected tokens are dealt out evenly: CTA r attends to rows [r, r + 1) * ktot / cs of the
+  // index list, whoever selected them (scores cluster by position, so the CTAs' own selections
+  // can differ several times in size); this costs one cluster barrier, after which the list
+  // written by the peers is visible.
+  cluster.sync();               // the index list is complete
+  const int a0 = (int)(((long long)ktot * crank) / cs);
+  const int a1 = (int)(((long long)ktot * (crank + 1)) / cs);
+  // The attention phase's working arrays take over the key / histogram area: every read of
+  // it, local or remote, happened before the selection's last barrier or the block barrier above.
+  float* s_acc = reinterpret_cast<float*>(smem_raw + sl.acc);                        // [kFW][HP][128]
+  float (*s_part)[kPartStride + 2] = reinterpret_cast<float (*)[kPartStride + 2]>(smem_raw + sl.part);
+  float (*s_p)[16] = reinterpret_cast<float (*)[16]>(smem_raw + sl.p);
+  float (*s_al)[HP] = reinterpret_cast<float (*)[HP]>(smem_raw + sl.al);
+  float (*s_m)[HP] = reinterpret_cast<float (*)[HP]>(smem_raw + sl.m);
+  float (*s_l)[HP] = reinterpret_cast<float (*)[HP]>(smem_raw + sl.l);
   const int n_hp = (p.group + HP - 1) / HP;
   for (int hp = 0; hp < n_hp; ++hp) {                          // uniform
     float2 acc[HP][2];
@@ -753,7 +934,7 @@ fused_decode_kernel(const FusedParams p) {
       dst[(crank * GP + g) * 2 + 0] = s_part[g][0];
       dst[(crank * GP + g) * 2 + 1] = s_part[g][1];
     }
-    cluster.sync();   // barrier 5: every CTA's partial results have arrived
+    cluster.sync();   // the merge barrier: every CTA's partial results have arrived
     const int opp = kFT / cs;                // outputs per pass (cs is a power of two <= 16)
     const int r = tid % cs, tl = tid / cs;
     for (int t0 = 0; t0 < per_o; t0 += opp) {   // uniform trip count
@@ -783,11 +964,7 @@ fused_decode_kernel(const FusedParams p) {
   }
 }
 
-size_t fused_smem_bytes(int cap) {
-  const size_t sel = (size_t)cap * 4 + 2 * kFBins * 4;
-  const size_t att = (size_t)kFW * 4 * FASA_HEAD_DIM * 4;
-  return sel > att ? sel : att;
-}
+size_t fused_smem_bytes(int cap) { return (size_t)fused_smem_layout(cap).total; }
 
 using FusedFn = void (*)(const FusedParams);
 
