@@ -1,23 +1,28 @@
 #!/usr/bin/env python
 """Benchmark of the FASA decode hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c1] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c2] [--impl reference]
 
 One step = one pass of the whole hot path over one batch: append one token per sequence
 (K, V and proxy-K rows), score every cached key on the dominant FCs, select the top-budget
 tokens, run exact attention over the selected rows and merge the splits.  The step is one
-call, fasa_append_decode_step (one cluster kernel: append -> score -> select -> attention);
-the stand-alone calls (fasa_kv_append, fasa_fc_score, fasa_topk, fasa_sparse_decode_attn)
-and the dense path are timed beside it, and the large batched workloads are reported under
-`other_workloads`.  Inputs are
-synthetic (paper_2602_03152_b200.synth) and resident in HBM before the timed region; L2 is
-flushed between steps.  Rank 0 prints one JSON line.
+call, fasa_append_decode_step (one cluster kernel: append -> score -> select -> attention, or
+that kernel ending after the selection + the split-K attention kernels where the selection is
+large); the stand-alone calls (fasa_kv_append, fasa_fc_score, fasa_topk,
+fasa_sparse_decode_attn) and the dense path are timed beside it.  The headline workload is
+the largest single-GPU configuration (c2: batch 16, 64K-128K contexts, 8 GiB of K/V); the
+smaller configurations ride along under `other_workloads`, and the budget row of
+configuration 4 under `budget_row`.  Inputs are synthetic (paper_2602_03152_b200.synth) and
+resident in HBM before the timed region; L2 is flushed between steps.  Rank 0 prints one JSON
+line.
 
 Headline metric: effective HBM GB/s = algorithmic bytes of the step (proxy bytes of every
 cached token + K/V rows of the selected tokens + q + out) / device time, summed over ranks;
 `us_per_step`, the dense-path time and the speedup ride along.  `roofline` describes the
-dominant kernel (the one-launch decode step, or the FC scoring stream where the step runs as
-three kernels), `cpu_baseline` the fp64 oracle timed on the host.
+dominant kernel (the cluster kernel: the whole step where it is one launch, scoring +
+selection where attention is handed to the split-K kernel), `kernels` the three calls the
+method names, `cpu_baseline` the fp64 oracle timed on the host, `parity` one unit of the timed
+configuration checked against that oracle.
 """
 from __future__ import annotations
 
@@ -40,26 +45,35 @@ UNIT = "GB/s"
 L2_FLUSH_BYTES = 256 << 20
 
 
-# DRAM traffic of the dominant kernel, from the ncu capture summarised in
-# profiles/fused_decode_kernel_c4.md: read + write bytes per launch over the launch's algorithmic
-# bytes.  Traffic follows the tokens processed, so the ratio carries over to other workloads of
-# the same kernel; it is reported only while the kernel sources are the captured ones.
-TRAFFIC_CAPTURE = {"kernel": "fused_decode_kernel", "workload": "c4", "dram_bytes": 281.33e6, "algorithmic_bytes": 277.02e6,
+# DRAM traffic of the dominant kernel from one ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum per launch) at the workload named here, next to that launch's algorithmic
+# bytes.  Traffic follows the tokens processed, so for another workload of the same kernel the
+# captured ratio is applied to its own algorithmic bytes and the figure is labelled
+# "extrapolated"; it is reported only while the kernel sources are the captured ones.
+TRAFFIC_CAPTURE = {"kernel": "fused_decode_kernel", "workload": "c4_sweep_llama3_8b_64k", "dram_bytes": None,
+                   "algorithmic_bytes": None,
                    "sources": ("paper_2602_03152_b200/csrc/fasa_fused.cu", "paper_2602_03152_b200/csrc/fasa_score_core.cuh"),
-                   "sha1": "581807e7fbd2071aa25b429937d6ecd98d2c144d"}
+                   "sha1": None}
 
 
-def _traffic(bytes_per_launch):
+def _traffic(bytes_per_launch, workload):
+    """(traffic bytes per launch or None, how it was obtained)."""
     import hashlib
+    if not TRAFFIC_CAPTURE["sha1"]:
+        return None, "no counters taken since the kernel last changed"
     h = hashlib.sha1()
     try:
         for f in TRAFFIC_CAPTURE["sources"]:
             h.update(open(os.path.join(ROOT, f), "rb").read())
     except OSError:
-        return None
+        return None, "kernel sources not found"
     if h.hexdigest() != TRAFFIC_CAPTURE["sha1"]:
-        return None     # the kernel changed since the counters were taken
-    return bytes_per_launch * TRAFFIC_CAPTURE["dram_bytes"] / TRAFFIC_CAPTURE["algorithmic_bytes"]
+        return None, "the kernel changed since the counters were taken"
+    ratio = TRAFFIC_CAPTURE["dram_bytes"] / TRAFFIC_CAPTURE["algorithmic_bytes"]
+    if workload == TRAFFIC_CAPTURE["workload"]:
+        return bytes_per_launch * ratio, "ncu counters of this workload and kernel"
+    return bytes_per_launch * ratio, ("extrapolated: DRAM bytes per algorithmic byte from an ncu capture of the same kernel at "
+                                      + TRAFFIC_CAPTURE["workload"] + ", applied to this launch's algorithmic bytes")
 
 
 def _peaks():
@@ -134,12 +148,31 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+# ---------------------------------------------------------------- shared by both arms ----
+
+def config_dict(w, lens=None):
+    """What both arms print under `config`: the workload, by name and by its numbers."""
+    lens = [w.len_lo, w.len_hi] if lens is None else lens
+    return {"workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
+            "context_lo": int(min(lens)), "context_hi": int(max(lens)), "max_len": w.max_len, "n_dom": w.n_dom,
+            "budget": w.budget, "n_sink": w.n_sink, "n_recent": w.n_recent, "heads_per_index_set": w.heads_per_set,
+            "l2": f"GPU arm: flushed before every step ({L2_FLUSH_BYTES >> 20} MiB write) and K/V + proxy larger than L2; "
+                  "CPU arm: none",
+            "per_rank": "each rank runs its own batch of independent units, no collective"}
+
+
+def oracle_sample(w):
+    """The bounded sample of a workload that the oracle is timed on: the units of sequence 0,
+    context cut to 32768 rows where longer (about a second of CPU work per pass on a few cores)."""
+    L = min(w.max_len, 32768)
+    return w.replace(batch=1, max_len=L, len_lo=min(w.len_lo, L), len_hi=min(w.len_hi, L))
+
+
 # ---------------------------------------------------------------- reference arm ----
 
 def run_reference(args, w):
     """Times the fp64 CPU oracle, as it stands, on the host cores: each step is one oracle
     pass (score -> select -> attention) over a bounded sample of the workload's units."""
-    import numpy as np
     from oracle import fasa_oracle as O
     from paper_2602_03152_b200 import synth
 
@@ -147,8 +180,7 @@ def run_reference(args, w):
     if rank != 0:
         return
     cores = os.cpu_count() or 1
-    # sample: at most 8 units, sequences cut to 32768 rows (about a second of CPU work per step)
-    sw = w.replace(batch=1, max_len=min(w.max_len, 32768), len_lo=min(w.len_lo, 32768), len_hi=min(w.len_hi, 32768))
+    sw = oracle_sample(w)
     t = synth.make_inputs(sw, "cpu")
     qb, kb, vb = synth.bf16_bits(t["q"]), synth.bf16_bits(t["k"]), synth.bf16_bits(t["v"])
     lens, dom = t["seq_lens"].numpy(), t["dom"].numpy()
@@ -163,12 +195,11 @@ def run_reference(args, w):
     dt = (time.perf_counter() - t0) / steps
     by = step_bytes(sw, lens, int(r["n_sel"].sum()))
     val = by["fasa"] / dt / 1e9
-    sample = f"{sw.n_kv_heads} units (batch 1 of {w.batch}), context {int(lens[0])}, one oracle pass per step"
+    sample = f"{sw.n_kv_heads} units (sequence 0 of {w.batch}), context {int(lens[0])}, one oracle pass per step"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "sample": sample},
+        "dtype": "f64", "data": "synthetic", "config": config_dict(w), "sample": sample,
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": int(r["threads"]), "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }), flush=True)
@@ -176,10 +207,12 @@ def run_reference(args, w):
 
 # ---------------------------------------------------------------- our arm ----
 
-def measure(w, K, W, dev, world, step_mode=None, sampler_factory=None, want_e2e=True, t=None, lens=None):
+def measure(w, K, W, dev, world, step_mode=None, sampler_factory=None, want_e2e=True, t=None, lens=None,
+            min_region_s=0.0, want_parts=True, want_dense=True):
     """Times one workload on this rank's GPU; returns a dict of measurements (durations are
     max over ranks where that matters).  `t` reuses inputs drawn earlier (their dominant-FC
-    list is redrawn for w.n_dom); `lens` overrides the sequence lengths."""
+    list is redrawn for w.n_dom); `lens` overrides the sequence lengths.  The timed region is
+    one block of exactly K steps, repeated until it has run for min_region_s of device time."""
     import torch
     import torch.distributed as dist
 
@@ -259,39 +292,55 @@ def measure(w, K, W, dev, world, step_mode=None, sampler_factory=None, want_e2e=
     if sampler is not None:
         sampler.mark()
 
-    # ---- timed region: K whole steps ------------------------------------------------
+    # ---- timed region: blocks of exactly K whole steps ----------------------------------
     timed(fasa_step, 0, W)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     l0 = f.launch_count()
-    step_us = timed(fasa_step, K, 0)
+    blocks = [timed(fasa_step, K, 0)]
     torch.cuda.synchronize()
     launches = f.launch_count() - l0
+    while sum(sum(b_) for b_ in blocks) * 1e-6 < min_region_s and len(blocks) < 200 and world == 1:
+        blocks.append(timed(fasa_step, K, 0))
+    torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    us_per_step = rank_max(sum(step_us)) / K
+    block_us = [sum(b_) / K for b_ in blocks]
+    us_per_step = rank_max(sum(block_us) / len(block_us))
+    all_steps = [x for b_ in blocks for x in b_]
 
     n_sel_total = int(n_sel.sum().item())
     by = step_bytes(w, lens_full.cpu().tolist(), n_sel_total)
+    Kk = min(K, 200)
+
+    # ---- the dominant kernel alone, where the step is several launches --------------------
+    launches_per_step = launches / max(K, 1)
+    select_us = None
+    if fused and launches_per_step > 1:
+        select_us = statistics.mean(timed(lambda: f.select_step(q, k, v, proxy, lens, w.budget, None, idx, n_sel, k_new, v_new),
+                                          Kk, W))
+        lens.copy_(lens_start)
+        fasa_step()                                # (leave idx / n_sel / out as the whole step writes them)
 
     # ---- the stand-alone calls, one C-ABI call at a time ---------------------------------
-    parts = {"kv_append": [], "fc_score": [], "topk": [], "sparse_attn": []}
-    Kk = min(K, 200)
-    for i in range(W + Kk):
-        lens.copy_(lens_start)
-        flush.fill_(i & 0xff)
-        e = [ev() for _ in range(5)]
-        e[0].record(); f.kv_append(k, v, proxy, lens, k_new, v_new)
-        e[1].record(); f.fc_score(q, proxy, lens, scores)
-        e[2].record(); f.topk(scores, lens, w.budget, idx, n_sel, ws)
-        e[3].record(); f.sparse_decode_attn(q, k, v, idx, n_sel, out, ws)
-        e[4].record(); e[4].synchronize()
-        if i >= W:
-            for j, name in enumerate(parts):
-                parts[name].append(e[j].elapsed_time(e[j + 1]) * 1e3)
-    kern_us = {n: statistics.mean(v_) for n, v_ in parts.items()}
-    dense_us = statistics.mean(timed(dense_step, Kk, W))
+    kern_us = None
+    if want_parts:
+        parts = {"kv_append": [], "fc_score": [], "topk": [], "sparse_attn": []}
+        for i in range(W + Kk):
+            lens.copy_(lens_start)
+            flush.fill_(i & 0xff)
+            e = [ev() for _ in range(5)]
+            e[0].record(); f.kv_append(k, v, proxy, lens, k_new, v_new)
+            e[1].record(); f.fc_score(q, proxy, lens, scores)
+            e[2].record(); f.topk(scores, lens, w.budget, idx, n_sel, ws)
+            e[3].record(); f.sparse_decode_attn(q, k, v, idx, n_sel, out, ws)
+            e[4].record(); e[4].synchronize()
+            if i >= W:
+                for j, name in enumerate(parts):
+                    parts[name].append(e[j].elapsed_time(e[j + 1]) * 1e3)
+        kern_us = {n: statistics.mean(v_) for n, v_ in parts.items()}
+    dense_us = statistics.mean(timed(dense_step, min(Kk, 50), W)) if want_dense else None
 
     # ---- end to end from host buffers ---------------------------------------------------
     e2e_us = h2d = d2h = None
@@ -307,39 +356,65 @@ def measure(w, K, W, dev, world, step_mode=None, sampler_factory=None, want_e2e=
         e2e_us = rank_max(statistics.mean(timed(e2e_step, Kk, W)))
         h2d = qh.numel() * 2 + knh.numel() * 2 + vnh.numel() * 2
         d2h = oh.numel() * 4
+    # one more whole step, whose outputs the parity check reads
+    lens.copy_(lens_start)
+    fasa_step()
+    torch.cuda.synchronize()
     status = f.device_status()
     clocks = sampler.stop() if sampler else None
-    return dict(w=w, t=t, by=by, us_per_step=us_per_step, step_us_median=statistics.median(step_us), launches=launches,
-                kern_us=kern_us, dense_us=dense_us, e2e_us=e2e_us, h2d=h2d, d2h=d2h, status=status, clocks=clocks,
-                fused=fused, cluster_size=f.step_cluster_size(), launches_per_step=launches / max(K, 1), n_sel_total=n_sel_total, lens_full=lens_full)
+    return dict(w=w, t=t, by=by, us_per_step=us_per_step, step_us_median=statistics.median(all_steps),
+                block_us=block_us, launches=launches, kern_us=kern_us, dense_us=dense_us, e2e_us=e2e_us, h2d=h2d,
+                d2h=d2h, status=status, clocks=clocks, fused=fused, cluster_size=f.step_cluster_size(),
+                launches_per_step=launches_per_step, select_us=select_us, n_sel_total=n_sel_total,
+                lens_full=lens_full, last=dict(idx=idx, n_sel=n_sel, out=out))
+
+
+def kernel_rooflines(m, peak):
+    """The three calls the method names, each against its own bytes: `bytes` counts what the
+    call must move including its unavoidable scratch (the fp32 score per token that scoring
+    writes and the selection reads, the index list), `bytes_method` only what the byte model of
+    the method counts for that stage (proxy rows; nothing for the selection; K/V rows)."""
+    w, by, ku = m["w"], m["by"], m["kern_us"]
+    tokens = by["proxy"] // (4 * w.n_dom) * w.n_sets // w.n_kv_heads      # scored positions: one fp32 per (set, token)
+    sel = m["n_sel_total"]
+    rows = {
+        "fasa_fc_score": (by["proxy"] + 4 * tokens + by["qo"] // 3, by["proxy"], ku["fc_score"]),
+        "fasa_topk": (4 * tokens + 4 * sel, 0, ku["topk"]),
+        "fasa_sparse_decode_attn": (by["gathered"] + 4 * sel + by["qo"], by["gathered"], ku["sparse_attn"]),
+    }
+    out = {}
+    for name, (b_all, b_method, us) in rows.items():
+        out[name] = {"us": us, "bytes": b_all, "gbs": b_all / us / 1e3, "frac": b_all / us / 1e3 / peak, "bound": "hbm",
+                     "bytes_method": b_method, "frac_method_bytes": b_method / us / 1e3 / peak}
+    return out
 
 
 def summarize(m, peak):
     """The figures every workload reports (the headline workload adds the contract's keys)."""
-    w, by, ku = m["w"], m["by"], m["kern_us"]
+    w, by = m["w"], m["by"]
     gbs = lambda nbytes, us: nbytes / (us * 1e-6) / 1e9
-    score_bytes = by["proxy"]
-    topk_bytes = by["proxy"] // w.n_dom           # one fp32 score per cached token
-    return {
+    r = {
         "workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
         "context": int(m["lens_full"].max()), "context_mean": float(m["lens_full"].float().mean()),
         "n_dom": w.n_dom, "budget": w.budget, "n_sink": w.n_sink, "n_recent": w.n_recent,
         "n_sel_per_unit": m["n_sel_total"] / (w.batch * w.n_sets), "heads_per_index_set": w.heads_per_set,
         "step_mode": ("three kernels" if not m["fused"] else
                       f"one cluster kernel (cluster of {m['cluster_size']})" if m["launches_per_step"] == 1 else
-                      f"cluster kernel (cluster of {m['cluster_size']}) + split-K tensor-core attention"),
+                      f"cluster kernel (cluster of {m['cluster_size']}, ends after the selection) + split-K tensor-core attention + merge"),
         "launches_per_step": m["launches_per_step"],
-        "us_per_step": m["us_per_step"], "step_bytes": by["fasa"],
+        "us_per_step": m["us_per_step"], "us_per_step_median": m["step_us_median"], "step_bytes": by["fasa"],
         "step_gbs": gbs(by["fasa"], m["us_per_step"]), "step_frac_of_peak": gbs(by["fasa"], m["us_per_step"]) / peak,
-        "dense_us_per_step": m["dense_us"], "dense_bytes": by["dense"],
-        "dense_frac_of_peak": gbs(by["dense"], m["dense_us"]) / peak,
-        "speedup_vs_dense": m["dense_us"] / m["us_per_step"], "byte_ratio_dense_over_fasa": by["dense"] / by["fasa"],
-        "standalone_us": ku,
-        "standalone_frac_of_peak": {"fc_score": gbs(score_bytes, ku["fc_score"]) / peak,
-                                    "topk": gbs(topk_bytes, ku["topk"]) / peak,
-                                    "sparse_attn": gbs(by["gathered"], ku["sparse_attn"]) / peak},
         "device_status": m["status"],
     }
+    if m["dense_us"] is not None:
+        r.update({"dense_us_per_step": m["dense_us"], "dense_bytes": by["dense"],
+                  "dense_frac_of_peak": gbs(by["dense"], m["dense_us"]) / peak,
+                  "speedup_vs_dense": m["dense_us"] / m["us_per_step"],
+                  "byte_ratio_dense_over_fasa": by["dense"] / by["fasa"]})
+    if m["kern_us"] is not None:
+        r["standalone_us"] = m["kern_us"]
+        r["kernels"] = kernel_rooflines(m, peak)
+    return r
 
 
 def run_fasa(args, w):
@@ -368,63 +443,97 @@ def run_fasa(args, w):
     # Weak scaling: every rank holds its own batch of independent (batch, KV head) units.
     wl = w.replace(index=w.index + 100 * rank)
     sampler = ClockSampler(gpu_id) if rank == 0 else None     # started early, marked at the timed region
-    m = measure(wl, K, W, dev, world, args.step_mode, (lambda: sampler) if rank == 0 else None)
+    m = measure(wl, K, W, dev, world, args.step_mode, (lambda: sampler) if rank == 0 else None,
+                min_region_s=args.min_region_s)
 
-    # Other configurations of the same path, a few steps each (single GPU only): the large
-    # batched shapes, where the stream is long enough to approach the HBM roofline.
-    others = []
+    peak, peak_src = _peaks()
+    line_extra = {}
+    if world == 1 and rank == 0 and not args.no_cpu_baseline:
+        line_extra = cpu_baseline(wl, m)                       # (reads the inputs: before they are released)
+    m.pop("t")
+    m.pop("last")
+    torch.cuda.empty_cache()
+
+    # Other configurations of the same path, a few steps each (single GPU only).
+    others, budget_row = [], []
     if world == 1 and not args.no_extras:
         for name in args.extras.split(","):
             if name and name in synth.CONFIGS and name != args.config:
-                mo = measure(synth.CONFIGS[name], 30, 3, dev, 1, args.step_mode, None, want_e2e=False)
-                mo.pop("t")
-                others.append(mo)
+                mo = measure(synth.CONFIGS[name], 50, 3, dev, 1, args.step_mode, None, want_e2e=False, min_region_s=0.05)
+                mo.pop("t"); mo.pop("last")
+                others.append(summarize(mo, peak))
+                del mo
+                torch.cuda.empty_cache()
+    if world == 1 and not args.no_budget_row:
+        # configuration 4 at 16 dominant FCs, every budget of its grid: the step and the dense
+        # path at each point ("speed-up over dense at every budget")
+        base = synth.CONFIGS["c4"]
+        tb = synth.make_inputs(base, dev)
+        for kb in (64, 128, 256, 512, 1024, 2048, 4096):
+            mo = measure(base.replace(budget=kb), 12, 3, dev, 1, args.step_mode, None, want_e2e=False, t=tb,
+                         want_parts=False, want_dense=True)
+            sm = summarize(mo, peak)
+            budget_row.append({k_: sm[k_] for k_ in ("budget", "us_per_step", "step_bytes", "step_frac_of_peak", "dense_us_per_step",
+                                                     "speedup_vs_dense", "byte_ratio_dense_over_fasa", "launches_per_step", "device_status")})
+            del mo
+        del tb
+        torch.cuda.empty_cache()
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    peak, peak_src = _peaks()
     by, us_per_step = m["by"], m["us_per_step"]
     head = summarize(m, peak)
     roof_us = by["fasa"] / (peak * 1e9) * 1e6
-    if m["fused"]:
+    if m["fused"] and m["launches_per_step"] == 1:
         # dominant kernel = the whole step in one launch: its algorithmic bytes are the step's
-        roofline = {"kernel": "fused_decode_kernel", "bound": "hbm", "achieved": head["step_gbs"], "peak": peak,
-                    "unit": "GB/s", "frac": head["step_frac_of_peak"],
-                    "traffic": _traffic(by["fasa"]) if m["launches_per_step"] == 1 else None,
-                    "traffic_source": "ncu capture at workload c4 scaled by algorithmic bytes (profiles/fused_decode_kernel_c4.md)",
+        tr, tr_src = _traffic(by["fasa"], wl.name)
+        roofline = {"kernel": "fused_decode_kernel (whole step)", "bound": "hbm", "achieved": head["step_gbs"], "peak": peak,
+                    "unit": "GB/s", "frac": head["step_frac_of_peak"], "traffic": tr, "traffic_source": tr_src,
                     "bytes_per_launch": by["fasa"], "us_per_launch": us_per_step, "peak_source": peak_src,
                     "cluster_size": m["cluster_size"]}
+    elif m["fused"]:
+        # dominant kernel = the cluster kernel ending after the selection (append + scoring + selection
+        # in one launch): it moves the proxy rows of every token, q and the index lists it writes
+        kb = by["proxy"] + by["qo"] // 3 + 4 * m["n_sel_total"]
+        us = m["select_us"]
+        tr, tr_src = _traffic(kb, wl.name)
+        roofline = {"kernel": "fused_decode_kernel (append + scoring + selection)", "bound": "hbm",
+                    "achieved": kb / us / 1e3, "peak": peak, "unit": "GB/s", "frac": kb / us / 1e3 / peak,
+                    "traffic": tr, "traffic_source": tr_src, "bytes_per_launch": kb, "us_per_launch": us,
+                    "share_of_step_time": us / us_per_step, "peak_source": peak_src, "cluster_size": m["cluster_size"]}
     else:
         fc_us = m["kern_us"]["fc_score"]
         roofline = {"kernel": "fc_score_kernel", "bound": "hbm", "achieved": by["proxy"] / (fc_us * 1e-6) / 1e9,
                     "peak": peak, "unit": "GB/s", "frac": by["proxy"] / (fc_us * 1e-6) / 1e9 / peak, "traffic": None,
-                    "bytes_per_launch": by["proxy"], "us_per_launch": fc_us, "peak_source": peak_src}
+                    "traffic_source": "no counters taken", "bytes_per_launch": by["proxy"], "us_per_launch": fc_us,
+                    "peak_source": peak_src}
     roofline["frac_of_nominal_8tbs"] = roofline["achieved"] / 8000.0      # context: the DGX figure for HBM3e
-    cfg = {k_: head[k_] for k_ in ("workload", "batch", "n_q_heads", "n_kv_heads", "context", "context_mean", "n_dom",
-                                   "budget", "n_sink", "n_recent", "n_sel_per_unit", "step_mode")}
-    cfg["l2"] = f"flushed before every step ({L2_FLUSH_BYTES >> 20} MiB write)"
-    cfg["per_rank"] = "each rank runs its own batch of independent units, no collective"
+    cfg = config_dict(w, m["lens_full"].cpu().tolist())
+    cfg["step_mode"] = head["step_mode"]
+    clocks = m["clocks"]
     line = {
         "metric": METRIC, "value": world * by["fasa"] / (us_per_step * 1e-6) / 1e9, "unit": UNIT,
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": us_per_step / 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, f32 accumulate",
         "data": "synthetic", "config": cfg,
-        "us_per_step": us_per_step, "us_per_step_median": m["step_us_median"],
+        "timed_blocks": len(m["block_us"]), "us_per_step": us_per_step,
+        "us_per_step_median_block": statistics.median(m["block_us"]), "us_per_step_median": m["step_us_median"],
+        "us_per_step_x_sm_mhz": (us_per_step * clocks["sm_mhz"]) if clocks and clocks.get("sm_mhz") else None,
+        "n_sel_per_unit": head["n_sel_per_unit"],
         "step_bytes": by["fasa"], "step_roofline_us": roof_us, "step_frac_of_roofline": roof_us / us_per_step,
         "dense_us_per_step": m["dense_us"], "dense_bytes": by["dense"], "dense_frac_of_roofline": head["dense_frac_of_peak"],
         "speedup_vs_dense": head["speedup_vs_dense"], "byte_ratio_dense_over_fasa": head["byte_ratio_dense_over_fasa"],
-        "standalone_kernels_us": m["kern_us"], "standalone_kernels_frac_of_peak": head["standalone_frac_of_peak"],
+        "standalone_kernels_us": m["kern_us"], "kernels": head["kernels"],
         "roofline": roofline,
         "e2e": {"value": world * by["fasa"] / (m["e2e_us"] * 1e-6) / 1e9, "unit": UNIT, "us_per_step": m["e2e_us"],
                 "h2d_bytes_per_step": m["h2d"], "d2h_bytes_per_step": m["d2h"]},
-        "gpu_launches": int(m["launches"]), "device_status": m["status"], "clocks": m["clocks"],
-        "other_workloads": [summarize(mo, peak) for mo in others],
+        "gpu_launches": int(m["launches"]), "device_status": m["status"], "clocks": clocks,
+        "other_workloads": others, "budget_row": {"workload": "c4_sweep_llama3_8b_64k", "n_dom": 16, "rows": budget_row},
     }
-    if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(wl, m["t"], by)
+    line.update(line_extra)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -455,7 +564,7 @@ def run_sweep(args):
             sm = summarize(m, peak)
             rows.append({k_: sm[k_] for k_ in ("n_dom", "budget", "us_per_step", "step_bytes", "step_gbs", "step_frac_of_peak",
                                                "dense_us_per_step", "speedup_vs_dense", "byte_ratio_dense_over_fasa",
-                                               "standalone_us", "standalone_frac_of_peak", "step_mode", "launches_per_step",
+                                               "standalone_us", "kernels", "step_mode", "launches_per_step",
                                                "device_status")})
             del m
     print(json.dumps({"sweep": base.name, "batch": base.batch, "context": base.max_len,
@@ -865,30 +974,65 @@ def run_longcot(args):
     print(json.dumps(res), flush=True)
 
 
-def cpu_baseline(w, t, by):
-    """The fp64 oracle, as it stands, timed on the host cores on a bounded sample: the units
-    of the first sequence, one whole pass (score -> select -> attention)."""
+def cpu_baseline(w, m):
+    """The fp64 oracle, as it stands, on the host: (1) timed on a bounded sample of the workload
+    (the units of sequence 0, context cut to 32768 rows where longer), on all cores and on one;
+    (2) one unit of the TIMED configuration at its full length, checked against the step's last
+    outputs with the parity rules of the tests.  Returns the `cpu_baseline` and `parity` objects."""
+    import math
+
+    import numpy as np
+
     from oracle import fasa_oracle as O
+    from oracle import parity as P
     from paper_2602_03152_b200 import synth
 
+    t = m["t"]
     cores = os.cpu_count() or 1
-    L = int(t["seq_lens"][0])
+    L = min(int(t["seq_lens"][0]), 32768)
     qb = synth.bf16_bits(t["q"][:1])
     kb = synth.bf16_bits(t["k"][:1, :, :L])
     vb = synth.bf16_bits(t["v"][:1, :, :L])
-    lens = t["seq_lens"][:1].cpu().numpy()
-    kw = dict(pairing=w.pairing, group_reduce=w.group_reduce, n_sink=w.n_sink, n_recent=w.n_recent,
-              budget=w.budget, n_sel_max=w.n_sel_max(), n_threads=cores, want_scores=False, want_dense=False)
-    r = O.decode_bf16(qb, kb, vb, lens, t["dom"].numpy(), **kw)      # warm-up, page in
-    reps, t0 = 0, time.perf_counter()
-    while reps < 3 or (time.perf_counter() - t0 < 10.0 and reps < 2000):
-        r = O.decode_bf16(qb, kb, vb, lens, t["dom"].numpy(), **kw)
-        reps += 1
-    dt = (time.perf_counter() - t0) / reps
+    lens = np.array([L], dtype=np.int32)
+    dom = t["dom"].numpy()
+    res = {}
+    for label, threads, budget_s in (("all", cores, 10.0), ("one", 1, 6.0)):
+        kw = dict(pairing=w.pairing, group_reduce=w.group_reduce, n_sink=w.n_sink, n_recent=w.n_recent,
+                  budget=w.budget, n_sel_max=w.n_sel_max(), n_threads=threads, want_scores=False, want_dense=False)
+        r = O.decode_bf16(qb, kb, vb, lens, dom, **kw)      # warm-up, page in
+        reps, t0 = 0, time.perf_counter()
+        while reps < 2 or (time.perf_counter() - t0 < budget_s and reps < 2000):
+            r = O.decode_bf16(qb, kb, vb, lens, dom, **kw)
+            reps += 1
+        res[label] = ((time.perf_counter() - t0) / reps, int(r["threads"]), reps)
     sb = step_bytes(w.replace(batch=1), [L], int(r["n_sel"].sum()))
-    return {"value": sb["fasa"] / dt / 1e9, "unit": UNIT, "cores": int(r["threads"]), "kind": "oracle",
-            "us_per_step_sample": dt * 1e6,
-            "sample": f"{w.n_kv_heads} units of sequence 0 (context {L}) out of batch {w.batch}, {reps} passes"}
+    dt, used, reps = res["all"]
+    base = {"value": sb["fasa"] / dt / 1e9, "unit": UNIT, "cores": used, "kind": "oracle", "us_per_step_sample": dt * 1e6,
+            "single_thread": {"value": sb["fasa"] / res["one"][0] / 1e9, "unit": UNIT, "cores": 1,
+                              "us_per_step_sample": res["one"][0] * 1e6, "passes": res["one"][2]},
+            "sample": f"{w.n_kv_heads} units of sequence 0 (context {L}"
+                      + (f", cut from {int(t['seq_lens'][0])}" if L < int(t["seq_lens"][0]) else "")
+                      + f") out of batch {w.batch}, {reps} passes"}
+
+    # parity of the timed configuration: unit (sequence 0, index set 0) at its full length
+    last = m["last"]
+    G = w.heads_per_set
+    h = 0
+    Lf = int(t["seq_lens"][0])
+    par = {"unit": [0, 0], "context": Lf, "ok": False}
+    try:
+        rep = P.check_step(t["q"][:1, :G].cpu().double().numpy(), t["k"][:1, :1, :Lf].cpu().double().numpy(),
+                           t["v"][:1, :1, :Lf].cpu().double().numpy(), [Lf], np.sort(dom, axis=1)[h:h + 1], pairing=w.pairing,
+                           group_reduce=w.group_reduce, n_sink=w.n_sink, n_recent=w.n_recent, budget=w.budget,
+                           scale=1.0 / math.sqrt(128.0), idx=last["idx"][:1, :1].cpu().numpy(),
+                           n_sel=last["n_sel"][:1, :1].cpu().numpy(), out=last["out"][:1, :G].cpu().numpy(),
+                           sel_heads=w.sel_heads, what="bench")
+        par.update(ok=True, index_set_identical=bool(rep["sets_identical"]), attn_max_abs_err=rep["attn_err"],
+                   attn_tolerance=P.ATTN_ABS, n_sel=int(last["n_sel"][0, 0]),
+                   rule="index set bit-exact outside the 1e-3 tie band; attention max-abs <= 2e-3 against the oracle on the GPU's set")
+    except AssertionError as e:
+        par["error"] = str(e)[:300]
+    return {"cpu_baseline": base, "parity": par}
 
 
 def main():
@@ -897,14 +1041,17 @@ def main():
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="fasa", choices=["fasa", "reference"])
-    ap.add_argument("--config", default="c1", help="workload: c0, c1 (default), c2, c4")
+    ap.add_argument("--config", default="c2", help="workload: c0, c1, c2 (default: the largest single-GPU one), c4")
     ap.add_argument("--budget", type=int, default=None)
     ap.add_argument("--n-dom", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (profiling)")
     ap.add_argument("--select-heads", type=int, default=None,
                     help="query heads sharing one index set (default: all heads of a KV head; 1 = a set per head)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--extras", default="c4,c2", help="other workloads reported under other_workloads (30 steps each)")
+    ap.add_argument("--extras", default="c1,c4", help="other workloads reported under other_workloads (50 steps each)")
+    ap.add_argument("--no-budget-row", action="store_true", help="skip configuration 4's budget row")
+    ap.add_argument("--min-region-s", type=float, default=0.4,
+                    help="repeat the block of --steps steps until the timed region has run this long on the device")
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="config 4 grid (budget x dominant FCs) instead of the bench line")
     ap.add_argument("--longcot", action="store_true", help="config 3 (long-CoT decode) instead of the bench line")

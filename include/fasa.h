@@ -70,6 +70,12 @@
  *   - Data-dependent problems (a sequence longer than max_len, an index out of
  *     range) never fault: the kernel clamps and ORs a bit into a device status
  *     word read by fasa_get_device_status.
+ *   - One context, one stream order.  The status word and the per-sequence arrival
+ *     counters with which the appending calls update seq_lens belong to the context.
+ *     Calls on the same context must therefore be ordered on the device (one stream, or
+ *     streams joined by events): two appending calls of one context that overlap corrupt
+ *     the length update without any error.  Different contexts are independent (apart from
+ *     the shared array of fasa_sparse_decode_attn_static, see there).
  */
 #ifndef FASA_H_
 #define FASA_H_
@@ -234,7 +240,10 @@ int32_t fasa_full_decode_attn(fasa_ctx_t* ctx, const void* q, const void* k_cach
  *     enqueued.  Configuration 1 of the benchmarks needs 0.1 MB, configuration 2 1.4 MB.
  *   - The context's device must be current (FASA_ERR_INVALID_ARG otherwise).  The first
  *     call on a device looks up the array's device address (a CUDA runtime query, no
- *     allocation); make that first call before any stream capture begins.
+ *     allocation; where the CUDA runtime loads modules lazily, that query is also what
+ *     places the library's module, array included, on the device); make that first call
+ *     before any stream capture begins.  The address is remembered per device for the
+ *     life of the process and does not survive a cudaDeviceReset.
  *   - All calls in the process share the one array per device.  Nothing in it has to
  *     start at zero (every partial that is read was written by the same call), but
  *     two calls whose kernels overlap on the GPU (different streams, or different
@@ -289,11 +298,28 @@ int32_t fasa_append_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_ne
                                 float* scores, int32_t* idx, int32_t* n_sel, float* out,
                                 float* lse, void* workspace, void* stream);
 
+/* Token importance prediction and selection of one step in ONE launch (TIP then TopK-I,
+ * Sec. 4.1): what fasa_decode_step does before it attends, for callers that run their own
+ * attention over the selected rows (or want the index sets alone).  Outputs idx, n_sel and,
+ * unless NULL, scores, exactly as fasa_fc_score followed by fasa_topk give them.  k_new and
+ * v_new (both NULL, or both bf16 [batch][n_kv_heads][1][128]) make it the appending form:
+ * UpdateCache first, as in fasa_append_decode_step, and seq_lens[b] += 1.  Only the cluster
+ * kernel provides this: FASA_ERR_UNSUPPORTED when fasa_step_cluster_size is 0. */
+int32_t fasa_select_step(fasa_ctx_t* ctx, const void* q, const void* k_new, const void* v_new,
+                         void* k_cache, void* v_cache, void* proxy_k, int32_t* seq_lens,
+                         int32_t budget, int32_t n_sel_max, float* scores, int32_t* idx,
+                         int32_t* n_sel, void* stream);
+
 /* End-to-end step from HOST buffers: q_host, k_new_host, v_new_host (layouts as
  * fasa_kv_append with n_new = 1) -> fasa_append_decode_step -> out copied to out_host
  * (fp32 [batch][n_q_heads][128]); synchronises the stream.  Inputs in pinned (page-locked,
- * mapped) host memory are read by the kernels in place, across the host link; pageable
- * inputs are first copied to the device staging area dev_stage (>= fasa_stage_bytes). */
+ * mapped) host memory need no copy call: a step that is one launch of one wave of CTAs reads
+ * them in place, across the host link; otherwise one small kernel brings them to the device
+ * staging area dev_stage (>= fasa_stage_bytes) first.  Pageable inputs are copied there with
+ * three asynchronous copies.  A pinned out_host is written by the step's last kernel itself.
+ * The context remembers what the driver said about the last four host pointers it saw, so a
+ * loop that passes the same buffers asks once; a buffer must therefore not change its kind
+ * (pageable / page-locked) while keeping its address between two calls. */
 int32_t fasa_stage_bytes(const fasa_ctx_t* ctx, size_t* out_bytes);
 int32_t fasa_decode_step_host(fasa_ctx_t* ctx, const void* q_host, const void* k_new_host,
                               const void* v_new_host, void* dev_stage, void* k_cache,

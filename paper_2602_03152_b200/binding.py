@@ -26,7 +26,7 @@ SYMBOLS = [
     "fasa_kv_append", "fasa_proxy_build", "fasa_fc_score", "fasa_topk", "fasa_sparse_decode_attn",
     "fasa_full_decode_attn", "fasa_decode_step", "fasa_stage_bytes", "fasa_decode_step_host",
     "fasa_sparse_decode_attn_static", "fasa_set_step_mode", "fasa_step_cluster_size",
-    "fasa_append_decode_step", "fasa_proxy_bytes",
+    "fasa_append_decode_step", "fasa_proxy_bytes", "fasa_select_step",
     "fasa_calib_workspace_bytes", "fasa_calib_accumulate", "fasa_calib_select", "fasa_set_block_table",
 ]
 
@@ -84,6 +84,7 @@ def load_library() -> ctypes.CDLL:
         "fasa_set_step_mode": (i32, [vp, i32]),
         "fasa_step_cluster_size": (i32, [vp]),
         "fasa_append_decode_step": (i32, [vp] * 8 + [i32, i32] + [vp] * 7),
+        "fasa_select_step": (i32, [vp] * 8 + [i32, i32] + [vp] * 4),
         "fasa_stage_bytes": (i32, [vp, ctypes.POINTER(ctypes.c_size_t)]),
         "fasa_decode_step_host": (i32, [vp] * 9 + [i32, i32] + [vp] * 7),
         "fasa_calib_workspace_bytes": (i32, [vp, i32, ctypes.POINTER(ctypes.c_size_t)]),
@@ -293,6 +294,14 @@ class Fasa:
             k_cache.data_ptr(), v_cache.data_ptr(), _dp(proxy_k), _dp(seq_lens, torch.int32), budget, n_sel_max,
             _dp(scores, torch.float32), _dp(idx, torch.int32), _dp(n_sel, torch.int32), _dp(out, torch.float32),
             _dp(lse), _dp(workspace), _stream()), "fasa_append_decode_step")
+
+    def select_step(self, q, k_cache, v_cache, proxy_k, seq_lens, budget, scores, idx, n_sel, k_new=None, v_new=None):
+        """Scoring and selection in one launch, no attention (appending form when k_new / v_new are given)."""
+        n_sel_max = idx.shape[-1]
+        self._check(self._lib.fasa_select_step(
+            self._h, _dp(q, torch.bfloat16), _dp(k_new, torch.bfloat16), _dp(v_new, torch.bfloat16),
+            k_cache.data_ptr(), v_cache.data_ptr(), _dp(proxy_k), _dp(seq_lens, torch.int32), budget, n_sel_max,
+            _dp(scores, torch.float32), _dp(idx, torch.int32), _dp(n_sel, torch.int32), _stream()), "fasa_select_step")
 
     # -- offline calibration (Algorithm 1) ---------------------------------------
     def calib_workspace_bytes(self, top_k: int) -> int:

@@ -213,6 +213,15 @@ extern "C" int32_t fasa_workspace_bytes(const fasa_ctx_t* ctx, int32_t n_sel_max
   return FASA_OK;
 }
 
+// What fasa_fc_score, fasa_topk and fasa_sparse_decode_attn require of the arguments they share
+// with the composite calls.
+static bool three_kernel_args_ok(const fasa_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                                 const void* proxy_k, const float* scores, const void* workspace) {
+  return scores && workspace && fasa_pages_ready(ctx) && !((uintptr_t)proxy_k & 15) && !((uintptr_t)q & 15) &&
+         !((uintptr_t)scores & 3) && !((uintptr_t)k_cache & 15) && !((uintptr_t)v_cache & 15) &&
+         !((uintptr_t)workspace & 255);
+}
+
 extern "C" int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_cache,
                                     const void* v_cache, const void* proxy_k,
                                     const int32_t* seq_lens, int32_t budget, int32_t n_sel_max,
@@ -225,7 +234,9 @@ extern "C" int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* 
     if (((uintptr_t)proxy_k & 15) || ((uintptr_t)q & 15) || ((uintptr_t)k_cache & 15) ||
         ((uintptr_t)v_cache & 15) || (scores && ((uintptr_t)scores & 3)))
       return FASA_ERR_INVALID_ARG;
+    if (!fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
     if (fasa_attend_separately(ctx, n_sel_max, workspace)) {
+      if ((uintptr_t)workspace & 255) return FASA_ERR_INVALID_ARG;   // (what the second launch would refuse)
       int32_t st2 = fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
                                       idx, n_sel, out, lse, nullptr, nullptr, (cudaStream_t)stream, false);
       if (st2 != FASA_OK) return st2;
@@ -234,7 +245,8 @@ extern "C" int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* 
     return fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
                              idx, n_sel, out, lse, nullptr, nullptr, (cudaStream_t)stream);
   }
-  if (!scores || !workspace) return FASA_ERR_INVALID_ARG;
+  // three kernels: everything any of them would refuse is refused before the first is enqueued
+  if (!three_kernel_args_ok(ctx, q, k_cache, v_cache, proxy_k, scores, workspace)) return FASA_ERR_INVALID_ARG;
   int32_t st = fasa_fc_score(ctx, q, proxy_k, seq_lens, scores, stream);
   if (st != FASA_OK) return st;
   st = fasa_topk(ctx, scores, seq_lens, budget, n_sel_max, idx, n_sel, workspace, stream);
@@ -260,16 +272,24 @@ static int32_t append_decode_step_impl(fasa_ctx_t* ctx, const void* q, const voi
         ((uintptr_t)v_cache & 15) || ((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15) ||
         (scores && ((uintptr_t)scores & 3)))
       return FASA_ERR_INVALID_ARG;
+    if (!fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
     if (fasa_attend_separately(ctx, n_sel_max, workspace)) {
+      if ((uintptr_t)workspace & 255) return FASA_ERR_INVALID_ARG;   // (what the second launch would refuse)
       int32_t st2 = fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
                                       idx, n_sel, out, lse, k_new, v_new, (cudaStream_t)stream, false);
       if (st2 != FASA_OK) return st2;
-      return fasa_sparse_decode_attn(ctx, q, k_cache, v_cache, idx, n_sel, n_sel_max, out, lse, workspace, stream);
+      return fasa_sparse_attn_mirrored(ctx, q, k_cache, v_cache, idx, n_sel, n_sel_max, out, lse, workspace,
+                                       (cudaStream_t)stream, out_mirror, mirrored);
     }
     *mirrored = out_mirror != nullptr;
     return fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
                              idx, n_sel, out, lse, k_new, v_new, (cudaStream_t)stream, true, out_mirror);
   }
+  // append + three kernels: the arguments of all four calls are checked before the cache grows,
+  // so that a caller who repairs an argument and retries does not append the token twice
+  if (!three_kernel_args_ok(ctx, q, k_cache, v_cache, proxy_k, scores, workspace) || ((uintptr_t)k_new & 15) ||
+      ((uintptr_t)v_new & 15))
+    return FASA_ERR_INVALID_ARG;
   int32_t st = fasa_kv_append(ctx, k_cache, v_cache, proxy_k, seq_lens, k_new, v_new, 1, stream);
   if (st != FASA_OK) return st;
   return fasa_decode_step(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores, idx,
@@ -285,6 +305,22 @@ extern "C" int32_t fasa_append_decode_step(fasa_ctx_t* ctx, const void* q, const
   bool mirrored;
   return append_decode_step_impl(ctx, q, k_new, v_new, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max,
                                  scores, idx, n_sel, out, lse, workspace, stream, nullptr, &mirrored);
+}
+
+extern "C" int32_t fasa_select_step(fasa_ctx_t* ctx, const void* q, const void* k_new,
+                                    const void* v_new, void* k_cache, void* v_cache, void* proxy_k,
+                                    int32_t* seq_lens, int32_t budget, int32_t n_sel_max,
+                                    float* scores, int32_t* idx, int32_t* n_sel, void* stream) {
+  if (!ctx || !q || !k_cache || !v_cache || !proxy_k || !seq_lens || !idx || !n_sel || budget == 0 ||
+      budget < -1000 || n_sel_max <= 0 || (k_new == nullptr) != (v_new == nullptr))
+    return FASA_ERR_INVALID_ARG;
+  if (!(ctx->use_fused && ctx->fused_step_ok && ctx->fused_cs > 0)) return FASA_ERR_UNSUPPORTED;
+  if (((uintptr_t)proxy_k & 15) || ((uintptr_t)q & 15) || ((uintptr_t)k_cache & 15) || ((uintptr_t)v_cache & 15) ||
+      ((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15) || (scores && ((uintptr_t)scores & 3)) ||
+      !fasa_pages_ready(ctx))
+    return FASA_ERR_INVALID_ARG;
+  return fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores, idx, n_sel,
+                           nullptr, nullptr, k_new, v_new, (cudaStream_t)stream, false);
 }
 
 extern "C" int32_t fasa_stage_bytes(const fasa_ctx_t* ctx, size_t* out_bytes) {
@@ -312,22 +348,36 @@ extern "C" int32_t fasa_decode_step_host(fasa_ctx_t* ctx, const void* q_host,
   char* dq = (char*)dev_stage;
   char* dk = dq + fasa_align_up(q_bytes, 256);
   char* dv = dk + fasa_align_up(kv_bytes, 256);
-  // Pinned (page-locked, mapped) host buffers are read by the kernels in place: the few KB of
-  // a step cross the host link inside the step's only launch instead of in three copies that
-  // each cost more than the transfer.  Anything else is copied to the staging area first.
-  auto mapped = [](const void* hp) -> const void* {
+  // Pinned (page-locked, mapped) host buffers need no copy call: where the step is a single wave
+  // of one launch its kernel reads them in place (the few KB cross the host link inside the
+  // launch); where it is several launches or several waves of CTAs, one small kernel first
+  // brings all three to the staging area, so that no CTA's start waits on the link.  Anything
+  // else is copied to the staging area with cudaMemcpyAsync.  The driver is asked about a
+  // pointer once: a decode loop passes the same buffers every step.
+  auto mapped = [&](int slot, const void* hp) -> void* {
+    if (ctx->host_seen[slot] == hp) return ctx->host_mapped[slot];
     cudaPointerAttributes at;
-    if (cudaPointerGetAttributes(&at, hp) != cudaSuccess) {
+    void* dp = nullptr;
+    if (cudaPointerGetAttributes(&at, hp) == cudaSuccess) {
+      if (at.type == cudaMemoryTypeHost) dp = at.devicePointer;
+    } else {
       cudaGetLastError();
-      return nullptr;
     }
-    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+    ctx->host_seen[slot] = hp;
+    ctx->host_mapped[slot] = dp;
+    return dp;
   };
-  const void* mq = mapped(q_host);
-  const void* mk = mapped(k_new_host);
-  const void* mv = mapped(v_new_host);
-  if (mq && mk && mv && !((uintptr_t)mq & 15) && !((uintptr_t)mk & 15) && !((uintptr_t)mv & 15)) {
+  const void* mq = mapped(0, q_host);
+  const void* mk = mapped(1, k_new_host);
+  const void* mv = mapped(2, v_new_host);
+  const bool all_mapped = mq && mk && mv && !((uintptr_t)mq & 15) && !((uintptr_t)mk & 15) && !((uintptr_t)mv & 15);
+  const bool one_wave_one_launch = ctx->use_fused && ctx->fused_cs > 0 && !fasa_attend_separately(ctx, n_sel_max, workspace) &&
+                                   (long long)c.batch * ctx->n_sets * ctx->fused_cs <= 2ll * ctx->n_sm;
+  if (all_mapped && one_wave_one_launch) {
     dq = (char*)mq; dk = (char*)mk; dv = (char*)mv;
+  } else if (all_mapped) {
+    FASA_CUDA_TRY(ctx, fasa_stage_from_mapped(dq, mq, q_bytes, dk, mk, dv, mv, kv_bytes, s));
+    ctx->launches += 1;
   } else {
     FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
     FASA_CUDA_TRY(ctx, cudaMemcpyAsync(dk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s));
@@ -335,7 +385,7 @@ extern "C" int32_t fasa_decode_step_host(fasa_ctx_t* ctx, const void* q_host,
   }
   // A pinned out_host is written by the step's kernel itself (next to `out`), where the path
   // taken has a single kernel to do it; otherwise `out` is copied back.
-  float* mo = (float*)mapped(out_host);
+  float* mo = (float*)mapped(3, out_host);
   if ((uintptr_t)mo & 3) mo = nullptr;
   bool mirrored = false;
   int32_t st = append_decode_step_impl(ctx, dq, dk, dv, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max,

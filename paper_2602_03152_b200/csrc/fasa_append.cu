@@ -219,3 +219,29 @@ extern "C" int32_t fasa_proxy_build(fasa_ctx_t* ctx, const void* k_cache, void* 
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
 }
+
+// ---- staging of the host-buffer step ---------------------------------------------------------
+namespace {
+// Copies three device-addressable (mapped host) buffers to device memory in one launch, 16 bytes
+// per thread and iteration; sizes are multiples of 16 bytes.
+__global__ void __launch_bounds__(256)
+stage_copy_kernel(uint4* __restrict__ d0, const uint4* __restrict__ s0, int n0, uint4* __restrict__ d1,
+                  const uint4* __restrict__ s1, uint4* __restrict__ d2, const uint4* __restrict__ s2, int n12) {
+  const int total = n0 + 2 * n12;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    if (i < n0) d0[i] = s0[i];
+    else if (i < n0 + n12) d1[i - n0] = s1[i - n0];
+    else d2[i - n0 - n12] = s2[i - n0 - n12];
+  }
+}
+}  // namespace
+
+cudaError_t fasa_stage_from_mapped(void* dq, const void* sq, size_t q_bytes, void* dk, const void* sk, void* dv,
+                                   const void* sv, size_t kv_bytes, cudaStream_t stream) {
+  const int n0 = (int)(q_bytes / 16), n12 = (int)(kv_bytes / 16);
+  const int total = n0 + 2 * n12;
+  const int blocks = total < 256 * 256 ? (total + 255) / 256 : 256;
+  stage_copy_kernel<<<blocks > 0 ? blocks : 1, 256, 0, stream>>>((uint4*)dq, (const uint4*)sq, n0, (uint4*)dk, (const uint4*)sk,
+                                                               (uint4*)dv, (const uint4*)sv, n12);
+  return cudaGetLastError();
+}

@@ -13,10 +13,16 @@
 //     merged by the coalescer).  Logits of a batch of 8 rows are completed with a transposing
 //     xor-shuffle reduction (8 shuffles per head per batch); probabilities travel back to all
 //     lanes through shared memory.  All multiply-adds are packed two-wide fp32 FMAs.
-// decode_attn_merge_kernel then combines the splits of every (sequence, query head).
+// decode_attn_merge_kernel then combines the splits of every (sequence, query head).  Where a
+// unit needs at most 8 splits (selections up to 16384 rows), the splits of a unit form one
+// thread-block cluster instead and merge through distributed shared memory inside the same
+// launch: no partial result touches HBM, no second launch, no workspace.
 #include <mutex>
 
+#include "fasa_cluster_merge.cuh"
 #include "fasa_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -37,6 +43,9 @@ struct AttnParams {
   const int32_t* idx;      // sparse: [units][n_sel_max]
   const int32_t* n_rows;   // sparse: n_sel [units]; dense: seq_lens [batch]
   float* partial;          // [batch][n_q_heads][n_splits][kPartialStride]
+  float* out;              // (cluster form: merged in the same launch)
+  float* out_mirror;       // (cluster form, nullable: a second copy of out, e.g. mapped host memory)
+  float* lse;
   int32_t* status;
   int n_q_heads, n_kv_heads, n_sets, group, max_len, n_sel_max, n_cap, chunk, n_splits;   // a unit = `group` query heads; n_sets units per sequence
   int64_t ksb, ksh, kst, vsb, vsh, vst;
@@ -332,26 +341,37 @@ struct MmaSmem {
 __device__ __forceinline__ void pdl_wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_release_successor() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// cluster_x > 0: the CTAs of a grid row form one thread-block cluster of that size.
 template <typename Kernel, typename... Args>
 cudaError_t launch_after_predecessor(Kernel kernel, dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
-                                     Args... args) {
+                                     int cluster_x, Args... args) {
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (cluster_x > 0) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)cluster_x;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
+  cfg.attrs = attr;
   return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
-template <bool SPARSE, bool PAGED>
+// CLUSTER: the splits of a unit are the CTAs of one cluster (grid.x = cluster size) and merge
+// in the same launch; otherwise each split writes its partial result for the merge kernel.
+template <bool SPARSE, bool PAGED, bool CLUSTER>
 __global__ void __launch_bounds__(kMmaThreads)
 decode_attn_mma_kernel(const AttnParams p) {
+  __shared__ ClusterMergeSmem s_merge;              // (CLUSTER only: written by the peers)
   pdl_wait_for_predecessor();
   pdl_release_successor();
   const int u = blockIdx.y;
@@ -369,8 +389,8 @@ decode_attn_mma_kernel(const AttnParams p) {
     n = clamp_len(p.n_rows[b], p.max_len, p.status);
   }
   const int split = blockIdx.x;
-  const int r0 = split * p.chunk;
-  if (r0 >= n) return;
+  const int r0 = min(n, split * p.chunk);
+  if (!CLUSTER && r0 >= n) return;                  // (in a cluster an empty split still joins the merge)
   const int r1 = min(n, r0 + p.chunk);
 
   const int lane = threadIdx.x & 31;
@@ -541,6 +561,8 @@ decode_attn_mma_kernel(const AttnParams p) {
   }
   __syncthreads();
   const int cch = threadIdx.x;                      // one channel per thread
+  // (CLUSTER: this CTA's partial per head goes to shared memory behind the combine area)
+  float (*s_part)[kMergePartStride] = reinterpret_cast<float (*)[kMergePartStride]>(s_ml + kMmaWarps * 8 * 2);
   for (int gl = 0; gl < p.group; ++gl) {
     float mx = -INFINITY;
 #pragma unroll
@@ -553,13 +575,17 @@ decode_attn_mma_kernel(const AttnParams p) {
       a += wt * s_acc[(w * 8 + gl) * FASA_HEAD_DIM + cch];
       l += wt * s_ml[(w * 8 + gl) * 2 + 1];
     }
-    float* dst = p.partial +
-                 ((su.q0 + gl) * p.n_splits + split) * kPartialStride;
+    float* dst = CLUSTER ? &s_part[gl][0] : p.partial + ((su.q0 + gl) * p.n_splits + split) * kPartialStride;
     dst[2 + cch] = a;
     if (cch == 0) {
       dst[0] = mx;
       dst[1] = l;
     }
+  }
+  if constexpr (CLUSTER) {
+    __syncthreads();
+    cg::cluster_group cluster = cg::this_cluster();
+    cluster_merge_store<kMmaThreads>(cluster, s_part, s_merge, p.group, su.q0, p.out, p.out_mirror, p.lse);
   }
 }
 
@@ -622,10 +648,14 @@ decode_attn_merge_kernel(const float* __restrict__ partial, const int32_t* __res
     lse[bh] = (ns > 0 && l_all > 0.f) ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
 }
 
+// out_mirror (nullable): a second destination of out; *mirrored tells whether it was written
+// (only the form that merges inside the attention launch can do that).
 template <bool SPARSE>
 int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
                     const int32_t* idx, const int32_t* n_rows, int n_upper, int n_sel_max,
-                    float* out, float* lse, void* workspace, cudaStream_t s) {
+                    float* out, float* lse, void* workspace, cudaStream_t s, float* out_mirror = nullptr,
+                    bool* mirrored = nullptr) {
+  if (mirrored) *mirrored = false;
   const fasa_config_t& c = ctx->cfg;
   if (!fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
   // the dense pass treats a KV head with all its query heads as the unit
@@ -634,7 +664,7 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   const fasa_split_plan plan = fasa_plan_splits(ctx, n_upper, c.batch * n_sets);
   AttnParams p;
   p.q = (const uint16_t*)q; p.k = (const uint16_t*)k; p.v = (const uint16_t*)v;
-  p.idx = idx; p.n_rows = n_rows; p.partial = (float*)workspace; p.status = ctx->d_status;
+  p.idx = idx; p.n_rows = n_rows; p.partial = (float*)workspace; p.out = nullptr; p.out_mirror = nullptr; p.lse = nullptr; p.status = ctx->d_status;
   p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.n_sets = n_sets; p.group = G;
   p.max_len = c.max_len; p.n_sel_max = n_sel_max; p.n_cap = n_upper; p.chunk = plan.chunk; p.n_splits = plan.n_splits;
   p.ksb = c.k_stride_b; p.ksh = c.k_stride_h; p.kst = c.k_stride_t;
@@ -643,13 +673,30 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
   dim3 grid((unsigned)plan.n_splits, (unsigned)(c.batch * n_sets));
   if (ctx->use_fused) {   // default: the tensor-core kernel (mode 0 keeps the scalar one)
-    static_assert(sizeof(MmaSmem) >= (size_t)kMmaWarps * 8 * (FASA_HEAD_DIM + 2) * sizeof(float), "combine area");
-    auto fn = c.page_size > 0 ? decode_attn_mma_kernel<SPARSE, true> : decode_attn_mma_kernel<SPARSE, false>;
+    static_assert(sizeof(MmaSmem) >= ((size_t)kMmaWarps * 8 * (FASA_HEAD_DIM + 2) + 8 * kMergePartStride) * sizeof(float),
+                  "combine area");
+    const int max_smem = (int)(sizeof(MmaSmem) + 2080 * sizeof(int32_t));
+    // One launch where the splits of a unit fit a portable cluster: the split count becomes a
+    // power of two <= 8 (the nearest to the planned one) and the cluster merges by itself.
+    int cs = 1;
+    while (cs < 8 && cs * 3 < plan.n_splits * 2) cs *= 2;          // nearest power of two, ties up
+    int cchunk = ((n_upper + cs - 1) / cs + 31) / 32 * 32;
+    while (cs < 8 && cchunk > 2048) { cs *= 2; cchunk = ((n_upper + cs - 1) / cs + 31) / 32 * 32; }
+    if (cchunk <= 2048) {
+      p.chunk = cchunk; p.n_splits = cs; p.out = out; p.out_mirror = out_mirror; p.lse = lse;
+      if (mirrored) *mirrored = out_mirror != nullptr;
+      auto fn = c.page_size > 0 ? decode_attn_mma_kernel<SPARSE, true, true> : decode_attn_mma_kernel<SPARSE, false, true>;
+      const size_t smem = sizeof(MmaSmem) + (SPARSE ? (size_t)cchunk * sizeof(int32_t) : 0);
+      FASA_CUDA_TRY(ctx, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+      FASA_CUDA_TRY(ctx, launch_after_predecessor(fn, dim3((unsigned)cs, grid.y), dim3(kMmaThreads), smem, s, cs, p));
+      FASA_LAUNCH_CHECK(ctx);
+      return FASA_OK;
+    }
+    auto fn = c.page_size > 0 ? decode_attn_mma_kernel<SPARSE, true, false> : decode_attn_mma_kernel<SPARSE, false, false>;
     // (+ the slice of the index list: chunk <= 2048 rows)
     const size_t smem = sizeof(MmaSmem) + (SPARSE ? (size_t)plan.chunk * sizeof(int32_t) : 0);
-    FASA_CUDA_TRY(ctx, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)(sizeof(MmaSmem) + 2080 * sizeof(int32_t))));
-    FASA_CUDA_TRY(ctx, launch_after_predecessor(fn, grid, dim3(kMmaThreads), smem, s, p));
+    FASA_CUDA_TRY(ctx, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
+    FASA_CUDA_TRY(ctx, launch_after_predecessor(fn, grid, dim3(kMmaThreads), smem, s, 0, p));
   } else if (G == 1) decode_attn_kernel<1, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   else if (G == 2) decode_attn_kernel<2, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   else if (G == 3) decode_attn_kernel<3, 1, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
@@ -659,7 +706,7 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   FASA_LAUNCH_CHECK(ctx);
   FASA_CUDA_TRY(ctx, launch_after_predecessor(
       decode_attn_merge_kernel<SPARSE>, dim3((unsigned)(c.batch * c.n_q_heads)), dim3(FASA_HEAD_DIM * kMergeWays),
-      (size_t)0, s, (const float*)workspace, n_rows, out, lse, ctx->d_status, (int)c.n_q_heads, (int)n_sets,
+      (size_t)0, s, 0, (const float*)workspace, n_rows, out, lse, ctx->d_status, (int)c.n_q_heads, (int)n_sets,
       (int)G, (int)c.max_len, (int)n_upper, (int)plan.chunk, (int)plan.n_splits));
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
@@ -680,6 +727,15 @@ extern "C" int32_t fasa_sparse_decode_attn(fasa_ctx_t* ctx, const void* q, const
   const int n_upper = n_sel_max < ctx->cfg.max_len ? n_sel_max : ctx->cfg.max_len;
   return launch_attn<true>(ctx, q, k_cache, v_cache, idx, n_sel, n_upper, n_sel_max, out, lse,
                            workspace, (cudaStream_t)stream);
+}
+
+// fasa_sparse_decode_attn with a second destination for the output (the host-buffer step).
+int32_t fasa_sparse_attn_mirrored(fasa_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                                  const int32_t* idx, const int32_t* n_sel, int32_t n_sel_max, float* out,
+                                  float* lse, void* workspace, cudaStream_t stream, float* out_mirror, bool* mirrored) {
+  const int n_upper = n_sel_max < ctx->cfg.max_len ? n_sel_max : ctx->cfg.max_len;
+  return launch_attn<true>(ctx, q, k_cache, v_cache, idx, n_sel, n_upper, n_sel_max, out, lse, workspace, stream,
+                           out_mirror, mirrored);
 }
 
 extern "C" int32_t fasa_full_decode_attn(fasa_ctx_t* ctx, const void* q, const void* k_cache,

@@ -32,6 +32,10 @@ struct fasa_ctx {
   int fused_step_ok;      // the one-launch step supports this configuration
   size_t fused_smem;      // its dynamic shared memory
   int use_fused;          // fasa_decode_step takes the one-launch kernel when it is available
+  // host-buffer step: the last host pointers seen and what the device can use in their place
+  // (null: not page-locked + mapped), so that a decode loop with fixed buffers asks the driver once
+  const void* host_seen[4];
+  void* host_mapped[4];
   long long launches;     // kernels launched through this context
   char cuda_err[256];
 };
@@ -86,6 +90,13 @@ static inline bool fasa_attend_separately(const fasa_ctx* ctx, int n_sel_max, co
   return workspace != nullptr &&
          (rows >= 2048 || (several_waves && rows >= 256) || (rows >= 512 && all_rows >= 24576));
 }
+
+cudaError_t fasa_stage_from_mapped(void* dq, const void* sq, size_t q_bytes, void* dk, const void* sk, void* dv,
+                                   const void* sv, size_t kv_bytes, cudaStream_t stream);
+
+int32_t fasa_sparse_attn_mirrored(fasa_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                                  const int32_t* idx, const int32_t* n_sel, int32_t n_sel_max, float* out,
+                                  float* lse, void* workspace, cudaStream_t stream, float* out_mirror, bool* mirrored);
 
 int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
                                int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,

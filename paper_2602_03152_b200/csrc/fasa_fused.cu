@@ -36,6 +36,7 @@
 // selection, after which no CTA touches a peer's shared memory.  No thread spins on anything.
 #include <cooperative_groups.h>
 
+#include "fasa_cluster_merge.cuh"
 #include "fasa_common.cuh"
 #include "fasa_score_core.cuh"
 
@@ -47,10 +48,10 @@ constexpr int kFT = 512;               // threads per CTA; two CTAs share an SM 
                                        // what one SM can pull from HBM grows with its resident warps
 constexpr int kFW = kFT / 32;          // warps per CTA
 constexpr int kFBins = 2048;           // bins of the widest radix pass
-constexpr int kPartStride = FASA_HEAD_DIM + 2;   // m, l, acc[128]
+constexpr int kPartStride = kMergePartStride - 2;   // m, l, acc[128] (+ 2 words of padding in shared memory)
 constexpr int kCapMax = 22528;         // keys a CTA can hold (88 KB of shared memory)
 constexpr int kCapPair = 16384;        // ... and still leave room for a second CTA on the SM
-constexpr int kMaxCs = 16;             // CTAs per cluster at most
+constexpr int kMaxCs = kMergeMaxCs;     // CTAs per cluster at most
 constexpr int kGroups = kFBins / 32;   // 32-bin groups of the widest radix pass
 constexpr int kCandCap = 4096;         // keys of one bin that the cluster finishes locally
 constexpr int kFinBits = 7;            // bits per block-level pass of that local finish
@@ -193,8 +194,7 @@ fused_decode_kernel(const FusedParams p) {
   __shared__ __align__(16) float s_q[GP][FASA_HEAD_DIM];
   __shared__ __align__(16) uint16_t s_qraw[GP][FASA_HEAD_DIM];   // the unit's query rows as stored (scoring operand)
   __shared__ int16_t s_chan[8 * FASA_MAX_DOM / 4];               // the head's channel table
-  __shared__ float s_racc[FASA_MAX_GROUP * FASA_HEAD_DIM + 16];   // pushed by the cluster: accumulators of this CTA's outputs
-  __shared__ float s_rml[kMaxCs][FASA_MAX_GROUP][2];              // ... and every CTA's (m, l) per head
+  __shared__ ClusterMergeSmem s_merge;                            // pushed by the cluster: the partial results this CTA finishes
 
   // ---- slices -------------------------------------------------------------------------
   // Append-then-step: one thread reads the length for the whole CTA, so that the CTA's arrival
@@ -916,52 +916,8 @@ fused_decode_kernel(const FusedParams p) {
     }
     __syncthreads();                                           // s_acc / s_m are reused by the next pass
   }
-  // ---- 5b. merge across the cluster ------------------------------------------------------------
-  // CTA r finishes outputs [r * per_o, (r + 1) * per_o).  Every CTA PUSHES its partial values
-  // for those outputs into r's shared memory; after the barrier r combines from local memory
-  // only, so no CTA reads a peer afterwards and none has to wait for the others to leave.
-  {
-    const int n_out = p.group * FASA_HEAD_DIM;
-    const int per_o = (n_out + cs - 1) / cs;
-    for (int o = tid; o < n_out; o += kFT) {
-      const int r = o / per_o, ol = o % per_o;
-      float* dst = cluster.map_shared_rank(&s_racc[0], r);
-      dst[crank * per_o + ol] = s_part[o / FASA_HEAD_DIM][2 + o % FASA_HEAD_DIM];
-    }
-    for (int i = tid; i < cs * GP; i += kFT) {
-      const int r = i / GP, g = i % GP;
-      float* dst = cluster.map_shared_rank(&s_rml[0][0][0], r);
-      dst[(crank * GP + g) * 2 + 0] = s_part[g][0];
-      dst[(crank * GP + g) * 2 + 1] = s_part[g][1];
-    }
-    cluster.sync();   // the merge barrier: every CTA's partial results have arrived
-    const int opp = kFT / cs;                // outputs per pass (cs is a power of two <= 16)
-    const int r = tid % cs, tl = tid / cs;
-    for (int t0 = 0; t0 < per_o; t0 += opp) {   // uniform trip count
-      const int t = t0 + tl;
-      const int o = crank * per_o + t;
-      const bool ok = t < per_o && o < n_out;
-      const int g = ok ? o / FASA_HEAD_DIM : 0;
-      const float ms = s_rml[r][g][0], ls = s_rml[r][g][1];
-      const float as = ok ? s_racc[r * per_o + t] : 0.f;
-      float mx = ms;
-      for (int off = cs >> 1; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-      const float wt = ms == -INFINITY ? 0.f : exp2f(ms - mx);
-      float av = wt * as, l = wt * ls;
-      for (int off = cs >> 1; off > 0; off >>= 1) {
-        av += __shfl_xor_sync(0xffffffffu, av, off);
-        l += __shfl_xor_sync(0xffffffffu, l, off);
-      }
-      if (ok && r == 0) {
-        const int c = o % FASA_HEAD_DIM;
-        const int64_t hq = su.q0 + g;
-        const float ov = l > 0.f ? av / l : 0.f;
-        p.out[hq * FASA_HEAD_DIM + c] = ov;
-        if (p.out_mirror) p.out_mirror[hq * FASA_HEAD_DIM + c] = ov;
-        if (p.lse && c == 0) p.lse[hq] = l > 0.f ? (mx + log2f(l)) * 0.6931471805599453f : -INFINITY;
-      }
-    }
-  }
+  // ---- 5b. merge across the cluster (one barrier; see fasa_cluster_merge.cuh) -------------------
+  cluster_merge_store<kFT>(cluster, s_part, s_merge, p.group, su.q0, p.out, p.out_mirror, p.lse);
 }
 
 size_t fused_smem_bytes(int cap) { return (size_t)fused_smem_layout(cap).total; }

@@ -267,9 +267,41 @@ def test_append_decode_step_equals_append_then_step(mode):
                       n_sel=b.n_sel.cpu().numpy(), out=b.out.cpu().numpy(), what="append+step", **b.oracle_kwargs())
 
 
+def test_select_step_gives_the_index_sets_of_the_separate_calls():
+    w = C["c2"].replace(batch=3, max_len=9000, len_lo=4000, len_hi=8999, budget=300, n_sink=2, n_recent=9)
+    r = Run(w)
+    r.build_proxy()
+    r.step()                                                   # fasa_fc_score + fasa_topk + attention
+    ref = (r.scores.clone(), r.idx.clone(), r.n_sel.clone())
+    r.reset_outputs()
+    n0 = r.fasa.launch_count()
+    r.fasa.select_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel)
+    torch.cuda.synchronize()
+    assert r.fasa.launch_count() == n0 + 1
+    assert torch.equal(r.scores, ref[0]) and torch.equal(r.idx, ref[1]) and torch.equal(r.n_sel, ref[2])
+    assert torch.all(r.out == SENTINEL)                        # no attention ran
+    # appending form: the cache's own next row appended again, lengths grow by one
+    lens0 = r.seq_lens.clone()
+    bi = torch.arange(w.batch, device="cuda")
+    k_new = r.k[bi, :, lens0.long()].unsqueeze(2).contiguous()
+    v_new = r.v[bi, :, lens0.long()].unsqueeze(2).contiguous()
+    r.fasa.select_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, None, r.idx, r.n_sel, k_new, v_new)
+    torch.cuda.synchronize()
+    assert torch.equal(r.seq_lens, lens0 + 1)
+    idx_a, n_a = r.idx.clone(), r.n_sel.clone()
+    r.fasa.fc_score(r.q, r.proxy, r.seq_lens, r.scores)
+    r.fasa.topk(r.scores, r.seq_lens, w.budget, r.idx, r.n_sel, r.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(r.idx, idx_a) and torch.equal(r.n_sel, n_a)
+    assert r.fasa.device_status() == 0
+    with pytest.raises(binding.FasaError):                     # k_new without v_new
+        r.fasa.select_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, None, r.idx, r.n_sel, k_new, None)
+
+
 def test_large_selection_is_attended_by_the_split_k_kernel():
     # n_sel_max * ceil(G / 4) >= 2048 and a workspace: cluster kernel without its attention
-    # phase, then the split-K tensor-core attention (3 launches); same results as one launch
+    # phase, then the split-K tensor-core attention whose splits merge inside their own cluster
+    # (2 launches); same results as one launch
     w = C["c3"].replace(batch=2, max_len=6000, len_lo=5000, len_hi=6000, budget=-300)
     r = Run(w)
     r.build_proxy()
@@ -279,7 +311,7 @@ def test_large_selection_is_attended_by_the_split_k_kernel():
     n0 = r.fasa.launch_count()
     r.fasa.decode_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel, r.out, r.ws, r.lse)
     torch.cuda.synchronize()
-    assert r.fasa.launch_count() - n0 == 3
+    assert r.fasa.launch_count() - n0 == 2
     for x, y in zip(one[:3], (r.scores, r.idx, r.n_sel)):
         assert torch.equal(x, y)
     assert float((one[3] - r.out).abs().max()) <= 1e-4 and float((one[4] - r.lse).abs().max()) <= 1e-4
@@ -361,7 +393,7 @@ def test_index_sets_per_query_head_large_selection_and_static_scratch():
     n0 = r.fasa.launch_count()
     r.fasa.decode_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, r.scores, r.idx, r.n_sel, r.out, r.ws, r.lse)
     torch.cuda.synchronize()
-    assert r.fasa.launch_count() - n0 == 3
+    assert r.fasa.launch_count() - n0 == 2
     h = r.host()
     parity.check_step(h["q"], h["k"], h["v"], h["seq_lens"], h["dom"], scores=h["scores"], idx=h["idx"],
                       n_sel=h["n_sel"], out=h["out"], what="split attention, sets per head", **r.oracle_kwargs())
@@ -405,6 +437,35 @@ def test_calibration_counts_match_the_oracle(cfg, kw, top_k):
     assert np.array_equal(used, u_or) and used.min() >= 1
     assert np.array_equal(counts, c_or)
     assert counts.max() <= used.max() * top_k
+
+
+def test_calibration_counts_against_the_fp64_statement_of_eq4():
+    # The bit-exact test above decides set membership in binary32, as the kernel does.  Against the
+    # plain fp64 statement of Eq. 4 the count of a (query head, FC) pair may differ only through
+    # positions whose score lies within 1e-3 (relative) of the K-th score of the full-score list or
+    # of that FC's list: those are the only memberships a rounding can flip.
+    w = C["c1"].replace(batch=1, n_q_heads=8, n_kv_heads=2, max_len=3000, len_lo=3000, len_hi=3000)
+    t = synth.make_inputs(w, "cpu")
+    top_k = 100
+    counts, used, _, _ = _calib(w, t, top_k)
+    q64, k64 = t["q"].double().numpy(), t["k"].double().numpy()
+
+    def band(s):
+        o = np.sort(s)[::-1]
+        tol = 1e-3 * max(abs(o[top_k - 1]), abs(o[top_k]))
+        return int(np.sum(np.abs(s - o[top_k - 1]) <= tol)) - 1          # the K-th position itself cannot flip alone
+
+    worst = 0
+    for hq in range(w.n_q_heads):
+        K = k64[0, hq // w.group, :3000]
+        c64 = O.ca_counts(q64[0, hq], K, top_k, w.pairing, f32=False)
+        a = O.fc_partial_logits(q64[0, hq], K, w.pairing)                 # [64][L]
+        b_full = band(a.sum(axis=0))
+        for i in range(64):
+            slack = b_full + band(a[i])
+            assert abs(int(counts[hq, i]) - int(c64[i])) <= slack, (hq, i, counts[hq, i], c64[i], slack)
+            worst = max(worst, abs(int(counts[hq, i]) - int(c64[i])))
+    assert used.tolist() == [1] * w.n_q_heads and worst <= 3
 
 
 def test_calibration_accumulates_and_skips_short_sequences():
@@ -470,7 +531,7 @@ def test_decode_loop_replays_from_a_cuda_graph():
     n0 = graphed.fasa.launch_count()
     with torch.cuda.graph(g):
         run(graphed, outs_g)
-    assert graphed.fasa.launch_count() - n0 == 3 + 2
+    assert graphed.fasa.launch_count() - n0 == 3 + 1          # (the dense pass of this size merges inside its clusters)
     for rounds in range(2):
         g.replay()
         run(eager, outs_e)
@@ -1018,7 +1079,7 @@ def test_config4_point_full_length_sampled_units():
                           what="c4", **r.oracle_kwargs())
 
 
-def _full_size_sampled(w, units, budget=None, append=False):
+def _full_size_sampled(w, units, budget=None, append=False, keep=None):
     """A benchmark workload at its full size, inputs drawn on the device, run as bench.py runs
     it (one fasa_append_decode_step / fasa_decode_step call) and checked against the oracle on
     a few (batch, KV head) units whose K/V are copied to the host."""
@@ -1061,6 +1122,13 @@ def _full_size_sampled(w, units, budget=None, append=False):
                                 idx=idx[b:b + 1, h:h + 1].cpu().numpy(), n_sel=n_sel[b:b + 1, h:h + 1].cpu().numpy(),
                                 out=out[b:b + 1, h * G:(h + 1) * G].cpu().numpy(), what=f"{w.name} unit ({b},{h})")
         assert rep["units"] == 1
+        if keep is not None:
+            keep.setdefault("q", {})[(b, h)] = q[b, h * G:(h + 1) * G].cpu().double().numpy()
+            keep.setdefault("k", {})[(b, h)] = k[b, h, :L].cpu().double().numpy()
+            keep.setdefault("idx", {})[(b, h)] = idx[b, h].cpu().numpy()
+            keep.setdefault("n_sel", {})[(b, h)] = int(n_sel[b, h])
+    if keep is not None:
+        keep.update(t=t, proxy=proxy, idx_dev=idx, n_sel_dev=n_sel, out_dev=out)
     return f
 
 
@@ -1070,11 +1138,84 @@ def test_config2_full_size_sampled_units():
     assert f.step_cluster_size() == 8
 
 
-def test_config3_full_size_sampled_units_with_append():
-    # long-CoT shape at its last step: batch 32, G = 7, 16384 rows, budget 18.9 %; the selection is
-    # large, so the step is the cluster kernel without attention + the split-K tensor-core kernel
-    w = C["c3"].replace(len_lo=16384, len_hi=16384)
+@pytest.mark.parametrize("layer", [0, 1])
+@pytest.mark.parametrize("step", [1, 512, 4096, 15360])
+def test_config3_full_size_sampled_units_with_append(step, layer):
+    # long-CoT shape: batch 32, G = 7, prompt 1024 + `step` generated tokens, budget 18.9 % of the
+    # current length; two layers = two contexts with their own dominant-FC tables and caches.  Small
+    # selections are attended inside the cluster kernel, large ones by the split-K kernel.
+    L = 1024 + step
+    w = C["c3"].replace(len_lo=L, len_hi=L, index=C["c3"].index + 1000 * layer)
     _full_size_sampled(w, [(0, 0), (31, 3), (13, 2)], append=True)
+
+
+@pytest.mark.parametrize("budget", [256, 4096])
+def test_config4_full_size_in_the_launch_shape_of_the_benchmark(budget):
+    # batch 8 x 8 KV heads = 64 units, clusters of 4 with 16384 keys per CTA, the appending form:
+    # budget 256 is one launch, budget 4096 the select-only cluster kernel + the split-K kernel
+    f = _full_size_sampled(C["c4"].replace(budget=budget), [(0, 0), (3, 5), (7, 7)], append=True)
+    assert f.step_cluster_size() == 4
+
+
+@pytest.mark.parametrize("F,budget", [(4, 64), (64, 4096)])
+def test_config4_sweep_corners_at_full_length(F, budget):
+    # the corners of the budget x dominant-FC grid at the full 65536 context; with all 64 FCs the
+    # score is the full logit, so the selection must also be the dense top-k (the "Oracle"
+    # baseline of Sec. 5.1), taken here from a plain fp64 matrix product
+    w = C["c4"].replace(n_dom=F, budget=budget)
+    units = [(1, 2), (6, 0)]
+    got = {}
+    f = _full_size_sampled(w, units, keep=got)
+    if F == 64:
+        G = w.group
+        for (b, h) in units:
+            full = got["k"][(b, h)] @ got["q"][(b, h)].sum(axis=0)                  # sum over the group of q_g . k_j
+            n = int(got["n_sel"][(b, h)])
+            assert n == budget
+            parity.check_selection(got["idx"][(b, h)][:n], full, 65536, budget, 0, 0, f"dense top-k ({b},{h})")
+
+
+def test_config4_full_size_paged_and_host_resident_caches():
+    # the benchmark's c4 point (budget 256) once more with (a) 64-token pages in random order and
+    # (b) K and V in page-locked host memory (FASA-M): both must give the bits of the contiguous,
+    # device-resident run, which is checked against the oracle on sampled units
+    w = C["c4"]
+    got = {}
+    f = _full_size_sampled(w, [(2, 3), (5, 6)], keep=got)
+    t = got["t"]
+    B, Hq, Hkv, Lm, P = w.batch, w.n_q_heads, w.n_kv_heads, w.max_len, 64
+    n_sel_max = w.n_sel_max()
+
+    def fresh():
+        return (torch.full((B, Hkv, n_sel_max), -7, dtype=torch.int32, device="cuda"), torch.full((B, Hkv), -7, dtype=torch.int32, device="cuda"),
+                torch.full((B, Hq, 128), SENTINEL, dtype=torch.float32, device="cuda"))
+
+    # (a) paged
+    pps = Lm // P
+    n_pages = B * pps
+    table = torch.randperm(n_pages, generator=torch.Generator().manual_seed(3)).to(torch.int32).view(B, pps).cuda()
+    fp = binding.Fasa(B, Hq, Hkv, Lm, t["dom"], rope_pairing=w.pairing, group_reduce=w.group_reduce, n_sink=w.n_sink,
+                      n_recent=w.n_recent, page_size=P, n_pages=n_pages)
+    fp.set_block_table(table)
+    kp, vp = fp.alloc_paged_cache(), fp.alloc_paged_cache()
+    for src, dst in ((t["k"], kp), (t["v"], vp)):
+        dst[table.long().view(-1)] = src.view(B, Hkv, pps, P, 128).permute(0, 2, 1, 3, 4).reshape(n_pages, Hkv, P, 128)
+    proxy = fp.alloc_proxy()
+    fp.proxy_build(kp, proxy, t["seq_lens"])
+    idx, n_sel, out = fresh()
+    fp.decode_step(t["q"], kp, vp, proxy, t["seq_lens"], w.budget, None, idx, n_sel, out, None)
+    torch.cuda.synchronize()
+    assert fp.device_status() == 0
+    assert torch.equal(idx, got["idx_dev"]) and torch.equal(n_sel, got["n_sel_dev"]) and torch.equal(out, got["out_dev"])
+    del kp, vp, proxy, fp
+    # (b) host-resident K and V, the proxy on the GPU
+    kh, vh = f.alloc_host_cache(), f.alloc_host_cache()
+    kh.copy_(t["k"]); vh.copy_(t["v"])
+    idx, n_sel, out = fresh()
+    f.decode_step(t["q"], kh, vh, got["proxy"], t["seq_lens"], w.budget, None, idx, n_sel, out, None)
+    torch.cuda.synchronize()
+    assert f.device_status() == 0
+    assert torch.equal(idx, got["idx_dev"]) and torch.equal(n_sel, got["n_sel_dev"]) and torch.equal(out, got["out_dev"])
 
 
 def test_contexts_of_different_sizes_coexist():

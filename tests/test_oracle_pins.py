@@ -494,9 +494,29 @@ def test_calibration_recovers_planted_dominant_fcs():
     assert mean[:, planted].min() > 1.5 * np.delete(mean, planted, axis=1).max()
 
 
-def test_byte_model_fraction():
-    # Sec. 4.4: fraction of KV bytes loaded = N_tip/d + N_fac/t.
-    for F, k, L in ((16, 256, 32768), (8, 256, 4096), (64, 4096, 65536)):
-        fasa = L * 4 * F + k * 512
-        dense = L * 512
-        assert math.isclose(fasa / dense, F / 128 + k / L, rel_tol=1e-15)
+def test_byte_model_of_the_benchmark():
+    # bench.step_bytes is the denominator of every reported roofline fraction.  Sec. 4.4: the
+    # fraction of the KV cache that a step loads is N_tip/d + N_fac/t (N_tip counted in FCs of
+    # two channels each, d = 128 channels); q and out are the only other terms.  Checked
+    # against that closed form and against the configuration's byte counts worked by hand.
+    import bench
+    from paper_2602_03152_b200 import synth
+    for name, lens, n_sel_unit in (("c1", [32768], 324), ("c4", [65536] * 8, 256), ("c2", [65536 + 977 * b for b in range(16)], 1024),
+                                   ("c3", [16384] * 32, 3097)):
+        w = synth.CONFIGS[name]
+        units = w.batch * w.n_kv_heads
+        by = bench.step_bytes(w, lens, n_sel_unit * units)
+        qo = w.batch * w.n_q_heads * 128 * (2 + 4)                  # bf16 query in, fp32 output back
+        assert by["qo"] == qo and by["fasa"] == by["proxy"] + by["gathered"] + qo
+        t_mean = sum(lens) / len(lens)
+        frac = (by["fasa"] - qo) / (by["dense"] - qo)
+        assert math.isclose(frac, w.n_dom / 128 + n_sel_unit / t_mean, rel_tol=1e-12), name
+        assert by["dense"] - qo == sum(lens) * w.n_kv_heads * 2 * 128 * 2       # every K and V row, bf16
+    # configuration 1 by hand: 8 units x 32768 tokens x 16 FCs x 4 bytes of proxy, 8 x 324 rows of 512 bytes, q + out
+    by = bench.step_bytes(synth.CONFIGS["c1"], [32768], 8 * 324)
+    assert (by["proxy"], by["gathered"], by["qo"], by["fasa"]) == (16777216, 1327104, 24576, 18128896)
+    assert by["dense"] == 134217728 + 24576
+    # index sets per query head gather more rows but stream the proxy once per KV head
+    w1 = synth.CONFIGS["c4"].replace(sel_heads=1)
+    b1 = bench.step_bytes(w1, [65536] * 8, 256 * 8 * 32)
+    assert b1["proxy"] == bench.step_bytes(synth.CONFIGS["c4"], [65536] * 8, 0)["proxy"] and b1["gathered"] == 256 * 256 * 512

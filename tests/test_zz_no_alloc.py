@@ -32,11 +32,21 @@ def test_static_scratch_variant_matches_workspace_variant_twice():
             ref_out, ref_lse = r.out.clone(), r.lse.clone()
         out = torch.full_like(r.out, SENTINEL)
         lse = torch.full_like(r.lse, SENTINEL)
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
         r.fasa.sparse_decode_attn_static(r.q, r.k, r.v, r.idx, r.n_sel, out, lse)
         torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
         assert r.fasa.device_status() == 0
+        if call == 1:
+            # (the first call on a device may load the library's module, which is where the
+            # array lives; from the second call on nothing on the device may change size)
+            assert free_after == free_before
         assert float((out - ref_out).abs().max()) <= ATTN_ABS
         assert float((lse - ref_lse).abs().max()) <= ATTN_ABS
+        # both variants run the same kernels with the same split plan: anything of the first
+        # call's partials leaking into the second would show as a difference in the bits
+        assert torch.equal(out, ref_out) and torch.equal(lse, ref_lse)
 
 
 def test_static_scratch_variant_rejects_what_does_not_fit():
