@@ -251,3 +251,31 @@ def decode_bf16(q_bits, K_bits, V_bits, seq_lens, dom, *, pairing=0, group_reduc
         raise ValueError("sel_heads must divide the group")
     return {"scores": scores, "idx": idx, "n_sel": n_sel, "band": band, "out": out, "lse": lse,
             "dense_out": dout, "dense_lse": dlse, "threads": int(used)}
+
+
+def decode_batched_bf16(q_bits, K_bits, V_bits, seq_lens, dom, **kw):
+    """A block of T query tokens per sequence (speculative / multi-token decoding).
+
+    The method defines token importance prediction and focused attention for ONE query q_t
+    (Sec. 4.1-4.2: S_t, T_t and Eq. 6-7 all carry the index t).  A block of T queries is
+    therefore T decode steps, nothing else: query t of the block (0 <= t < T) is the query of
+    the cache position L - T + t, where L = seq_lens[b] counts the rows cached INCLUDING the
+    block's own T keys; it sees the rows at positions <= its own (rows j < L - (T - 1 - t)),
+    and has its own scores, its own index set and its own output.  Written out as exactly that:
+    T calls of decode_bf16 on the shortened caches.
+
+    q_bits [B,T,Hq,d]; K_bits, V_bits, seq_lens, dom and the keyword arguments as decode_bf16.
+    Returns the dict of decode_bf16 with a token axis after the batch axis ([B,T,...]).
+    """
+    q_bits = np.ascontiguousarray(q_bits, dtype=np.uint16)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    B, T = q_bits.shape[:2]
+    steps = []
+    for t in range(T):
+        lens_t = np.maximum(seq_lens - (T - 1 - t), 0).astype(np.int32)
+        steps.append(decode_bf16(q_bits[:, t], K_bits, V_bits, lens_t, dom, **kw))
+    out = {"threads": steps[0]["threads"]}
+    for key in ("scores", "idx", "n_sel", "band", "out", "lse", "dense_out", "dense_lse"):
+        out[key] = None if steps[0][key] is None else np.stack([s_[key] for s_ in steps], axis=1)
+    return out
+

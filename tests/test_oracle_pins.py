@@ -494,6 +494,83 @@ def test_calibration_recovers_planted_dominant_fcs():
     assert mean[:, planted].min() > 1.5 * np.delete(mean, planted, axis=1).max()
 
 
+def _batched_case(seed, B=2, T=4, Hq=4, Hkv=2, L=90, F=6, budget=11, n_sink=1, n_recent=3):
+    rng = np.random.default_rng(seed)
+    q = torch.from_numpy(rng.standard_normal((B, T, Hq, 128))).to(torch.bfloat16)
+    k = torch.from_numpy(rng.standard_normal((B, Hkv, L, 128))).to(torch.bfloat16)
+    v = torch.from_numpy(rng.standard_normal((B, Hkv, L, 128))).to(torch.bfloat16)
+    lens = np.array([L, L - 17][:B], dtype=np.int32)
+    dom = np.stack([np.sort(rng.choice(64, F, replace=False)) for _ in range(Hkv)]).astype(np.int32)
+    return q, k, v, lens, dom, dict(budget=budget, n_sink=n_sink, n_recent=n_recent)
+
+
+def test_batched_queries_with_one_token_are_the_decode_step():
+    from paper_2602_03152_b200 import synth
+    q, k, v, lens, dom, kw = _batched_case(3, T=1)
+    a = O.decode_batched_bf16(synth.bf16_bits(q), synth.bf16_bits(k), synth.bf16_bits(v), lens, dom, **kw)
+    b = O.decode_bf16(synth.bf16_bits(q[:, 0]), synth.bf16_bits(k), synth.bf16_bits(v), lens, dom, **kw)
+    for key in ("scores", "idx", "n_sel", "out", "lse", "dense_out"):
+        assert np.array_equal(a[key][:, 0], b[key], equal_nan=True), key
+
+
+def test_batched_queries_against_the_masked_dense_formulation():
+    # The same block computed the way a dense framework would: ONE matrix product of all T queries
+    # against the dominant channels of the keys, a causal mask over the block (the query whose own
+    # key sits at cache row L - T + t sees rows <= that one), library top-k on the masked scores,
+    # then ONE masked scaled-dot-product attention over all rows with a boolean mask holding the T
+    # index sets.  Sink and recent positions are relative to each query's own visible range.
+    from paper_2602_03152_b200 import synth
+    q, k, v, lens, dom, kw = _batched_case(4)
+    B, T, Hq = q.shape[:3]
+    Hkv, G = k.shape[1], q.shape[2] // k.shape[1]
+    r = O.decode_batched_bf16(synth.bf16_bits(q), synth.bf16_bits(k), synth.bf16_bits(v), lens, dom, **kw)
+    q64, k64, v64 = q.double(), k.double(), v.double()
+    for b in range(B):
+        L = int(lens[b])
+        for h in range(Hkv):
+            ch = np.concatenate([dom[h], dom[h] + 64])
+            qsum = q64[b, :, h * G:(h + 1) * G].sum(dim=1)                         # [T,128]: sum over the group
+            S = qsum[:, ch] @ k64[b, h, :L][:, ch].T                               # [T,L]
+            own = torch.arange(T) + (L - T)                                         # cache row of each query's own key
+            visible = torch.arange(L)[None, :] <= own[:, None]
+            mask = torch.zeros((T, L), dtype=torch.bool)
+            for t in range(T):
+                Lt = int(own[t]) + 1
+                assert np.allclose(r["scores"][b, t, h, :Lt], S[t, :Lt].numpy(), rtol=1e-12, atol=1e-12)
+                forced = torch.zeros(L, dtype=torch.bool)
+                forced[:kw["n_sink"]] = True
+                forced[Lt - kw["n_recent"]:Lt] = True
+                cand = S[t].clone()
+                cand[~visible[t] | forced] = -float("inf")
+                top = torch.topk(cand, kw["budget"]).indices
+                sel = torch.sort(torch.cat([torch.nonzero(forced).flatten(), top])).values
+                n = int(r["n_sel"][b, t, h])
+                assert n == kw["budget"] + kw["n_sink"] + kw["n_recent"]
+                assert np.array_equal(r["idx"][b, t, h, :n], sel.numpy()), (b, h, t)
+                mask[t, sel] = True
+            for g in range(G):
+                hq = h * G + g
+                o = torch.nn.functional.scaled_dot_product_attention(q64[b, :, hq][None], k64[b, h, :L][None], v64[b, h, :L][None],
+                                                                     attn_mask=mask[None])[0]
+                assert np.allclose(r["out"][b, :, hq], o.numpy(), rtol=1e-11, atol=1e-12)
+            # the last query of the block is the ordinary decode step on the whole cache
+    last = O.decode_bf16(synth.bf16_bits(q[:, -1]), synth.bf16_bits(k), synth.bf16_bits(v), lens, dom, **kw)
+    assert np.array_equal(r["idx"][:, -1], last["idx"]) and np.array_equal(r["out"][:, -1], last["out"])
+
+
+def test_batched_queries_do_not_see_later_keys_of_their_block():
+    # planting a huge key at the block's last position changes the last query's result only
+    from paper_2602_03152_b200 import synth
+    q, k, v, lens, dom, kw = _batched_case(5, B=1, T=3, n_recent=0)
+    base = O.decode_batched_bf16(synth.bf16_bits(q), synth.bf16_bits(k), synth.bf16_bits(v), lens, dom, **kw)
+    k2, v2 = k.clone(), v.clone()
+    k2[0, :, int(lens[0]) - 1] *= 50.0
+    v2[0, :, int(lens[0]) - 1] += 7.0
+    moved = O.decode_batched_bf16(synth.bf16_bits(q), synth.bf16_bits(k2), synth.bf16_bits(v2), lens, dom, **kw)
+    assert np.array_equal(base["out"][:, :2], moved["out"][:, :2]) and np.array_equal(base["idx"][:, :2], moved["idx"][:, :2])
+    assert not np.array_equal(base["out"][:, 2], moved["out"][:, 2])
+
+
 def test_byte_model_of_the_benchmark():
     # bench.step_bytes is the denominator of every reported roofline fraction.  Sec. 4.4: the
     # fraction of the KV cache that a step loads is N_tip/d + N_fac/t (N_tip counted in FCs of
