@@ -892,6 +892,86 @@ def run_paged(args):
                       **res}), flush=True)
 
 
+def run_batched(args):
+    """Blocks of query tokens (q_len > 1) on --config's shape: the three batched calls (scoring of all
+    queries of a block in one pass over the proxy on the tcgen05 tensor cores, selection and attention
+    per query) next to q_len repetitions of the single-query calls.  One JSON object."""
+    import numpy as np
+    import torch
+
+    from paper_2602_03152_b200 import binding, build, synth
+
+    build.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    w = synth.CONFIGS[args.config]
+    if args.budget is not None:
+        w = w.replace(budget=args.budget)
+    if args.batch is not None:
+        w = w.replace(batch=args.batch)
+    t = synth.make_inputs(w, dev)
+    f = binding.Fasa.from_workload(w, t["dom"])
+    B, Hq, Hs, Lm = w.batch, w.n_q_heads, w.n_sets, w.max_len
+    n_sel_max = w.n_sel_max()
+    proxy = f.alloc_proxy(dev)
+    f.proxy_build(t["k"], proxy, t["seq_lens"])
+    ws = f.alloc_workspace(n_sel_max, dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    peak, peak_src = _peaks()
+    tokens = int(sum(t["seq_lens"].cpu().tolist()))
+
+    def timed(fn):
+        ts = []
+        for i in range(args.warmup + args.steps):
+            flush.fill_(i & 1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            b.synchronize()
+            if i >= args.warmup:
+                ts.append(a.elapsed_time(b) * 1e3)
+        return float(np.mean(ts))
+
+    s1 = torch.zeros((B, Hs, Lm), dtype=torch.float32, device=dev)
+    i1 = torch.zeros((B, Hs, n_sel_max), dtype=torch.int32, device=dev)
+    n1 = torch.zeros((B, Hs), dtype=torch.int32, device=dev)
+    o1 = torch.zeros((B, Hq, 128), dtype=torch.float32, device=dev)
+    single = {"fc_score": timed(lambda: f.fc_score(t["q"], proxy, t["seq_lens"], s1)),
+              "topk": timed(lambda: f.topk(s1, t["seq_lens"], w.budget, i1, n1, ws)),
+              "sparse_attn": timed(lambda: f.sparse_decode_attn(t["q"], t["k"], t["v"], i1, n1, o1, ws))}
+    rows = []
+    for T in (1, 2, 4, 8):
+        if T * w.heads_per_set > 64:
+            continue
+        q = torch.stack([synth.make_step_inputs(w, 40 + j, dev)["q"] for j in range(T)], dim=1).contiguous()
+        sc = torch.zeros((B, T, Hs, Lm), dtype=torch.float32, device=dev)
+        idx = torch.zeros((B, T, Hs, n_sel_max), dtype=torch.int32, device=dev)
+        n_sel = torch.zeros((B, T, Hs), dtype=torch.int32, device=dev)
+        out = torch.zeros((B, T, Hq, 128), dtype=torch.float32, device=dev)
+        us = {"fc_score_batched": timed(lambda: f.fc_score_batched(q, proxy, t["seq_lens"], sc)),
+              "topk_batched": timed(lambda: f.topk_batched(sc, t["seq_lens"], w.budget, idx, n_sel)),
+              "sparse_attn_batched": timed(lambda: f.sparse_decode_attn_batched(q, t["k"], t["v"], idx, n_sel, out, ws)),
+              "step_batched": timed(lambda: f.decode_step_batched(q, t["k"], t["v"], proxy, t["seq_lens"], w.budget, sc, idx, n_sel,
+                                                                  out, ws))}
+        sel = int(n_sel.sum().item())
+        # scoring: the proxy once for all queries, one fp32 score per (query, set, token), the queries
+        score_bytes = tokens * w.n_kv_heads * 4 * w.n_dom + 4 * tokens * Hs * T + B * T * Hq * 256
+        flops = 2.0 * tokens * w.n_kv_heads * (2 * w.n_dom) * (w.group * T)
+        step_bytes_ = tokens * w.n_kv_heads * 4 * w.n_dom + sel * 512 + B * T * Hq * 128 * 6
+        rows.append({"q_len": T, "columns": T * w.heads_per_set, "us": us, "n_sel_per_query_unit": sel / (B * T * Hs),
+                     "fc_score_batched": {"bytes": score_bytes, "gbs": score_bytes / us["fc_score_batched"] / 1e3,
+                                          "frac": score_bytes / us["fc_score_batched"] / 1e3 / peak, "bound": "hbm",
+                                          "tflops": flops / us["fc_score_batched"] / 1e6,
+                                          "speedup_vs_q_len_single_calls": T * single["fc_score"] / us["fc_score_batched"]},
+                     "step_batched": {"bytes_method": step_bytes_, "frac_method_bytes": step_bytes_ / us["step_batched"] / 1e3 / peak,
+                                      "speedup_vs_q_len_single_steps": T * sum(single.values()) / us["step_batched"]},
+                     "device_status": f.device_status()})
+        del q, sc, idx, n_sel, out
+    print(json.dumps({"batched_queries": w.name, "budget": w.budget, "n_dom": w.n_dom, "steps": args.steps, "peak_gbs": peak,
+                      "peak_source": peak_src, "single_query_calls_us": single, "rows": rows}), flush=True)
+
+
 def run_longcot(args):
     """Workload c3 (long-CoT shape, Qwen2.5-7B-like attention): 28 layers, batch 32, prompt
     1024 then 15360 decode steps, budget 18.9 % of the current length, 16 dominant FCs.  One
@@ -1061,6 +1141,8 @@ def main():
                     help="FASA-M (Algorithm 2): K/V caches in page-locked host memory, instead of the bench line")
     ap.add_argument("--paged", type=int, default=0, metavar="PAGE_SIZE",
                     help="paged caches with this page size (a power of two >= 16) against contiguous ones, instead of the bench line")
+    ap.add_argument("--batched", action="store_true",
+                    help="blocks of query tokens (q_len 1..8) on --config's shape instead of the bench line")
     ap.add_argument("--no-resident", action="store_true", help="--longcot: skip the 28-layer resident measurement")
     ap.add_argument("--sweep-steps", type=int, default=20)
     ap.add_argument("--step-mode", type=int, default=None, choices=[0, 1],
@@ -1077,6 +1159,8 @@ def main():
         return run_offload(args)
     if args.paged:
         return run_paged(args)
+    if args.batched:
+        return run_batched(args)
     from paper_2602_03152_b200 import synth
     w = synth.CONFIGS[args.config]
     if args.budget is not None:

@@ -100,6 +100,8 @@ extern "C" {
 #define FASA_DEV_IDX_CLAMPED    4   /* sparse attention met an index outside [0, max_len)  */
 #define FASA_DEV_NSEL_CLAMPED   8   /* n_sel exceeded n_sel_max                            */
 #define FASA_DEV_PAGE_CLAMPED  16   /* a block-table entry was < 0 or >= n_pages           */
+#define FASA_DEV_TIMEOUT       32   /* a bounded wait inside a kernel ran out; results of  */
+                                    /* that launch are undefined, the context stays usable */
 
 typedef struct fasa_ctx fasa_ctx_t;
 
@@ -309,6 +311,45 @@ int32_t fasa_select_step(fasa_ctx_t* ctx, const void* q, const void* k_new, cons
                          void* k_cache, void* v_cache, void* proxy_k, int32_t* seq_lens,
                          int32_t budget, int32_t n_sel_max, float* scores, int32_t* idx,
                          int32_t* n_sel, void* stream);
+
+/* ---- blocks of query tokens (q_len > 1) ----------------------------------- */
+
+/* Most query tokens per sequence that the batched calls take. */
+#define FASA_MAX_QLEN 8
+
+/* The method is defined per query token q_t (Sec. 4.1: S_t, T_t; Sec. 4.2, Eq. 6-7), so a block
+ * of q_len queries per sequence - speculative or multi-token decoding - is q_len decode steps
+ * over one cache: query t (0 <= t < q_len) is the query of cache row seq_lens[b] - q_len + t
+ * (the block's own keys are already appended, e.g. by fasa_kv_append with n_new = q_len), it
+ * sees rows j < seq_lens[b] - (q_len - 1 - t), sink / recent positions are those of that range,
+ * and it has its own scores, its own index set and its own output.  Layouts gain a query axis
+ * after the batch axis: q bf16 [batch][q_len][n_q_heads][128]; scores fp32
+ * [batch][q_len][n_sets][max_len]; idx [batch][q_len][n_sets][n_sel_max]; n_sel
+ * [batch][q_len][n_sets]; out fp32 [batch][q_len][n_q_heads][128]; lse [batch][q_len][n_q_heads].
+ * What the q_len steps share is the proxy stream: fasa_fc_score_batched reads it ONCE and
+ * scores all queries as one matrix product P[L x 2F] . Q[2F x (heads per set * q_len)] on the
+ * tcgen05 tensor cores (fp32 accumulation in tensor memory), then reduces each query's heads
+ * (sum, or max with group_reduce = 1).  q_len = 1 gives the results of the single-query calls
+ * up to the rounding order of the fp32 accumulation.  fasa_topk_batched and
+ * fasa_sparse_decode_attn_batched are fasa_topk and fasa_sparse_decode_attn over the
+ * (sequence, query) pairs; fasa_decode_step_batched runs the three on one stream (scores and
+ * workspace required).  Status FASA_ERR_UNSUPPORTED: q_len outside [1, FASA_MAX_QLEN],
+ * batch * q_len * n_sets > 65535, (selection) a context without
+ * a cluster shape (fasa_step_cluster_size == 0), or (attention, q_len > 1) n_sel_max > 16384. */
+int32_t fasa_fc_score_batched(fasa_ctx_t* ctx, const void* q, const void* proxy_k,
+                              const int32_t* seq_lens, int32_t q_len, float* scores, void* stream);
+int32_t fasa_topk_batched(fasa_ctx_t* ctx, const float* scores, const int32_t* seq_lens,
+                          int32_t q_len, int32_t budget, int32_t n_sel_max, int32_t* idx,
+                          int32_t* n_sel, void* stream);
+int32_t fasa_sparse_decode_attn_batched(fasa_ctx_t* ctx, const void* q, const void* k_cache,
+                                        const void* v_cache, const int32_t* idx,
+                                        const int32_t* n_sel, int32_t q_len, int32_t n_sel_max,
+                                        float* out, float* lse, void* workspace, void* stream);
+int32_t fasa_decode_step_batched(fasa_ctx_t* ctx, const void* q, const void* k_cache,
+                                 const void* v_cache, const void* proxy_k, const int32_t* seq_lens,
+                                 int32_t q_len, int32_t budget, int32_t n_sel_max, float* scores,
+                                 int32_t* idx, int32_t* n_sel, float* out, float* lse,
+                                 void* workspace, void* stream);
 
 /* End-to-end step from HOST buffers: q_host, k_new_host, v_new_host (layouts as
  * fasa_kv_append with n_new = 1) -> fasa_append_decode_step -> out copied to out_host

@@ -17,7 +17,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libfasa.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
-DEV_LEN_CLAMPED, DEV_APPEND_FULL, DEV_IDX_CLAMPED, DEV_NSEL_CLAMPED, DEV_PAGE_CLAMPED = 1, 2, 4, 8, 16
+DEV_LEN_CLAMPED, DEV_APPEND_FULL, DEV_IDX_CLAMPED, DEV_NSEL_CLAMPED, DEV_PAGE_CLAMPED, DEV_TIMEOUT = 1, 2, 4, 8, 16, 32
 
 # Every entry point include/fasa.h declares.
 SYMBOLS = [
@@ -27,6 +27,7 @@ SYMBOLS = [
     "fasa_full_decode_attn", "fasa_decode_step", "fasa_stage_bytes", "fasa_decode_step_host",
     "fasa_sparse_decode_attn_static", "fasa_set_step_mode", "fasa_step_cluster_size",
     "fasa_append_decode_step", "fasa_proxy_bytes", "fasa_select_step",
+    "fasa_fc_score_batched", "fasa_topk_batched", "fasa_sparse_decode_attn_batched", "fasa_decode_step_batched",
     "fasa_calib_workspace_bytes", "fasa_calib_accumulate", "fasa_calib_select", "fasa_set_block_table",
 ]
 
@@ -85,6 +86,10 @@ def load_library() -> ctypes.CDLL:
         "fasa_step_cluster_size": (i32, [vp]),
         "fasa_append_decode_step": (i32, [vp] * 8 + [i32, i32] + [vp] * 7),
         "fasa_select_step": (i32, [vp] * 8 + [i32, i32] + [vp] * 4),
+        "fasa_fc_score_batched": (i32, [vp, vp, vp, vp, i32, vp, vp]),
+        "fasa_topk_batched": (i32, [vp, vp, vp, i32, i32, i32, vp, vp, vp]),
+        "fasa_sparse_decode_attn_batched": (i32, [vp] * 6 + [i32, i32] + [vp] * 4),
+        "fasa_decode_step_batched": (i32, [vp] * 6 + [i32, i32, i32] + [vp] * 7),
         "fasa_stage_bytes": (i32, [vp, ctypes.POINTER(ctypes.c_size_t)]),
         "fasa_decode_step_host": (i32, [vp] * 9 + [i32, i32] + [vp] * 7),
         "fasa_calib_workspace_bytes": (i32, [vp, i32, ctypes.POINTER(ctypes.c_size_t)]),
@@ -302,6 +307,28 @@ class Fasa:
             self._h, _dp(q, torch.bfloat16), _dp(k_new, torch.bfloat16), _dp(v_new, torch.bfloat16),
             k_cache.data_ptr(), v_cache.data_ptr(), _dp(proxy_k), _dp(seq_lens, torch.int32), budget, n_sel_max,
             _dp(scores, torch.float32), _dp(idx, torch.int32), _dp(n_sel, torch.int32), _stream()), "fasa_select_step")
+
+    # -- blocks of query tokens: tensors carry a query axis after the batch axis ------
+    def fc_score_batched(self, q, proxy_k, seq_lens, scores):
+        self._check(self._lib.fasa_fc_score_batched(self._h, _dp(q, torch.bfloat16), _dp(proxy_k), _dp(seq_lens, torch.int32),
+                                                    q.shape[1], _dp(scores, torch.float32), _stream()), "fasa_fc_score_batched")
+
+    def topk_batched(self, scores, seq_lens, budget, idx, n_sel):
+        self._check(self._lib.fasa_topk_batched(self._h, _dp(scores, torch.float32), _dp(seq_lens, torch.int32), scores.shape[1],
+                                                budget, idx.shape[-1], _dp(idx, torch.int32), _dp(n_sel, torch.int32), _stream()),
+                    "fasa_topk_batched")
+
+    def sparse_decode_attn_batched(self, q, k_cache, v_cache, idx, n_sel, out, workspace, lse=None):
+        self._check(self._lib.fasa_sparse_decode_attn_batched(
+            self._h, _dp(q, torch.bfloat16), k_cache.data_ptr(), v_cache.data_ptr(), _dp(idx, torch.int32),
+            _dp(n_sel, torch.int32), q.shape[1], idx.shape[-1], _dp(out, torch.float32), _dp(lse), _dp(workspace), _stream()),
+            "fasa_sparse_decode_attn_batched")
+
+    def decode_step_batched(self, q, k_cache, v_cache, proxy_k, seq_lens, budget, scores, idx, n_sel, out, workspace, lse=None):
+        self._check(self._lib.fasa_decode_step_batched(
+            self._h, _dp(q, torch.bfloat16), k_cache.data_ptr(), v_cache.data_ptr(), _dp(proxy_k), _dp(seq_lens, torch.int32),
+            q.shape[1], budget, idx.shape[-1], _dp(scores, torch.float32), _dp(idx, torch.int32), _dp(n_sel, torch.int32),
+            _dp(out, torch.float32), _dp(lse), _dp(workspace), _stream()), "fasa_decode_step_batched")
 
     # -- offline calibration (Algorithm 1) ---------------------------------------
     def calib_workspace_bytes(self, top_k: int) -> int:

@@ -51,6 +51,8 @@ struct AttnParams {
   int64_t ksb, ksh, kst, vsb, vsh, vst;
   PageMap pm;              // paged caches (all zero: contiguous)
   float scale_log2;        // softmax_scale * log2(e)
+  int q_len;               // blocks of queries (tensor-core kernel, sparse form): a "sequence" of the grid is a
+                           // (sequence, query) pair and reads the cache of sequence b / q_len; 1 otherwise
 };
 
 // GP: heads per half-warp (1..4).  HWS: half-warps sharing a row (1: group <= 4, 2: group <= 8).
@@ -442,8 +444,9 @@ decode_attn_mma_kernel(const AttnParams p) {
   // logits), so memory stays busy while the warp computes.  One cp.async group per buffer
   // fill, an empty group when there is no next tile, so "all but the newest group" always
   // names the buffer that is needed next.
-  const uint16_t* kunit = PAGED ? p.k : p.k + b * p.ksb + h * p.ksh;
-  const uint16_t* vunit = PAGED ? p.v : p.v + b * p.vsb + h * p.vsh;
+  const int bc = b / p.q_len;                       // the sequence whose cache this unit reads
+  const uint16_t* kunit = PAGED ? p.k : p.k + bc * p.ksb + h * p.ksh;
+  const uint16_t* vunit = PAGED ? p.v : p.v + bc * p.vsb + h * p.vsh;
   auto stage = [&](uint16_t (*dst)[kRowPad], const uint16_t* unit, int64_t sb, int64_t sh, int64_t st, int base) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
@@ -452,7 +455,7 @@ decode_attn_mma_kernel(const AttnParams p) {
       const int tok = SPARSE ? s_idx[r - r0] : r;
       const int c8 = (lane & 15) * 8;
       // (contiguous caches keep the plain address arithmetic: the page map costs registers)
-      if constexpr (PAGED) cp_async16(&dst[row][c8], unit + cache_row(p.pm, b, h, tok, sb, sh, st, p.status) + c8);
+      if constexpr (PAGED) cp_async16(&dst[row][c8], unit + cache_row(p.pm, bc, h, tok, sb, sh, st, p.status) + c8);
       else cp_async16(&dst[row][c8], unit + (int64_t)tok * st + c8);
     }
   };
@@ -654,15 +657,17 @@ template <bool SPARSE>
 int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
                     const int32_t* idx, const int32_t* n_rows, int n_upper, int n_sel_max,
                     float* out, float* lse, void* workspace, cudaStream_t s, float* out_mirror = nullptr,
-                    bool* mirrored = nullptr) {
+                    bool* mirrored = nullptr, int q_len = 1) {
   if (mirrored) *mirrored = false;
   const fasa_config_t& c = ctx->cfg;
   if (!fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
   // the dense pass treats a KV head with all its query heads as the unit
   const int n_sets = SPARSE ? ctx->n_sets : c.n_kv_heads;
   const int G = SPARSE ? ctx->sel_heads : ctx->group;
-  const fasa_split_plan plan = fasa_plan_splits(ctx, n_upper, c.batch * n_sets);
+  const int n_seq = c.batch * q_len;                // rows of the grid's "batch" axis
+  const fasa_split_plan plan = fasa_plan_splits(ctx, n_upper, n_seq * n_sets);
   AttnParams p;
+  p.q_len = q_len;
   p.q = (const uint16_t*)q; p.k = (const uint16_t*)k; p.v = (const uint16_t*)v;
   p.idx = idx; p.n_rows = n_rows; p.partial = (float*)workspace; p.out = nullptr; p.out_mirror = nullptr; p.lse = nullptr; p.status = ctx->d_status;
   p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.n_sets = n_sets; p.group = G;
@@ -671,7 +676,7 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   p.vsb = c.v_stride_b; p.vsh = c.v_stride_h; p.vst = c.v_stride_t;
   p.pm = fasa_page_map(ctx);
   p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
-  dim3 grid((unsigned)plan.n_splits, (unsigned)(c.batch * n_sets));
+  dim3 grid((unsigned)plan.n_splits, (unsigned)(n_seq * n_sets));
   if (ctx->use_fused) {   // default: the tensor-core kernel (mode 0 keeps the scalar one)
     static_assert(sizeof(MmaSmem) >= ((size_t)kMmaWarps * 8 * (FASA_HEAD_DIM + 2) + 8 * kMergePartStride) * sizeof(float),
                   "combine area");
@@ -705,7 +710,7 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   else decode_attn_kernel<4, 2, SPARSE><<<grid, kAttnThreads, 0, s>>>(p);
   FASA_LAUNCH_CHECK(ctx);
   FASA_CUDA_TRY(ctx, launch_after_predecessor(
-      decode_attn_merge_kernel<SPARSE>, dim3((unsigned)(c.batch * c.n_q_heads)), dim3(FASA_HEAD_DIM * kMergeWays),
+      decode_attn_merge_kernel<SPARSE>, dim3((unsigned)(n_seq * c.n_q_heads)), dim3(FASA_HEAD_DIM * kMergeWays),
       (size_t)0, s, 0, (const float*)workspace, n_rows, out, lse, ctx->d_status, (int)c.n_q_heads, (int)n_sets,
       (int)G, (int)c.max_len, (int)n_upper, (int)plan.chunk, (int)plan.n_splits));
   FASA_LAUNCH_CHECK(ctx);
@@ -736,6 +741,24 @@ int32_t fasa_sparse_attn_mirrored(fasa_ctx* ctx, const void* q, const void* k_ca
   const int n_upper = n_sel_max < ctx->cfg.max_len ? n_sel_max : ctx->cfg.max_len;
   return launch_attn<true>(ctx, q, k_cache, v_cache, idx, n_sel, n_upper, n_sel_max, out, lse, workspace, stream,
                            out_mirror, mirrored);
+}
+
+extern "C" int32_t fasa_sparse_decode_attn_batched(fasa_ctx_t* ctx, const void* q, const void* k_cache,
+                                                   const void* v_cache, const int32_t* idx, const int32_t* n_sel,
+                                                   int32_t q_len, int32_t n_sel_max, float* out, float* lse,
+                                                   void* workspace, void* stream) {
+  if (!ctx || !q || !k_cache || !v_cache || !idx || !n_sel || !out || !workspace || n_sel_max <= 0)
+    return FASA_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(workspace, 256))
+    return FASA_ERR_INVALID_ARG;
+  if (q_len < 1 || q_len > FASA_MAX_QLEN || !ctx->use_fused) return FASA_ERR_UNSUPPORTED;   // (tensor-core kernel only)
+  if ((long long)ctx->cfg.batch * q_len * ctx->n_sets > 65535) return FASA_ERR_UNSUPPORTED;
+  const int n_upper = n_sel_max < ctx->cfg.max_len ? n_sel_max : ctx->cfg.max_len;
+  // (beyond 16384 rows per unit the splits no longer merge inside one cluster, and the workspace
+  // is sized for single queries)
+  if (q_len > 1 && n_upper > 16384) return FASA_ERR_UNSUPPORTED;
+  return launch_attn<true>(ctx, q, k_cache, v_cache, idx, n_sel, n_upper, n_sel_max, out, lse, workspace,
+                           (cudaStream_t)stream, nullptr, nullptr, q_len);
 }
 
 extern "C" int32_t fasa_full_decode_attn(fasa_ctx_t* ctx, const void* q, const void* k_cache,

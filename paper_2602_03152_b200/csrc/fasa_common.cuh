@@ -102,9 +102,11 @@ int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t
                                int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
                                cudaStream_t stream);
 
+// q_len > 1: the rows of a sequence are (query, set) pairs, query-major, and query t of the
+// block sees seq_lens[b] - (q_len - 1 - t) positions.
 int32_t fasa_fused_topk_rows(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
                              int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
-                             int rows_per_seq, int n_sink, int n_recent, cudaStream_t stream);
+                             int rows_per_seq, int n_sink, int n_recent, cudaStream_t stream, int q_len = 1);
 
 // Paged caches: how a (sequence, token) pair finds its page.  All zero = contiguous caches.
 struct PageMap {

@@ -118,6 +118,8 @@ struct FusedParams {
   int32_t* status;
   int n_q_heads, n_kv_heads, n_sets, group, max_len, chunks, n_sink, n_recent, budget, n_sel_max;   // group: query heads of a unit
   int max_reduce;          // score of a KV head = max over its query heads instead of their sum
+  int q_len;               // select-only form over blocks of queries: rows per sequence are (query, set) pairs,
+                           // query t sees q_len - 1 - t fewer positions (0 or 1: plain rows)
   int64_t ksb, ksh, kst, vsb, vsh, vst;
   float scale_log2;        // softmax_scale * log2(e)
   PageMap pm;              // paged caches (all zero: contiguous)
@@ -212,6 +214,10 @@ fused_decode_kernel(const FusedParams p) {
     q_stage = *reinterpret_cast<const uint4*>(p.q + su.q0 * FASA_HEAD_DIM + tid * 8);
   int16_t chan_stage = -1;
   if (MODE != 1 && tid < p.chunks * 8) chan_stage = p.chan[h * p.chunks * 8 + tid];
+  if (MODE == 1 && p.q_len > 1) {
+    const int t = (u % p.n_sets) / (p.n_sets / p.q_len);        // the query of this row
+    if (len_raw >= 0 && len_raw <= p.max_len) len_raw = max(0, len_raw - (p.q_len - 1 - t));   // (a bad length is left for clamp_len to flag)
+  }
   int len_old;
   if (append) {
     if (tid == 0) s_len_old = clamp_len(len_raw, p.max_len, p.status);
@@ -1028,6 +1034,7 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
   p.chunks = ctx->chunks; p.n_sink = c.n_sink; p.n_recent = c.n_recent; p.budget = budget;
   p.n_sel_max = n_sel_max;
   p.max_reduce = c.group_reduce;
+  p.q_len = 1;
   p.ksb = c.k_stride_b; p.ksh = c.k_stride_h; p.kst = c.k_stride_t;
   p.vsb = c.v_stride_b; p.vsh = c.v_stride_h; p.vst = c.v_stride_t;
   p.scale_log2 = c.softmax_scale * 1.4426950408889634f;
@@ -1067,7 +1074,7 @@ int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t
 // r / rows_per_seq), with the given forced positions instead of the context's.
 int32_t fasa_fused_topk_rows(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
                              int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
-                             int rows_per_seq, int n_sink, int n_recent, cudaStream_t stream) {
+                             int rows_per_seq, int n_sink, int n_recent, cudaStream_t stream, int q_len) {
   const fasa_config_t& c = ctx->cfg;
   FusedParams p;
   memset(&p, 0, sizeof(p));
@@ -1077,6 +1084,7 @@ int32_t fasa_fused_topk_rows(fasa_ctx* ctx, const float* scores, const int32_t* 
   p.n_q_heads = rows_per_seq; p.n_kv_heads = 1; p.n_sets = rows_per_seq; p.group = 1; p.max_len = c.max_len;
   p.chunks = ctx->chunks; p.n_sink = n_sink; p.n_recent = n_recent; p.budget = budget;
   p.n_sel_max = n_sel_max;
+  p.q_len = q_len;
   // The context's cluster size suits its own number of rows (few rows: wide clusters, so the
   // whole GPU works on them).  A launch with many more rows takes the narrowest cluster that
   // holds a row's keys: more rows are then resident at once.

@@ -298,6 +298,76 @@ def test_select_step_gives_the_index_sets_of_the_separate_calls():
         r.fasa.select_step(r.q, r.k, r.v, r.proxy, r.seq_lens, w.budget, None, r.idx, r.n_sel, k_new, None)
 
 
+# ------------------------------------------------------------------ blocks of queries ----
+
+def _batched_run(w, T, budget=None, seed=0):
+    """Runs fasa_decode_step_batched on a block of T queries per sequence and checks every (sequence,
+    query) pair against the oracle: query t sees the rows up to its own position."""
+    r = Run(w)
+    r.build_proxy()
+    budget = w.budget if budget is None else budget
+    B, Hq, Hs, Lm = w.batch, w.n_q_heads, w.n_sets, w.max_len
+    q = torch.stack([synth.make_step_inputs(w.replace(index=w.index + seed), 40 + t, "cuda")["q"] for t in range(T)], dim=1).contiguous()
+    scores = torch.full((B, T, Hs, Lm), SENTINEL, dtype=torch.float32, device="cuda")
+    idx = torch.full((B, T, Hs, r.n_sel_max), -7, dtype=torch.int32, device="cuda")
+    n_sel = torch.full((B, T, Hs), -7, dtype=torch.int32, device="cuda")
+    out = torch.full((B, T, Hq, 128), SENTINEL, dtype=torch.float32, device="cuda")
+    lse = torch.full((B, T, Hq), SENTINEL, dtype=torch.float32, device="cuda")
+    r.fasa.decode_step_batched(q, r.k, r.v, r.proxy, r.seq_lens, budget, scores, idx, n_sel, out, r.ws, lse)
+    torch.cuda.synchronize()
+    assert r.fasa.device_status() == 0
+    h = r.host()
+    qh = q.cpu().double().numpy()
+    for t in range(T):
+        lens_t = np.maximum(h["seq_lens"] - (T - 1 - t), 0)
+        parity.check_step(qh[:, t], h["k"], h["v"], lens_t, h["dom"], scores=scores[:, t].cpu().numpy(), idx=idx[:, t].cpu().numpy(),
+                          n_sel=n_sel[:, t].cpu().numpy(), out=out[:, t].cpu().numpy(), what=f"{w.name} query {t} of {T}",
+                          **r.oracle_kwargs(budget))
+        for b in range(B):                       # rows at and past what the query sees are never written
+            assert torch.all(scores[b, t, :, int(lens_t[b]):] == SENTINEL)
+    return r, q, scores, idx, n_sel, out, lse
+
+
+@pytest.mark.parametrize("T", [1, 2, 4, 8])
+def test_batched_queries_match_the_oracle(T):
+    w = C["c1"].replace(batch=2, max_len=3000, len_lo=1500, len_hi=2999, budget=100, n_sink=2, n_recent=5)
+    r, q, scores, idx, n_sel, out, lse = _batched_run(w, T)
+    if T == 1:
+        # one query per block: the single-query calls on the same inputs (scores up to the
+        # rounding order of the fp32 accumulation, everything after them the same kernels)
+        r.q = q[:, 0].contiguous()
+        r.step()
+        assert torch.allclose(scores[:, 0], r.scores, rtol=0, atol=2e-4 * float(r.scores[r.scores != SENTINEL].abs().max()))
+        assert float((out[:, 0] - r.out).abs().max()) <= 1e-3
+
+
+@pytest.mark.parametrize("cfg,kw,T", [
+    ("c3", dict(batch=2, max_len=2000, len_lo=900, len_hi=1999, budget=-150), 8),          # group of 7 x 8 queries = 56 columns, no RoPE
+    ("c1", dict(batch=1, n_q_heads=8, n_kv_heads=1, max_len=1500, len_lo=1500, len_hi=1500, budget=64), 8),   # 8 x 8 = 64 columns
+    ("c1", dict(batch=2, max_len=1000, len_lo=3, len_hi=999, n_dom=3, budget=40), 3),     # one 8-channel block, padded K
+    ("c1", dict(batch=1, max_len=2500, len_lo=2400, len_hi=2400, n_dom=5, budget=40, pairing=1), 5),   # odd chunk count
+    ("c1", dict(batch=1, max_len=2100, len_lo=2100, len_hi=2100, n_dom=64, budget=77), 2),  # all FCs: 8 blocks of 16 channels
+    ("c1", dict(batch=2, max_len=1300, len_lo=600, len_hi=1300, n_dom=13, budget=50, group_reduce=1), 4),   # max over the group
+    ("c4", dict(batch=2, n_q_heads=8, n_kv_heads=2, max_len=1800, len_lo=700, len_hi=1800, budget=33, sel_heads=1), 6),   # a set per head
+])
+def test_batched_queries_shapes(cfg, kw, T):
+    _batched_run(C[cfg].replace(**kw), T)
+
+
+def test_batched_queries_reject_what_they_cannot_take():
+    w = C["c1"].replace(batch=1, n_q_heads=16, n_kv_heads=1, max_len=600, len_lo=600, len_hi=600)   # 16 heads per set? no: group 16 > 8
+    w = C["c3"].replace(batch=1, max_len=600, len_lo=600, len_hi=600)
+    r = Run(w)
+    r.build_proxy()
+    for T in (9, 0):
+        q = torch.zeros((1, max(T, 1), w.n_q_heads, 128), dtype=torch.bfloat16, device="cuda")
+        st = r.fasa._lib.fasa_fc_score_batched(r.fasa._h, q.data_ptr(), r.proxy.data_ptr(), r.seq_lens.data_ptr(), T,
+                                               r.scores.data_ptr(), None)
+        assert st == binding.ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+    assert r.fasa.device_status() == 0
+
+
 def test_large_selection_is_attended_by_the_split_k_kernel():
     # n_sel_max * ceil(G / 4) >= 2048 and a workspace: cluster kernel without its attention
     # phase, then the split-K tensor-core attention whose splits merge inside their own cluster
