@@ -769,9 +769,8 @@ def run_offload(args):
     lens = t["seq_lens"].clone()
     start = (t["seq_lens"] - 1).clamp_(min=0)
 
-    # Without a workspace the step stays one launch whatever the selection size: over the host
-    # link the cluster kernel's own gather (plain 8-byte loads) runs about twice as fast as the
-    # split-K kernel's 16-byte asynchronous copies (717 vs 1477 us at workload c4, budget 1024).
+    # Without a workspace the step stays one launch whatever the selection size (the cluster
+    # kernel's own gather); the tensor-core attention route is measured beside it.
     def step(k, v):
         return lambda: f.append_decode_step(s["q"], s["k_new"], s["v_new"], k, v, proxy, lens, w.budget, None, idx,
                                             n_sel, out, None)
@@ -779,6 +778,23 @@ def run_offload(args):
     reset = lambda: lens.copy_(start)
     us_host, _ = timed(step(kh, vh), args.steps, args.warmup, reset)
     out_host = out.clone()
+    # the same caches through the tensor-core attention kernel (a workspace hands the attention over)
+    us_host_ws, _ = timed(lambda: f.append_decode_step(s["q"], s["k_new"], s["v_new"], kh, vh, proxy, lens, w.budget, None, idx,
+                                                       n_sel, out, ws), args.steps, args.warmup, reset)
+    # the split key cache of Algorithm 2: only the non-dominant channels of the selected keys cross the link
+    split = None
+    if w.n_dom % 4 == 0:
+        knd = f.alloc_host_nondom()
+        f.m_split(t["k"], knd, t["seq_lens"])
+        torch.cuda.synchronize()
+        us_split, _ = timed(lambda: f.m_decode_step(s["q"], knd, vh, proxy, lens, w.budget, None, idx, n_sel, out, ws, None,
+                                                    s["k_new"], s["v_new"]), args.steps, args.warmup, reset)
+        nsel = int(n_sel.sum().item())
+        split_link = nsel * (512 - 4 * w.n_dom) + w.batch * w.n_kv_heads * (512 - 4 * w.n_dom)
+        split = {"us_per_step": us_split, "link_bytes_per_step": split_link, "link_bytes_per_selected_token": 512 - 4 * w.n_dom,
+                 "achieved_gbs": split_link / us_split / 1e3, "frac_of_link": split_link / us_split / 1e3 / link_gbs,
+                 "max_abs_diff_vs_whole_rows": float((out - out_host).abs().max())}
+        del knd
     n_sel_total = int(n_sel.sum().item())
     us_dev, _ = timed(step(t["k"], t["v"]), args.steps, args.warmup, reset)
     same = bool(torch.equal(out, out_host))
@@ -798,6 +814,9 @@ def run_offload(args):
                      "frac": link_bytes / us_host / 1e3 / link_gbs,
                      "peak_source": "measured here: 256 MiB page-locked host -> device copy, best of 5",
                      "step_bound_us": bound_us, "step_frac_of_bound": bound_us / us_host},
+        "whole_rows_tensor_core_attention": {"us_per_step": us_host_ws, "achieved_gbs": link_bytes / us_host_ws / 1e3,
+                                             "frac_of_link": link_bytes / us_host_ws / 1e3 / link_gbs},
+        "split_key_cache": split,
         "dense_over_host_resident_caches_us": us_dense_host,
         "speedup_vs_dense_over_host_resident_caches": us_dense_host / us_host,
         "gpu_bytes_per_cached_token": {"fasa_m": f.row_elems * 2, "full_cache": 512 + f.row_elems * 2},

@@ -351,6 +351,48 @@ int32_t fasa_decode_step_batched(fasa_ctx_t* ctx, const void* q, const void* k_c
                                  int32_t* idx, int32_t* n_sel, float* out, float* lse,
                                  void* workspace, void* stream);
 
+/* ---- memory-optimised variant with a split key cache (FASA-M, Algorithm 2) -------------- */
+
+/* Algorithm 2 keeps the dominant part of the key cache on the GPU (here: the proxy-K buffer)
+ * and moves the rest - the non-dominant key channels and the values - to the CPU; per step it
+ * selects on the GPU, transfers K^nondom_T and V_T for the selected tokens only, and Combines
+ * the key rows before the attention.  Besides handing whole-row caches in host memory to the
+ * ordinary calls (see "Where the caches live"), the library therefore takes the key cache in
+ * that split form:
+ *   k_nondom  bf16 [batch][n_kv_heads][max_len][fasa_m_nondom_row_elems(n_dom)]: of every key
+ *             the 128 - 2 n_dom channels that are NOT dominant for its head, ascending; meant
+ *             for page-locked, device-addressable host memory (device memory works too);
+ *   v_cache   as everywhere else, likewise in host memory; proxy_k on the GPU.
+ * A selected token then costs 512 - 4 n_dom bytes on the host link instead of 512, and a group
+ * of up to 8 query heads reads each row once.  Requirements: n_dom a multiple of 4 (otherwise
+ * fasa_m_nondom_row_elems returns 0 and the calls FASA_ERR_UNSUPPORTED), contiguous caches.
+ *   fasa_m_split        Split of an existing full key cache: writes k_nondom rows j < seq_lens[b]
+ *                       (the proxy comes from fasa_proxy_build).
+ *   fasa_m_kv_append    Split + UpdateCache of n_new new tokens per sequence: their dominant pairs
+ *                       to the proxy, the other channels to k_nondom, the value rows to v_cache;
+ *                       seq_lens[b] += n_new.  Arguments as fasa_kv_append.
+ *   fasa_m_sparse_decode_attn   Combine + FAC (Eq. 6-7): the key rows of idx are assembled in
+ *                       shared memory from k_nondom and the proxy.  The logits are the same dot
+ *                       products as in fasa_sparse_decode_attn, summed in another channel order
+ *                       (results agree to fp32 rounding, not bit for bit).
+ *   fasa_m_decode_step  Algorithm 2's loop body: (k_new / v_new non-NULL: Split + UpdateCache,)
+ *                       TIP and TopK-I on the proxy (the cluster kernel, one launch), then the
+ *                       call above.  Needs a cluster shape (fasa_step_cluster_size > 0). */
+int32_t fasa_m_nondom_row_elems(int32_t n_dom);
+int32_t fasa_m_split(fasa_ctx_t* ctx, const void* k_cache, void* k_nondom, const int32_t* seq_lens,
+                     void* stream);
+int32_t fasa_m_kv_append(fasa_ctx_t* ctx, void* k_nondom, void* v_cache, void* proxy_k,
+                         int32_t* seq_lens, const void* k_new, const void* v_new, int32_t n_new,
+                         void* stream);
+int32_t fasa_m_sparse_decode_attn(fasa_ctx_t* ctx, const void* q, const void* k_nondom,
+                                  const void* v_cache, const void* proxy_k, const int32_t* idx,
+                                  const int32_t* n_sel, int32_t n_sel_max, float* out, float* lse,
+                                  void* workspace, void* stream);
+int32_t fasa_m_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_new, const void* v_new,
+                           void* k_nondom, void* v_cache, void* proxy_k, int32_t* seq_lens,
+                           int32_t budget, int32_t n_sel_max, float* scores, int32_t* idx,
+                           int32_t* n_sel, float* out, float* lse, void* workspace, void* stream);
+
 /* End-to-end step from HOST buffers: q_host, k_new_host, v_new_host (layouts as
  * fasa_kv_append with n_new = 1) -> fasa_append_decode_step -> out copied to out_host
  * (fp32 [batch][n_q_heads][128]); synchronises the stream.  Inputs in pinned (page-locked,

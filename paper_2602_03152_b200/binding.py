@@ -27,6 +27,7 @@ SYMBOLS = [
     "fasa_full_decode_attn", "fasa_decode_step", "fasa_stage_bytes", "fasa_decode_step_host",
     "fasa_sparse_decode_attn_static", "fasa_set_step_mode", "fasa_step_cluster_size",
     "fasa_append_decode_step", "fasa_proxy_bytes", "fasa_select_step",
+    "fasa_m_nondom_row_elems", "fasa_m_split", "fasa_m_kv_append", "fasa_m_sparse_decode_attn", "fasa_m_decode_step",
     "fasa_fc_score_batched", "fasa_topk_batched", "fasa_sparse_decode_attn_batched", "fasa_decode_step_batched",
     "fasa_calib_workspace_bytes", "fasa_calib_accumulate", "fasa_calib_select", "fasa_set_block_table",
 ]
@@ -86,6 +87,11 @@ def load_library() -> ctypes.CDLL:
         "fasa_step_cluster_size": (i32, [vp]),
         "fasa_append_decode_step": (i32, [vp] * 8 + [i32, i32] + [vp] * 7),
         "fasa_select_step": (i32, [vp] * 8 + [i32, i32] + [vp] * 4),
+        "fasa_m_nondom_row_elems": (i32, [i32]),
+        "fasa_m_split": (i32, [vp] * 5),
+        "fasa_m_kv_append": (i32, [vp] * 7 + [i32, vp]),
+        "fasa_m_sparse_decode_attn": (i32, [vp] * 7 + [i32] + [vp] * 4),
+        "fasa_m_decode_step": (i32, [vp] * 8 + [i32, i32] + [vp] * 7),
         "fasa_fc_score_batched": (i32, [vp, vp, vp, vp, i32, vp, vp]),
         "fasa_topk_batched": (i32, [vp, vp, vp, i32, i32, i32, vp, vp, vp]),
         "fasa_sparse_decode_attn_batched": (i32, [vp] * 6 + [i32, i32] + [vp] * 4),
@@ -307,6 +313,38 @@ class Fasa:
             self._h, _dp(q, torch.bfloat16), _dp(k_new, torch.bfloat16), _dp(v_new, torch.bfloat16),
             k_cache.data_ptr(), v_cache.data_ptr(), _dp(proxy_k), _dp(seq_lens, torch.int32), budget, n_sel_max,
             _dp(scores, torch.float32), _dp(idx, torch.int32), _dp(n_sel, torch.int32), _stream()), "fasa_select_step")
+
+    # -- memory-optimised variant with a split key cache (Algorithm 2) -----------------
+    def alloc_host_nondom(self) -> torch.Tensor:
+        """Page-locked host tensor [batch][n_kv_heads][max_len][128 - 2 n_dom] for the non-dominant key channels."""
+        nd = int(self._lib.fasa_m_nondom_row_elems(self.n_dom))
+        if nd == 0:
+            raise FasaError(ERR_UNSUPPORTED, "fasa_m_nondom_row_elems", "n_dom must be a multiple of 4")
+        t = torch.zeros((self.batch, self.n_kv_heads, self.max_len, nd), dtype=torch.bfloat16).pin_memory()
+        return t
+
+    def m_split(self, k_cache, k_nondom, seq_lens):
+        self._check(self._lib.fasa_m_split(self._h, k_cache.data_ptr(), k_nondom.data_ptr(), _dp(seq_lens, torch.int32), _stream()),
+                    "fasa_m_split")
+
+    def m_kv_append(self, k_nondom, v_cache, proxy_k, seq_lens, k_new, v_new):
+        self._check(self._lib.fasa_m_kv_append(self._h, k_nondom.data_ptr(), v_cache.data_ptr(), _dp(proxy_k), _dp(seq_lens, torch.int32),
+                                               _dp(k_new, torch.bfloat16), _dp(v_new, torch.bfloat16), k_new.shape[2], _stream()),
+                    "fasa_m_kv_append")
+
+    def m_sparse_decode_attn(self, q, k_nondom, v_cache, proxy_k, idx, n_sel, out, workspace, lse=None):
+        self._check(self._lib.fasa_m_sparse_decode_attn(self._h, _dp(q, torch.bfloat16), k_nondom.data_ptr(), v_cache.data_ptr(),
+                                                        _dp(proxy_k), _dp(idx, torch.int32), _dp(n_sel, torch.int32), idx.shape[-1],
+                                                        _dp(out, torch.float32), _dp(lse), _dp(workspace), _stream()),
+                    "fasa_m_sparse_decode_attn")
+
+    def m_decode_step(self, q, k_nondom, v_cache, proxy_k, seq_lens, budget, scores, idx, n_sel, out, workspace, lse=None,
+                      k_new=None, v_new=None):
+        self._check(self._lib.fasa_m_decode_step(
+            self._h, _dp(q, torch.bfloat16), _dp(k_new, torch.bfloat16), _dp(v_new, torch.bfloat16), k_nondom.data_ptr(),
+            v_cache.data_ptr(), _dp(proxy_k), _dp(seq_lens, torch.int32), budget, idx.shape[-1], _dp(scores, torch.float32),
+            _dp(idx, torch.int32), _dp(n_sel, torch.int32), _dp(out, torch.float32), _dp(lse), _dp(workspace), _stream()),
+            "fasa_m_decode_step")
 
     # -- blocks of query tokens: tensors carry a query axis after the batch axis ------
     def fc_score_batched(self, q, proxy_k, seq_lens, scores):

@@ -103,6 +103,20 @@ extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_h
     }
   }
 
+  // the complement of each head's dominant channels, ascending (split key cache)
+  std::vector<int16_t> ndchan;
+  if (c.n_dom % 4 == 0 && c.n_dom < FASA_HEAD_DIM / 2 && c.page_size == 0) {
+    const int nd = FASA_HEAD_DIM - 2 * c.n_dom;
+    ndchan.resize((size_t)c.n_kv_heads * nd);
+    for (int h = 0; h < c.n_kv_heads; ++h) {
+      bool dom[FASA_HEAD_DIM] = {false};
+      for (int i = 0; i < 2 * c.n_dom; ++i) dom[chan[(size_t)h * ctx->row_elems + i]] = true;
+      int n = 0;
+      for (int ch = 0; ch < FASA_HEAD_DIM; ++ch)
+        if (!dom[ch]) ndchan[(size_t)h * nd + n++] = (int16_t)ch;
+    }
+  }
+
   cudaError_t e = cudaGetDevice(&ctx->device);
   cudaDeviceProp prop;
   if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, ctx->device);
@@ -118,9 +132,14 @@ extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_h
   if (e == cudaSuccess)
     e = cudaMemcpy(ctx->d_chan, chan.data(), chan.size() * sizeof(int16_t), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
+  if (e == cudaSuccess && !ndchan.empty()) {
+    e = cudaMalloc(&ctx->d_ndchan, ndchan.size() * sizeof(int16_t));
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->d_ndchan, ndchan.data(), ndchan.size() * sizeof(int16_t), cudaMemcpyHostToDevice);
+  }
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     cudaFree(ctx->d_chan);
+    cudaFree(ctx->d_ndchan);
     cudaFree(ctx->d_status);
     cudaFree(ctx->d_arrive);
     delete ctx;
@@ -132,6 +151,19 @@ extern "C" int32_t fasa_create(const fasa_config_t* cfg, const int32_t* dom_fc_h
   return FASA_OK;
 }
 
+// Whether a K/V cache pointer is host memory (the memory-optimised variant keeps the caches in
+// page-locked host memory): asked of the driver once per pointer, a decode loop passes the same one.
+bool fasa_on_host(fasa_ctx* ctx, const void* p) {
+  if (ctx->cache_seen == p && p) return ctx->cache_on_host != 0;
+  cudaPointerAttributes at;
+  bool host = false;
+  if (cudaPointerGetAttributes(&at, p) == cudaSuccess) host = at.type == cudaMemoryTypeHost;
+  else cudaGetLastError();
+  ctx->cache_seen = p;
+  ctx->cache_on_host = host ? 1 : 0;
+  return host;
+}
+
 extern "C" int32_t fasa_set_block_table(fasa_ctx_t* ctx, const int32_t* block_table) {
   if (!ctx || !block_table || ctx->cfg.page_size == 0) return FASA_ERR_INVALID_ARG;
   ctx->block_table = block_table;
@@ -141,6 +173,7 @@ extern "C" int32_t fasa_set_block_table(fasa_ctx_t* ctx, const int32_t* block_ta
 extern "C" int32_t fasa_destroy(fasa_ctx_t* ctx) {
   if (!ctx) return FASA_ERR_INVALID_ARG;
   cudaFree(ctx->d_chan);
+  cudaFree(ctx->d_ndchan);
   cudaFree(ctx->d_status);
   cudaFree(ctx->d_arrive);
   delete ctx;
@@ -213,6 +246,15 @@ extern "C" int32_t fasa_workspace_bytes(const fasa_ctx_t* ctx, int32_t n_sel_max
   return FASA_OK;
 }
 
+// The cluster kernel attends to groups of more than four query heads in two passes over the
+// selected rows.  From HBM the second pass hits L2; from caches in page-locked host memory every
+// row would cross the host link twice (measured at 28 / 4 heads: 531 us against 282 us through
+// the tensor-core kernel, which reads a row once for up to eight heads): given a workspace, such
+// steps hand the attention over whatever the selection size.
+static bool fasa_host_rows_twice(fasa_ctx* ctx, const void* k_cache, const void* workspace) {
+  return workspace != nullptr && ctx->sel_heads > 4 && ctx->cfg.page_size == 0 && fasa_on_host(ctx, k_cache);
+}
+
 // What fasa_fc_score, fasa_topk and fasa_sparse_decode_attn require of the arguments they share
 // with the composite calls.
 static bool three_kernel_args_ok(const fasa_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
@@ -235,7 +277,7 @@ extern "C" int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* 
         ((uintptr_t)v_cache & 15) || (scores && ((uintptr_t)scores & 3)))
       return FASA_ERR_INVALID_ARG;
     if (!fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
-    if (fasa_attend_separately(ctx, n_sel_max, workspace)) {
+    if (fasa_attend_separately(ctx, n_sel_max, workspace) || fasa_host_rows_twice(ctx, k_cache, workspace)) {
       if ((uintptr_t)workspace & 255) return FASA_ERR_INVALID_ARG;   // (what the second launch would refuse)
       int32_t st2 = fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
                                       idx, n_sel, out, lse, nullptr, nullptr, (cudaStream_t)stream, false);
@@ -273,7 +315,7 @@ static int32_t append_decode_step_impl(fasa_ctx_t* ctx, const void* q, const voi
         (scores && ((uintptr_t)scores & 3)))
       return FASA_ERR_INVALID_ARG;
     if (!fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
-    if (fasa_attend_separately(ctx, n_sel_max, workspace)) {
+    if (fasa_attend_separately(ctx, n_sel_max, workspace) || fasa_host_rows_twice(ctx, k_cache, workspace)) {
       if ((uintptr_t)workspace & 255) return FASA_ERR_INVALID_ARG;   // (what the second launch would refuse)
       int32_t st2 = fasa_fused_launch(ctx, q, k_cache, v_cache, proxy_k, seq_lens, budget, n_sel_max, scores,
                                       idx, n_sel, out, lse, k_new, v_new, (cudaStream_t)stream, false);

@@ -21,6 +21,7 @@
 
 #include "fasa_cluster_merge.cuh"
 #include "fasa_common.cuh"
+#include "fasa_score_core.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -51,6 +52,7 @@ struct AttnParams {
   int64_t ksb, ksh, kst, vsb, vsh, vst;
   PageMap pm;              // paged caches (all zero: contiguous)
   float scale_log2;        // softmax_scale * log2(e)
+  fasa_ksplit ks;          // split key cache (KSPLIT kernels): k holds the non-dominant channels only
   int q_len;               // blocks of queries (tensor-core kernel, sparse form): a "sequence" of the grid is a
                            // (sequence, query) pair and reads the cache of sequence b / q_len; 1 otherwise
 };
@@ -304,6 +306,15 @@ __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)
 __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst)), "l"(src) : "memory");
 }
+// The same through L1 ("cache all levels"): rows that live in page-locked HOST memory cross the
+// host link in full 128-byte requests this way, at twice the rate of the L2-only form (measured:
+// 50 vs 25 GB/s of a 55 GB/s link); for rows in HBM the L2-only form above is the faster one.
+__device__ __forceinline__ void cp_async16_ca(void* dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_addr(dst)), "l"(src) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 // waits until at most N of this thread's committed groups are still in flight
 template <int N>
@@ -370,7 +381,13 @@ cudaError_t launch_after_predecessor(Kernel kernel, dim3 grid, dim3 block, size_
 
 // CLUSTER: the splits of a unit are the CTAs of one cluster (grid.x = cluster size) and merge
 // in the same launch; otherwise each split writes its partial result for the merge kernel.
-template <bool SPARSE, bool PAGED, bool CLUSTER>
+// HOSTMEM: K and V rows are copied through L1 (caches in page-locked host memory).  KSPLIT
+// (Algorithm 2's Combine; sparse, contiguous, HOSTMEM): a key row is assembled in shared memory
+// from its non-dominant channels (p.k, ascending channel order, the part that crosses the host
+// link) followed by its dominant channels in proxy order (from the GPU-resident proxy); the
+// query operand is loaded in the same channel order, so the logits are the same dot products
+// summed in another order.
+template <bool SPARSE, bool PAGED, bool CLUSTER, bool HOSTMEM = false, bool KSPLIT = false>
 __global__ void __launch_bounds__(kMmaThreads)
 decode_attn_mma_kernel(const AttnParams p) {
   __shared__ ClusterMergeSmem s_merge;              // (CLUSTER only: written by the peers)
@@ -406,10 +423,21 @@ decode_attn_mma_kernel(const AttnParams p) {
   uint32_t qb[8][2];
   {
     const uint16_t* qh = p.q + (su.q0 + (g < p.group ? g : 0)) * FASA_HEAD_DIM;
+    // position c of an assembled key row holds channel ndchan[c] (c < nd) or chan[c - nd]
+    auto q_at = [&](int c) -> uint32_t {
+      const int ch = c < p.ks.nd ? p.ks.ndchan[h * p.ks.nd + c] : p.ks.chan[h * p.ks.chunks * 8 + c - p.ks.nd];
+      return qh[ch];
+    };
 #pragma unroll
     for (int kb = 0; kb < 8; ++kb) {
-      const uint32_t w0 = *reinterpret_cast<const uint32_t*>(qh + kb * 16 + 2 * t);
-      const uint32_t w1 = *reinterpret_cast<const uint32_t*>(qh + kb * 16 + 2 * t + 8);
+      uint32_t w0, w1;
+      if constexpr (KSPLIT) {
+        w0 = q_at(kb * 16 + 2 * t) | (q_at(kb * 16 + 2 * t + 1) << 16);
+        w1 = q_at(kb * 16 + 2 * t + 8) | (q_at(kb * 16 + 2 * t + 9) << 16);
+      } else {
+        w0 = *reinterpret_cast<const uint32_t*>(qh + kb * 16 + 2 * t);
+        w1 = *reinterpret_cast<const uint32_t*>(qh + kb * 16 + 2 * t + 8);
+      }
       qb[kb][0] = g < p.group ? w0 : 0u;
       qb[kb][1] = g < p.group ? w1 : 0u;
     }
@@ -456,11 +484,32 @@ decode_attn_mma_kernel(const AttnParams p) {
       const int c8 = (lane & 15) * 8;
       // (contiguous caches keep the plain address arithmetic: the page map costs registers)
       if constexpr (PAGED) cp_async16(&dst[row][c8], unit + cache_row(p.pm, bc, h, tok, sb, sh, st, p.status) + c8);
+      else if constexpr (HOSTMEM) cp_async16_ca(&dst[row][c8], unit + (int64_t)tok * st + c8);
       else cp_async16(&dst[row][c8], unit + (int64_t)tok * st + c8);
     }
   };
+  // Combine: the 16 key rows of a tile from their two homes
+  const ProxyGeom ks_pg = proxy_geom(KSPLIT ? p.ks.chunks : 1);
+  const unsigned char* ks_proxy = KSPLIT ? p.ks.proxy + (int64_t)su.kv * ((p.max_len + 15) >> 4) * ks_pg.tile_bytes : nullptr;
+  auto stage_split_k = [&](uint16_t (*dst)[kRowPad], int base) {
+    const int nd_chunks = p.ks.nd >> 3, words = 4 * p.ks.chunks;
+    for (int c = lane; c < 16 * nd_chunks; c += 32) {                 // the part that crosses the link
+      const int row = c / nd_chunks, ch = c % nd_chunks;
+      const int tok = s_idx[min(base + row, r1 - 1) - r0];
+      cp_async16_ca(&dst[row][ch * 8], kunit + (int64_t)tok * p.kst + ch * 8);
+    }
+    for (int c = lane; c < 16 * words; c += 32) {                     // the dominant pairs, from the proxy
+      const int row = c / words, w = c % words;
+      const int tok = s_idx[min(base + row, r1 - 1) - r0];
+      cp_async4(&dst[row][p.ks.nd + 2 * w], ks_proxy + proxy_word_offset(ks_pg, tok, w));
+    }
+  };
+  auto stage_k = [&](int base) {
+    if constexpr (KSPLIT) stage_split_k(sm.k[warp], base);
+    else stage(sm.k[warp], kunit, p.ksb, p.ksh, p.kst, base);
+  };
   constexpr int kTileStep = kMmaWarps * 16;
-  if (r0 + warp * 16 < r1) stage(sm.k[warp], kunit, p.ksb, p.ksh, p.kst, r0 + warp * 16);
+  if (r0 + warp * 16 < r1) stage_k(r0 + warp * 16);
   cp_async_commit();
   if (r0 + warp * 16 < r1) stage(sm.v[warp], vunit, p.vsb, p.vsh, p.vst, r0 + warp * 16);
   cp_async_commit();
@@ -511,7 +560,7 @@ decode_attn_mma_kernel(const AttnParams p) {
       sm.p_lo[warp][head][row] = (uint16_t)f32_to_bf16_bits(rest);
     }
     __syncwarp();                                   // P is visible; every lane is done with the K buffer
-    if (more) stage(sm.k[warp], kunit, p.ksb, p.ksh, p.kst, base + kTileStep);
+    if (more) stage_k(base + kTileStep);
     cp_async_commit();
     cp_async_wait<1>();                             // this tile's V rows have landed
     __syncwarp();
@@ -657,7 +706,7 @@ template <bool SPARSE>
 int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
                     const int32_t* idx, const int32_t* n_rows, int n_upper, int n_sel_max,
                     float* out, float* lse, void* workspace, cudaStream_t s, float* out_mirror = nullptr,
-                    bool* mirrored = nullptr, int q_len = 1) {
+                    bool* mirrored = nullptr, int q_len = 1, const fasa_ksplit* ksplit = nullptr) {
   if (mirrored) *mirrored = false;
   const fasa_config_t& c = ctx->cfg;
   if (!fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
@@ -668,6 +717,10 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
   const fasa_split_plan plan = fasa_plan_splits(ctx, n_upper, n_seq * n_sets);
   AttnParams p;
   p.q_len = q_len;
+  memset(&p.ks, 0, sizeof(p.ks));
+  if (ksplit) p.ks = *ksplit;
+  // caches in page-locked host memory are copied through L1 (contiguous caches, tensor-core kernel)
+  const bool host = c.page_size == 0 && ctx->use_fused && (ksplit != nullptr || fasa_on_host(ctx, k));
   p.q = (const uint16_t*)q; p.k = (const uint16_t*)k; p.v = (const uint16_t*)v;
   p.idx = idx; p.n_rows = n_rows; p.partial = (float*)workspace; p.out = nullptr; p.out_mirror = nullptr; p.lse = nullptr; p.status = ctx->d_status;
   p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.n_sets = n_sets; p.group = G;
@@ -691,6 +744,8 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
       p.chunk = cchunk; p.n_splits = cs; p.out = out; p.out_mirror = out_mirror; p.lse = lse;
       if (mirrored) *mirrored = out_mirror != nullptr;
       auto fn = c.page_size > 0 ? decode_attn_mma_kernel<SPARSE, true, true> : decode_attn_mma_kernel<SPARSE, false, true>;
+      if (host) fn = decode_attn_mma_kernel<SPARSE, false, true, true>;
+      if constexpr (SPARSE) { if (ksplit) fn = decode_attn_mma_kernel<true, false, true, true, true>; }
       const size_t smem = sizeof(MmaSmem) + (SPARSE ? (size_t)cchunk * sizeof(int32_t) : 0);
       FASA_CUDA_TRY(ctx, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
       FASA_CUDA_TRY(ctx, launch_after_predecessor(fn, dim3((unsigned)cs, grid.y), dim3(kMmaThreads), smem, s, cs, p));
@@ -698,6 +753,8 @@ int32_t launch_attn(fasa_ctx* ctx, const void* q, const void* k, const void* v,
       return FASA_OK;
     }
     auto fn = c.page_size > 0 ? decode_attn_mma_kernel<SPARSE, true, false> : decode_attn_mma_kernel<SPARSE, false, false>;
+    if (host) fn = decode_attn_mma_kernel<SPARSE, false, false, true>;
+    if constexpr (SPARSE) { if (ksplit) fn = decode_attn_mma_kernel<true, false, false, true, true>; }
     // (+ the slice of the index list: chunk <= 2048 rows)
     const size_t smem = sizeof(MmaSmem) + (SPARSE ? (size_t)plan.chunk * sizeof(int32_t) : 0);
     FASA_CUDA_TRY(ctx, cudaFuncSetAttribute((const void*)fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem));
@@ -741,6 +798,28 @@ int32_t fasa_sparse_attn_mirrored(fasa_ctx* ctx, const void* q, const void* k_ca
   const int n_upper = n_sel_max < ctx->cfg.max_len ? n_sel_max : ctx->cfg.max_len;
   return launch_attn<true>(ctx, q, k_cache, v_cache, idx, n_sel, n_upper, n_sel_max, out, lse, workspace, stream,
                            out_mirror, mirrored);
+}
+
+// FAC over a split key cache (Algorithm 2: Combine, then Eq. 6-7): k_nondom holds the non-dominant
+// channels of every key, the proxy their dominant ones.
+int32_t fasa_attn_split_keys(fasa_ctx* ctx, const void* q, const void* k_nondom, const void* v_cache, const void* proxy_k,
+                             const int32_t* idx, const int32_t* n_sel, int32_t n_sel_max, float* out, float* lse,
+                             void* workspace, cudaStream_t stream) {
+  const fasa_config_t& c = ctx->cfg;
+  fasa_ksplit ks;
+  ks.proxy = (const unsigned char*)proxy_k; ks.ndchan = ctx->d_ndchan; ks.chan = ctx->d_chan;
+  ks.chunks = ctx->chunks; ks.nd = FASA_HEAD_DIM - 2 * c.n_dom;
+  // (the kernel addresses k_nondom with the K strides: rows of nd elements, dense per unit)
+  fasa_ctx tmp = *ctx;
+  tmp.cfg.k_stride_t = ks.nd;
+  tmp.cfg.k_stride_h = (int64_t)c.max_len * ks.nd;
+  tmp.cfg.k_stride_b = tmp.cfg.k_stride_h * c.n_kv_heads;
+  const int n_upper = n_sel_max < c.max_len ? n_sel_max : c.max_len;
+  int32_t st = launch_attn<true>(&tmp, q, k_nondom, v_cache, idx, n_sel, n_upper, n_sel_max, out, lse, workspace, stream,
+                                 nullptr, nullptr, 1, &ks);
+  ctx->launches = tmp.launches;
+  memcpy(ctx->cuda_err, tmp.cuda_err, sizeof(ctx->cuda_err));
+  return st;
 }
 
 extern "C" int32_t fasa_sparse_decode_attn_batched(fasa_ctx_t* ctx, const void* q, const void* k_cache,

@@ -26,6 +26,8 @@ struct fasa_ctx {
   int page_shift;         // log2(page_size), 0 for contiguous caches
   int pages_per_seq;      // ceil(max_len / page_size)
   int16_t* d_chan;        // device [n_kv_heads][row_elems]: K channel of each proxy element, -1 = padding
+  int16_t* d_ndchan;      // device [n_kv_heads][128 - 2 n_dom]: the other channels of each head, ascending (null
+                          // unless n_dom is a multiple of 4: the split key cache of the memory-optimised variant)
   int32_t* d_status;      // device status word (FASA_DEV_* bits)
   int32_t* d_arrive;      // device [batch]: CTAs of a sequence that have read its length (append-then-step)
   int fused_cs;           // cluster size of the cluster kernel (step and top-k), 0 = not available
@@ -36,6 +38,8 @@ struct fasa_ctx {
   // (null: not page-locked + mapped), so that a decode loop with fixed buffers asks the driver once
   const void* host_seen[4];
   void* host_mapped[4];
+  const void* cache_seen;   // the last K/V cache pointer asked about, and whether it is host memory
+  int cache_on_host;
   long long launches;     // kernels launched through this context
   char cuda_err[256];
 };
@@ -97,6 +101,18 @@ cudaError_t fasa_stage_from_mapped(void* dq, const void* sq, size_t q_bytes, voi
 int32_t fasa_sparse_attn_mirrored(fasa_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                                   const int32_t* idx, const int32_t* n_sel, int32_t n_sel_max, float* out,
                                   float* lse, void* workspace, cudaStream_t stream, float* out_mirror, bool* mirrored);
+
+// Split key cache (memory-optimised variant): what the attention kernels need besides k_nondom.
+struct fasa_ksplit {
+  const unsigned char* proxy;   // the dominant part, on the GPU
+  const int16_t* ndchan;        // [n_kv_heads][nd]
+  const int16_t* chan;          // [n_kv_heads][2 n_dom]
+  int chunks, nd;               // 16-byte chunks per proxy row; non-dominant channels per key
+};
+int32_t fasa_attn_split_keys(fasa_ctx* ctx, const void* q, const void* k_nondom, const void* v_cache, const void* proxy_k,
+                             const int32_t* idx, const int32_t* n_sel, int32_t n_sel_max, float* out, float* lse,
+                             void* workspace, cudaStream_t stream);
+bool fasa_on_host(fasa_ctx* ctx, const void* p);
 
 int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
                                int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,

@@ -658,6 +658,78 @@ def test_fasa_m_caches_in_pinned_host_memory():
     assert host.fasa.device_status() == 0
 
 
+@pytest.mark.parametrize("cfg,kw,budget", [
+    ("c3", dict(batch=2, max_len=3000, len_lo=1400, len_hi=2900), -150),                     # group of 7: one pass over the link
+    ("c1", dict(batch=2, max_len=2500, len_lo=900, len_hi=2400, n_dom=8, pairing=1), 200),  # sinks and recent rows, 8 FCs
+    ("c4", dict(batch=1, n_q_heads=8, n_kv_heads=2, max_len=1900, len_lo=1890, len_hi=1890, n_dom=32), 64),
+])
+def test_fasa_m_split_key_cache(cfg, kw, budget):
+    # Algorithm 2 as stated: the dominant channels of the keys stay on the GPU (the proxy), the other
+    # channels and the values live in page-locked host memory; Split on append, Combine in the
+    # attention kernel.  Layout bit for bit, index sets equal to the whole-row path, outputs against
+    # the oracle and within fp32 rounding of the whole-row path (same products, another order).
+    w = C[cfg].replace(**kw)
+    r = Run(w)
+    r.build_proxy()
+    f = r.fasa
+    knd, vh = f.alloc_host_nondom(), f.alloc_host_cache()
+    assert knd.is_pinned() and knd.shape[-1] == 128 - 2 * w.n_dom
+    vh.copy_(r.t["v"])
+    f.m_split(r.k, knd, r.seq_lens)
+    torch.cuda.synchronize()
+    dom = np.sort(r.dom.numpy(), axis=1)
+    lens = r.t["seq_lens"].tolist()
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            d = np.concatenate([dom[h], dom[h] + 64]) if w.pairing == 0 else np.concatenate([2 * dom[h], 2 * dom[h] + 1])
+            rest = np.setdiff1d(np.arange(128), d)                     # ascending
+            L = lens[b]
+            assert torch.equal(knd[b, h, :L], r.t["k"][b, h, :L][:, torch.from_numpy(rest)])
+            assert torch.all(knd[b, h, L:] == 0)
+    # one appended token through Split + UpdateCache, against the whole-row append
+    s = synth.make_step_inputs(w, 2, "cuda")
+    proxy2, lens2 = r.proxy.clone(), r.seq_lens.clone()
+    f.m_kv_append(knd, vh, proxy2, lens2, s["k_new"], s["v_new"])
+    f.kv_append(r.k, r.v, r.proxy, r.seq_lens, s["k_new"], s["v_new"])
+    torch.cuda.synchronize()
+    assert torch.equal(proxy2, r.proxy) and torch.equal(lens2, r.seq_lens) and torch.equal(vh, r.v.cpu())
+    knd_ref = f.alloc_host_nondom()
+    f.m_split(r.k, knd_ref, r.seq_lens)
+    torch.cuda.synchronize()
+    assert torch.equal(knd, knd_ref)
+    # the step: whole-row path on the device, split path over the link
+    r.reset_outputs()
+    r.fasa.decode_step(s["q"], r.k, r.v, r.proxy, r.seq_lens, budget, r.scores, r.idx, r.n_sel, r.out, None, r.lse)
+    ref = [x.clone() for x in (r.scores, r.idx, r.n_sel, r.out, r.lse)]
+    r.reset_outputs()
+    n0 = f.launch_count()
+    f.m_decode_step(s["q"], knd, vh, proxy2, lens2, budget, r.scores, r.idx, r.n_sel, r.out, r.ws, r.lse)
+    torch.cuda.synchronize()
+    assert f.launch_count() - n0 == 2 and f.device_status() == 0
+    assert torch.equal(r.scores, ref[0]) and torch.equal(r.idx, ref[1]) and torch.equal(r.n_sel, ref[2])
+    assert float((r.out - ref[3]).abs().max()) <= 1e-4
+    h = r.host()
+    parity.check_step(s["q"].cpu().double().numpy(), r.k.cpu().double().numpy(), r.v.cpu().double().numpy(), r.seq_lens.cpu().numpy(),
+                      h["dom"], idx=h["idx"], n_sel=h["n_sel"], out=h["out"], what="split key cache", **r.oracle_kwargs(budget))
+    # appending form of the step (Algorithm 2's loop body): equals append + step
+    s3 = synth.make_step_inputs(w, 3, "cuda")
+    f.kv_append(r.k, r.v, r.proxy, r.seq_lens, s3["k_new"], s3["v_new"])
+    f.decode_step(s3["q"], r.k, r.v, r.proxy, r.seq_lens, budget, None, r.idx, r.n_sel, r.out, None)
+    ref_idx, ref_out = r.idx.clone(), r.out.clone()
+    f.m_decode_step(s3["q"], knd, vh, proxy2, lens2, budget, None, r.idx, r.n_sel, r.out, r.ws, None, s3["k_new"], s3["v_new"])
+    torch.cuda.synchronize()
+    assert torch.equal(lens2, r.seq_lens) and torch.equal(r.idx, ref_idx) and float((r.out - ref_out).abs().max()) <= 1e-4
+
+
+def test_fasa_m_split_needs_whole_chunks():
+    w = C["c1"].replace(batch=1, max_len=600, len_lo=600, len_hi=600, n_dom=6)
+    r = Run(w)
+    assert r.fasa._lib.fasa_m_nondom_row_elems(6) == 0 and r.fasa._lib.fasa_m_nondom_row_elems(16) == 96
+    buf = torch.zeros(1 << 16, dtype=torch.bfloat16, device="cuda")
+    st = r.fasa._lib.fasa_m_split(r.fasa._h, r.k.data_ptr(), buf.data_ptr(), r.seq_lens.data_ptr(), None)
+    assert st == binding.ERR_UNSUPPORTED
+
+
 def _random_workloads(n, seed):
     rng = np.random.default_rng(seed)
     out = []
