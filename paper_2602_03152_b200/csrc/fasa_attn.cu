@@ -408,9 +408,14 @@ decode_attn_mma_kernel(const AttnParams p) {
     n = clamp_len(p.n_rows[b], p.max_len, p.status);
   }
   const int split = blockIdx.x;
-  const int r0 = min(n, split * p.chunk);
-  if (!CLUSTER && r0 >= n) return;                  // (in a cluster an empty split still joins the merge)
-  const int r1 = min(n, r0 + p.chunk);
+  // In a cluster the splits share the rows the unit actually has (every CTA stays for the merge
+  // anyway, and with rows far below the bound a fixed split size would leave most of them idle
+  // while they hold their place on an SM); otherwise the split size is the planned one, which
+  // the merge kernel knows.
+  const int chunk = CLUSTER ? min(p.chunk, max(32, ((n + (int)gridDim.x - 1) / (int)gridDim.x + 31) & ~31)) : p.chunk;
+  const int r0 = min(n, split * chunk);
+  if (!CLUSTER && r0 >= n) return;
+  const int r1 = min(n, r0 + chunk);
 
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
