@@ -354,6 +354,44 @@ def test_batched_queries_shapes(cfg, kw, T):
     _batched_run(C[cfg].replace(**kw), T)
 
 
+def test_batched_queries_on_paged_caches_equal_the_contiguous_results():
+    # a block of 4 queries after a 4-token append, page pools in random order: the batched calls read
+    # the proxy and the K/V rows through the block table and must give the contiguous bits
+    w = C["c1"].replace(batch=2, max_len=2000, len_lo=700, len_hi=1900, budget=60, n_sink=1, n_recent=4)
+    t = synth.make_inputs(w, "cpu")
+    P, T = 64, 4
+    r, f, kp, vp, tab, table, need = _paged_twin(w, t, P, extra_tokens=T)
+    proxy_p, lens_p = f.alloc_proxy(), r.seq_lens.clone()
+    r.build_proxy()
+    f.proxy_build(kp, proxy_p, lens_p)
+    g = torch.Generator().manual_seed(4)
+    kn = torch.randn((w.batch, w.n_kv_heads, T, 128), generator=g).to(torch.bfloat16).cuda()
+    vn = torch.randn((w.batch, w.n_kv_heads, T, 128), generator=g).to(torch.bfloat16).cuda()
+    r.fasa.kv_append(r.k, r.v, r.proxy, r.seq_lens, kn, vn)
+    f.kv_append(kp, vp, proxy_p, lens_p, kn, vn)
+    q = torch.stack([synth.make_step_inputs(w, 70 + j, "cuda")["q"] for j in range(T)], dim=1).contiguous()
+    B, Hq, Hs, Lm = w.batch, w.n_q_heads, w.n_sets, w.max_len
+    res = []
+    for fa, k, v, px, ln in ((r.fasa, r.k, r.v, r.proxy, r.seq_lens), (f, kp, vp, proxy_p, lens_p)):
+        scores = torch.full((B, T, Hs, Lm), SENTINEL, dtype=torch.float32, device="cuda")
+        idx = torch.full((B, T, Hs, r.n_sel_max), -7, dtype=torch.int32, device="cuda")
+        n_sel = torch.full((B, T, Hs), -7, dtype=torch.int32, device="cuda")
+        out = torch.full((B, T, Hq, 128), SENTINEL, dtype=torch.float32, device="cuda")
+        fa.decode_step_batched(q, k, v, px, ln, w.budget, scores, idx, n_sel, out, r.ws)
+        torch.cuda.synchronize()
+        assert fa.device_status() == 0
+        res.append((scores, idx, n_sel, out))
+    for x, y in zip(*res):
+        assert torch.equal(x, y)
+    # and the contiguous run against the oracle, on the grown caches
+    kh, vh = r.k.cpu().double().numpy(), r.v.cpu().double().numpy()
+    lens = r.seq_lens.cpu().numpy()
+    for tq in range(T):
+        parity.check_step(q[:, tq].cpu().double().numpy(), kh, vh, np.maximum(lens - (T - 1 - tq), 0), np.sort(r.dom.numpy(), axis=1),
+                          scores=res[0][0][:, tq].cpu().numpy(), idx=res[0][1][:, tq].cpu().numpy(), n_sel=res[0][2][:, tq].cpu().numpy(),
+                          out=res[0][3][:, tq].cpu().numpy(), what=f"paged block, query {tq}", **r.oracle_kwargs())
+
+
 def test_batched_queries_reject_what_they_cannot_take():
     w = C["c1"].replace(batch=1, n_q_heads=16, n_kv_heads=1, max_len=600, len_lo=600, len_hi=600)   # 16 heads per set? no: group 16 > 8
     w = C["c3"].replace(batch=1, max_len=600, len_lo=600, len_hi=600)
