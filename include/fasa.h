@@ -35,6 +35,10 @@
  *     proxy_row_elems * 2 (64 at n_dom = 16); a step then moves n_sel * 512 bytes per
  *     (batch, KV head) over the link, which bounds it.  The dense path over host-resident
  *     caches streams the whole cache over the link and is only useful as a reference.
+ *     The attention calls ask the driver once per k_cache pointer whether it is host memory
+ *     (rows in host memory are copied through L1, which doubles the link's throughput) and
+ *     remember the answer for the last pointer seen: k_cache and v_cache must be of the same
+ *     kind, and a buffer must not change its kind while keeping its address.
  *   - Paged caches (page_size > 0).  K, V and the proxy are pools of n_pages pages of
  *     page_size tokens, shared by the sequences; a block table, int32
  *     [batch][ceil(max_len / page_size)] on the device, names the physical page of every

@@ -1214,6 +1214,29 @@ def test_topk_exact_on_heavy_ties():
     _assert_topk_exact(torch.full((1, 2, 3000), -1.5), [2999], -189)
 
 
+def test_topk_exact_on_crowded_bins():
+    # The select phase finishes on the candidates of the k-th key's bin when that bin holds at most
+    # 4096 keys cluster-wide.  Scores crowded into one bin of the first pass (same sign, exponent and
+    # two leading mantissa bits) take a second cluster pass before the candidates are few enough;
+    # scores crowded into one bin of the second pass as well take all three.
+    g = torch.Generator().manual_seed(12)
+    sc1 = 1.0 + 0.2 * torch.rand((2, 2, 20000), generator=g)                  # one 11-bit bin, ~12 keys per 22-bit bin
+    sc2 = 1.0 + 1e-4 * torch.rand((1, 2, 20000), generator=g)                 # one 22-bit bin: every radix pass runs
+    sc3 = torch.cat([sc1[:1, :, :10000], -sc1[:1, :, 10000:]], dim=2)         # the crowd split over a positive and a negative bin
+    for sc in (sc1, sc2, sc3):
+        lens = [20000 - 37 * b for b in range(sc.shape[0])]
+        for budget in (1, 300, 4096, 9000, 19990):
+            _assert_topk_exact(sc, lens, budget)
+        _assert_topk_exact(sc, lens, 500, n_sink=3, n_recent=100)
+        _assert_topk_exact(sc, lens, -189)
+    # exactly 4096 / 4097 keys in the bin (the capacity of the candidate area), the rest far below
+    for n_in in (4096, 4097):
+        sc = torch.full((1, 1, 30000), -5.0)
+        sc[0, 0, torch.randperm(30000, generator=g)[:n_in]] = 1.0 + 0.2 * torch.rand(n_in, generator=g)
+        for budget in (1, 2048, n_in - 1, n_in, n_in + 5):
+            _assert_topk_exact(sc, [30000], budget)
+
+
 def test_topk_exact_on_special_values():
     g = torch.Generator().manual_seed(6)
     sc = torch.randn(1, 4, 4096, generator=g)
