@@ -214,7 +214,9 @@ int32_t fasa_topk(fasa_ctx_t* ctx, const float* scores, const int32_t* seq_lens,
  * the n_sel[b][h] rows listed in idx (any order, rows used as stored).  fp32
  * accumulation; out fp32 [batch][n_q_heads][128]; lse (nullable) fp32
  * [batch][n_q_heads] = log sum_j exp(logit_j).  n_sel == 0 gives out = 0,
- * lse = -inf.  Split over the selection, merged by a second kernel. */
+ * lse = -inf.  Split over the selection; the splits of a unit merge inside the same launch (they
+ * form one thread-block cluster) up to n_sel_max = 16384, through `workspace` and a second
+ * kernel beyond. */
 int32_t fasa_sparse_decode_attn(fasa_ctx_t* ctx, const void* q, const void* k_cache,
                                 const void* v_cache, const int32_t* idx, const int32_t* n_sel,
                                 int32_t n_sel_max, float* out, float* lse, void* workspace,
@@ -273,7 +275,10 @@ int32_t fasa_sparse_decode_attn_static(fasa_ctx_t* ctx, const void* q, const voi
  * >= 2048; >= 512 when all units together reach 24576 such rows; >= 256 when the cluster
  * kernel's grid exceeds two CTAs per SM), mode 1 ends the
  * cluster kernel after the selection and attends with the split-K tensor-core kernel of
- * fasa_sparse_decode_attn (three launches instead of one).
+ * fasa_sparse_decode_attn (two launches instead of one; three beyond 16384 selected rows).  The
+ * same hand-over happens, whatever the selection size, when the caches are page-locked host
+ * memory and an index set serves more than four query heads (the cluster kernel would fetch
+ * every row twice over the host link).
  * Mode 0, and every configuration mode 1 cannot take: fasa_fc_score -> fasa_topk ->
  * fasa_sparse_decode_attn; scores and workspace are then required (INVALID_ARG if NULL).
  * Both modes select identical index sets; outputs agree to fp32 rounding.
