@@ -203,7 +203,7 @@ extern "C" int32_t fasa_set_step_mode(fasa_ctx_t* ctx, int32_t mode) {
 }
 
 extern "C" int32_t fasa_step_cluster_size(const fasa_ctx_t* ctx) {
-  return ctx && ctx->use_fused && ctx->fused_step_ok ? ctx->fused_cs : 0;
+  return ctx && ctx->use_fused && ctx->fused_step_ok ? (ctx->fused_cs > 0 ? ctx->step_cs : 0) : 0;
 }
 
 extern "C" int64_t fasa_launch_count(const fasa_ctx_t* ctx) { return ctx ? ctx->launches : 0; }

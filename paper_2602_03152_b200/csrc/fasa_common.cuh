@@ -33,6 +33,9 @@ struct fasa_ctx {
   int fused_cs;           // cluster size of the cluster kernel (step and top-k), 0 = not available
   int fused_step_ok;      // the one-launch step supports this configuration
   size_t fused_smem;      // its dynamic shared memory
+  int step_threads;       // the decode step's own shape: 512 threads with fused_cs CTAs per cluster, or the wide
+  int step_cs;            // form (1024 threads, one CTA per SM, half the cluster) where that evens out the stream
+  size_t step_smem;
   int use_fused;          // fasa_decode_step takes the one-launch kernel when it is available
   // host-buffer step: the last host pointers seen and what the device can use in their place
   // (null: not page-locked + mapped), so that a decode loop with fixed buffers asks the driver once

@@ -46,7 +46,6 @@ namespace {
 
 constexpr int kFT = 512;               // threads per CTA; two CTAs share an SM (64 registers per thread):
                                        // what one SM can pull from HBM grows with its resident warps
-constexpr int kFW = kFT / 32;          // warps per CTA
 constexpr int kFBins = 2048;           // bins of the widest radix pass
 constexpr int kPartStride = kMergePartStride - 2;   // m, l, acc[128] (+ 2 words of padding in shared memory)
 constexpr int kCapMax = 22528;         // keys a CTA can hold (88 KB of shared memory)
@@ -71,7 +70,7 @@ struct FusedSmem {
   int acc, part, p, al, m, l, att_end;
   int total;
 };
-__host__ __device__ inline FusedSmem fused_smem_layout(int cap) {
+__host__ __device__ inline FusedSmem fused_smem_layout(int cap, int kFW = kFT / 32) {   // kFW: warps per CTA
   FusedSmem L;
   L.keys = 0;
   L.hist1 = cap * 4;
@@ -169,9 +168,12 @@ __device__ __forceinline__ bool warp_find_kth(uint32_t v, uint32_t kth, int lane
 // tensor-core kernel instead).
 // PAGED: K, V and the proxy are page pools behind a block table (compiled separately, so that
 // the contiguous form keeps its plain address arithmetic within 64 registers).
-template <int KB, int NG, int MODE, bool PAGED = false>
-__global__ void __launch_bounds__(kFT, 2)
+// NT: threads per CTA: 512 (two CTAs per SM) or 1024 (one CTA per SM with twice the slice).
+template <int KB, int NG, int MODE, bool PAGED = false, int NT = 512>
+__global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1)
 fused_decode_kernel(const FusedParams p) {
+  constexpr int kFT = NT;                  // (shadow the file-level constants inside this kernel)
+  constexpr int kFW = NT / 32;
   cg::cluster_group cluster = cg::this_cluster();
   const int cs = (int)cluster.num_blocks();
   const int crank = (int)cluster.block_rank();
@@ -242,7 +244,7 @@ fused_decode_kernel(const FusedParams p) {
   const int c1 = min(len, c0 + per);
   const int nloc = c1 - c0;
   const int cap = (((p.max_len + cs - 1) / cs) + 31) & ~31;
-  const FusedSmem sl = fused_smem_layout(cap);
+  const FusedSmem sl = fused_smem_layout(cap, kFW);
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + sl.keys);
   uint32_t* hist0 = reinterpret_cast<uint32_t*>(smem_raw + sl.hist0);
   uint32_t* hist1 = reinterpret_cast<uint32_t*>(smem_raw + sl.hist1);
@@ -337,9 +339,9 @@ fused_decode_kernel(const FusedParams p) {
     }
   }
   for (int i = tid; i < kFBins; i += kFT) { hist0[i] = 0u; hist1[i] = 0u; }
-  if (tid < 3 * kFinBins) (&s_fin[0][0])[tid] = 0u;
-  if (tid < 3 * 2 * kGroups) (&s_gsum[0][0][0])[tid] = 0u;
-  if (tid < 3 * 2 * 32) (&s_fine[0][0][0])[tid] = 0u;
+  for (int i = tid; i < 3 * kFinBins; i += kFT) (&s_fin[0][0])[i] = 0u;
+  for (int i = tid; i < 3 * 2 * kGroups; i += kFT) (&s_gsum[0][0][0])[i] = 0u;
+  for (int i = tid; i < 3 * 2 * 32; i += kFT) (&s_fine[0][0][0])[i] = 0u;
   if (tid == 0) { s_ncand = 0u; s_cgt = 0u; s_ceq = 0u; }
   if (MODE != 1 && tid < GP * (FASA_HEAD_DIM / 8))
     *reinterpret_cast<uint4*>(&s_qraw[tid / (FASA_HEAD_DIM / 8)][(tid % (FASA_HEAD_DIM / 8)) * 8]) = q_stage;
@@ -945,6 +947,19 @@ FusedFn fused_fn(int chunks, bool paged = false) {
 
 FusedFn topk_fn() { return fused_decode_kernel<1, 1, 1>; }
 
+// The wide form of the step: 1024 threads, one CTA per SM.
+template <int MODE, bool PAGED>
+FusedFn wide_variant(int chunks) {
+  const int nb = (chunks + 1) / 2;
+  if (nb <= 1) return fused_decode_kernel<1, 1, MODE, PAGED, 1024>;
+  if (nb <= 2) return fused_decode_kernel<2, 1, MODE, PAGED, 1024>;
+  if (nb <= 4) return fused_decode_kernel<4, 1, MODE, PAGED, 1024>;
+  return fused_decode_kernel<4, 2, MODE, PAGED, 1024>;
+}
+FusedFn wide_fn(int chunks, bool paged) { return paged ? wide_variant<0, true>(chunks) : wide_variant<0, false>(chunks); }
+FusedFn wide_select_fn(int chunks, bool paged) { return paged ? wide_variant<2, true>(chunks) : wide_variant<2, false>(chunks); }
+constexpr int kCapWide = 40960;        // keys a 1024-thread CTA can hold (one CTA per SM)
+
 FusedFn select_fn(int chunks, bool paged = false) {         // the step without attention
   return paged ? fused_variant<2, true>(chunks) : fused_variant<2, false>(chunks);
 }
@@ -1011,6 +1026,45 @@ int fasa_fused_plan(fasa_ctx* ctx) {
     }
     ctx->fused_cs = cs;
     ctx->fused_smem = smem;
+    // The wide form.  When the 512-thread grid has more CTAs than SMs, SMs hold pairs of CTAs that
+    // share their ~44 GB/s while lone CTAs (in a single wave: batch 8 x 8 heads at 64 K) end their
+    // stream at 28 us against 50 us, and grids of several rounds run twice as many select chains.
+    // Half as many CTAs of 1024 threads with twice the slice each sit alone on their SMs and
+    // stream at the same rate: 74 -> 70 us there, 68 -> 57 us for batch 5, 210 -> 203 us for the
+    // four-round grid of batch 16 at 64-128 K.
+    ctx->step_threads = kFT;
+    ctx->step_cs = cs;
+    ctx->step_smem = smem;
+    const long long ctas = (long long)units * cs;
+    // (not down to clusters of one CTA: batch 32 x 4 heads of 7 query heads at 16 K lost 3-6 % that way)
+    if (cs >= 4 && ctas > ctx->n_sm && cap_of(cs / 2) <= kCapWide) {
+      const int cs_w = cs / 2;
+      const size_t smem_w = (size_t)fused_smem_layout(cap_of(cs_w), 32).total;
+      const int limit_w = (int)fused_smem_layout(kCapWide, 32).total;
+      FusedFn fw = wide_fn(ctx->chunks, paged), fs = wide_select_fn(ctx->chunks, paged);
+      cudaLaunchConfig_t cw;
+      memset(&cw, 0, sizeof(cw));
+      cw.gridDim = dim3((unsigned)cs_w, (unsigned)units, 1);
+      cw.blockDim = dim3(1024, 1, 1);
+      cw.dynamicSmemBytes = smem_w;
+      cudaLaunchAttribute aw[1];
+      aw[0].id = cudaLaunchAttributeClusterDimension;
+      aw[0].val.clusterDim.x = (unsigned)cs_w;
+      aw[0].val.clusterDim.y = 1;
+      aw[0].val.clusterDim.z = 1;
+      cw.attrs = aw;
+      cw.numAttrs = 1;
+      int n_w = 0;
+      if (cudaFuncSetAttribute((const void*)fw, cudaFuncAttributeMaxDynamicSharedMemorySize, limit_w) == cudaSuccess &&
+          cudaFuncSetAttribute((const void*)fs, cudaFuncAttributeMaxDynamicSharedMemorySize, limit_w) == cudaSuccess &&
+          cudaOccupancyMaxActiveClusters(&n_w, (const void*)fw, &cw) == cudaSuccess && n_w >= 1) {
+        ctx->step_threads = 1024;
+        ctx->step_cs = cs_w;
+        ctx->step_smem = smem_w;
+      } else {
+        cudaGetLastError();
+      }
+    }
     return cs;
   }
   return 0;
@@ -1042,16 +1096,21 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
   if (!fasa_pages_ready(ctx)) return FASA_ERR_INVALID_ARG;
   const bool paged = c.page_size > 0;
   FusedFn fn = with_attention ? fused_fn(ctx->chunks, paged) : select_fn(ctx->chunks, paged);
+  // (the step's own shape: 512 threads and the context's cluster size, or the wide form)
+  const bool wide = ctx->step_threads == 1024;
+  if (wide) fn = with_attention ? wide_fn(ctx->chunks, paged) : wide_select_fn(ctx->chunks, paged);
+  const int threads = wide ? 1024 : kFT, cs_l = wide ? ctx->step_cs : ctx->fused_cs;
+  const size_t smem_l = wide ? ctx->step_smem : ctx->fused_smem;
 
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3((unsigned)ctx->fused_cs, (unsigned)(c.batch * ctx->n_sets), 1);
-  cfg.blockDim = dim3(kFT, 1, 1);
-  cfg.dynamicSmemBytes = ctx->fused_smem;
+  cfg.gridDim = dim3((unsigned)cs_l, (unsigned)(c.batch * ctx->n_sets), 1);
+  cfg.blockDim = dim3((unsigned)threads, 1, 1);
+  cfg.dynamicSmemBytes = smem_l;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)ctx->fused_cs;
+  attr[0].val.clusterDim.x = (unsigned)cs_l;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;

@@ -1336,9 +1336,10 @@ def _full_size_sampled(w, units, budget=None, append=False, keep=None):
 
 
 def test_config2_full_size_sampled_units():
-    # batch 16, ragged 64K-128K contexts, 8 GiB of K/V on the device: the cluster kernel in clusters of 8
+    # batch 16, ragged 64K-128K contexts, 8 GiB of K/V on the device: the cluster kernel in its wide
+    # form (clusters of 4 CTAs of 1024 threads, up to 32768 keys each), several rounds of CTAs
     f = _full_size_sampled(C["c2"], [(0, 0), (7, 5), (15, 7)])
-    assert f.step_cluster_size() == 8
+    assert f.step_cluster_size() == 4
 
 
 @pytest.mark.parametrize("layer", [0, 1])
@@ -1356,8 +1357,10 @@ def test_config3_full_size_sampled_units_with_append(step, layer):
 def test_config4_full_size_in_the_launch_shape_of_the_benchmark(budget):
     # batch 8 x 8 KV heads = 64 units, clusters of 4 with 16384 keys per CTA, the appending form:
     # budget 256 is one launch, budget 4096 the select-only cluster kernel + the split-K kernel
+    # (64 units x clusters of 4 would put one 512-thread CTA on some SMs and two on others: the plan
+    # takes the wide form, clusters of 2 CTAs of 1024 threads with 32768 keys each)
     f = _full_size_sampled(C["c4"].replace(budget=budget), [(0, 0), (3, 5), (7, 7)], append=True)
-    assert f.step_cluster_size() == 4
+    assert f.step_cluster_size() == 2
 
 
 @pytest.mark.parametrize("F,budget", [(4, 64), (64, 4096)])
