@@ -19,12 +19,15 @@
 //     tiles with coalesced 16-byte loads and scatters their four 4-byte words per lane into the
 //     core-matrix layout (conflict-free: the 32 lanes of a store fill 128 contiguous bytes);
 //   - one thread issues K / 16 tcgen05.mma (M 128, N 16..64, bf16 x bf16 -> fp32) and commits
-//     them to an mbarrier; the loads of the next tile are issued before the CTA waits on it;
-//   - epilogue: thread r owns token row r: tcgen05.ld of its N columns, sum (or max) over the G
-//     heads of each query, rows past a query's own position are not written.
-// Several CTAs share an SM (64 TMEM columns each), which overlaps one CTA's loads with another's
-// product and epilogue.  The wait on the mbarrier is bounded: on expiry the kernel raises
-// FASA_DEV_TIMEOUT, frees its tensor memory and returns.
+//     them to an mbarrier;
+//   - epilogue: thread r owns token row r: tcgen05.ld of its N columns (column 8 g + t = head g,
+//     query t, so the registers of a head are indexed statically), sum (or max) over the G heads
+//     of each query, rows past a query's own position are not written.
+// Two A buffers, two accumulators (32 or 64 TMEM columns each) and two register stages: the
+// product of tile i+1 is issued before the epilogue of tile i, while the loads of tiles i+2 and
+// i+3 travel.  Several CTAs share an SM (64 or 128 TMEM columns each; the shared memory is padded
+// so that the CTAs of an SM never ask for more than its 512 columns).  The wait on the mbarrier
+// is bounded: on expiry the kernel raises FASA_DEV_TIMEOUT, frees its tensor memory and returns.
 //
 // Selection and attention of the block reuse the cluster kernel's selection phases and the
 // split-K tensor-core attention with (sequence, query) pairs as rows.
