@@ -36,6 +36,8 @@
 // selection, after which no CTA touches a peer's shared memory.  No thread spins on anything.
 #include <cooperative_groups.h>
 
+#include <type_traits>
+
 #include "fasa_cluster_merge.cuh"
 #include "fasa_common.cuh"
 #include "fasa_score_core.cuh"
@@ -393,46 +395,78 @@ fused_decode_kernel(const FusedParams p) {
   } else {
     if (own_new) fetch(a, T, 0);                              // (the new row is in place now)
     locate(tp_next, T + step);
-    while (T * 16 < c1) {       // uniform over the warp
-      float c[TPI][4];
+    // The loop exists twice.  When the head's dominant channels fill whole 16-channel blocks and
+    // exactly the KB x NG blocks this kernel is compiled for (4 n_dom = 32 KB NG: 8, 16, 32 or 64
+    // FCs), a tile's loads and products need no run-time test of the geometry: the loads of a batch
+    // then leave back to back, which is worth a quarter of what one SM can pull on its own.
+    auto stream = [&](auto exact_tag) {
+      constexpr bool EXACT = decltype(exact_tag)::value;
+      auto fetch_x = [&](uint4 (&aa)[TPI][KB], int TT, int grp) {
+        if constexpr (EXACT) {
 #pragma unroll
-      for (int j = 0; j < TPI; ++j) c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.f;
+          for (int j = 0; j < TPI; ++j) {
+            const unsigned char* tile;
+            if constexpr (PAGED) tile = tp[j];
+            else tile = unit + (int64_t)(TT + j) * (KB * NG * 512);
+            const bool ok = (TT + j) * 16 < c1;
 #pragma unroll
-      for (int grp = 0; grp < NG; ++grp) {
-#pragma unroll
-        for (int j = 0; j < TPI; ++j) mma_tile<KB>(c[j], a[j], f[grp], n_blocks - grp * KB);
-        // the registers are free again: the next group, or the next batch of tiles, at once
-        if (grp + 1 < NG) {
-          fetch(a, T, grp + 1);
-        } else if ((T + step) * 16 < c1) {
-          if constexpr (PAGED) {
-#pragma unroll
-            for (int j = 0; j < TPI; ++j) tp[j] = tp_next[j];
+            for (int i = 0; i < KB; ++i)
+              aa[j][i] = ok ? ld_proxy_u4(tile + (grp * KB + i) * 512 + lane * 16) : make_uint4(0u, 0u, 0u, 0u);
           }
-          fetch(a, T + step, 0);
-          locate(tp_next, T + 2 * step);
-        }
-      }
-#pragma unroll
-      for (int pr = 0; pr < TPI / 2; ++pr) {
-        float a_lo, a_hi, b_lo, b_hi, sc;
-        if (p.max_reduce) {     // uniform
-          reduce_heads<true>(c[2 * pr], p.group, lane, a_lo, a_hi);
-          reduce_heads<true>(c[2 * pr + 1], p.group, lane, b_lo, b_hi);
         } else {
-          reduce_heads<false>(c[2 * pr], p.group, lane, a_lo, a_hi);
-          reduce_heads<false>(c[2 * pr + 1], p.group, lane, b_lo, b_hi);
+          fetch(aa, TT, grp);
         }
-        const int row = (T + 2 * pr) * 16 + pick_row_of_pair(lane, a_lo, a_hi, b_lo, b_hi, sc);
-        if (row < c1) {
-          const uint32_t key = fasa_item_key(sc, row, len, p.n_sink, p.n_recent);
-          atomicAdd(&hist0[key >> 21], 1u);
-          keys[row - c0] = key;
-          if (srow) srow[row] = sc;
+      };
+      while (T * 16 < c1) {       // uniform over the warp
+        float c[TPI][4];
+#pragma unroll
+        for (int j = 0; j < TPI; ++j) c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.f;
+#pragma unroll
+        for (int grp = 0; grp < NG; ++grp) {
+#pragma unroll
+          for (int j = 0; j < TPI; ++j) {
+            if constexpr (EXACT) {
+#pragma unroll
+              for (int kb = 0; kb < KB; ++kb) mma_bf16_16816(c[j], a[j][kb], f[grp].b[kb]);
+            } else {
+              mma_tile<KB>(c[j], a[j], f[grp], n_blocks - grp * KB);
+            }
+          }
+          // the registers are free again: the next group, or the next batch of tiles, at once
+          if (grp + 1 < NG) {
+            fetch_x(a, T, grp + 1);
+          } else if ((T + step) * 16 < c1) {
+            if constexpr (PAGED) {
+#pragma unroll
+              for (int j = 0; j < TPI; ++j) tp[j] = tp_next[j];
+            }
+            fetch_x(a, T + step, 0);
+            locate(tp_next, T + 2 * step);
+          }
         }
+#pragma unroll
+        for (int pr = 0; pr < TPI / 2; ++pr) {
+          float a_lo, a_hi, b_lo, b_hi, sc;
+          if (p.max_reduce) {     // uniform
+            reduce_heads<true>(c[2 * pr], p.group, lane, a_lo, a_hi);
+            reduce_heads<true>(c[2 * pr + 1], p.group, lane, b_lo, b_hi);
+          } else {
+            reduce_heads<false>(c[2 * pr], p.group, lane, a_lo, a_hi);
+            reduce_heads<false>(c[2 * pr + 1], p.group, lane, b_lo, b_hi);
+          }
+          const int row = (T + 2 * pr) * 16 + pick_row_of_pair(lane, a_lo, a_hi, b_lo, b_hi, sc);
+          if (row < c1) {
+            const uint32_t key = fasa_item_key(sc, row, len, p.n_sink, p.n_recent);
+            atomicAdd(&hist0[key >> 21], 1u);
+            keys[row - c0] = key;
+            if (srow) srow[row] = sc;
+          }
+        }
+        T += step;
       }
-      T += step;
-    }
+    };
+    if (pg.n8 == 0 && pg.n16 == KB * NG) stream(std::true_type{});
+    else stream(std::false_type{});
   }
   __syncthreads();
 

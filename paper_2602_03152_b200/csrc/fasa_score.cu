@@ -4,6 +4,8 @@
 // channels x up to 8 query heads into partial scores with one mma.sync; several tiles are in
 // flight per warp, and the first batch of loads is issued before the sequence length, the
 // channel table and the query are known.
+#include <type_traits>
+
 #include "fasa_common.cuh"
 #include "fasa_score_core.cuh"
 
@@ -78,25 +80,50 @@ fc_score_kernel(const uint16_t* __restrict__ q, const unsigned char* __restrict_
   };
   look_ahead(T + kScoreWarps * TPI);
 
-  while (T * 16 < row1) {       // uniform over the warp
-    float s_lo[TPI], s_hi[TPI];
+  // The loop exists twice: when the dominant channels fill exactly KB whole 16-channel blocks
+  // (8, 16, 32 FCs), loads and products need no run-time test of the tile geometry.
+  auto stream = [&](auto exact_tag) {
+    constexpr bool EXACT = decltype(exact_tag)::value;
+    while (T * 16 < row1) {       // uniform over the warp
+      float s_lo[TPI], s_hi[TPI];
 #pragma unroll
-    for (int j = 0; j < TPI; ++j) score_tile<KB, MAXRED>(a[j], f, n_blocks, group, lane, s_lo[j], s_hi[j]);
-    const int next = T + kScoreWarps * TPI;
-    if (next * 16 < row1) {
+      for (int j = 0; j < TPI; ++j) {
+        if constexpr (EXACT) {
+          float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int j = 0; j < TPI; ++j)
-        load_tile<KB>(a[j], PAGED ? ahead[j] : tile_at(next + j, nullptr), pg, lane, (next + j) * 16 < row1);
-      look_ahead(next + kScoreWarps * TPI);
+          for (int kb = 0; kb < KB; ++kb) mma_bf16_16816(c, a[j][kb], f.b[kb]);
+          reduce_heads<MAXRED>(c, group, lane, s_lo[j], s_hi[j]);
+        } else {
+          score_tile<KB, MAXRED>(a[j], f, n_blocks, group, lane, s_lo[j], s_hi[j]);
+        }
+      }
+      const int next = T + kScoreWarps * TPI;
+      if (next * 16 < row1) {
+#pragma unroll
+        for (int j = 0; j < TPI; ++j) {
+          const unsigned char* tile = PAGED ? ahead[j] : tile_at(next + j, nullptr);
+          const bool ok = (next + j) * 16 < row1;
+          if constexpr (EXACT) {
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb)
+              a[j][kb] = ok ? ld_proxy_u4(tile + kb * 512 + lane * 16) : make_uint4(0u, 0u, 0u, 0u);
+          } else {
+            load_tile<KB>(a[j], tile, pg, lane, ok);
+          }
+        }
+        look_ahead(next + kScoreWarps * TPI);
+      }
+#pragma unroll
+      for (int p = 0; p < TPI / 2; ++p) {
+        float v;
+        const int row = (T + 2 * p) * 16 + pick_row_of_pair(lane, s_lo[2 * p], s_hi[2 * p], s_lo[2 * p + 1], s_hi[2 * p + 1], v);
+        if (row < row1) srow[row] = v;
+      }
+      T = next;
     }
-#pragma unroll
-    for (int p = 0; p < TPI / 2; ++p) {
-      float v;
-      const int row = (T + 2 * p) * 16 + pick_row_of_pair(lane, s_lo[2 * p], s_hi[2 * p], s_lo[2 * p + 1], s_hi[2 * p + 1], v);
-      if (row < row1) srow[row] = v;
-    }
-    T = next;
-  }
+  };
+  if (pg.n8 == 0 && pg.n16 == KB) stream(std::true_type{});
+  else stream(std::false_type{});
 }
 
 template <int KB>
