@@ -31,6 +31,8 @@
 //
 // Selection and attention of the block reuse the cluster kernel's selection phases and the
 // split-K tensor-core attention with (sequence, query) pairs as rows.
+#include <type_traits>
+
 #include "fasa_common.cuh"
 #include "fasa_score_core.cuh"
 
@@ -92,7 +94,10 @@ __device__ __forceinline__ uint32_t operand_word(int r, int w, int chunks_pad) {
 // KB: 16-channel blocks per proxy tile rounded up to 1, 2, 4 or 8 (the registers of the loads in
 // flight).  Columns of the product: n = 8 g + t for head g of the set and query t of the block
 // (a fixed 8 columns per head, so that the reduction over the heads indexes registers statically).
-template <int KB, bool MAXRED>
+// EXACT: contiguous caches whose dominant channels fill exactly KB whole 16-channel blocks (8, 16,
+// 32, 64 FCs), so loads and stores need no run-time test of the tile geometry or of a page map
+// (the kernel is bound by the instructions it issues per tile, not by HBM).
+template <int KB, bool MAXRED, bool EXACT>
 __global__ void __launch_bounds__(kBT)
 fc_score_batched_kernel(const BatchedParams p) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -155,15 +160,23 @@ fc_score_batched_kernel(const BatchedParams p) {
   // a warp brings proxy tiles 2 warp, 2 warp + 1 of every 128-token tile (16 tokens each)
   // two register stages: tile i + 1 waits in one while the loads of tile i + 2 fill the other
   uint4 a0[2][KB], a1[2][KB];
+  const unsigned char* unit_base = p.proxy + (int64_t)su.kv * tiles_alloc * (KB * 512);   // (EXACT)
+  float* const score_row0 = p.scores + ((int64_t)b * p.q_len * p.n_sets + hs) * p.max_len;    // query 0 of this unit
+  const int64_t score_stride = (int64_t)p.n_sets * p.max_len;                                // one query to the next
   auto fetch = [&](uint4 (&a)[2][KB], int mt) {
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
       const int T16 = mt * 8 + warp * 2 + j;
       const bool ok = T16 < tiles_alloc && T16 * 16 < len;
       const unsigned char* tile = p.proxy;
-      if (ok) tile += proxy_tile_offset(p.pm, b, h, p.n_kv_heads, T16, tiles_alloc, pg.tile_bytes, p.status);
+      if constexpr (EXACT) tile = unit_base + (int64_t)T16 * (KB * 512);
+      else if (ok) tile += proxy_tile_offset(p.pm, b, h, p.n_kv_heads, T16, tiles_alloc, pg.tile_bytes, p.status);
 #pragma unroll
       for (int kb = 0; kb < KB; ++kb) {
+        if constexpr (EXACT) {
+          a[j][kb] = ok ? ld_proxy_u4(tile + kb * 512 + lane * 16) : make_uint4(0u, 0u, 0u, 0u);
+          continue;
+        }
         a[j][kb] = make_uint4(0u, 0u, 0u, 0u);
         if (ok && kb < pg.n16) {
           a[j][kb] = ld_proxy_u4(tile + kb * 512 + lane * 16);
@@ -184,10 +197,10 @@ fc_score_batched_kernel(const BatchedParams p) {
       unsigned char* rowg = base + ((warp * 2 + j) * 2) * group_stride;   // rows g and (next group) g + 8 of this 16-token tile
 #pragma unroll
       for (int kb = 0; kb < KB; ++kb) {
-        if (kb < n_blocks) {
+        if (EXACT || kb < n_blocks) {
           *reinterpret_cast<uint32_t*>(rowg + kb * 256) = a[j][kb].x;
           *reinterpret_cast<uint32_t*>(rowg + group_stride + kb * 256) = a[j][kb].y;
-          if (kb < pg.n16) {
+          if (EXACT || kb < pg.n16) {
             *reinterpret_cast<uint32_t*>(rowg + kb * 256 + 128) = a[j][kb].z;
             *reinterpret_cast<uint32_t*>(rowg + group_stride + kb * 256 + 128) = a[j][kb].w;
           }
@@ -257,7 +270,7 @@ fc_score_batched_kernel(const BatchedParams p) {
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
       if (t < T && j < len - (T - 1 - t))
-        p.scores[(((int64_t)b * T + t) * p.n_sets + hs) * p.max_len + j] = red[t] + 0.0f;   // (-0 becomes +0)
+        score_row0[t * score_stride + j] = red[t] + 0.0f;   // (-0 becomes +0)
     }
   };
   fetch(a0, mt0);
@@ -320,11 +333,18 @@ extern "C" int32_t fasa_fc_score_batched(fasa_ctx_t* ctx, const void* q, const v
     return cudaGetLastError();
   };
   const bool mx = c.group_reduce != 0;
+  const int kb_of = nb <= 1 ? 1 : (nb <= 2 ? 2 : (nb <= 4 ? 4 : 8));
+  const bool exact = ctx->chunks % 2 == 0 && ctx->chunks / 2 == kb_of && c.page_size == 0;
+  auto pick = [&](auto kb_tag) -> cudaError_t {
+    constexpr int K = decltype(kb_tag)::value;
+    if (exact) return mx ? go(fc_score_batched_kernel<K, true, true>) : go(fc_score_batched_kernel<K, false, true>);
+    return mx ? go(fc_score_batched_kernel<K, true, false>) : go(fc_score_batched_kernel<K, false, false>);
+  };
   cudaError_t e;
-  if (nb <= 1) e = mx ? go(fc_score_batched_kernel<1, true>) : go(fc_score_batched_kernel<1, false>);
-  else if (nb <= 2) e = mx ? go(fc_score_batched_kernel<2, true>) : go(fc_score_batched_kernel<2, false>);
-  else if (nb <= 4) e = mx ? go(fc_score_batched_kernel<4, true>) : go(fc_score_batched_kernel<4, false>);
-  else e = mx ? go(fc_score_batched_kernel<8, true>) : go(fc_score_batched_kernel<8, false>);
+  if (kb_of == 1) e = pick(std::integral_constant<int, 1>{});
+  else if (kb_of == 2) e = pick(std::integral_constant<int, 2>{});
+  else if (kb_of == 4) e = pick(std::integral_constant<int, 4>{});
+  else e = pick(std::integral_constant<int, 8>{});
   FASA_CUDA_TRY(ctx, e);
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
