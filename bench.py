@@ -794,6 +794,22 @@ def run_offload(args):
         split = {"us_per_step": us_split, "link_bytes_per_step": split_link, "link_bytes_per_selected_token": 512 - 4 * w.n_dom,
                  "achieved_gbs": split_link / us_split / 1e3, "frac_of_link": split_link / us_split / 1e3 / link_gbs,
                  "max_abs_diff_vs_whole_rows": float((out - out_host).abs().max())}
+        # the forced rows (sinks + recent window) kept on the GPU: they no longer cross the link
+        if w.n_sink + w.n_recent > 0:
+            out_split = out.clone()
+            res_buf = f.alloc_resident()
+            f.m_resident_build(knd, vh, proxy, t["seq_lens"])
+            torch.cuda.synchronize()
+            us_res, _ = timed(lambda: f.m_decode_step(s["q"], knd, vh, proxy, lens, w.budget, None, idx, n_sel, out, ws, None,
+                                                      s["k_new"], s["v_new"]), args.steps, args.warmup, reset)
+            forced = sum(min(int(L), w.n_sink + w.n_recent) for L in t["seq_lens"].cpu().tolist()) * w.n_kv_heads
+            res_link = (nsel - forced) * (512 - 4 * w.n_dom) + w.batch * w.n_kv_heads * (512 - 4 * w.n_dom)
+            split["resident_forced_rows"] = {
+                "us_per_step": us_res, "link_bytes_per_step": res_link, "rows_kept_on_gpu_per_unit": w.n_sink + w.n_recent,
+                "gpu_bytes": int(res_buf.numel()), "achieved_gbs": res_link / us_res / 1e3,
+                "frac_of_link": res_link / us_res / 1e3 / link_gbs, "outputs_identical": bool(torch.equal(out, out_split))}
+            f.m_set_resident(None)
+            del res_buf
         del knd
     n_sel_total = int(n_sel.sum().item())
     us_dev, _ = timed(step(t["k"], t["v"]), args.steps, args.warmup, reset)

@@ -402,6 +402,33 @@ int32_t fasa_m_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_new, co
                            int32_t budget, int32_t n_sel_max, float* scores, int32_t* idx,
                            int32_t* n_sel, float* out, float* lse, void* workspace, void* stream);
 
+/* Rows that need not cross the host link (Sec. 4.3 pairs the memory-optimised variant with
+ * prefetching; Algorithm 2, appendix).  The only rows of a step that are known before its
+ * selection ends are the forced ones: the n_sink first positions and the n_recent last ones
+ * (Sec. 4.1's T_t always contains them here).  With a resident buffer registered they are kept
+ * on the GPU for good instead of being fetched every step: fasa_m_kv_append stores every
+ * appended row that is a sink position or among the last n_recent of the grown sequence into
+ * its slot (a slot per sink position, a ring of n_recent slots behind them, each tagged with
+ * the position it holds), and fasa_m_sparse_decode_attn / fasa_m_decode_step copy a selected
+ * row from there whenever the tag of its slot names it, from the host otherwise.  Outputs are
+ * bit-identical with and without the buffer.
+ *   fasa_m_resident_bytes   size of the buffer: per (sequence, KV head) n_sink + n_recent slots of
+ *                           512 bytes (the key row as the kernel assembles it + the value row)
+ *                           and a 4-byte tag each; 0 when n_sink + n_recent = 0 or the split key
+ *                           cache is not available for this configuration.
+ *   fasa_m_set_resident     registers the caller's DEVICE buffer (16-byte aligned, kept by
+ *                           reference, caller-owned; NULL switches the feature off) and enqueues
+ *                           the clearing of its tags on `stream`.  UNSUPPORTED when
+ *                           fasa_m_resident_bytes is 0.
+ *   fasa_m_resident_build   fills the slots from split caches that already hold tokens (after
+ *                           fasa_m_split, or after the buffer was registered late): reads the
+ *                           forced rows of the current lengths from k_nondom / v_cache / proxy_k.
+ * Like the block table, the buffer belongs to the calls of one context in stream order. */
+int64_t fasa_m_resident_bytes(const fasa_ctx_t* ctx);
+int32_t fasa_m_set_resident(fasa_ctx_t* ctx, void* resident, void* stream);
+int32_t fasa_m_resident_build(fasa_ctx_t* ctx, const void* k_nondom, const void* v_cache,
+                              const void* proxy_k, const int32_t* seq_lens, void* stream);
+
 /* End-to-end step from HOST buffers: q_host, k_new_host, v_new_host (layouts as
  * fasa_kv_append with n_new = 1) -> fasa_append_decode_step -> out copied to out_host
  * (fp32 [batch][n_q_heads][128]); synchronises the stream.  Inputs in pinned (page-locked,

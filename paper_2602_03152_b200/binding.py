@@ -28,6 +28,7 @@ SYMBOLS = [
     "fasa_sparse_decode_attn_static", "fasa_set_step_mode", "fasa_step_cluster_size",
     "fasa_append_decode_step", "fasa_proxy_bytes", "fasa_select_step",
     "fasa_m_nondom_row_elems", "fasa_m_split", "fasa_m_kv_append", "fasa_m_sparse_decode_attn", "fasa_m_decode_step",
+    "fasa_m_resident_bytes", "fasa_m_set_resident", "fasa_m_resident_build",
     "fasa_fc_score_batched", "fasa_topk_batched", "fasa_sparse_decode_attn_batched", "fasa_decode_step_batched",
     "fasa_calib_workspace_bytes", "fasa_calib_accumulate", "fasa_calib_select", "fasa_set_block_table",
 ]
@@ -92,6 +93,9 @@ def load_library() -> ctypes.CDLL:
         "fasa_m_kv_append": (i32, [vp] * 7 + [i32, vp]),
         "fasa_m_sparse_decode_attn": (i32, [vp] * 7 + [i32] + [vp] * 4),
         "fasa_m_decode_step": (i32, [vp] * 8 + [i32, i32] + [vp] * 7),
+        "fasa_m_resident_bytes": (i64, [vp]),
+        "fasa_m_set_resident": (i32, [vp, vp, vp]),
+        "fasa_m_resident_build": (i32, [vp] * 6),
         "fasa_fc_score_batched": (i32, [vp, vp, vp, vp, i32, vp, vp]),
         "fasa_topk_batched": (i32, [vp, vp, vp, i32, i32, i32, vp, vp, vp]),
         "fasa_sparse_decode_attn_batched": (i32, [vp] * 6 + [i32, i32] + [vp] * 4),
@@ -345,6 +349,24 @@ class Fasa:
             v_cache.data_ptr(), _dp(proxy_k), _dp(seq_lens, torch.int32), budget, idx.shape[-1], _dp(scores, torch.float32),
             _dp(idx, torch.int32), _dp(n_sel, torch.int32), _dp(out, torch.float32), _dp(lse), _dp(workspace), _stream()),
             "fasa_m_decode_step")
+
+    def alloc_resident(self) -> torch.Tensor:
+        """Device buffer for the GPU-resident sink / recent rows of the memory-optimised variant, registered."""
+        n = int(self._lib.fasa_m_resident_bytes(self._h))
+        if n == 0:
+            raise FasaError(ERR_UNSUPPORTED, "fasa_m_resident_bytes", "no forced positions, or no split key cache")
+        buf = torch.empty(n, dtype=torch.uint8, device="cuda")
+        self.m_set_resident(buf)
+        return buf
+
+    def m_set_resident(self, buf):
+        self._check(self._lib.fasa_m_set_resident(self._h, None if buf is None else buf.data_ptr(), _stream()),
+                    "fasa_m_set_resident")
+        self._resident = buf                       # (kept by reference in the library)
+
+    def m_resident_build(self, k_nondom, v_cache, proxy_k, seq_lens):
+        self._check(self._lib.fasa_m_resident_build(self._h, k_nondom.data_ptr(), v_cache.data_ptr(), _dp(proxy_k),
+                                                    _dp(seq_lens, torch.int32), _stream()), "fasa_m_resident_build")
 
     # -- blocks of query tokens: tensors carry a query axis after the batch axis ------
     def fc_score_batched(self, q, proxy_k, seq_lens, scores):

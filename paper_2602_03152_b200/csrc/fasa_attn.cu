@@ -465,6 +465,13 @@ decode_attn_mma_kernel(const AttnParams p) {
         atomicOr(p.status, FASA_DEV_IDX_CLAMPED);
         tok = 0;
       }
+      if constexpr (KSPLIT) {
+        // a row that is resident on the GPU is entered as -1 - slot: it is then copied from there
+        if (p.ks.res.tags != nullptr) {
+          const int slot = fasa_resident_slot(p.ks.res, tok);
+          if (slot >= 0 && p.ks.res.tags[(int64_t)su.kv * p.ks.res.slots_pad + slot] == tok) tok = -1 - slot;
+        }
+      }
       s_idx[i] = tok;
     }
     __syncthreads();
@@ -496,18 +503,39 @@ decode_attn_mma_kernel(const AttnParams p) {
   // Combine: the 16 key rows of a tile from their two homes
   const ProxyGeom ks_pg = proxy_geom(KSPLIT ? p.ks.chunks : 1);
   const unsigned char* ks_proxy = KSPLIT ? p.ks.proxy + (int64_t)su.kv * ((p.max_len + 15) >> 4) * ks_pg.tile_bytes : nullptr;
+  const uint16_t* res_rows = KSPLIT && p.ks.res.tags ? p.ks.res.rows + (int64_t)su.kv * p.ks.res.slots * 2 * FASA_HEAD_DIM : nullptr;
   auto stage_split_k = [&](uint16_t (*dst)[kRowPad], int base) {
     const int nd_chunks = p.ks.nd >> 3, words = 4 * p.ks.chunks;
     for (int c = lane; c < 16 * nd_chunks; c += 32) {                 // the part that crosses the link
       const int row = c / nd_chunks, ch = c % nd_chunks;
       const int tok = s_idx[min(base + row, r1 - 1) - r0];
-      cp_async16_ca(&dst[row][ch * 8], kunit + (int64_t)tok * p.kst + ch * 8);
+      if (tok >= 0) cp_async16_ca(&dst[row][ch * 8], kunit + (int64_t)tok * p.kst + ch * 8);
     }
     for (int c = lane; c < 16 * words; c += 32) {                     // the dominant pairs, from the proxy
       const int row = c / words, w = c % words;
       const int tok = s_idx[min(base + row, r1 - 1) - r0];
-      cp_async4(&dst[row][p.ks.nd + 2 * w], ks_proxy + proxy_word_offset(ks_pg, tok, w));
+      if (tok >= 0) cp_async4(&dst[row][p.ks.nd + 2 * w], ks_proxy + proxy_word_offset(ks_pg, tok, w));
     }
+    if (res_rows != nullptr) {                                        // resident rows: whole assembled key rows
+      for (int c = lane; c < 16 * 16; c += 32) {
+        const int row = c >> 4, ch = c & 15;
+        const int tok = s_idx[min(base + row, r1 - 1) - r0];
+        if (tok < 0) cp_async16(&dst[row][ch * 8], res_rows + (int64_t)(-1 - tok) * 2 * FASA_HEAD_DIM + ch * 8);
+      }
+    }
+  };
+  // value rows of a tile with a split key cache: from the host, or from the resident rows
+  auto stage_split_v = [&](uint16_t (*dst)[kRowPad], int base) {
+    for (int c = lane; c < 16 * 16; c += 32) {
+      const int row = c >> 4, ch = c & 15;
+      const int tok = s_idx[min(base + row, r1 - 1) - r0];
+      if (tok >= 0) cp_async16_ca(&dst[row][ch * 8], vunit + (int64_t)tok * p.vst + ch * 8);
+      else cp_async16(&dst[row][ch * 8], res_rows + (int64_t)(-1 - tok) * 2 * FASA_HEAD_DIM + FASA_HEAD_DIM + ch * 8);
+    }
+  };
+  auto stage_v = [&](int base) {
+    if constexpr (KSPLIT) stage_split_v(sm.v[warp], base);
+    else stage(sm.v[warp], vunit, p.vsb, p.vsh, p.vst, base);
   };
   auto stage_k = [&](int base) {
     if constexpr (KSPLIT) stage_split_k(sm.k[warp], base);
@@ -516,7 +544,7 @@ decode_attn_mma_kernel(const AttnParams p) {
   constexpr int kTileStep = kMmaWarps * 16;
   if (r0 + warp * 16 < r1) stage_k(r0 + warp * 16);
   cp_async_commit();
-  if (r0 + warp * 16 < r1) stage(sm.v[warp], vunit, p.vsb, p.vsh, p.vst, r0 + warp * 16);
+  if (r0 + warp * 16 < r1) stage_v(r0 + warp * 16);
   cp_async_commit();
 
   for (int base = r0 + warp * 16; base < r1; base += kTileStep) {   // uniform over the warp
@@ -587,7 +615,7 @@ decode_attn_mma_kernel(const AttnParams p) {
       mma16816(acc[cb], a, pl0, pl1);
     }
     __syncwarp();                                   // every lane is done with the V buffer
-    if (more) stage(sm.v[warp], vunit, p.vsb, p.vsh, p.vst, base + kTileStep);
+    if (more) stage_v(base + kTileStep);
     cp_async_commit();
   }
   cp_async_wait<0>();
@@ -814,6 +842,7 @@ int32_t fasa_attn_split_keys(fasa_ctx* ctx, const void* q, const void* k_nondom,
   fasa_ksplit ks;
   ks.proxy = (const unsigned char*)proxy_k; ks.ndchan = ctx->d_ndchan; ks.chan = ctx->d_chan;
   ks.chunks = ctx->chunks; ks.nd = FASA_HEAD_DIM - 2 * c.n_dom;
+  ks.res = fasa_resident_of(ctx);
   // (the kernel addresses k_nondom with the K strides: rows of nd elements, dense per unit)
   fasa_ctx tmp = *ctx;
   tmp.cfg.k_stride_t = ks.nd;

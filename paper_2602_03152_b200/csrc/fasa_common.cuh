@@ -26,6 +26,7 @@ struct fasa_ctx {
   int page_shift;         // log2(page_size), 0 for contiguous caches
   int pages_per_seq;      // ceil(max_len / page_size)
   int16_t* d_chan;        // device [n_kv_heads][row_elems]: K channel of each proxy element, -1 = padding
+  void* m_resident;       // memory-optimised variant: the caller's buffer of GPU-resident sink / recent rows (null: none)
   int16_t* d_ndchan;      // device [n_kv_heads][128 - 2 n_dom]: the other channels of each head, ascending (null
                           // unless n_dom is a multiple of 4: the split key cache of the memory-optimised variant)
   int32_t* d_status;      // device status word (FASA_DEV_* bits)
@@ -106,12 +107,27 @@ int32_t fasa_sparse_attn_mirrored(fasa_ctx* ctx, const void* q, const void* k_ca
                                   float* lse, void* workspace, cudaStream_t stream, float* out_mirror, bool* mirrored);
 
 // Split key cache (memory-optimised variant): what the attention kernels need besides k_nondom.
+// The rows every step attends to (the sink positions and the recent window) can stay on the GPU:
+// a slot per sink position and a ring of n_recent slots for the positions behind them, each
+// tagged with the position it holds.  A slot holds the key row as the attention kernel
+// assembles it (non-dominant channels, then the dominant pairs in proxy order) and the value row.
+struct fasa_resident {
+  int32_t* tags;                // [batch * n_kv_heads][slots_pad]: position held by each slot, -1 = none
+  uint16_t* rows;               // [batch * n_kv_heads][slots][2][128]
+  int slots, slots_pad, n_sink, n_recent;   // tags == nullptr: no resident rows
+};
+__host__ __device__ inline int fasa_resident_slot(const fasa_resident& r, int tok) {
+  if (tok < r.n_sink) return tok;
+  return r.n_recent > 0 ? r.n_sink + (tok - r.n_sink) % r.n_recent : -1;
+}
 struct fasa_ksplit {
   const unsigned char* proxy;   // the dominant part, on the GPU
   const int16_t* ndchan;        // [n_kv_heads][nd]
   const int16_t* chan;          // [n_kv_heads][2 n_dom]
   int chunks, nd;               // 16-byte chunks per proxy row; non-dominant channels per key
+  fasa_resident res;            // rows that need not cross the host link
 };
+fasa_resident fasa_resident_of(const fasa_ctx* ctx);
 int32_t fasa_attn_split_keys(fasa_ctx* ctx, const void* q, const void* k_nondom, const void* v_cache, const void* proxy_k,
                              const int32_t* idx, const int32_t* n_sel, int32_t n_sel_max, float* out, float* lse,
                              void* workspace, cudaStream_t stream);

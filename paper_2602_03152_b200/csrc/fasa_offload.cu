@@ -28,7 +28,7 @@ split_rows_kernel(const uint16_t* __restrict__ k_src, const uint16_t* __restrict
                   int32_t* seq_lens_w, int32_t* arrive, const int16_t* __restrict__ chan,
                   const int16_t* __restrict__ ndchan, int32_t* __restrict__ status, int n_new, int n_kv_heads,
                   int max_len, int chunks, int nd, int64_t ksb, int64_t ksh, int64_t kst, int64_t vsb, int64_t vsh,
-                  int64_t vst) {
+                  int64_t vst, const fasa_resident res) {
   __shared__ __align__(16) uint16_t s_k[kSplitRows][FASA_HEAD_DIM];
   const int u = blockIdx.y, h = u % n_kv_heads, b = u / n_kv_heads, tid = threadIdx.x;
   const int len = clamp_len(seq_lens[b], max_len, status);
@@ -47,6 +47,15 @@ split_rows_kernel(const uint16_t* __restrict__ k_src, const uint16_t* __restrict
   const int n_src = APPEND ? n_new : len;
   const int first = APPEND ? len + n0 : n0;              // destination row of source row n0
   if (n0 >= n_src) return;
+  // Resident rows (APPEND): an appended row that is a sink position, or one of the last n_recent of
+  // the grown sequence, is also kept on the GPU, assembled as the attention kernel reads it.
+  const int grown_len = min(max_len, len + n_new);
+  auto res_slot_of = [&](int pos) -> int {
+    if (!APPEND || res.tags == nullptr || pos >= max_len) return -1;
+    if (pos >= res.n_sink && pos < grown_len - res.n_recent) return -1;
+    return fasa_resident_slot(res, pos);
+  };
+  uint16_t* res_unit = APPEND && res.tags ? res.rows + (int64_t)u * res.slots * 2 * FASA_HEAD_DIM : nullptr;
   if (APPEND && first + min(kSplitRows, n_src - n0) > max_len && tid == 0) atomicOr(status, FASA_DEV_APPEND_FULL);
   const int r = tid >> 4, c8 = (tid & 15) * 8;
   const bool row_ok = n0 + r < n_src && first + r < max_len;
@@ -55,9 +64,15 @@ split_rows_kernel(const uint16_t* __restrict__ k_src, const uint16_t* __restrict
     const uint16_t* ks = APPEND ? k_src + ((int64_t)u * n_new + n0 + r) * FASA_HEAD_DIM
                                 : k_src + b * ksb + h * ksh + (int64_t)(first + r) * kst;
     kx = *reinterpret_cast<const uint4*>(ks + c8);
-    if (APPEND)
-      *reinterpret_cast<uint4*>(v_cache + b * vsb + h * vsh + (int64_t)(first + r) * vst + c8) =
-          *reinterpret_cast<const uint4*>(v_src + ((int64_t)u * n_new + n0 + r) * FASA_HEAD_DIM + c8);
+    if (APPEND) {
+      const uint4 vx = *reinterpret_cast<const uint4*>(v_src + ((int64_t)u * n_new + n0 + r) * FASA_HEAD_DIM + c8);
+      *reinterpret_cast<uint4*>(v_cache + b * vsb + h * vsh + (int64_t)(first + r) * vst + c8) = vx;
+      const int slot = res_slot_of(first + r);
+      if (slot >= 0) {
+        *reinterpret_cast<uint4*>(res_unit + (int64_t)slot * 2 * FASA_HEAD_DIM + FASA_HEAD_DIM + c8) = vx;
+        if (c8 == 0) res.tags[(int64_t)u * res.slots_pad + slot] = first + r;
+      }
+    }
   }
   *reinterpret_cast<uint4*>(&s_k[r][c8]) = kx;
   __syncthreads();
@@ -69,6 +84,8 @@ split_rows_kernel(const uint16_t* __restrict__ k_src, const uint16_t* __restrict
     if (n0 + rr >= n_src || first + rr >= max_len) continue;
     const uint32_t lo = s_k[rr][nch[2 * w]], hi = s_k[rr][nch[2 * w + 1]];
     *reinterpret_cast<uint32_t*>(dst_unit + (int64_t)(first + rr) * nd + 2 * w) = lo | (hi << 16);
+    const int slot = res_slot_of(first + rr);
+    if (slot >= 0) *reinterpret_cast<uint32_t*>(res_unit + (int64_t)slot * 2 * FASA_HEAD_DIM + 2 * w) = lo | (hi << 16);
   }
   if (APPEND) {
     const ProxyGeom pg = proxy_geom(chunks);
@@ -80,7 +97,45 @@ split_rows_kernel(const uint16_t* __restrict__ k_src, const uint16_t* __restrict
       if (n0 + rr >= n_src || first + rr >= max_len) continue;
       const uint32_t lo = s_k[rr][ch[2 * w]], hi = s_k[rr][ch[2 * w + 1]];
       *reinterpret_cast<uint32_t*>(punit + proxy_word_offset(pg, first + rr, w)) = lo | (hi << 16);
+      const int slot = res_slot_of(first + rr);
+      if (slot >= 0) *reinterpret_cast<uint32_t*>(res_unit + (int64_t)slot * 2 * FASA_HEAD_DIM + nd + 2 * w) = lo | (hi << 16);
     }
+  }
+}
+
+// Fills the resident rows of one (batch, KV head) unit from the split caches as they stand: the
+// sink positions and the last n_recent positions of the sequence.  One warp per row.
+__global__ void __launch_bounds__(256)
+resident_build_kernel(const uint16_t* __restrict__ k_nondom, const uint16_t* __restrict__ v_cache,
+                      const unsigned char* __restrict__ proxy, const int32_t* __restrict__ seq_lens,
+                      int32_t* __restrict__ status, int n_kv_heads, int max_len, int chunks, int nd, int64_t vsb,
+                      int64_t vsh, int64_t vst, const fasa_resident res) {
+  const int u = blockIdx.x, h = u % n_kv_heads, b = u / n_kv_heads;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int len = clamp_len(seq_lens[b], max_len, status);
+  const ProxyGeom pg = proxy_geom(chunks);
+  const unsigned char* punit = proxy + (int64_t)u * ((max_len + 15) >> 4) * pg.tile_bytes;
+  for (int s = warp; s < res.slots; s += 8) {
+    // the position this slot holds now, if any
+    int pos = -1;
+    if (s < res.n_sink) {
+      if (s < len) pos = s;
+    } else if (len > res.n_sink) {
+      const int lo = max(res.n_sink, len - res.n_recent);       // first position of the window
+      const int cand = lo + ((s - res.n_sink) - (lo - res.n_sink) % res.n_recent + res.n_recent) % res.n_recent;
+      if (cand < len) pos = cand;
+    }
+    uint16_t* row = res.rows + ((int64_t)u * res.slots + s) * 2 * FASA_HEAD_DIM;
+    if (pos >= 0) {
+      for (int c = lane; c < nd / 2; c += 32)
+        reinterpret_cast<uint32_t*>(row)[c] = reinterpret_cast<const uint32_t*>(k_nondom + ((int64_t)u * max_len + pos) * nd)[c];
+      for (int w = lane; w < 4 * chunks; w += 32)
+        reinterpret_cast<uint32_t*>(row + nd)[w] = *reinterpret_cast<const uint32_t*>(punit + proxy_word_offset(pg, pos, w));
+      for (int c = lane; c < FASA_HEAD_DIM / 2; c += 32)
+        reinterpret_cast<uint32_t*>(row + FASA_HEAD_DIM)[c] =
+            reinterpret_cast<const uint32_t*>(v_cache + b * vsb + h * vsh + (int64_t)pos * vst)[c];
+    }
+    if (lane == 0) res.tags[(int64_t)u * res.slots_pad + s] = pos;
   }
 }
 
@@ -103,7 +158,7 @@ extern "C" int32_t fasa_m_split(fasa_ctx_t* ctx, const void* k_cache, void* k_no
   split_rows_kernel<false><<<grid, 256, 0, (cudaStream_t)stream>>>(
       (const uint16_t*)k_cache, nullptr, (uint16_t*)k_nondom, nullptr, nullptr, seq_lens, nullptr, nullptr, ctx->d_chan,
       ctx->d_ndchan, ctx->d_status, 0, c.n_kv_heads, c.max_len, ctx->chunks, FASA_HEAD_DIM - 2 * c.n_dom, c.k_stride_b,
-      c.k_stride_h, c.k_stride_t, c.v_stride_b, c.v_stride_h, c.v_stride_t);
+      c.k_stride_h, c.k_stride_t, c.v_stride_b, c.v_stride_h, c.v_stride_t, fasa_resident{});
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
 }
@@ -120,7 +175,60 @@ extern "C" int32_t fasa_m_kv_append(fasa_ctx_t* ctx, void* k_nondom, void* v_cac
       (const uint16_t*)k_new, (const uint16_t*)v_new, (uint16_t*)k_nondom, (uint16_t*)v_cache, (unsigned char*)proxy_k,
       seq_lens, seq_lens, ctx->d_arrive, ctx->d_chan, ctx->d_ndchan, ctx->d_status, n_new, c.n_kv_heads, c.max_len,
       ctx->chunks, FASA_HEAD_DIM - 2 * c.n_dom, c.k_stride_b, c.k_stride_h, c.k_stride_t, c.v_stride_b, c.v_stride_h,
-      c.v_stride_t);
+      c.v_stride_t, fasa_resident_of(ctx));
+  FASA_LAUNCH_CHECK(ctx);
+  return FASA_OK;
+}
+
+// ---- GPU-resident copies of the rows every step attends to -------------------------------------
+fasa_resident fasa_resident_of(const fasa_ctx* ctx) {
+  fasa_resident r;
+  memset(&r, 0, sizeof(r));
+  if (ctx->m_resident == nullptr) return r;
+  const fasa_config_t& c = ctx->cfg;
+  r.n_sink = c.n_sink;
+  r.n_recent = c.n_recent;
+  r.slots = c.n_sink + c.n_recent;
+  r.slots_pad = (r.slots + 3) & ~3;
+  r.tags = (int32_t*)ctx->m_resident;
+  r.rows = (uint16_t*)((unsigned char*)ctx->m_resident + (size_t)c.batch * c.n_kv_heads * r.slots_pad * sizeof(int32_t));
+  return r;
+}
+
+extern "C" int64_t fasa_m_resident_bytes(const fasa_ctx_t* ctx) {
+  if (!ctx || !split_ok(ctx)) return 0;
+  const fasa_config_t& c = ctx->cfg;
+  const int64_t slots = c.n_sink + c.n_recent, slots_pad = (slots + 3) & ~3;
+  if (slots == 0) return 0;
+  return (int64_t)c.batch * c.n_kv_heads * (slots_pad * 4 + slots * 2 * FASA_HEAD_DIM * 2);
+}
+
+extern "C" int32_t fasa_m_set_resident(fasa_ctx_t* ctx, void* resident, void* stream) {
+  if (!ctx) return FASA_ERR_INVALID_ARG;
+  if (resident == nullptr) {
+    ctx->m_resident = nullptr;
+    return FASA_OK;
+  }
+  if (!aligned16(resident)) return FASA_ERR_INVALID_ARG;
+  if (fasa_m_resident_bytes(ctx) == 0) return FASA_ERR_UNSUPPORTED;
+  const fasa_config_t& c = ctx->cfg;
+  const size_t tag_bytes = (size_t)c.batch * c.n_kv_heads * (((size_t)c.n_sink + c.n_recent + 3) & ~(size_t)3) * sizeof(int32_t);
+  FASA_CUDA_TRY(ctx, cudaMemsetAsync(resident, 0xff, tag_bytes, (cudaStream_t)stream));   // every tag -1: nothing held
+  ctx->m_resident = resident;
+  return FASA_OK;
+}
+
+extern "C" int32_t fasa_m_resident_build(fasa_ctx_t* ctx, const void* k_nondom, const void* v_cache, const void* proxy_k,
+                                         const int32_t* seq_lens, void* stream) {
+  if (!ctx || !k_nondom || !v_cache || !proxy_k || !seq_lens || !aligned16(k_nondom) || !aligned16(v_cache) ||
+      !aligned16(proxy_k))
+    return FASA_ERR_INVALID_ARG;
+  if (!split_ok(ctx) || ctx->m_resident == nullptr) return FASA_ERR_UNSUPPORTED;
+  const fasa_config_t& c = ctx->cfg;
+  resident_build_kernel<<<(unsigned)(c.batch * c.n_kv_heads), 256, 0, (cudaStream_t)stream>>>(
+      (const uint16_t*)k_nondom, (const uint16_t*)v_cache, (const unsigned char*)proxy_k, seq_lens, ctx->d_status,
+      c.n_kv_heads, c.max_len, ctx->chunks, FASA_HEAD_DIM - 2 * c.n_dom, c.v_stride_b, c.v_stride_h, c.v_stride_t,
+      fasa_resident_of(ctx));
   FASA_LAUNCH_CHECK(ctx);
   return FASA_OK;
 }

@@ -759,6 +759,132 @@ def test_fasa_m_split_key_cache(cfg, kw, budget):
     assert torch.equal(lens2, r.seq_lens) and torch.equal(r.idx, ref_idx) and float((r.out - ref_out).abs().max()) <= 1e-4
 
 
+def _resident_expect(w, dom_sorted_h, k_rows, v_rows):
+    """Rows of the resident buffer for the given K / V rows [n][128] of one KV head."""
+    if w.pairing == 0:
+        c0, c1 = dom_sorted_h, dom_sorted_h + 64
+    else:
+        c0, c1 = 2 * dom_sorted_h, 2 * dom_sorted_h + 1
+    rest = np.setdiff1d(np.arange(128), np.concatenate([c0, c1]))
+    pairs = np.stack([c0, c1], axis=1).reshape(-1)                    # proxy order: (c0, c1) per dominant FC, ascending
+    kk = torch.cat([k_rows[:, torch.from_numpy(rest)], k_rows[:, torch.from_numpy(pairs)]], dim=1)
+    return torch.stack([kk, v_rows], dim=1)                            # [n][2][128]
+
+
+def _check_resident(w, f, buf, dom, k_dev, v_dev, lens):
+    S, Sp = w.n_sink + w.n_recent, (w.n_sink + w.n_recent + 3) & ~3
+    units = w.batch * w.n_kv_heads
+    tags = buf[:units * Sp * 4].view(torch.int32).view(units, Sp).cpu()
+    rows = buf[units * Sp * 4:].view(torch.bfloat16).view(units, S, 2, 128).cpu()
+    dom_sorted = np.sort(dom.numpy(), axis=1)
+    for b in range(w.batch):
+        L = int(lens[b])
+        want = sorted(set(range(min(w.n_sink, L))) | set(range(max(w.n_sink, L - w.n_recent), L)))
+        for h in range(w.n_kv_heads):
+            u = b * w.n_kv_heads + h
+            held = sorted(int(x) for x in tags[u, :S] if x >= 0)
+            assert held == want, (b, h, L)
+            for s_ in range(S):
+                pos = int(tags[u, s_])
+                if pos < 0:
+                    continue
+                assert s_ == (pos if pos < w.n_sink else w.n_sink + (pos - w.n_sink) % w.n_recent)
+                exp = _resident_expect(w, dom_sorted[h], k_dev[b, h, pos:pos + 1].cpu(), v_dev[b, h, pos:pos + 1].cpu())[0]
+                assert torch.equal(rows[u, s_], exp), (b, h, s_, pos)
+
+
+@pytest.mark.parametrize("kw,budget", [
+    (dict(batch=2, max_len=2500, len_lo=900, len_hi=2400), 200),                          # 16 FCs, 4 sinks + 64 recent
+    (dict(batch=3, max_len=700, len_lo=20, len_hi=640, n_dom=8, pairing=1, n_sink=3, n_recent=30), 40),   # a sequence shorter than the window
+])
+def test_fasa_m_resident_forced_rows(kw, budget):
+    # The sink positions and the recent window are part of every selection: with a resident buffer
+    # they stay on the GPU (a slot per position, tagged) and never cross the host link.  The buffer
+    # holds exactly those rows after a build, after single appends and after a bulk append; the
+    # step's results do not change bit for bit; and they still do not change when the host copies
+    # of those rows are overwritten with garbage, which shows where the kernel reads them.
+    w = C["c1"].replace(**kw)
+    r = Run(w)
+    r.build_proxy()
+    f = r.fasa
+    knd, vh = f.alloc_host_nondom(), f.alloc_host_cache()
+    vh.copy_(r.t["v"])
+    f.m_split(r.k, knd, r.seq_lens)
+    s = synth.make_step_inputs(w, 5, "cuda")
+    r.reset_outputs()
+    f.m_decode_step(s["q"], knd, vh, r.proxy, r.seq_lens, budget, None, r.idx, r.n_sel, r.out, r.ws, r.lse)
+    ref = [x.clone() for x in (r.idx, r.n_sel, r.out, r.lse)]
+    assert f._lib.fasa_m_resident_bytes(f._h) == w.batch * w.n_kv_heads * (((w.n_sink + w.n_recent + 3) & ~3) * 4 + (w.n_sink + w.n_recent) * 512)
+    buf = f.alloc_resident()
+    f.m_resident_build(knd, vh, r.proxy, r.seq_lens)
+    torch.cuda.synchronize()
+    _check_resident(w, f, buf, r.dom, r.k, r.v, r.seq_lens.tolist())
+
+    def poison_host(lens):
+        for b in range(w.batch):
+            L = int(lens[b])
+            for lo, hi in ((0, min(w.n_sink, L)), (max(w.n_sink, L - w.n_recent), L)):
+                knd[b, :, lo:hi] = float("nan")
+                vh[b, :, lo:hi] = float("nan")
+
+    for poisoned in (False, True):
+        if poisoned:
+            poison_host(r.seq_lens.tolist())
+        r.reset_outputs()
+        f.m_decode_step(s["q"], knd, vh, r.proxy, r.seq_lens, budget, None, r.idx, r.n_sel, r.out, r.ws, r.lse)
+        torch.cuda.synchronize()
+        assert f.device_status() == 0
+        for x, y in zip((r.idx, r.n_sel, r.out, r.lse), ref):
+            assert torch.equal(x, y), poisoned
+    vh.copy_(r.v)                                  # (the host copies whole again: those rows leave the window below)
+    f.m_split(r.k, knd, r.seq_lens)
+    torch.cuda.synchronize()
+    # three single appends through the step, then a bulk append longer than the window; the whole-row
+    # device caches follow with the ordinary calls and give the reference
+    lens2 = r.seq_lens.clone()
+    for i in range(3):
+        si = synth.make_step_inputs(w, 10 + i, "cuda")
+        f.kv_append(r.k, r.v, r.proxy.clone(), r.seq_lens, si["k_new"], si["v_new"])          # (device caches + lengths)
+        f.m_decode_step(si["q"], knd, vh, r.proxy, lens2, budget, None, r.idx, r.n_sel, r.out, r.ws, None, si["k_new"], si["v_new"])
+        torch.cuda.synchronize()
+        assert torch.equal(lens2, r.seq_lens)
+        _check_resident(w, f, buf, r.dom, r.k, r.v, lens2.tolist())
+    room = w.max_len - int(r.seq_lens.max())
+    n_bulk = min(room, w.n_recent + 37)
+    if n_bulk > 0:
+        g = torch.Generator(device="cuda").manual_seed(77)
+        kb = torch.randn(w.batch, w.n_kv_heads, n_bulk, 128, device="cuda", generator=g).to(torch.bfloat16)
+        vb = torch.randn(w.batch, w.n_kv_heads, n_bulk, 128, device="cuda", generator=g).to(torch.bfloat16)
+        f.kv_append(r.k, r.v, r.proxy.clone(), r.seq_lens, kb, vb)
+        f.m_kv_append(knd, vh, r.proxy, lens2, kb, vb)
+        torch.cuda.synchronize()
+        assert torch.equal(lens2, r.seq_lens)
+        _check_resident(w, f, buf, r.dom, r.k, r.v, lens2.tolist())
+    poison_host(lens2.tolist())
+    s9 = synth.make_step_inputs(w, 9, "cuda")
+    r.reset_outputs()
+    f.decode_step(s9["q"], r.k, r.v, r.proxy, r.seq_lens, budget, None, r.idx, r.n_sel, r.out, None)
+    ref_idx, ref_out = r.idx.clone(), r.out.clone()
+    r.reset_outputs()
+    f.m_decode_step(s9["q"], knd, vh, r.proxy, lens2, budget, None, r.idx, r.n_sel, r.out, r.ws, None)
+    torch.cuda.synchronize()
+    assert f.device_status() == 0 and torch.equal(r.idx, ref_idx)
+    assert bool(torch.isfinite(r.out).all()) and float((r.out - ref_out).abs().max()) <= 1e-4
+    # switched off again: the poisoned host rows are read, which the outputs show
+    f.m_set_resident(None)
+    f.m_decode_step(s9["q"], knd, vh, r.proxy, lens2, budget, None, r.idx, r.n_sel, r.out, r.ws, None)
+    torch.cuda.synchronize()
+    assert not float((r.out - ref_out).abs().max()) <= 1e-2     # (NaN logits: the kernel writes zeros, or NaN)
+
+
+def test_fasa_m_resident_needs_forced_positions():
+    w = C["c4"].replace(batch=1, n_q_heads=8, n_kv_heads=2, max_len=600, len_lo=600, len_hi=600)
+    r = Run(w)
+    assert w.n_sink + w.n_recent == 0 and r.fasa._lib.fasa_m_resident_bytes(r.fasa._h) == 0
+    buf = torch.zeros(1 << 12, dtype=torch.uint8, device="cuda")
+    assert r.fasa._lib.fasa_m_set_resident(r.fasa._h, buf.data_ptr(), None) == binding.ERR_UNSUPPORTED
+
+
 def test_fasa_m_split_needs_whole_chunks():
     w = C["c1"].replace(batch=1, max_len=600, len_lo=600, len_hi=600, n_dom=6)
     r = Run(w)
