@@ -1180,8 +1180,9 @@ def main():
                     help="blocks of query tokens (q_len 1..8) on --config's shape instead of the bench line")
     ap.add_argument("--no-resident", action="store_true", help="--longcot: skip the 28-layer resident measurement")
     ap.add_argument("--sweep-steps", type=int, default=20)
-    ap.add_argument("--step-mode", type=int, default=None, choices=[0, 1],
-                    help="0: fasa_decode_step as three kernels; 1 (default): one cluster kernel where available")
+    ap.add_argument("--step-mode", type=int, default=None, choices=[0, 1, 2],
+                    help="0: fasa_decode_step as three kernels; 1 (default): one cluster kernel where available; "
+                         "2: as 1, with the one-CTA-per-row kernel behind fasa_topk")
     args = ap.parse_args()
 
     if args.sweep:

@@ -288,7 +288,11 @@ int32_t fasa_sparse_decode_attn_static(fasa_ctx_t* ctx, const void* q, const voi
  * max_len; idx is addressed with whatever n_sel_max is passed as its row stride. */
 int32_t fasa_set_step_mode(fasa_ctx_t* ctx, int32_t mode);
 /* (The mode also selects the kernel behind fasa_topk: the cluster kernel's selection phases
- * in mode 1, a register-resident cluster kernel in mode 0; the results are identical.) */
+ * in mode 1, a register-resident cluster kernel in mode 0; the results are identical.  Launches
+ * with more score rows than the step has units - fasa_topk_batched, the calibration - take a
+ * third kernel, one CTA per row, which re-reads the row once per radix level instead of
+ * holding its keys; mode 2 is mode 1 with that kernel behind fasa_topk as well, for rows of
+ * up to 524288 tokens.) */
 /* Cluster size mode 1 runs with for this context; 0 = fasa_decode_step uses mode 0. */
 int32_t fasa_step_cluster_size(const fasa_ctx_t* ctx);
 int32_t fasa_decode_step(fasa_ctx_t* ctx, const void* q, const void* k_cache,

@@ -198,7 +198,8 @@ class Fasa:
         return int(out.value)
 
     def set_step_mode(self, mode: int):
-        """1: decode_step runs as one cluster kernel where available; 0: three separate calls."""
+        """1: decode_step runs as one cluster kernel where available; 0: three separate calls; 2: as 1, with the
+        one-CTA-per-row kernel behind topk."""
         self._check(self._lib.fasa_set_step_mode(self._h, mode), "fasa_set_step_mode")
 
     def step_cluster_size(self) -> int:

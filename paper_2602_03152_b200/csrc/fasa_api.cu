@@ -197,8 +197,9 @@ extern "C" const char* fasa_last_cuda_error(const fasa_ctx_t* ctx) {
 }
 
 extern "C" int32_t fasa_set_step_mode(fasa_ctx_t* ctx, int32_t mode) {
-  if (!ctx || (mode != 0 && mode != 1)) return FASA_ERR_INVALID_ARG;
-  ctx->use_fused = mode;
+  if (!ctx || mode < 0 || mode > 2) return FASA_ERR_INVALID_ARG;
+  ctx->use_fused = mode != 0;
+  ctx->topk_rows = mode == 2;
   return FASA_OK;
 }
 

@@ -38,6 +38,7 @@ struct fasa_ctx {
   int step_cs;            // form (1024 threads, one CTA per SM, half the cluster) where that evens out the stream
   size_t step_smem;
   int use_fused;          // fasa_decode_step takes the one-launch kernel when it is available
+  int topk_rows;          // fasa_topk by the one-CTA-per-row kernel whatever the number of rows (fasa_set_step_mode 2)
   // host-buffer step: the last host pointers seen and what the device can use in their place
   // (null: not page-locked + mapped), so that a decode loop with fixed buffers asks the driver once
   const void* host_seen[4];
@@ -133,6 +134,10 @@ int32_t fasa_attn_split_keys(fasa_ctx* ctx, const void* q, const void* k_nondom,
                              void* workspace, cudaStream_t stream);
 bool fasa_on_host(fasa_ctx* ctx, const void* p);
 
+bool fasa_topk_row_ok(const fasa_ctx* ctx);
+int32_t fasa_topk_row_launch(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens, int32_t budget,
+                             int32_t n_sel_max, int32_t* idx, int32_t* n_sel, int rows_per_seq, int n_sink,
+                             int n_recent, cudaStream_t stream, int q_len);
 int32_t fasa_fused_topk_launch(fasa_ctx* ctx, const float* scores, const int32_t* seq_lens,
                                int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
                                cudaStream_t stream);

@@ -1298,7 +1298,7 @@ def test_device_status_bits_instead_of_faults():
 # ------------------------------------------------------------------ top-k alone ----
 
 def _topk_only(scores_cpu, lens, budget, n_sink, n_recent, n_sel_max, mode=1):
-    """mode 1: the cluster kernel's selection phases; mode 0: the register-resident kernel."""
+    """mode 1: the cluster kernel's selection phases; mode 0: the register-resident kernel; mode 2: one CTA per row."""
     B, H, Lm = scores_cpu.shape
     dom = torch.arange(4, dtype=torch.int32).repeat(H, 1)
     f = binding.Fasa(B, H, H, Lm, dom, n_sink=n_sink, n_recent=n_recent)
@@ -1318,8 +1318,9 @@ def _assert_topk_exact(scores_cpu, lens, budget, n_sink=0, n_recent=0, n_sel_max
     B, H, Lm = scores_cpu.shape
     n_sel_max = n_sel_max or Lm
     idx, ns = _topk_only(scores_cpu, lens, budget, n_sink, n_recent, n_sel_max, 1)
-    idx0, ns0 = _topk_only(scores_cpu, lens, budget, n_sink, n_recent, n_sel_max, 0)
-    assert np.array_equal(idx, idx0) and np.array_equal(ns, ns0)      # both kernels, bit for bit
+    for other in (0, 2):                                               # all three kernels, bit for bit
+        idx0, ns0 = _topk_only(scores_cpu, lens, budget, n_sink, n_recent, n_sel_max, other)
+        assert np.array_equal(idx, idx0) and np.array_equal(ns, ns0), other
     for b in range(B):
         L = lens[b]
         k = budget if budget > 0 else (-budget * L + 999) // 1000
@@ -1355,8 +1356,9 @@ def test_topk_exact_on_crowded_bins():
             _assert_topk_exact(sc, lens, budget)
         _assert_topk_exact(sc, lens, 500, n_sink=3, n_recent=100)
         _assert_topk_exact(sc, lens, -189)
-    # exactly 4096 / 4097 keys in the bin (the capacity of the candidate area), the rest far below
-    for n_in in (4096, 4097):
+    # exactly 4096 / 4097 keys in the bin (the capacity of the cluster kernel's candidate area), and
+    # 8192 / 8193 (that of the one-CTA-per-row kernel's list), the rest far below
+    for n_in in (4096, 4097, 8192, 8193):
         sc = torch.full((1, 1, 30000), -5.0)
         sc[0, 0, torch.randperm(30000, generator=g)[:n_in]] = 1.0 + 0.2 * torch.rand(n_in, generator=g)
         for budget in (1, 2048, n_in - 1, n_in, n_in + 5):
