@@ -1169,14 +1169,14 @@ int32_t fasa_fused_topk_rows(fasa_ctx* ctx, const float* scores, const int32_t* 
                              int32_t budget, int32_t n_sel_max, int32_t* idx, int32_t* n_sel,
                              int rows_per_seq, int n_sink, int n_recent, cudaStream_t stream, int q_len) {
   const fasa_config_t& c = ctx->cfg;
-  // More rows than the step has units, at least one per SM, and long ones (blocks of queries,
-  // calibration): clusters would run in rounds, each paying the whole chain of cluster barriers; one
-  // CTA per row is faster there (calibration of 512 samples at 64-128 K: 18.5 -> 13.4 ms; eight
-  // queries per sequence at batch 8, 64 K: 133 -> 127 us).  For the step's own rows, for few rows and
-  // for short ones the cluster form wins (batch 8 at 64 K: 21 against 36 us; 64 rows of 32 K: 23
-  // against 28 us; 2080 rows of 32 K: 387 against 420 us).
+  // Many long rows (batch 16 at 64-128 K, blocks of queries, calibration): clusters would run in
+  // rounds, each paying the whole chain of cluster barriers; one CTA per row is faster there (128 rows
+  // of 64-128 K: 64 -> 53 us; calibration of 512 samples at 64-128 K: 18.5 -> 11.6 ms; eight queries
+  // per sequence at batch 8, 64 K: 133 -> 105 us).  For few rows and for short ones the cluster form
+  // wins (64 rows of 64 K: 21 against 31 us; 8 rows of 32 K: 16 against 23 us; 2080 rows of 32 K: 387
+  // against 420 us).
   if (fasa_topk_row_ok(ctx) &&
-      ((rows_per_seq > ctx->n_sets && (long long)c.batch * rows_per_seq >= ctx->n_sm && c.max_len >= 65536) || ctx->topk_rows))
+      (((long long)c.batch * rows_per_seq >= ctx->n_sm * 3 / 4 && c.max_len >= 65536) || ctx->topk_rows))
     return fasa_topk_row_launch(ctx, scores, seq_lens, budget, n_sel_max, idx, n_sel, rows_per_seq, n_sink, n_recent, stream, q_len);
   FusedParams p;
   memset(&p, 0, sizeof(p));

@@ -127,6 +127,12 @@ __global__ void __launch_bounds__(kRT, 1) topk_row_kernel(const RowParams p) {
   // A thread keeps kRU 16-byte loads in flight (2 KB per warp) and asks for the next batch before it
   // works on the one that has arrived: what an SM can pull follows the bytes its warps have
   // outstanding, and a row is read at most a handful of times, each time in full.
+  // positions [free_lo, free_hi) are not forced: their key is the score's order key, capped below the forced one
+  const int free_lo = sink, free_hi = len - min(p.n_recent, len - sink);
+  auto plain_key = [](float sc) -> uint32_t {
+    const uint32_t k = fasa_order_key(sc);
+    return k == 0xffffffffu ? 0xfffffffeu : k;
+  };
   auto load_batch = [&](float4 (&v)[kRU], int i0) {
 #pragma unroll
     for (int r = 0; r < kRU; ++r) {
@@ -151,11 +157,19 @@ __global__ void __launch_bounds__(kRT, 1) topk_row_kernel(const RowParams p) {
       for (int r = 0; r < kRU; ++r) {
         const int i = i0 + r * kRT * 4;
         const float sv[4] = {v[r].x, v[r].y, v[r].z, v[r].w};
+        if (i >= free_lo && i + 3 < free_hi) {     // no forced position among the four: the plain key
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (i + e < len) {
-            const uint32_t key = fasa_item_key(sv[e], i + e, len, p.n_sink, p.n_recent);
+          for (int e = 0; e < 4; ++e) {
+            const uint32_t key = plain_key(sv[e]);
             if (above >= 32 || (key >> above) == prefix) atomicAdd(&hist[(key >> shift) & mask], 1u);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            if (i + e < len) {
+              const uint32_t key = fasa_item_key(sv[e], i + e, len, p.n_sink, p.n_recent);
+              if (above >= 32 || (key >> above) == prefix) atomicAdd(&hist[(key >> shift) & mask], 1u);
+            }
           }
         }
       }
@@ -209,32 +223,56 @@ __global__ void __launch_bounds__(kRT, 1) topk_row_kernel(const RowParams p) {
       sv[e] = i < len ? srow[i] : 0.f;
     }
   };
+  // The step's body exists in three forms: two for blocks without forced positions or a ragged end
+  // (threshold known / only its leading bits known), where a key costs a handful of instructions, and
+  // the general one.
+  auto emit = [&](uint32_t ma, uint32_t mc, int w, bool same, uint32_t key) {
+    if (lane == 0) { s_mg[w] = ma; s_me[w] = mc; }
+    if (collect && mc) {
+      uint32_t base = 0;
+      if (lane == 0) base = atomicAdd(&s_ncand, (uint32_t)__popc(mc));
+      base = __shfl_sync(0xffffffffu, base, 0);
+      const uint32_t slot = base + __popc(mc & ((1u << lane) - 1u));
+      if (same && slot < (uint32_t)kRCand) cand[slot] = key;
+    }
+  };
   float sv[8], sv_next[8];
   load_blocks(sv, warp * 2);
   for (int blk0 = warp * 2; blk0 * 128 < len; blk0 += kRW * 2) {    // uniform over the warp; two blocks of 128 tokens
     load_blocks(sv_next, blk0 + kRW * 2);                           // (past the end: no loads)
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int i = blk0 * 128 + 32 * e + lane;
-      const bool in = i < len;
-      const uint32_t key = in ? fasa_item_key(sv[e], i, len, p.n_sink, p.n_recent) : 0u;
-      bool above, same;
+    const int first = blk0 * 128;
+    if (first >= free_lo && first + 256 <= free_hi) {               // uniform over the warp
       if (done) {
-        above = in && key > thr;
-        same = in && key == thr;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const uint32_t key = plain_key(sv[e]);
+          const bool same = key == thr;
+          emit(__ballot_sync(0xffffffffu, key > thr), __ballot_sync(0xffffffffu, same), blk0 * 4 + e, same, key);
+        }
       } else {
-        above = in && (key >> shift) > prefix;
-        same = in && (key >> shift) == prefix;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const uint32_t key = plain_key(sv[e]), top = key >> shift;
+          const bool same = top == prefix;
+          emit(__ballot_sync(0xffffffffu, top > prefix), __ballot_sync(0xffffffffu, same), blk0 * 4 + e, same, key);
+        }
       }
-      const uint32_t ma = __ballot_sync(0xffffffffu, above), mc = __ballot_sync(0xffffffffu, same);
-      const int w = blk0 * 4 + e;
-      if (lane == 0 && w < n_words) { s_mg[w] = ma; s_me[w] = mc; }
-      if (collect && mc) {
-        uint32_t base = 0;
-        if (lane == 0) base = atomicAdd(&s_ncand, (uint32_t)__popc(mc));
-        base = __shfl_sync(0xffffffffu, base, 0);
-        const uint32_t slot = base + __popc(mc & ((1u << lane) - 1u));
-        if (same && slot < (uint32_t)kRCand) cand[slot] = key;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int i = first + 32 * e + lane;
+        const bool in = i < len;
+        const uint32_t key = in ? fasa_item_key(sv[e], i, len, p.n_sink, p.n_recent) : 0u;
+        bool above, same;
+        if (done) {
+          above = in && key > thr;
+          same = in && key == thr;
+        } else {
+          above = in && (key >> shift) > prefix;
+          same = in && (key >> shift) == prefix;
+        }
+        const uint32_t ma = __ballot_sync(0xffffffffu, above), mc = __ballot_sync(0xffffffffu, same);
+        if (blk0 * 4 + e < n_words) emit(ma, mc, blk0 * 4 + e, same, key);
       }
     }
 #pragma unroll
