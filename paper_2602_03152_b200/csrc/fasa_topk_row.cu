@@ -26,6 +26,8 @@ constexpr int kRCand = 8192;            // keys of one bin that the CTA finishes
 constexpr int kRFinBits = 7;
 constexpr int kRFinBins = 1 << kRFinBits;
 constexpr int kRU = 4;                  // 16-byte loads a thread keeps in flight
+constexpr int kRRep = 4;                // copies of the histogram: lane l adds to copy l % 4, so that the keys a warp
+constexpr int kRStride = kRBins + 8;    // crowds into one bin collide four times less; copies start 8 banks apart
 
 struct RowParams {
   const float* scores;                  // [rows][max_len]
@@ -63,7 +65,12 @@ __device__ __forceinline__ void row_block_find(const uint32_t* hist, int nb, uin
                                                int lane, uint32_t* bin, uint32_t* residual, uint32_t* in_bin) {
   const int ng = nb / 32;
   for (int g = warp; g < kRGroups; g += kRW) {
-    const uint32_t v = __reduce_add_sync(0xffffffffu, g < ng ? hist[g * 32 + lane] : 0u);
+    uint32_t x = 0;
+    if (g < ng) {
+#pragma unroll
+      for (int r = 0; r < kRRep; ++r) x += hist[r * kRStride + g * 32 + lane];
+    }
+    const uint32_t v = __reduce_add_sync(0xffffffffu, x);
     if (lane == 0) s_grp[g] = v;
   }
   __syncthreads();
@@ -74,7 +81,9 @@ __device__ __forceinline__ void row_block_find(const uint32_t* hist, int nb, uin
   const uint32_t first = __shfl_sync(0xffffffffu, hi, hit);
   int g = kRGroups - 1 - 2 * hit;
   if (first < res) { res -= first; --g; }
-  const uint32_t v = hist[g * 32 + 31 - lane];      // lane 0 = highest bin of the group
+  uint32_t v = 0;                                   // lane 0 = highest bin of the group
+#pragma unroll
+  for (int r = 0; r < kRRep; ++r) v += hist[r * kRStride + g * 32 + 31 - lane];
   int hit2 = 31;
   uint32_t res2 = 1;
   if (!row_find_kth(v, res, lane, &hit2, &res2)) { hit2 = 31; res2 = 1; }
@@ -93,7 +102,8 @@ __global__ void __launch_bounds__(kRT, 1) topk_row_kernel(const RowParams p) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int u = blockIdx.x, b = u / p.rows_per_seq;
   uint32_t* hist = reinterpret_cast<uint32_t*>(rsm);
-  uint32_t* cand = hist + kRBins;
+  uint32_t* cand = hist + kRRep * kRStride;
+  uint32_t* my_hist = hist + (lane & (kRRep - 1)) * kRStride;
   uint32_t* s_mg = cand + kRCand;                   // keys above the threshold (first: in higher bins)
   uint32_t* s_me = s_mg + (p.max_len >> 5) + 1;     // keys equal to it (first: the candidates)
 
@@ -116,7 +126,7 @@ __global__ void __launch_bounds__(kRT, 1) topk_row_kernel(const RowParams p) {
     if (tid == 0) p.n_sel[u] = 0;
     return;
   }
-  for (int i = tid; i < kRBins; i += kRT) hist[i] = 0u;
+  for (int i = tid; i < kRRep * kRStride; i += kRT) hist[i] = 0u;
   for (int i = tid; i < 3 * kRFinBins; i += kRT) (&s_fin[0][0])[i] = 0u;
   if (tid == 0) s_ncand = 0u;
   __syncthreads();
@@ -161,14 +171,14 @@ __global__ void __launch_bounds__(kRT, 1) topk_row_kernel(const RowParams p) {
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const uint32_t key = plain_key(sv[e]);
-            if (above >= 32 || (key >> above) == prefix) atomicAdd(&hist[(key >> shift) & mask], 1u);
+            if (above >= 32 || (key >> above) == prefix) atomicAdd(&my_hist[(key >> shift) & mask], 1u);
           }
         } else {
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             if (i + e < len) {
               const uint32_t key = fasa_item_key(sv[e], i + e, len, p.n_sink, p.n_recent);
-              if (above >= 32 || (key >> above) == prefix) atomicAdd(&hist[(key >> shift) & mask], 1u);
+              if (above >= 32 || (key >> above) == prefix) atomicAdd(&my_hist[(key >> shift) & mask], 1u);
             }
           }
         }
@@ -186,7 +196,7 @@ __global__ void __launch_bounds__(kRT, 1) topk_row_kernel(const RowParams p) {
   for (int level = 0; level < 3; ++level) {
     const int bits = level == 2 ? 10 : 11;
     if (level > 0) {
-      for (int i = tid; i < kRBins; i += kRT) hist[i] = 0u;
+      for (int i = tid; i < kRRep * kRStride; i += kRT) hist[i] = 0u;
       __syncthreads();
     }
     count_pass(prefix, shift, shift - bits, (1u << bits) - 1u);
@@ -404,9 +414,9 @@ int32_t fasa_topk_row_launch(fasa_ctx* ctx, const float* scores, const int32_t* 
   p.scores = scores; p.seq_lens = seq_lens; p.idx = idx; p.n_sel = n_sel; p.status = ctx->d_status;
   p.rows_per_seq = rows_per_seq; p.max_len = c.max_len; p.n_sink = n_sink; p.n_recent = n_recent;
   p.budget = budget; p.n_sel_max = n_sel_max; p.q_len = q_len;
-  const size_t smem = (size_t)(kRBins + kRCand) * 4 + 2 * ((size_t)(c.max_len >> 5) + 1) * 4;
+  const size_t smem = (size_t)(kRRep * kRStride + kRCand) * 4 + 2 * ((size_t)(c.max_len >> 5) + 1) * 4;
   cudaError_t e = cudaFuncSetAttribute((const void*)topk_row_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)((size_t)(kRBins + kRCand) * 4 + 2 * ((size_t)(kTopkRowMaxLen >> 5) + 1) * 4));
+                                       (int)((size_t)(kRRep * kRStride + kRCand) * 4 + 2 * ((size_t)(kTopkRowMaxLen >> 5) + 1) * 4));
   if (e == cudaSuccess) {
     topk_row_kernel<<<(unsigned)(c.batch * rows_per_seq), kRT, smem, stream>>>(p);
     e = cudaGetLastError();
