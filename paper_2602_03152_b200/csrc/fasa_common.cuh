@@ -37,6 +37,7 @@ struct fasa_ctx {
   int step_threads;       // the decode step's own shape: 512 threads with fused_cs CTAs per cluster, or the wide
   int step_cs;            // form (1024 threads, one CTA per SM, half the cluster) where that evens out the stream
   size_t step_smem;
+  int step_resident;      // clusters of the step's shape that the device holds at once
   int use_fused;          // fasa_decode_step takes the one-launch kernel when it is available
   int topk_rows;          // fasa_topk by the one-CTA-per-row kernel whatever the number of rows (fasa_set_step_mode 2)
   // host-buffer step: the last host pointers seen and what the device can use in their place

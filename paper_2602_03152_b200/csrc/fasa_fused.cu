@@ -110,6 +110,7 @@ struct FusedParams {
   unsigned char* proxy_w;
   int32_t* seq_lens_w;
   int32_t* arrive;
+  int shift_clusters, shift_ctas;   // phase shift of grids that run in rounds: clusters / CTAs resident at once (0: none)
   float* scores;           // nullable
   int32_t* idx;
   int32_t* n_sel;
@@ -245,6 +246,24 @@ fused_decode_kernel(const FusedParams p) {
   const int c0 = min(len, crank * per);
   const int c1 = min(len, c0 + per);
   const int nloc = c1 - c0;
+  // Phase shift.  A grid of several rounds of CTAs runs in lock-step: streams that run side by side
+  // share HBM evenly and end together, after which all their CTAs select at the same time and HBM
+  // idles for the length of a select chain, round after round.  Every second cluster of the FIRST
+  // round therefore starts late by a little under half the time the round's streams take (its own
+  // slice stands for the average; 6.4 bytes per ns is about what the memory delivers), which puts
+  // the two halves of the machine out of phase for the rest of the launch: one half streams while
+  // the other selects.  Measured: batch 16 at 64-128 K 177.9 -> 167.9 us, batch 32 at 64 K
+  // 225.9 -> 189.2 us.  The wait is a sleep bounded by the clock; nothing is waited for.
+  if (MODE != 1 && p.shift_ctas > 0 && (int)blockIdx.y < p.shift_clusters && (blockIdx.y & 1)) {
+    const float ns = 0.45f * (float)p.shift_ctas * (float)nloc * (float)(p.chunks * 16) * (1.0f / 6400.0f);
+    const unsigned long long want = (unsigned long long)fminf(ns, 200000.0f);
+    unsigned long long t0, t1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    do {
+      __nanosleep(1000);
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+    } while (t1 - t0 < want);
+  }
   const int cap = (((p.max_len + cs - 1) / cs) + 31) & ~31;
   const FusedSmem sl = fused_smem_layout(cap, kFW);
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + sl.keys);
@@ -1069,6 +1088,7 @@ int fasa_fused_plan(fasa_ctx* ctx) {
     ctx->step_threads = kFT;
     ctx->step_cs = cs;
     ctx->step_smem = smem;
+    ctx->step_resident = n_clusters;
     const long long ctas = (long long)units * cs;
     // (not down to clusters of one CTA: batch 32 x 4 heads of 7 query heads at 16 K lost 3-6 % that way)
     if (cs >= 4 && ctas > ctx->n_sm && cap_of(cs / 2) <= kCapWide) {
@@ -1095,6 +1115,7 @@ int fasa_fused_plan(fasa_ctx* ctx) {
         ctx->step_threads = 1024;
         ctx->step_cs = cs_w;
         ctx->step_smem = smem_w;
+        ctx->step_resident = n_w;
       } else {
         cudaGetLastError();
       }
@@ -1117,6 +1138,7 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
   p.k_new = (const uint16_t*)k_new; p.v_new = (const uint16_t*)v_new;
   p.k_w = (uint16_t*)k_cache; p.v_w = (uint16_t*)v_cache; p.proxy_w = (unsigned char*)proxy_k;
   p.seq_lens_w = (int32_t*)seq_lens; p.arrive = ctx->d_arrive;
+  p.shift_clusters = 0; p.shift_ctas = 0;
   p.scores = scores; p.idx = idx; p.n_sel = n_sel; p.out = out; p.lse = lse; p.status = ctx->d_status;
   p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.n_sets = ctx->n_sets; p.group = ctx->sel_heads; p.max_len = c.max_len;
   p.chunks = ctx->chunks; p.n_sink = c.n_sink; p.n_recent = c.n_recent; p.budget = budget;
@@ -1136,6 +1158,11 @@ int32_t fasa_fused_launch(fasa_ctx* ctx, const void* q, const void* k_cache, con
   const int threads = wide ? 1024 : kFT, cs_l = wide ? ctx->step_cs : ctx->fused_cs;
   const size_t smem_l = wide ? ctx->step_smem : ctx->fused_smem;
 
+  // (from one and a half rounds of CTAs on: see the kernel)
+  if (ctx->step_resident > 0 && 2ll * c.batch * ctx->n_sets >= 3ll * ctx->step_resident) {
+    p.shift_clusters = ctx->step_resident;
+    p.shift_ctas = ctx->step_resident * cs_l;
+  }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3((unsigned)cs_l, (unsigned)(c.batch * ctx->n_sets), 1);
