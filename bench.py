@@ -50,10 +50,10 @@ L2_FLUSH_BYTES = 256 << 20
 # bytes.  Traffic follows the tokens processed, so for another workload of the same kernel the
 # captured ratio is applied to its own algorithmic bytes and the figure is labelled
 # "extrapolated"; it is reported only while the kernel sources are the captured ones.
-TRAFFIC_CAPTURE = {"kernel": "fused_decode_kernel", "workload": "c4_sweep_llama3_8b_64k", "dram_bytes": 281.30e6,
+TRAFFIC_CAPTURE = {"kernel": "fused_decode_kernel", "workload": "c4_sweep_llama3_8b_64k", "dram_bytes": 281.39e6,
                    "algorithmic_bytes": 277.02e6,
                    "sources": ("paper_2602_03152_b200/csrc/fasa_fused.cu", "paper_2602_03152_b200/csrc/fasa_score_core.cuh"),
-                   "sha1": "e41b75d9a0a27cd120b1765fc9e72c23ef0fe952"}
+                   "sha1": "bcda1628a361a3d74946dc3064adc6dc087de2ef"}
 
 
 def _traffic(bytes_per_launch, workload):
