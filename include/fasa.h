@@ -96,7 +96,7 @@ extern "C" {
 #define FASA_ERR_UNSUPPORTED   -2   /* head_dim != 128, n_dom outside 1..64, group > 8 ... */
 #define FASA_ERR_WORKSPACE     -3   /* n_sel_max / budget larger than the workspace covers */
 #define FASA_ERR_CUDA          -4   /* a CUDA runtime call failed (see fasa_last_cuda_error) */
-#define FASA_ERR_TIMEOUT       -5   /* reserved: no kernel of this library waits           */
+#define FASA_ERR_TIMEOUT       -5   /* reserved: no kernel waits for another; see FASA_DEV_TIMEOUT */
 
 /* Bits of the device status word. */
 #define FASA_DEV_LEN_CLAMPED    1   /* a seq_lens entry was < 0 or > max_len               */
