@@ -1007,6 +1007,23 @@ def run_batched(args):
                       "peak_source": peak_src, "single_query_calls_us": single, "rows": rows}), flush=True)
 
 
+def partial_total(samples, points, key, n_layers):
+    """Seconds of the decode steps up to the last sampled context: per step n_layers x the step time,
+    linearly interpolated between the samples taken so far."""
+    acc = 0.0
+    for L in range(1025, samples[len(points) - 1] + 1):
+        j = 0
+        while j + 1 < len(points) and samples[j + 1] <= L:
+            j += 1
+        if j == len(points) - 1:
+            v = points[j][key]
+        else:
+            x0, x1 = samples[j], samples[j + 1]
+            v = points[j][key] + (points[j + 1][key] - points[j][key]) * (L - x0) / (x1 - x0)
+        acc += v * n_layers
+    return acc * 1e-6
+
+
 def run_longcot(args):
     """Workload c3 (long-CoT shape, Qwen2.5-7B-like attention): 28 layers, batch 32, prompt
     1024 then 15360 decode steps, budget 18.9 % of the current length, 16 dominant FCs.  One
@@ -1032,6 +1049,14 @@ def run_longcot(args):
                     "dense_frac_of_peak": sm["dense_frac_of_peak"], "speedup_vs_dense": sm["speedup_vs_dense"],
                     "device_status": sm["device_status"]})
         del m
+        # progress line (stderr): what a run that is cut short has measured so far
+        done_steps = max(0, min(L, 1024 + 15360) - 1024)
+        print(json.dumps({"longcot_progress": {"sampled_context": L, "decode_steps_covered": done_steps,
+                                               "us_per_step": pts[-1]["us_per_step"],
+                                               "dense_us_per_step": pts[-1]["dense_us_per_step"],
+                                               "fasa_seconds_so_far": partial_total(samples, pts, "us_per_step", 28),
+                                               "dense_seconds_so_far": partial_total(samples, pts, "dense_us_per_step", 28)}}),
+              file=sys.stderr, flush=True)
 
     def total(points, key, n_layers):
         acc = 0.0
